@@ -1,0 +1,136 @@
+/*
+ * gka.h — C ABI of the B200 (sm_100a) Gated KalmaNet hot path.
+ *
+ * The library computes the chunk-wise gated online ridge regression of the GKA layer:
+ * for every (batch, head) pair and token t
+ *
+ *     H_t = gamma_t H_{t-1} + k_t k_t^T          U_t = gamma_t U_{t-1} + v_t k_t^T
+ *     x_t = CH(H_t + lambda_t I, q_t, n_iter)    o_t = U_t x_t
+ *
+ * (forward recurrence, eq. (CH), Section 4.1), where CH is the Chebyshev Iteration of
+ * Algorithm 1 run for exactly n_iter matrix-vector products with eigenvalue bounds
+ * L = ||H_t||_F + lambda_t, mu = lambda_t (Section 4.1, "Adaptive Regularization").
+ * ||H_t||_F is evaluated per token inside each chunk from the chunk-initial state
+ * (Section 4.2.1).  The spec name M_t is the paper's U_t; this header uses U.
+ *
+ * Conventions shared by every call
+ *   - All data pointers are DEVICE pointers, 16-byte aligned, contiguous row-major.
+ *     The descriptor itself is a host struct.
+ *   - q, k : [B, T, heads, d_k];  v, out : [B, T, heads, d_v];  gate, lam : [B, T, heads] float32.
+ *     gate holds gamma_t in (0, 1]; lam holds lambda_t > 0 (absolute), or, with
+ *     GKA_FLAG_ADAPTIVE_LAMBDA, the constant a of lambda_t = a ||H_t||_F (Section 4.1).
+ *   - state / state_in / state_out : [B, heads, d_k*d_k + d_v*d_k] float32; per head first
+ *     H (d_k x d_k, row-major) then U (d_v x d_k, row-major, U[i][j] = sum v_i k_j).
+ *   - The caller owns every buffer.  The library allocates no device memory, keeps no state
+ *     between calls apart from cached device attributes, and never synchronises: work is
+ *     enqueued on desc->stream and the call returns.
+ *   - Argument errors are reported by the return value before anything is launched.  Nothing
+ *     throws or aborts.  Device-side waits are bounded; if one runs out the kernel stores
+ *     GKA_ERR_TIMEOUT into *desc->device_status (when given) and returns cleanly.
+ *   - Supported: d_k == d_v in {64, 128}; chunk == 64; T a multiple of chunk; n_iter >= 0.
+ */
+#ifndef GKA_H_
+#define GKA_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GKA_OK = 0,
+    GKA_ERR_NULL = 1,        /* a required pointer is NULL                                   */
+    GKA_ERR_SHAPE = 2,       /* non-positive size, T not a multiple of chunk, d_k != d_v     */
+    GKA_ERR_DTYPE = 3,       /* unknown io_dtype / precision value                           */
+    GKA_ERR_UNSUPPORTED = 4, /* a shape or mode outside the supported set                    */
+    GKA_ERR_WORKSPACE = 5,   /* workspace missing, misaligned or smaller than required       */
+    GKA_ERR_DOMAIN = 6,      /* reserved: input outside its domain                           */
+    GKA_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed (launch, attribute, map) */
+    GKA_ERR_TIMEOUT = 8,     /* written to *device_status by a kernel whose bounded wait ran out */
+    GKA_ERR_ALIGN = 9        /* a data pointer is not 16-byte aligned                        */
+} gka_status;
+
+typedef enum { GKA_F32 = 0, GKA_BF16 = 1 } gka_dtype;
+
+typedef enum {
+    GKA_PREC_NATIVE = 0, /* bf16 I/O: bf16 tensor-core operands, fp32 accumulation and masters;
+                            f32 I/O: fp32 arithmetic throughout                               */
+    GKA_PREC_HIGH = 1    /* fp32 arithmetic throughout, whatever the I/O dtype                */
+} gka_precision;
+
+enum {
+    GKA_FLAG_ADAPTIVE_LAMBDA = 1u /* lam[] holds a; lambda_t = a * ||H_t||_F (Section 4.1, eq. (4)) */
+};
+
+typedef struct {
+    int B;               /* batch (chunked forward) or number of sequences (decode)          */
+    int T;               /* tokens per sequence; ignored by gka_decode_step                  */
+    int heads;
+    int d_k, d_v;
+    int io_dtype;        /* gka_dtype of q, k, v, out                                         */
+    int precision;       /* gka_precision                                                     */
+    unsigned flags;      /* GKA_FLAG_*                                                        */
+    void *stream;        /* cudaStream_t, caller-owned; NULL = default stream                 */
+    void *workspace;     /* device scratch, >= gka_fwd_workspace_bytes(), 256-byte aligned    */
+    size_t workspace_bytes;
+    const float *state_in; /* optional initial state of the chunked forward; NULL = zero state */
+    int *device_status;  /* optional device int, set by kernels on a bounded-wait timeout     */
+    float *fro_out;      /* optional [B, T, heads] float32: ||H_t||_F per token (debug output) */
+    void *profile_start; /* optional cudaEvent_t recorded on the stream right before the dominant  */
+    void *profile_stop;  /* kernel (main forward kernel / decode kernel) and right after it        */
+} gka_desc;
+
+/*
+ * Scratch the chunked forward needs for this descriptor (segment summaries and segment start
+ * states of the cross-chunk state scan; Section 4.2.1 stores the initial state of every chunk,
+ * this library stores one state per work segment instead and carries the rest on chip).
+ * Returns 0 if the descriptor is invalid.  Pure host arithmetic; no CUDA call.
+ */
+size_t gka_fwd_workspace_bytes(const gka_desc *desc, int chunk);
+
+/*
+ * Chunk-wise forward (eq. (CH) evaluated chunk by chunk, Section 4.2.1; Algorithm 1 on whole
+ * chunks; chunk-wise Frobenius norms).  Writes out[B,T,heads,d_v] in io_dtype and, when
+ * state_out != NULL, the final (H_T, U_T) of every (batch, head) pair.  out and state_out must
+ * not alias any input.  Uses desc->workspace.  Returns GKA_OK once all kernels are enqueued.
+ */
+gka_status gka_fwd_chunked(const gka_desc *desc, const void *q, const void *k, const void *v,
+                           const float *gate, const float *lam, int n_iter, int chunk,
+                           void *out, float *state_out);
+
+/*
+ * Recurrent single-token step (eq. (CH) applied once): state is read, decayed by gate, updated
+ * with k k^T / v k^T and written back in place; out[B,heads,d_v] = U_t CH(H_t + lambda_t I, q_t).
+ * q, k : [B, heads, d_k]; v, out : [B, heads, d_v]; gate, lam : [B, heads].  Needs no workspace.
+ * The state written by gka_fwd_chunked(state_out) is a valid input here.
+ */
+gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, const void *k,
+                           const void *v, const float *gate, const float *lam, int n_iter,
+                           void *out);
+
+/* Static, human-readable name of a status code. */
+const char *gka_status_string(int status);
+
+/*
+ * Work decomposition of the chunked forward, for callers that size buffers or report launch
+ * counts: number of persistent work items (thread blocks) the main kernel uses for this
+ * descriptor on the current device, or a negative gka_status.
+ */
+int gka_fwd_num_work_items(const gka_desc *desc, int chunk);
+
+/*
+ * Introspection of the work decomposition (pure host arithmetic, no CUDA call): the flat list of
+ * B*heads*(T/chunk) chunks is split into num_items contiguous ranges; item `item` owns chunks
+ * [*first_chunk, *end_chunk).  *cut_in / *cut_out tell whether the range starts / ends inside a
+ * sequence (then its start state comes from the cross-item scan / its last run is summarised).
+ * Returns GKA_OK or an argument error.
+ */
+gka_status gka_fwd_work_range(const gka_desc *desc, int chunk, int num_items, int item,
+                              long long *first_chunk, long long *end_chunk, int *cut_in,
+                              int *cut_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GKA_H_ */

@@ -1,0 +1,172 @@
+// C ABI of the GKA library: argument validation, work planning and kernel dispatch.
+// Every step of the path runs in the kernels of this library; nothing here computes.
+#include <stdio.h>
+
+#include "gka_common.cuh"
+
+namespace gka {
+
+cudaError_t launch_fwd_tc(const FwdArgs &a, cudaStream_t stream);   // gka_tc.cu
+bool fwd_tc_available();
+
+namespace {
+
+int g_sm_count = 0;
+
+int sm_count() {
+    if (g_sm_count == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+        g_sm_count = n;
+    }
+    return g_sm_count;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+gka_status check_desc_common(const gka_desc *d) {
+    if (!d) return GKA_ERR_NULL;
+    if (d->B <= 0 || d->heads <= 0 || d->d_k <= 0 || d->d_v <= 0) return GKA_ERR_SHAPE;
+    if (d->d_k != d->d_v) return GKA_ERR_SHAPE;
+    if (d->io_dtype != GKA_F32 && d->io_dtype != GKA_BF16) return GKA_ERR_DTYPE;
+    if (d->precision != GKA_PREC_NATIVE && d->precision != GKA_PREC_HIGH) return GKA_ERR_DTYPE;
+    if (d->d_k != 64 && d->d_k != 128) return GKA_ERR_UNSUPPORTED;
+    if (d->flags & ~(unsigned)GKA_FLAG_ADAPTIVE_LAMBDA) return GKA_ERR_UNSUPPORTED;
+    return GKA_OK;
+}
+
+gka_status check_fwd_shape(const gka_desc *d, int chunk) {
+    gka_status s = check_desc_common(d);
+    if (s != GKA_OK) return s;
+    if (chunk != kChunk) return chunk <= 0 ? GKA_ERR_SHAPE : GKA_ERR_UNSUPPORTED;
+    if (d->T <= 0 || d->T % chunk != 0) return GKA_ERR_SHAPE;
+    return GKA_OK;
+}
+
+// Upper bound on work items used for sizing (independent of the device).
+int work_items_cap(const gka_desc *d, int chunk) {
+    long long nc = (long long)d->B * d->heads * (d->T / chunk);
+    return (int)(nc < kMaxWorkItems ? nc : kMaxWorkItems);
+}
+
+}  // namespace
+}  // namespace gka
+
+using namespace gka;
+
+extern "C" {
+
+const char *gka_status_string(int status) {
+    switch (status) {
+        case GKA_OK: return "GKA_OK";
+        case GKA_ERR_NULL: return "GKA_ERR_NULL: a required pointer is NULL";
+        case GKA_ERR_SHAPE: return "GKA_ERR_SHAPE: bad size (non-positive, T not a multiple of chunk, or d_k != d_v)";
+        case GKA_ERR_DTYPE: return "GKA_ERR_DTYPE: unknown io_dtype or precision";
+        case GKA_ERR_UNSUPPORTED: return "GKA_ERR_UNSUPPORTED: shape or mode outside the supported set";
+        case GKA_ERR_WORKSPACE: return "GKA_ERR_WORKSPACE: workspace missing, misaligned or too small";
+        case GKA_ERR_DOMAIN: return "GKA_ERR_DOMAIN: input outside its domain";
+        case GKA_ERR_CUDA: return "GKA_ERR_CUDA: a CUDA call failed";
+        case GKA_ERR_TIMEOUT: return "GKA_ERR_TIMEOUT: a bounded device-side wait ran out";
+        case GKA_ERR_ALIGN: return "GKA_ERR_ALIGN: a data pointer is not 16-byte aligned";
+        default: return "GKA_ERR_?: unknown status";
+    }
+}
+
+size_t gka_fwd_workspace_bytes(const gka_desc *desc, int chunk) {
+    if (check_fwd_shape(desc, chunk) != GKA_OK) return 0;
+    return workspace_bytes_for(work_items_cap(desc, chunk), desc->d_k, desc->d_v);
+}
+
+int gka_fwd_num_work_items(const gka_desc *desc, int chunk) {
+    gka_status s = check_fwd_shape(desc, chunk);
+    if (s != GKA_OK) return -(int)s;
+    const int sms = sm_count();
+    if (sms <= 0) return -(int)GKA_ERR_CUDA;
+    const int cap = work_items_cap(desc, chunk);
+    return sms < cap ? sms : cap;
+}
+
+gka_status gka_fwd_work_range(const gka_desc *desc, int chunk, int num_items, int item,
+                              long long *first_chunk, long long *end_chunk, int *cut_in,
+                              int *cut_out) {
+    gka_status s = check_fwd_shape(desc, chunk);
+    if (s != GKA_OK) return s;
+    if (!first_chunk || !end_chunk || !cut_in || !cut_out) return GKA_ERR_NULL;
+    WorkPlan p;
+    p.BH = desc->B * desc->heads;
+    p.N = desc->T / chunk;
+    p.NC = (long long)p.BH * p.N;
+    if (num_items <= 0 || num_items > p.NC || item < 0 || item >= num_items) return GKA_ERR_SHAPE;
+    p.G = num_items;
+    *first_chunk = p.lo(item);
+    *end_chunk = p.lo(item + 1);
+    *cut_in = p.cut_in(item) ? 1 : 0;
+    *cut_out = p.cut_out(item) ? 1 : 0;
+    return GKA_OK;
+}
+
+gka_status gka_fwd_chunked(const gka_desc *desc, const void *q, const void *k, const void *v,
+                           const float *gate, const float *lam, int n_iter, int chunk, void *out,
+                           float *state_out) {
+    gka_status s = check_fwd_shape(desc, chunk);
+    if (s != GKA_OK) return s;
+    if (!q || !k || !v || !gate || !lam || !out) return GKA_ERR_NULL;
+    if (n_iter < 0) return GKA_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(gate) || !aligned16(lam) ||
+        !aligned16(out) || !aligned16(state_out) || !aligned16(desc->state_in) ||
+        !aligned16(desc->fro_out))
+        return GKA_ERR_ALIGN;
+    const size_t need = gka_fwd_workspace_bytes(desc, chunk);
+    if (!desc->workspace || desc->workspace_bytes < need ||
+        (reinterpret_cast<uintptr_t>(desc->workspace) & 255u) != 0)
+        return GKA_ERR_WORKSPACE;
+    const int G = gka_fwd_num_work_items(desc, chunk);
+    if (G <= 0) return GKA_ERR_CUDA;
+
+    FwdArgs a;
+    a.q = q; a.k = k; a.v = v; a.gate = gate; a.lam = lam; a.out = out;
+    a.state_out = state_out;
+    a.state_in = desc->state_in;
+    a.fro_out = desc->fro_out;
+    a.device_status = desc->device_status;
+    a.B = desc->B; a.T = desc->T; a.heads = desc->heads;
+    a.n_iter = n_iter;
+    a.flags = desc->flags;
+    a.plan.BH = desc->B * desc->heads;
+    a.plan.N = desc->T / chunk;
+    a.plan.NC = (long long)a.plan.BH * a.plan.N;
+    a.plan.G = G;
+    a.ws = carve_workspace(desc->workspace, G, desc->d_k, desc->d_v);
+    a.ev_start = reinterpret_cast<cudaEvent_t>(desc->profile_start);
+    a.ev_stop = reinterpret_cast<cudaEvent_t>(desc->profile_stop);
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(desc->stream);
+
+    cudaError_t err;
+    const bool tensor_path = desc->io_dtype == GKA_BF16 && desc->precision == GKA_PREC_NATIVE &&
+                             desc->d_k == 128 && fwd_tc_available();
+    if (tensor_path)
+        err = launch_fwd_tc(a, stream);
+    else
+        err = launch_fwd_simt(a, desc->d_k, desc->io_dtype, stream);
+    return err == cudaSuccess ? GKA_OK : GKA_ERR_CUDA;
+}
+
+gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, const void *k,
+                           const void *v, const float *gate, const float *lam, int n_iter,
+                           void *out) {
+    gka_status s = check_desc_common(desc);
+    if (s != GKA_OK) return s;
+    if (!state || !q || !k || !v || !gate || !lam || !out) return GKA_ERR_NULL;
+    if (n_iter < 0) return GKA_ERR_SHAPE;
+    if (!aligned16(state) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+        return GKA_ERR_ALIGN;
+    cudaError_t err = launch_decode(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->heads,
+                                    desc->d_k, desc->io_dtype, desc->flags, desc->device_status,
+                                    reinterpret_cast<cudaEvent_t>(desc->profile_start),
+                                    reinterpret_cast<cudaEvent_t>(desc->profile_stop),
+                                    reinterpret_cast<cudaStream_t>(desc->stream));
+    return err == cudaSuccess ? GKA_OK : GKA_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,155 @@
+// Shared host/device helpers of the GKA library: work decomposition of the chunked
+// forward, workspace layout, I/O type conversion.  No method arithmetic lives here.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/gka.h"
+
+namespace gka {
+
+constexpr int kChunk = 64;            // tokens per chunk (C)
+constexpr int kMaxWorkItems = 296;    // upper bound on persistent work items (2 per SM on 148 SMs)
+
+// ---------------------------------------------------------------------------------------------
+// Work decomposition.  The B*heads sequences of N = T/C chunks each form one flat list of
+// NC = B*heads*N chunks; work item i of G owns the contiguous range [lo(i), lo(i+1)).  A range
+// may cover several sequences and may cut a sequence in the middle.  Where an item's range ends
+// inside a sequence the item's last run is summarised (decay product, delta-H, delta-U) by the
+// summary kernel, a scan turns summaries into the start state of the next item, and the main
+// kernel then processes all items independently, carrying (H, U) on chip inside each run.
+// ---------------------------------------------------------------------------------------------
+struct WorkPlan {
+    int BH;        // B * heads
+    int N;         // chunks per sequence
+    long long NC;  // total chunks
+    int G;         // work items
+    __host__ __device__ long long lo(int i) const { return ((long long)i * NC) / G; }
+    // start of the last run of item i (flat chunk index)
+    __host__ __device__ long long last_run_start(int i) const {
+        long long l = lo(i), h = lo(i + 1);
+        long long s = ((h - 1) / N) * N;
+        return s > l ? s : l;
+    }
+    __host__ __device__ bool cut_out(int i) const { return (lo(i + 1) % N) != 0; }
+    __host__ __device__ bool cut_in(int i) const { return (lo(i) % N) != 0; }
+};
+
+// Workspace layout (floats): start states [G][st], summaries [G][st], running masters [G][st],
+// decay products [G].  st = d_k*d_k + d_v*d_k.
+struct Workspace {
+    float *start;
+    float *delta;
+    float *cur;
+    float *decay;
+};
+
+__host__ __device__ inline size_t state_floats(int dk, int dv) {
+    return (size_t)dk * dk + (size_t)dv * dk;
+}
+
+inline size_t workspace_bytes_for(int G, int dk, int dv) {
+    size_t st = state_floats(dk, dv);
+    size_t fl = 3 * (size_t)G * st + (size_t)G;
+    return ((fl * sizeof(float) + 255) / 256) * 256;
+}
+
+inline Workspace carve_workspace(void *base, int G, int dk, int dv) {
+    size_t st = state_floats(dk, dv);
+    Workspace w;
+    w.start = reinterpret_cast<float *>(base);
+    w.delta = w.start + (size_t)G * st;
+    w.cur = w.delta + (size_t)G * st;
+    w.decay = w.cur + (size_t)G * st;
+    return w;
+}
+
+// ---------------------------------------------------------------------------------------------
+// I/O element access: T is float or __nv_bfloat16; arithmetic always sees float.
+// ---------------------------------------------------------------------------------------------
+template <typename T> struct Io;
+template <> struct Io<float> {
+    static __device__ __forceinline__ float4 load4(const float *p) {
+        return *reinterpret_cast<const float4 *>(p);
+    }
+    static __device__ __forceinline__ void store4(float *p, float4 v) {
+        *reinterpret_cast<float4 *>(p) = v;
+    }
+    static __device__ __forceinline__ float load1(const float *p) { return *p; }
+    static __device__ __forceinline__ void store1(float *p, float v) { *p = v; }
+};
+template <> struct Io<__nv_bfloat16> {
+    static __device__ __forceinline__ float4 load4(const __nv_bfloat16 *p) {
+        uint2 u = *reinterpret_cast<const uint2 *>(p);
+        __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162 *>(&u.x);
+        __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162 *>(&u.y);
+        float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+        return make_float4(fa.x, fa.y, fb.x, fb.y);
+    }
+    static __device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 v) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y);
+        __nv_bfloat162 b = __floats2bfloat162_rn(v.z, v.w);
+        uint2 u;
+        u.x = *reinterpret_cast<uint32_t *>(&a);
+        u.y = *reinterpret_cast<uint32_t *>(&b);
+        *reinterpret_cast<uint2 *>(p) = u;
+    }
+    static __device__ __forceinline__ float load1(const __nv_bfloat16 *p) {
+        return __bfloat162float(*p);
+    }
+    static __device__ __forceinline__ void store1(__nv_bfloat16 *p, float v) {
+        *p = __float2bfloat16_rn(v);
+    }
+};
+
+#ifdef __CUDACC__
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+// Wait for an mbarrier phase with a time limit (about one second of SM clocks).  Returns false if
+// the phase did not complete in time; the caller records GKA_ERR_TIMEOUT and leaves cleanly.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar_addr, uint32_t parity) {
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar_addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if (clock64() - t0 > 2000000000LL) return false;
+    }
+}
+#endif
+
+// Arguments shared by the chunked-forward kernels.
+struct FwdArgs {
+    const void *q, *k, *v;
+    const float *gate, *lam;
+    void *out;
+    float *state_out;
+    const float *state_in;
+    float *fro_out;
+    int *device_status;
+    int B, T, heads;
+    int n_iter;
+    unsigned flags;
+    WorkPlan plan;
+    Workspace ws;
+    cudaEvent_t ev_start, ev_stop;   // optional, recorded around the main kernel (host side only)
+};
+
+// Launchers implemented in the kernel translation units.  Each returns a cudaError_t.
+cudaError_t launch_fwd_simt(const FwdArgs &a, int d, int io_dtype, cudaStream_t stream);
+cudaError_t launch_decode(float *state, const void *q, const void *k, const void *v,
+                          const float *gate, const float *lam, int n_iter, void *out, int nseq,
+                          int heads, int d, int io_dtype, unsigned flags, int *device_status,
+                          cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream);
+
+}  // namespace gka

@@ -1,0 +1,508 @@
+// fp32 chunk-wise GKA forward on CUDA cores (sm_100a).
+//
+// This is the fp32-arithmetic path of gka_fwd_chunked: it serves f32 I/O and GKA_PREC_HIGH.
+// It follows the chunk-wise formulation of Section 4.2.1: per chunk of C = 64 tokens, with the
+// chunk-initial state (H_0, U_0), cumulative gates zeta and the decay mask
+// Gamma[c][j] = zeta_c / zeta_j (j <= c),
+//
+//     ||H_c||_F    from H_0, K and the Gram matrix K K^T                     (chunk-wise norms)
+//     Y = zeta o (X H_0) + (Gamma o (X K^T)) K + lambda o X                  (H_c x_c for all c)
+//     Algorithm 1 on all 64 tokens at once, L = ||H_c||_F + lambda_c, mu = lambda_c
+//     O = zeta o (X U_0^T) + (Gamma o (X K^T)) V
+//     H_C = zeta_C H_0 + K^T diag(Gamma[C]) K,  U_C = zeta_C U_0 + V^T diag(Gamma[C]) K
+//
+// Three kernels: segment summaries, a scan over segments, and the main kernel (gka_common.cuh
+// explains the work decomposition).  One thread block of 256 threads per work item.
+#include "gka_common.cuh"
+
+namespace gka {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int XS = 68;  // padded stride (floats) of tiles stored [channel][token]
+
+template <int D> struct Cfg {
+    static constexpr int DG = D / 64;   // float4 groups per thread along channels
+    static constexpr int NCH = 4 * DG;  // channels per thread
+    static constexpr int kSmemFloats = D * D + 2 * D * XS + 2 * kChunk * D + kChunk * XS + 8 * kChunk + 64;
+    static constexpr size_t kSmemBytes = (size_t)kSmemFloats * sizeof(float);
+};
+
+__device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ void st4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
+
+// acc[t][g*4+u] += sum_kk At[kk][4tc+t] * Bm[kk][64g + 4td + u]
+template <int D>
+__device__ __forceinline__ void gemm_tok_mat(float (&acc)[4][Cfg<D>::NCH], const float *At,
+                                             const float *Bm, int Kdim, int tc, int td) {
+#pragma unroll 4
+    for (int kk = 0; kk < Kdim; ++kk) {
+        float4 xv = ld4(At + kk * XS + 4 * tc);
+        float xa[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+        for (int g = 0; g < Cfg<D>::DG; ++g) {
+            float4 hv = ld4(Bm + kk * D + 64 * g + 4 * td);
+            float ha[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) acc[t][4 * g + u] = fmaf(xa[t], ha[u], acc[t][4 * g + u]);
+        }
+    }
+}
+
+// s[t][u] = sum_d At[d][4tc+t] * Bt[d][4td+u]
+template <int D>
+__device__ __forceinline__ void gemm_tok_tok(float (&s)[4][4], const float *At, const float *Bt,
+                                             int tc, int td) {
+#pragma unroll
+    for (int t = 0; t < 4; ++t)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) s[t][u] = 0.f;
+#pragma unroll 4
+    for (int d = 0; d < D; ++d) {
+        float4 xv = ld4(At + d * XS + 4 * tc);
+        float4 kv = ld4(Bt + d * XS + 4 * td);
+        float xa[4] = {xv.x, xv.y, xv.z, xv.w};
+        float ka[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t)
+#pragma unroll
+            for (int u = 0; u < 4; ++u) s[t][u] = fmaf(xa[t], ka[u], s[t][u]);
+    }
+}
+
+// M (global, [D][D]) <- zetaC * M + sum_j A[j][row] * w[j] * K[j][col];  A, K: smem [64][D].
+template <int D>
+__device__ __forceinline__ void state_update(float *M, const float *A, const float *K, const float *w,
+                                             float zetaC, bool first_is_zero) {
+    constexpr int DG = Cfg<D>::DG, NCH = Cfg<D>::NCH;
+    const int tr = threadIdx.x >> 4, tcn = threadIdx.x & 15;
+    float acc[NCH][NCH];
+#pragma unroll
+    for (int i = 0; i < NCH; ++i)
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) acc[i][j] = 0.f;
+#pragma unroll 2
+    for (int j = 0; j < kChunk; ++j) {
+        const float wj = w[j];
+        float ar[NCH], kc[NCH];
+#pragma unroll
+        for (int g = 0; g < DG; ++g) {
+            float4 a4 = ld4(A + j * D + 64 * g + 4 * tr);
+            float4 k4 = ld4(K + j * D + 64 * g + 4 * tcn);
+            ar[4 * g + 0] = a4.x * wj; ar[4 * g + 1] = a4.y * wj;
+            ar[4 * g + 2] = a4.z * wj; ar[4 * g + 3] = a4.w * wj;
+            kc[4 * g + 0] = k4.x; kc[4 * g + 1] = k4.y; kc[4 * g + 2] = k4.z; kc[4 * g + 3] = k4.w;
+        }
+#pragma unroll
+        for (int i = 0; i < NCH; ++i)
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) acc[i][c] = fmaf(ar[i], kc[c], acc[i][c]);
+    }
+#pragma unroll
+    for (int gi = 0; gi < DG; ++gi)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int row = 64 * gi + 4 * tr + i;
+#pragma unroll
+            for (int gc = 0; gc < DG; ++gc) {
+                float *p = M + (size_t)row * D + 64 * gc + 4 * tcn;
+                float4 o = first_is_zero ? make_float4(0.f, 0.f, 0.f, 0.f) : ld4(p);
+                o.x = fmaf(zetaC, o.x, acc[4 * gi + i][4 * gc + 0]);
+                o.y = fmaf(zetaC, o.y, acc[4 * gi + i][4 * gc + 1]);
+                o.z = fmaf(zetaC, o.z, acc[4 * gi + i][4 * gc + 2]);
+                o.w = fmaf(zetaC, o.w, acc[4 * gi + i][4 * gc + 3]);
+                st4(p, o);
+            }
+        }
+}
+
+// Load one chunk's rows of a [B,T,heads,D] tensor into smem row-major (dst) and, optionally,
+// transposed with stride XS (dstT[d][token]).
+template <int D, typename IoT>
+__device__ __forceinline__ void load_rows(const IoT *src, size_t row0_elem, size_t row_stride_elem,
+                                          float *dst, float *dstT) {
+    constexpr int F4 = D / 4;
+    for (int idx = threadIdx.x; idx < kChunk * F4; idx += kThreads) {
+        const int row = idx / F4, c4 = idx % F4;
+        float4 v = Io<IoT>::load4(src + row0_elem + (size_t)row * row_stride_elem + 4 * c4);
+        if (dst) st4(dst + row * D + 4 * c4, v);
+        if (dstT) {
+            dstT[(4 * c4 + 0) * XS + row] = v.x;
+            dstT[(4 * c4 + 1) * XS + row] = v.y;
+            dstT[(4 * c4 + 2) * XS + row] = v.z;
+            dstT[(4 * c4 + 3) * XS + row] = v.w;
+        }
+    }
+}
+
+__device__ __forceinline__ float block_sum(float v, float *red) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float t = 0.f;
+#pragma unroll
+    for (int i = 0; i < kThreads / 32; ++i) t += red[i];
+    return t;
+}
+
+// Gates of one chunk: G[c] = sum_{i<=c} log gamma_i (clamped), zeta = exp(G), w[j] = exp(G[C-1]-G[j]).
+__device__ __forceinline__ void load_gates(const float *gate, const float *lam, size_t tok0, int heads,
+                                           float *sG, float *sZeta, float *sLam, float *sW) {
+    const int c = threadIdx.x;
+    if (c < kChunk) {
+        sW[c] = fmaxf(logf(gate[tok0 + (size_t)c * heads]), -80.f);  // temporary: log gamma
+        sLam[c] = lam[tok0 + (size_t)c * heads];
+    }
+    __syncthreads();
+    float g = 0.f;
+    if (c < kChunk) {
+        for (int i = 0; i <= c; ++i) g += sW[i];
+    }
+    __syncthreads();
+    if (c < kChunk) {
+        sG[c] = g;
+        sZeta[c] = expf(g);
+    }
+    __syncthreads();
+    if (c < kChunk) sW[c] = expf(sG[kChunk - 1] - sG[c]);
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------
+// Segment summaries: for every work item whose range ends inside a sequence, the decay product
+// and the (delta-H, delta-U) of its last run, relative to a zero start state.
+// ------------------------------------------------------------------------------------------
+template <int D, typename IoT>
+__global__ void __launch_bounds__(kThreads, 1) fwd_simt_summary(FwdArgs a) {
+    extern __shared__ __align__(16) float smem[];
+    const WorkPlan &P = a.plan;
+    const int item = blockIdx.x;
+    if (!P.cut_out(item)) return;
+    float *sK = smem;
+    float *sV = sK + kChunk * D;
+    float *sG = sV + kChunk * D;
+    float *sZeta = sG + kChunk, *sLam = sZeta + kChunk, *sW = sLam + kChunk;
+    const size_t st = state_floats(D, D);
+    float *dH = a.ws.delta + (size_t)item * st;
+    float *dU = dH + (size_t)D * D;
+    const long long f0 = P.last_run_start(item), f1 = P.lo(item + 1);
+    const int seq = (int)(f0 / P.N), b = seq / a.heads, h = seq % a.heads;
+    const size_t rs = (size_t)a.heads * D;
+    float decay_log = 0.f;
+    for (long long f = f0; f < f1; ++f) {
+        const int n = (int)(f % P.N);
+        const size_t tok0 = ((size_t)b * a.T + (size_t)n * kChunk) * a.heads + h;
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, nullptr);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr);
+        load_gates(a.gate, a.lam, tok0, a.heads, sG, sZeta, sLam, sW);
+        const float zc = sZeta[kChunk - 1];
+        decay_log += sG[kChunk - 1];
+        state_update<D>(dH, sK, sK, sW, zc, f == f0);
+        state_update<D>(dU, sV, sK, sW, zc, f == f0);
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) a.ws.decay[item] = expf(decay_log);
+}
+
+// ------------------------------------------------------------------------------------------
+// Scan over work items: start state of item i+1 = decay_i * (start of item i's last run) + delta_i.
+// One thread per state element; the loop over items carries the running value.
+// ------------------------------------------------------------------------------------------
+__global__ void fwd_scan(FwdArgs a, int st) {
+    const WorkPlan &P = a.plan;
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= st) return;
+    float carry = 0.f;
+    for (int i = 0; i + 1 < P.G; ++i) {
+        if (!P.cut_out(i)) continue;
+        const long long rs = P.last_run_start(i);
+        float init;
+        if (rs % P.N == 0) {
+            const int seq = (int)(rs / P.N);
+            init = a.state_in ? a.state_in[(size_t)seq * st + e] : 0.f;
+        } else {
+            init = carry;
+        }
+        carry = fmaf(a.ws.decay[i], init, a.ws.delta[(size_t)i * st + e]);
+        a.ws.start[(size_t)(i + 1) * st + e] = carry;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Main kernel.
+// ------------------------------------------------------------------------------------------
+template <int D, typename IoT>
+__global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
+    constexpr int DG = Cfg<D>::DG, NCH = Cfg<D>::NCH;
+    extern __shared__ __align__(16) float smem[];
+    float *sH = smem;                      // [D][D]  H_0, later U_0^T
+    float *sXt = sH + D * D;               // [D][XS] X^T
+    float *sKt = sXt + D * XS;             // [D][XS] K^T
+    float *sK = sKt + D * XS;              // [64][D]
+    float *sV = sK + kChunk * D;           // [64][D]
+    float *sPt = sV + kChunk * D;          // [64][XS] P^T: sPt[j][c]
+    float *sG = sPt + kChunk * XS;
+    float *sZeta = sG + kChunk, *sLam = sZeta + kChunk, *sW = sLam + kChunk;
+    float *sF = sW + kChunk, *sA = sF + kChunk, *sDj = sA + kChunk, *sTmp = sDj + kChunk;
+    float *sRed = sTmp + kChunk;
+
+    const WorkPlan &P = a.plan;
+    const int item = blockIdx.x;
+    const int tid = threadIdx.x, tc = tid >> 4, td = tid & 15;
+    const size_t st = state_floats(D, D);
+    float *mH = a.ws.cur + (size_t)item * st;   // running masters of this work item
+    float *mU = mH + (size_t)D * D;
+    const IoT *gq = reinterpret_cast<const IoT *>(a.q);
+    IoT *gout = reinterpret_cast<IoT *>(a.out);
+    const size_t rs = (size_t)a.heads * D;
+    const bool adaptive = (a.flags & GKA_FLAG_ADAPTIVE_LAMBDA) != 0;
+
+    const long long f_lo = P.lo(item), f_hi = P.lo(item + 1);
+    for (long long f = f_lo; f < f_hi; ++f) {
+        const int seq = (int)(f / P.N), n = (int)(f % P.N);
+        const int b = seq / a.heads, h = seq % a.heads;
+        const size_t tok0 = ((size_t)b * a.T + (size_t)n * kChunk) * a.heads + h;
+
+        // ---- run start: fetch the start state into the running masters
+        if (f == f_lo || n == 0) {
+            const float *src = (n == 0) ? (a.state_in ? a.state_in + (size_t)seq * st : nullptr)
+                                        : a.ws.start + (size_t)item * st;
+            for (size_t e = 4 * (size_t)tid; e < st; e += 4 * kThreads)
+                st4(mH + e, src ? ld4(src + e) : make_float4(0.f, 0.f, 0.f, 0.f));
+        }
+        __syncthreads();
+
+        // ---- stage the chunk
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, sKt);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr);
+        for (int e = 4 * tid; e < D * D; e += 4 * kThreads) st4(sH + e, ld4(mH + e));
+        load_gates(a.gate, a.lam, tok0, a.heads, sG, sZeta, sLam, sW);  // ends with a barrier
+
+        // ---- chunk-wise Frobenius norms (Section 4.2.1), O(C^2) form:
+        //      f_c^2 = zeta_c^2 ||H_0||^2 + sum_{j<=c} Gamma[c][j]^2 d_j,
+        //      d_j   = 2 zeta_j k_j^T H_0 k_j + 2 sum_{i<j} Gamma[j][i] (k_j.k_i)^2 + (k_j.k_j)^2
+        float hh = 0.f;
+        for (int e = 4 * tid; e < D * D; e += 4 * kThreads) {
+            float4 v4 = ld4(sH + e);
+            hh += v4.x * v4.x + v4.y * v4.y + v4.z * v4.z + v4.w * v4.w;
+        }
+        hh = block_sum(hh, sRed);
+        {
+            float acc[4][NCH];
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+                for (int u = 0; u < NCH; ++u) acc[t][u] = 0.f;
+            gemm_tok_mat<D>(acc, sKt, sH, D, tc, td);   // (K H_0)[j][d]
+            float part[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                float s = 0.f;
+#pragma unroll
+                for (int g = 0; g < DG; ++g) {
+                    float4 kv = ld4(sK + (4 * tc + t) * D + 64 * g + 4 * td);
+                    s += acc[t][4 * g + 0] * kv.x + acc[t][4 * g + 1] * kv.y +
+                         acc[t][4 * g + 2] * kv.z + acc[t][4 * g + 3] * kv.w;
+                }
+                part[t] = s;
+            }
+            float gm[4][4];
+            gemm_tok_tok<D>(gm, sKt, sKt, tc, td);      // Gram[j][i], j = 4tc+t, i = 4td+u
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int j = 4 * tc + t;
+                float s = 2.f * sZeta[j] * part[t];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = 4 * td + u;
+                    const float g2 = gm[t][u] * gm[t][u];
+                    if (i < j) s += 2.f * expf(sG[j] - sG[i]) * g2;
+                    else if (i == j) s += g2;
+                }
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                if (td == 0) sDj[j] = s;
+            }
+        }
+        __syncthreads();
+        if (tid < kChunk) {
+            const int c = tid;
+            float s = sZeta[c] * sZeta[c] * hh;
+            for (int j = 0; j <= c; ++j) s += expf(2.f * (sG[c] - sG[j])) * sDj[j];
+            const float fc = sqrtf(fmaxf(s, 0.f));
+            sF[c] = fc;
+            if (adaptive) sLam[c] = sLam[c] * fc;
+            if (a.fro_out) a.fro_out[tok0 + (size_t)c * a.heads] = fc;
+        }
+        __syncthreads();
+
+        // ---- Algorithm 1 on the whole chunk
+        float xm[4][NCH], xp[4][NCH], qm[4][NCH];
+        float omega[4], rho2[4], s0[4], lamr[4], zet[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int c = 4 * tc + t;
+            const float fc = sF[c], lc = sLam[c];
+            const float Lpm = fc + 2.f * lc;            // L + mu
+            const float rho = fc / Lpm;                 // (L - mu) / (L + mu)
+            rho2[t] = rho * rho;
+            s0[t] = 2.f / Lpm;
+            lamr[t] = lc;
+            zet[t] = sZeta[c];
+            omega[t] = 2.f;
+#pragma unroll
+            for (int g = 0; g < DG; ++g) {
+                float4 qv = Io<IoT>::load4(gq + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td);
+                qm[t][4 * g + 0] = qv.x; qm[t][4 * g + 1] = qv.y;
+                qm[t][4 * g + 2] = qv.z; qm[t][4 * g + 3] = qv.w;
+            }
+#pragma unroll
+            for (int u = 0; u < NCH; ++u) {
+                xm[t][u] = s0[t] * qm[t][u];            // xi_0 = 2 q / (L + mu)
+                xp[t][u] = 0.f;                         // xi_{-1} = 0
+            }
+        }
+        auto publish_x = [&]() {
+#pragma unroll
+            for (int g = 0; g < DG; ++g)
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    st4(sXt + (64 * g + 4 * td + u) * XS + 4 * tc,
+                        make_float4(xm[0][4 * g + u], xm[1][4 * g + u], xm[2][4 * g + u], xm[3][4 * g + u]));
+        };
+        auto masked_scores = [&]() {   // sPt[j][c] = Gamma[c][j] * (x_c . k_j), j <= c
+            float s[4][4];
+            gemm_tok_tok<D>(s, sXt, sKt, tc, td);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int j = 4 * td + u;
+                float p[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int c = 4 * tc + t;
+                    p[t] = (j <= c) ? expf(sG[c] - sG[j]) * s[t][u] : 0.f;
+                }
+                st4(sPt + j * XS + 4 * tc, make_float4(p[0], p[1], p[2], p[3]));
+            }
+        };
+        publish_x();
+        __syncthreads();
+        for (int it = 0; it < a.n_iter; ++it) {
+            masked_scores();
+            __syncthreads();
+            float acc[4][NCH];
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+                for (int u = 0; u < NCH; ++u) acc[t][u] = 0.f;
+            gemm_tok_mat<D>(acc, sXt, sH, D, tc, td);          // X H_0
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+                for (int u = 0; u < NCH; ++u) acc[t][u] *= zet[t];
+            gemm_tok_mat<D>(acc, sPt, sK, kChunk, tc, td);     // + P K
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                omega[t] = 4.f / (4.f - rho2[t] * omega[t]);   // weight schedule
+                const float step = s0[t] * omega[t];
+                const float mom = omega[t] - 1.f;
+#pragma unroll
+                for (int u = 0; u < NCH; ++u) {
+                    const float y = fmaf(lamr[t], xm[t][u], acc[t][u]);       // (H_c + lambda_c I) x_c
+                    const float xn = xm[t][u] - step * (y - qm[t][u]) + mom * (xm[t][u] - xp[t][u]);
+                    xp[t][u] = xm[t][u];
+                    xm[t][u] = xn;
+                }
+            }
+            __syncthreads();      // every read of sXt / sPt of this iteration is done
+            publish_x();
+            __syncthreads();
+        }
+
+        // ---- output O = zeta o (X U_0^T) + P V
+        masked_scores();
+        for (int idx = tid; idx < D * (D / 4); idx += kThreads) {   // sH <- U_0^T
+            const int i = idx / (D / 4), e4 = idx % (D / 4);
+            float4 uv = ld4(mU + (size_t)i * D + 4 * e4);
+            sH[(4 * e4 + 0) * D + i] = uv.x;
+            sH[(4 * e4 + 1) * D + i] = uv.y;
+            sH[(4 * e4 + 2) * D + i] = uv.z;
+            sH[(4 * e4 + 3) * D + i] = uv.w;
+        }
+        __syncthreads();
+        {
+            float acc[4][NCH];
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+                for (int u = 0; u < NCH; ++u) acc[t][u] = 0.f;
+            gemm_tok_mat<D>(acc, sXt, sH, D, tc, td);
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+                for (int u = 0; u < NCH; ++u) acc[t][u] *= zet[t];
+            gemm_tok_mat<D>(acc, sPt, sV, kChunk, tc, td);
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int c = 4 * tc + t;
+#pragma unroll
+                for (int g = 0; g < DG; ++g)
+                    Io<IoT>::store4(gout + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td,
+                                    make_float4(acc[t][4 * g + 0], acc[t][4 * g + 1],
+                                                acc[t][4 * g + 2], acc[t][4 * g + 3]));
+            }
+        }
+
+        // ---- state carry
+        const float zc = sZeta[kChunk - 1];
+        state_update<D>(mH, sK, sK, sW, zc, false);
+        state_update<D>(mU, sV, sK, sW, zc, false);
+        __syncthreads();
+        if (n == P.N - 1 && a.state_out) {
+            float *dst = a.state_out + (size_t)seq * st;
+            for (size_t e = 4 * (size_t)tid; e < st; e += 4 * kThreads) st4(dst + e, ld4(mH + e));
+        }
+        __syncthreads();
+    }
+}
+
+template <int D, typename IoT>
+cudaError_t launch_typed(const FwdArgs &a, cudaStream_t stream) {
+    const int G = a.plan.G;
+    const int st = (int)state_floats(D, D);
+    cudaError_t err;
+    bool any_cut = false;
+    for (int i = 0; i + 1 < G; ++i) any_cut |= a.plan.cut_out(i);
+    if (any_cut) {
+        const size_t sm_sum = (size_t)(2 * kChunk * D + 4 * kChunk) * sizeof(float);
+        err = cudaFuncSetAttribute(fwd_simt_summary<D, IoT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)sm_sum);
+        if (err != cudaSuccess) return err;
+        fwd_simt_summary<D, IoT><<<G, kThreads, sm_sum, stream>>>(a);
+        fwd_scan<<<(st + 255) / 256, 256, 0, stream>>>(a, st);
+    }
+    err = cudaFuncSetAttribute(fwd_simt_main<D, IoT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)Cfg<D>::kSmemBytes);
+    if (err != cudaSuccess) return err;
+    if (a.ev_start) cudaEventRecord(a.ev_start, stream);
+    fwd_simt_main<D, IoT><<<G, kThreads, Cfg<D>::kSmemBytes, stream>>>(a);
+    if (a.ev_stop) cudaEventRecord(a.ev_stop, stream);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_fwd_simt(const FwdArgs &a, int d, int io_dtype, cudaStream_t stream) {
+    if (d == 128) {
+        return io_dtype == GKA_BF16 ? launch_typed<128, __nv_bfloat16>(a, stream)
+                                    : launch_typed<128, float>(a, stream);
+    }
+    return io_dtype == GKA_BF16 ? launch_typed<64, __nv_bfloat16>(a, stream)
+                                : launch_typed<64, float>(a, stream);
+}
+
+}  // namespace gka

@@ -1,0 +1,192 @@
+"""Thin ctypes binding of the GKA C ABI (include/gka.h).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of
+``libgka.so``.  PyTorch is used for device memory and streams.  There is no CPU
+fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgka.so")
+
+GKA_OK = 0
+GKA_F32, GKA_BF16 = 0, 1
+GKA_PREC_NATIVE, GKA_PREC_HIGH = 0, 1
+GKA_FLAG_ADAPTIVE_LAMBDA = 1
+GKA_ERR_TIMEOUT = 8
+
+EXPORTS = ("gka_fwd_workspace_bytes", "gka_fwd_chunked", "gka_decode_step", "gka_status_string",
+           "gka_fwd_num_work_items", "gka_fwd_work_range")
+
+
+class GkaDesc(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int), ("T", ctypes.c_int), ("heads", ctypes.c_int),
+        ("d_k", ctypes.c_int), ("d_v", ctypes.c_int),
+        ("io_dtype", ctypes.c_int), ("precision", ctypes.c_int), ("flags", ctypes.c_uint),
+        ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t), ("state_in", ctypes.c_void_p),
+        ("device_status", ctypes.c_void_p), ("fro_out", ctypes.c_void_p),
+        ("profile_start", ctypes.c_void_p), ("profile_stop", ctypes.c_void_p),
+    ]
+
+
+class GkaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)}")
+
+
+_lib = None
+
+
+def load_library():
+    """Load libgka.so (built in-tree by ``build.build_library``).  Raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2511_21016_b200.build` "
+                "(there is no CPU fallback)")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, ci = ctypes.c_void_p, ctypes.c_int
+        dp = ctypes.POINTER(GkaDesc)
+        lib.gka_fwd_workspace_bytes.argtypes = [dp, ci]
+        lib.gka_fwd_workspace_bytes.restype = ctypes.c_size_t
+        lib.gka_fwd_num_work_items.argtypes = [dp, ci]
+        lib.gka_fwd_num_work_items.restype = ci
+        lib.gka_fwd_chunked.argtypes = [dp, vp, vp, vp, vp, vp, ci, ci, vp, vp]
+        lib.gka_fwd_chunked.restype = ci
+        lib.gka_decode_step.argtypes = [dp, vp, vp, vp, vp, vp, vp, ci, vp]
+        lib.gka_decode_step.restype = ci
+        llp, ip = ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int)
+        lib.gka_fwd_work_range.argtypes = [dp, ci, ci, ci, llp, llp, ip, ip]
+        lib.gka_fwd_work_range.restype = ci
+        lib.gka_status_string.argtypes = [ci]
+        lib.gka_status_string.restype = ctypes.c_char_p
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load_library().gka_status_string(int(status)).decode()
+
+
+def _io_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return GKA_F32
+    if t.dtype == torch.bfloat16:
+        return GKA_BF16
+    raise TypeError(f"unsupported I/O dtype {t.dtype}")
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _check_cuda(*ts):
+    for t in ts:
+        if t is not None:
+            if not t.is_cuda:
+                raise ValueError("all tensors must live on the CUDA device (no CPU fallback)")
+            if not t.is_contiguous():
+                raise ValueError("tensors must be contiguous")
+
+
+def make_desc(B, T, heads, d_k, d_v, io_dtype, precision=GKA_PREC_NATIVE, flags=0, stream=None,
+              workspace=None, state_in=None, device_status=None, fro_out=None,
+              profile_events=None) -> GkaDesc:
+    d = GkaDesc()
+    d.B, d.T, d.heads, d.d_k, d.d_v = B, T, heads, d_k, d_v
+    d.io_dtype, d.precision, d.flags = io_dtype, precision, flags
+    d.stream = stream
+    d.workspace = _ptr(workspace)
+    d.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    d.state_in = _ptr(state_in)
+    d.device_status = _ptr(device_status)
+    d.fro_out = _ptr(fro_out)
+    if profile_events is not None:
+        d.profile_start, d.profile_stop = profile_events
+    return d
+
+
+def gka_fwd_workspace_bytes(B, T, heads, d, io_dtype=GKA_BF16, chunk=64) -> int:
+    desc = make_desc(B, T, heads, d, d, io_dtype)
+    return int(load_library().gka_fwd_workspace_bytes(ctypes.byref(desc), chunk))
+
+
+def gka_fwd_num_work_items(B, T, heads, d, io_dtype=GKA_BF16, chunk=64) -> int:
+    desc = make_desc(B, T, heads, d, d, io_dtype)
+    return int(load_library().gka_fwd_num_work_items(ctypes.byref(desc), chunk))
+
+
+def gka_fwd_work_range(B, T, heads, d, num_items, item, chunk=64):
+    """(first_chunk, end_chunk, cut_in, cut_out) of one work item; host arithmetic only."""
+    desc = make_desc(B, T, heads, d, d, GKA_BF16)
+    lo, hi = ctypes.c_longlong(), ctypes.c_longlong()
+    ci_, co_ = ctypes.c_int(), ctypes.c_int()
+    rc = load_library().gka_fwd_work_range(ctypes.byref(desc), chunk, num_items, item,
+                                           ctypes.byref(lo), ctypes.byref(hi), ctypes.byref(ci_),
+                                           ctypes.byref(co_))
+    if rc != GKA_OK:
+        raise GkaError(rc, "gka_fwd_work_range")
+    return lo.value, hi.value, bool(ci_.value), bool(co_.value)
+
+
+def alloc_workspace(B, T, heads, d, device, chunk=64) -> torch.Tensor:
+    n = gka_fwd_workspace_bytes(B, T, heads, d, chunk=chunk)
+    if n == 0:
+        raise GkaError(2, "gka_fwd_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def gka_fwd_chunked(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=None, *,
+                    state_in=None, workspace=None, precision=GKA_PREC_NATIVE, flags=0,
+                    fro_out=None, device_status=None, stream=None, profile_events=None):
+    """Chunk-wise GKA forward.  q,k,v: [B,T,heads,d] (f32 or bf16); gate, lam: [B,T,heads] f32.
+
+    Returns (out, state_out).  Work is enqueued on ``stream`` (default: torch's current stream).
+    """
+    _check_cuda(q, k, v, gate, lam, out, state_out, state_in, workspace, fro_out, device_status)
+    B, T, heads, d = q.shape
+    if out is None:
+        out = torch.empty_like(v)
+    if state_out is None:
+        state_out = torch.empty(B, heads, 2 * d * d, dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = alloc_workspace(B, T, heads, d, q.device, chunk)
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    desc = make_desc(B, T, heads, d, v.shape[-1], _io_code(q), precision, flags, stream, workspace,
+                     state_in, device_status, fro_out, profile_events)
+    rc = load_library().gka_fwd_chunked(ctypes.byref(desc), q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                        gate.data_ptr(), lam.data_ptr(), int(n_iter), int(chunk),
+                                        out.data_ptr(), _ptr(state_out))
+    if rc != GKA_OK:
+        raise GkaError(rc, "gka_fwd_chunked")
+    return out, state_out
+
+
+def gka_decode_step(state, q, k, v, gate, lam, n_iter, out=None, *, flags=0, device_status=None,
+                    stream=None, profile_events=None):
+    """One recurrent step.  state: [N,heads,2*d*d] f32, updated in place; q,k,v: [N,heads,d]."""
+    _check_cuda(state, q, k, v, gate, lam, out, device_status)
+    N, heads, d = q.shape
+    if out is None:
+        out = torch.empty_like(v)
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    desc = make_desc(N, 1, heads, d, v.shape[-1], _io_code(q), GKA_PREC_NATIVE, flags, stream,
+                     device_status=device_status, profile_events=profile_events)
+    rc = load_library().gka_decode_step(ctypes.byref(desc), state.data_ptr(), q.data_ptr(),
+                                        k.data_ptr(), v.data_ptr(), gate.data_ptr(), lam.data_ptr(),
+                                        int(n_iter), out.data_ptr())
+    if rc != GKA_OK:
+        raise GkaError(rc, "gka_decode_step")
+    return out

@@ -1,0 +1,141 @@
+"""Host-side checks that need no GPU: the C-ABI library loads, exports every symbol the header
+declares, validates arguments before any launch, and splits work as documented."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2511_21016_b200 import build, gka, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return gka.load_library()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "gka.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gka_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert {"gka_fwd_chunked", "gka_decode_step", "gka_fwd_workspace_bytes"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/gka.h but not exported"
+    assert set(gka.EXPORTS) <= set(names)
+
+
+def test_status_strings(lib):
+    assert gka.status_string(0) == "GKA_OK"
+    seen = {gka.status_string(i) for i in range(10)}
+    assert len(seen) == 10
+    assert "unknown" in gka.status_string(99)
+
+
+def test_workspace_bytes_arithmetic(lib):
+    st = 2 * 128 * 128
+    # 64 sequences x 64 chunks = 4096 chunks -> capped at 296 work items
+    n = gka.gka_fwd_workspace_bytes(4, 4096, 16, 128)
+    assert n == ((3 * 296 * st + 296) * 4 + 255) // 256 * 256
+    # tiny problem: 2 sequences x 4 chunks = 8 items
+    n = gka.gka_fwd_workspace_bytes(1, 256, 2, 64)
+    assert n == ((3 * 8 * 2 * 64 * 64 + 8) * 4 + 255) // 256 * 256
+    assert gka.gka_fwd_workspace_bytes(1, 100, 2, 64) == 0       # T not a multiple of 64
+    assert gka.gka_fwd_workspace_bytes(1, 128, 2, 96) == 0       # unsupported head dim
+
+
+def _call_fwd(lib, desc, ptrs, n_iter=1, chunk=64):
+    return lib.gka_fwd_chunked(ctypes.byref(desc), *ptrs[:5], n_iter, chunk, *ptrs[5:])
+
+
+def test_argument_errors_are_reported_before_any_launch(lib):
+    """None of these reaches a CUDA call, so they run without a GPU."""
+    ok = 256  # fake, aligned, non-null "device pointers": never dereferenced on these paths
+    ptrs = [ok] * 7
+    d = gka.make_desc(1, 128, 2, 64, 64, gka.GKA_F32)
+    assert _call_fwd(lib, d, [None] + ptrs[1:]) == 1                       # NULL
+    assert _call_fwd(lib, d, ptrs, n_iter=-1) == 2                         # negative n_iter
+    assert _call_fwd(lib, d, ptrs, chunk=32) == 4                          # unsupported chunk
+    assert _call_fwd(lib, d, ptrs, chunk=0) == 2
+    assert _call_fwd(lib, d, [ok + 4] + ptrs[1:]) == 9                     # misaligned q
+    assert _call_fwd(lib, d, ptrs) == 5                                    # no workspace
+    d.workspace, d.workspace_bytes = 256, 16
+    assert _call_fwd(lib, d, ptrs) == 5                                    # workspace too small
+    d2 = gka.make_desc(1, 100, 2, 64, 64, gka.GKA_F32)
+    assert _call_fwd(lib, d2, ptrs) == 2                                   # T % chunk != 0
+    d3 = gka.make_desc(1, 128, 2, 64, 128, gka.GKA_F32)
+    assert _call_fwd(lib, d3, ptrs) == 2                                   # d_k != d_v
+    d4 = gka.make_desc(1, 128, 2, 64, 64, 7)
+    assert _call_fwd(lib, d4, ptrs) == 3                                   # bad dtype
+    d5 = gka.make_desc(1, 128, 2, 64, 64, gka.GKA_F32, flags=0x10)
+    assert _call_fwd(lib, d5, ptrs) == 4                                   # unknown flag
+    dd = gka.make_desc(4, 1, 2, 128, 128, gka.GKA_BF16)
+    rc = lib.gka_decode_step(ctypes.byref(dd), None, ok, ok, ok, ok, ok, 3, ok)
+    assert rc == 1
+    rc = lib.gka_decode_step(ctypes.byref(dd), ok, ok, ok + 2, ok, ok, ok, 3, ok)
+    assert rc == 9
+    rc = lib.gka_decode_step(None, ok, ok, ok, ok, ok, ok, 3, ok)
+    assert rc == 1
+
+
+@pytest.mark.parametrize("B,T,heads,G", [(4, 4096, 16, 148), (1, 131072, 32, 148), (1, 256, 2, 8),
+                                         (1, 6400, 3, 148), (3, 192, 5, 7), (1, 64, 1, 1)])
+def test_work_ranges_partition_the_chunk_list(lib, B, T, heads, G):
+    N = T // 64
+    NC = B * heads * N
+    prev_hi = 0
+    sizes = []
+    for i in range(G):
+        lo, hi, cin, cout = gka.gka_fwd_work_range(B, T, heads, 128, G, i)
+        assert lo == prev_hi and hi > lo
+        assert cin == (lo % N != 0) and cout == (hi % N != 0)
+        sizes.append(hi - lo)
+        prev_hi = hi
+    assert prev_hi == NC
+    assert max(sizes) - min(sizes) <= 1          # balanced to within one chunk
+    with pytest.raises(gka.GkaError):
+        gka.gka_fwd_work_range(B, T, heads, 128, G, G)
+
+
+def test_missing_library_is_an_error(monkeypatch, tmp_path):
+    monkeypatch.setattr(gka, "_lib", None)
+    monkeypatch.setattr(gka, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(FileNotFoundError):
+        gka.load_library()
+
+
+def test_cpu_tensors_are_rejected():
+    import torch
+    t = torch.zeros(1, 64, 1, 64)
+    g = torch.ones(1, 64, 1)
+    with pytest.raises(ValueError):
+        gka.gka_fwd_chunked(t, t, t, g, g, 1)
+
+
+def test_synth_substreams_and_distributions():
+    cfg = synth.shrink(synth.CONFIGS[1], B=2, heads=3, T=128)
+    full = synth.make_inputs(cfg)
+    part = synth.make_inputs(cfg, pairs=[(1, 2)])
+    for key in full:
+        assert np.array_equal(full[key][1, :, 2], part[key][1, :, 2])
+    assert full["q"].shape == (2, 128, 3, 128) and full["gate"].shape == (2, 128, 3)
+    # bf16-representable, unit-norm up to bf16 rounding
+    assert np.array_equal(synth.round_bf16(full["k"]), full["k"])
+    assert np.allclose(np.linalg.norm(full["k"], axis=-1), 1.0, atol=2e-2)
+    assert np.all((full["gate"] > 0) & (full["gate"] <= 1)) and np.all(full["lam"] >= 1e-2)
+    # stress recipe: keys close to a rank-8 subspace, tiny lambda
+    c4 = synth.shrink(synth.CONFIGS[4], B=1, heads=1, T=512)
+    x = synth.make_inputs(c4)
+    sv = np.linalg.svd(x["k"][0, :, 0].astype(np.float64), compute_uv=False)
+    assert sv[8] < 0.05 * sv[7]
+    assert x["lam"].max() < 1e-3
+    # bf16 rounding helper: ties to even
+    assert synth.to_bf16_bits(np.array([1.0, 1.00390625, 1.01171875], np.float32)).tolist() == \
+        [0x3F80, 0x3F80, 0x3F82]
