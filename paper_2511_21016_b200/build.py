@@ -49,7 +49,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    cmd = [_nvcc(), "-shared", "-o", LIB, *objs, "-lcudart", "-lcuda"]
+    cmd = [_nvcc(), "-shared", "-o", LIB, *objs, "-lcudart"]
     subprocess.check_call(cmd)
     return LIB
 

@@ -147,6 +147,7 @@ struct FwdArgs {
 
 // Launchers implemented in the kernel translation units.  Each returns a cudaError_t.
 cudaError_t launch_fwd_simt(const FwdArgs &a, int d, int io_dtype, cudaStream_t stream);
+cudaError_t launch_fwd_summary_scan_bf16_d128(const FwdArgs &a, cudaStream_t stream);
 cudaError_t launch_decode(float *state, const void *q, const void *k, const void *v,
                           const float *gate, const float *lam, int n_iter, void *out, int nseq,
                           int heads, int d, int io_dtype, unsigned flags, int *device_status,

@@ -470,31 +470,41 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
     }
 }
 
+// Summary + scan pass (only when some work item starts inside a sequence).
 template <int D, typename IoT>
-cudaError_t launch_typed(const FwdArgs &a, cudaStream_t stream) {
+cudaError_t launch_summary_scan_typed(const FwdArgs &a, cudaStream_t stream) {
     const int G = a.plan.G;
     const int st = (int)state_floats(D, D);
-    cudaError_t err;
     bool any_cut = false;
     for (int i = 0; i + 1 < G; ++i) any_cut |= a.plan.cut_out(i);
-    if (any_cut) {
-        const size_t sm_sum = (size_t)(2 * kChunk * D + 4 * kChunk) * sizeof(float);
-        err = cudaFuncSetAttribute(fwd_simt_summary<D, IoT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   (int)sm_sum);
-        if (err != cudaSuccess) return err;
-        fwd_simt_summary<D, IoT><<<G, kThreads, sm_sum, stream>>>(a);
-        fwd_scan<<<(st + 255) / 256, 256, 0, stream>>>(a, st);
-    }
+    if (!any_cut) return cudaSuccess;
+    const size_t sm_sum = (size_t)(2 * kChunk * D + 4 * kChunk) * sizeof(float);
+    cudaError_t err = cudaFuncSetAttribute(fwd_simt_summary<D, IoT>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_sum);
+    if (err != cudaSuccess) return err;
+    fwd_simt_summary<D, IoT><<<G, kThreads, sm_sum, stream>>>(a);
+    fwd_scan<<<(st + 255) / 256, 256, 0, stream>>>(a, st);
+    return cudaGetLastError();
+}
+
+template <int D, typename IoT>
+cudaError_t launch_typed(const FwdArgs &a, cudaStream_t stream) {
+    cudaError_t err = launch_summary_scan_typed<D, IoT>(a, stream);
+    if (err != cudaSuccess) return err;
     err = cudaFuncSetAttribute(fwd_simt_main<D, IoT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)Cfg<D>::kSmemBytes);
     if (err != cudaSuccess) return err;
     if (a.ev_start) cudaEventRecord(a.ev_start, stream);
-    fwd_simt_main<D, IoT><<<G, kThreads, Cfg<D>::kSmemBytes, stream>>>(a);
+    fwd_simt_main<D, IoT><<<a.plan.G, kThreads, Cfg<D>::kSmemBytes, stream>>>(a);
     if (a.ev_stop) cudaEventRecord(a.ev_stop, stream);
     return cudaGetLastError();
 }
 
 }  // namespace
+
+cudaError_t launch_fwd_summary_scan_bf16_d128(const FwdArgs &a, cudaStream_t stream) {
+    return launch_summary_scan_typed<128, __nv_bfloat16>(a, stream);
+}
 
 cudaError_t launch_fwd_simt(const FwdArgs &a, int d, int io_dtype, cudaStream_t stream) {
     if (d == 128) {
