@@ -113,6 +113,12 @@ gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, co
 const char *gka_status_string(int status);
 
 /*
+ * Detail of the last GKA_ERR_CUDA returned to the calling thread (CUDA error name and text, and
+ * which call raised it); an empty string if there was none.  The pointer stays valid for the thread.
+ */
+const char *gka_last_error_detail(void);
+
+/*
  * Work decomposition of the chunked forward, for callers that size buffers or report launch
  * counts: number of persistent work items (thread blocks) the main kernel uses for this
  * descriptor on the current device, or a negative gka_status.

@@ -12,6 +12,14 @@ bool fwd_tc_available();
 namespace {
 
 int g_sm_count = 0;
+thread_local char g_detail[256] = "";
+
+gka_status cuda_result(cudaError_t err, const char *where) {
+    if (err == cudaSuccess) return GKA_OK;
+    snprintf(g_detail, sizeof(g_detail), "%s: %s (%s)", where, cudaGetErrorName(err), cudaGetErrorString(err));
+    (void)cudaGetLastError();   // clear the sticky launch error so that later calls are not poisoned
+    return GKA_ERR_CUDA;
+}
 
 int sm_count() {
     if (g_sm_count == 0) {
@@ -149,7 +157,7 @@ gka_status gka_fwd_chunked(const gka_desc *desc, const void *q, const void *k, c
         err = launch_fwd_tc(a, stream);
     else
         err = launch_fwd_simt(a, desc->d_k, desc->io_dtype, stream);
-    return err == cudaSuccess ? GKA_OK : GKA_ERR_CUDA;
+    return cuda_result(err, tensor_path ? "gka_fwd_chunked (tensor-core path)" : "gka_fwd_chunked (fp32 path)");
 }
 
 gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, const void *k,
@@ -166,7 +174,9 @@ gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, co
                                     reinterpret_cast<cudaEvent_t>(desc->profile_start),
                                     reinterpret_cast<cudaEvent_t>(desc->profile_stop),
                                     reinterpret_cast<cudaStream_t>(desc->stream));
-    return err == cudaSuccess ? GKA_OK : GKA_ERR_CUDA;
+    return cuda_result(err, "gka_decode_step");
 }
+
+const char *gka_last_error_detail(void) { return g_detail; }
 
 }  // extern "C"

@@ -109,22 +109,23 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
 
-// Wait for an mbarrier phase with a time limit (about one second of SM clocks).  Returns false if
-// the phase did not complete in time; the caller records GKA_ERR_TIMEOUT and leaves cleanly.
+// Wait for an mbarrier phase with a time limit (about a second).  The wait sleeps in hardware
+// (try_wait with a suspend-time hint), so a waiting warp leaves the issue slots to working warps.
+// Returns false if the phase did not complete in time; the caller records GKA_ERR_TIMEOUT and
+// leaves cleanly.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar_addr, uint32_t parity) {
-    const long long t0 = clock64();
-    for (;;) {
+    for (int tries = 0; tries < 200000; ++tries) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
-            : "r"(bar_addr), "r"(parity)
+            : "r"(bar_addr), "r"(parity), "r"(5000u)
             : "memory");
         if (done) return true;
-        if (clock64() - t0 > 2000000000LL) return false;
     }
+    return false;
 }
 #endif
 
@@ -147,7 +148,7 @@ struct FwdArgs {
 
 // Launchers implemented in the kernel translation units.  Each returns a cudaError_t.
 cudaError_t launch_fwd_simt(const FwdArgs &a, int d, int io_dtype, cudaStream_t stream);
-cudaError_t launch_fwd_summary_scan_bf16_d128(const FwdArgs &a, cudaStream_t stream);
+cudaError_t launch_fwd_scan(const FwdArgs &a, int st, cudaStream_t stream);   // cross-item scan of the summaries
 cudaError_t launch_decode(float *state, const void *q, const void *k, const void *v,
                           const float *gate, const float *lam, int n_iter, void *out, int nseq,
                           int heads, int d, int io_dtype, unsigned flags, int *device_status,

@@ -209,27 +209,30 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_summary(FwdArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------
-// Scan over work items: start state of item i+1 = decay_i * (start of item i's last run) + delta_i.
-// One thread per state element; the loop over items carries the running value.
+// Scan over work items: the start state of item i (when its range starts inside a sequence) is the
+// fold  state <- decay_j * state + delta_j  over the items j < i that hold the earlier part of the
+// same sequence, starting from the sequence's initial state.  A sequence spans few items, so every
+// item folds its own short chain independently: blockIdx.y = item, four state elements per thread.
 // ------------------------------------------------------------------------------------------
 __global__ void fwd_scan(FwdArgs a, int st) {
     const WorkPlan &P = a.plan;
-    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    const int i = blockIdx.y + 1;
+    if (!P.cut_in(i)) return;
+    const int e = 4 * (blockIdx.x * blockDim.x + threadIdx.x);
     if (e >= st) return;
-    float carry = 0.f;
-    for (int i = 0; i + 1 < P.G; ++i) {
-        if (!P.cut_out(i)) continue;
-        const long long rs = P.last_run_start(i);
-        float init;
-        if (rs % P.N == 0) {
-            const int seq = (int)(rs / P.N);
-            init = a.state_in ? a.state_in[(size_t)seq * st + e] : 0.f;
-        } else {
-            init = carry;
-        }
-        carry = fmaf(a.ws.decay[i], init, a.ws.delta[(size_t)i * st + e]);
-        a.ws.start[(size_t)(i + 1) * st + e] = carry;
+    int j0 = i - 1;                       // first item of the chain: the one that holds the sequence start
+    while (P.cut_in(j0)) --j0;
+    const int seq = (int)(P.lo(i) / P.N);
+    float4 carry = a.state_in ? ld4(a.state_in + (size_t)seq * st + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = j0; j < i; ++j) {
+        const float dcy = a.ws.decay[j];
+        const float4 d = ld4(a.ws.delta + (size_t)j * st + e);
+        carry.x = fmaf(dcy, carry.x, d.x);
+        carry.y = fmaf(dcy, carry.y, d.y);
+        carry.z = fmaf(dcy, carry.z, d.z);
+        carry.w = fmaf(dcy, carry.w, d.w);
     }
+    st4(a.ws.start + (size_t)i * st + e, carry);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -483,7 +486,7 @@ cudaError_t launch_summary_scan_typed(const FwdArgs &a, cudaStream_t stream) {
                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_sum);
     if (err != cudaSuccess) return err;
     fwd_simt_summary<D, IoT><<<G, kThreads, sm_sum, stream>>>(a);
-    fwd_scan<<<(st + 255) / 256, 256, 0, stream>>>(a, st);
+    if (G > 1) fwd_scan<<<dim3((st / 4 + 255) / 256, G - 1), 256, 0, stream>>>(a, st);
     return cudaGetLastError();
 }
 
@@ -502,8 +505,9 @@ cudaError_t launch_typed(const FwdArgs &a, cudaStream_t stream) {
 
 }  // namespace
 
-cudaError_t launch_fwd_summary_scan_bf16_d128(const FwdArgs &a, cudaStream_t stream) {
-    return launch_summary_scan_typed<128, __nv_bfloat16>(a, stream);
+cudaError_t launch_fwd_scan(const FwdArgs &a, int st, cudaStream_t stream) {
+    if (a.plan.G > 1) fwd_scan<<<dim3((st / 4 + 255) / 256, a.plan.G - 1), 256, 0, stream>>>(a, st);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_fwd_simt(const FwdArgs &a, int d, int io_dtype, cudaStream_t stream) {

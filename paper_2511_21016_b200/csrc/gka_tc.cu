@@ -1,9 +1,10 @@
 // tcgen05 / TMEM chunk-wise GKA forward (bf16 operands, fp32 accumulation) for sm_100a.
 //
 // One persistent thread block per SM walks its range of chunks (gka_common.cuh explains the work
-// decomposition).  The block has NSLOT "slots"; a slot is one warpgroup of 128 threads that owns one
-// chunk of C = 64 tokens at a time, so with NSLOT = 2 the tensor pipe works on one chunk while the
-// CUDA cores run the element-wise part of the other.  Slots take chunks alternately.
+// decomposition).  The block has two "slots"; a slot is a group of 256 threads that owns one chunk of
+// C = 64 tokens at a time, so the tensor pipe works on one chunk while the CUDA cores run the
+// element-wise part of the other.  Slots take chunks alternately.  One extra warp issues every
+// tcgen05.mma: the slots post requests to it through mbarriers, it answers with tcgen05.commit.
 //
 // Orientation: every product is computed transposed, so that TMEM lanes are channels and TMEM
 // columns are tokens (Section 4.2.1 in row form; Algorithm 1 on the whole chunk):
@@ -33,7 +34,10 @@ namespace {
 
 constexpr int D = 128;
 constexpr int C = kChunk;
-constexpr int WG = 128;
+constexpr int NSLOT = 2;
+constexpr int ST = 256;                       // threads per slot
+constexpr int kThreadsTc = NSLOT * ST + 128;  // 16 slot warps + one warpgroup that issues the MMAs
+constexpr int kRegsSlot = 112, kRegsIssuer = 32;   // register split after setmaxnreg (launch: 96 each)
 
 // ---- shared memory map of one slot (bytes; every operand buffer is 1024-byte aligned)
 constexpr uint32_t OFF_K = 0;          // K tile: 2 boxes [64 keys][64 ch], SW128
@@ -50,35 +54,48 @@ struct SlotScalars {
     float ac[C];        // G2_c - max(G2_c, -60): exponent correction of clamped tokens
     float w[C];         // zeta_C / zeta_j
     float s0[C];        // 2 / (L + mu)
+    float omega[C], rho2[C];   // weight schedule state of Algorithm 1
     float dj[C];        // Frobenius increments
-    float4 coef[2][C];  // per-iteration (sigma, beta, A, zt)
+    float part[3][2][C];  // partial sums of the Frobenius epilogue: [quantity][column half][key]
+    float4 coef[2][C];  // per-iteration (sigma zt, beta, A, -): x' <- A x' - beta x'_prev + sigma zt (q - y)
     float red[8];
     float hh;           // ||H_0||_F^2
     int clamped;        // chunk decays below 2^-60 somewhere
+    int req_op;         // request to the MMA issuer
 };
-constexpr uint32_t SLOT_BYTES = OFF_SC + 4096;
-static_assert(sizeof(SlotScalars) <= 4096, "scalar block too large");
+constexpr uint32_t SLOT_BYTES = OFF_SC + 7168;
+static_assert(sizeof(SlotScalars) <= 7168, "scalar block too large");
 
 // ---- TMEM columns
-constexpr uint32_t TM_H = 0, TM_U = 128, TM_Y0 = 256, TM_SPARE = 320, TM_Y1 = 384, TM_S = 448;
+// H, U: fp32 masters.  Y0 / Y1: the slots' Y^T / O^T accumulators.  Q: the slots' q tiles as packed bf16 pairs
+// (32 columns each).  S: the slots' score accumulators, M = 64 rows each, interleaved on lane halves.
+constexpr uint32_t TM_H = 0, TM_U = 128, TM_Y0 = 256, TM_Q = 320, TM_Y1 = 384, TM_S = 448;
 
-enum { BAR_TMA = 0, BAR_A, BAR_B, BAR_COUNT };   // per-slot mbarriers
+enum { BAR_TMA = 0, BAR_A, BAR_B, BAR_REQ, BAR_COUNT };   // per-slot mbarriers
+enum { OP_FROB = 1, OP_ITER1, OP_ITER1_LAST, OP_ITER2, OP_OUT, OP_EXIT };
 
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes,
-                                              uint32_t layout_type) {
-    return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16) |
-           ((uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32) | ((uint64_t)1 << 46) |
-           ((uint64_t)(layout_type & 7) << 61);
-}
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn, int b_mn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem), "l"(da), "l"(db),
-                 "r"(idesc), "r"(acc)
-                 : "memory");
+// Every operand of this kernel uses the 128-byte swizzle with 1024 bytes between 8-row groups, so all
+// shared-memory descriptors share one high word; the low word holds the start address and the leading offset.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+    return ((saddr >> 4) & 0x3FFF) | (((lbo_bytes >> 4) & 0x3FFF) << 16);
+}
+// a_step / b_step are added to the low words inside the asm block (as immediates), so that the compiler does
+// not keep one register per k-step alive in the issuer, which runs on a small register budget.
+template <int ACC>
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, int a_step, uint32_t b_lo, int b_step,
+                                       uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t.reg .b32 la, lb;\n\t"
+        "add.u32 la, %1, %5;\n\tadd.u32 lb, %2, %6;\n\t"
+        "mov.b64 da, {la, %4};\n\tmov.b64 db, {lb, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, %7;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc),
+        "r"(kDescHi), "r"(a_step), "r"(b_step), "n"(ACC)
+        : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -86,15 +103,44 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void wg_sync(int slot) { asm volatile("bar.sync %0, 128;" ::"r"(slot + 1) : "memory"); }
+__device__ __forceinline__ void slot_sync(int slot) { asm volatile("bar.sync %0, 256;" ::"r"(slot + 1) : "memory"); }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done != 0;
+}
 
 #define TMEM_LD16(taddr, r)                                                                                   \
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];" \
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),       \
                    "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])  \
                  : "r"(taddr)                                                                                             \
+                 : "memory")
+#define TMEM_LD8(taddr, r)                                                                                    \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"                                 \
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])        \
+                 : "r"(taddr)                                                                                             \
+                 : "memory")
+#define TMEM_LD2(taddr, r) \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(taddr) : "memory")
+#define TMEM_LD4(taddr, r)                                                                                    \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"                                             \
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])                                                         \
+                 : "r"(taddr)                                                                                             \
+                 : "memory")
+#define TMEM_ST16(taddr, r)                                                                                   \
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" \
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),   \
+                 "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])            \
                  : "memory")
 #define TMEM_LD32(taddr, r)                                                                                   \
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"         \
@@ -114,6 +160,14 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
                  "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),         \
                  "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])                      \
                  : "memory")
+// 16 lanes x 32 columns spread over the whole warp: thread l holds rows l/4 and l/4 + 8, and for column
+// block i (8 columns) the pair 2 (l % 4), 2 (l % 4) + 1: r[4 i + 2 h + e] = (row l/4 + 8 h, column 8 i + 2 (l%4) + e)
+#define TMEM_LD_16x256b_x4(taddr, r)                                                                          \
+    asm volatile("tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];" \
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),       \
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])  \
+                 : "r"(taddr)                                                                                             \
+                 : "memory")
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
@@ -127,77 +181,323 @@ __device__ __forceinline__ float ex2_fast(float x) {
     return y;
 }
 
-struct TcParams {
-    FwdArgs a;
-};
+#ifdef GKA_TC_TIMING
+// Debug build only: event trace of block 0 (thread 0 of each slot and the two issuer threads).
+__device__ long long g_trace[4][8192];
+__device__ int g_trace_n[4];
+#define TRACE_DECL int trace_n = 0
+#define TRACE(role, id)                                                                                        \
+    do {                                                                                                       \
+        if (blockIdx.x == 0 && trace_n < 8192) g_trace[role][trace_n++] = (clock64() << 8) | (long long)(id);  \
+    } while (0)
+#define TSTAMP(k)                   \
+    do {                            \
+        if (t == 0) TRACE(slot, k); \
+    } while (0)
+#else
+#define TRACE_DECL
+#define TRACE(role, id)
+#define TSTAMP(k)
+#endif
 
-// Everything one warpgroup needs to know about itself.
+// ---------------------------------------------------------------------------------------------
+// MMA issue.  One thread per slot (in the issuer warpgroup) runs the slot's tcgen05.mma batches.  Operand
+// descriptors are a base low word per operand plus a compile-time step per k-step (K = 16 per instruction):
+//   K-major tiles made of two 64-column boxes: k-step ks -> box ks / 4 (`box` bytes apart), 32 bytes per step;
+//   MN-major tiles: 16 k-rows = 2048 bytes per step.
+// ---------------------------------------------------------------------------------------------
+struct IssueCtx {
+    uint32_t K_k, K_mn, V_mn, Kw_mn, H_k, X_mn, P_mn;   // descriptor low words at k-step 0
+    uint32_t tm_y, tm_s, bars;
+};
+__host__ __device__ constexpr int kstep(int ks, int box_bytes) { return ((ks >> 2) * box_bytes + (ks & 3) * 32) >> 4; }
+__host__ __device__ constexpr int mnstep(int ks) { return (ks * 2048) >> 4; }
+
+// acc = A(K-major, 2 boxes `abox` apart) x B(MN-major) over 8 k-steps; first step overwrites when !ACC0
+template <int ACC0>
+__device__ __forceinline__ void mma_k8_kmaj_mn(uint32_t d, uint32_t a_lo, int abox, uint32_t b_lo, uint32_t idesc) {
+    mma_ss<ACC0>(d, a_lo, kstep(0, abox), b_lo, mnstep(0), idesc);
+#pragma unroll
+    for (int ks = 1; ks < 8; ++ks) mma_ss<1>(d, a_lo, kstep(ks, abox), b_lo, mnstep(ks), idesc);
+}
+// both operands K-major (8 k-steps); b_off is an extra row offset of B in 16-byte units
+template <int ACC0>
+__device__ __forceinline__ void mma_k8_kmaj_kmaj(uint32_t d, uint32_t a_lo, int abox, uint32_t b_lo, int bbox, int b_off,
+                                                 uint32_t idesc) {
+    mma_ss<ACC0>(d, a_lo, kstep(0, abox), b_lo, kstep(0, bbox) + b_off, idesc);
+#pragma unroll
+    for (int ks = 1; ks < 8; ++ks) mma_ss<1>(d, a_lo, kstep(ks, abox), b_lo, kstep(ks, bbox) + b_off, idesc);
+}
+// both operands MN-major over 4 k-steps (64 keys), accumulating
+__device__ __forceinline__ void mma_k4_mn_mn(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) mma_ss<1>(d, a_lo, mnstep(ks), b_lo, mnstep(ks), idesc);
+}
+
+__device__ __forceinline__ void issuer_run(const IssueCtx &s, int op, uint32_t tm_H, uint32_t tm_U) {
+    constexpr uint32_t I_S = make_idesc(64, 64, 0, 1);
+    constexpr uint32_t I_Y1 = make_idesc(128, 64, 0, 1);
+    constexpr uint32_t I_Y2 = make_idesc(128, 64, 1, 1);
+    constexpr uint32_t I_ADV = make_idesc(128, 128, 1, 1);
+    constexpr uint32_t I_GR = make_idesc(64, 64, 0, 0);
+    if (op == OP_ITER1 || op == OP_ITER1_LAST) {
+        mma_k8_kmaj_mn<0>(s.tm_s, s.K_k, 8192, s.X_mn, I_S);
+        mma_commit(s.bars + 8 * BAR_A);
+        if (op == OP_ITER1) mma_k8_kmaj_mn<0>(s.tm_y, s.H_k, 16384, s.X_mn, I_Y1);
+    } else if (op == OP_ITER2) {
+        mma_k4_mn_mn(s.tm_y, s.K_mn, s.P_mn, I_Y2);
+        mma_commit(s.bars + 8 * BAR_B);
+    } else if (op == OP_FROB) {
+        // H advance: Hm += K^T (w o K)
+        mma_k4_mn_mn(tm_H, s.K_mn, s.Kw_mn, I_ADV);
+        // (K H_0)[:, 0:64] -> Y columns, lanes +0;  (K H_0)[:, 64:128] -> the slot's S region;  Gram -> Y columns, lanes +16
+        mma_k8_kmaj_kmaj<0>(s.tm_y, s.K_k, 8192, s.H_k, 16384, 0, I_GR);
+        mma_k8_kmaj_kmaj<0>(s.tm_s, s.K_k, 8192, s.H_k, 16384, 8192 >> 4, I_GR);
+        mma_k8_kmaj_kmaj<0>(s.tm_y + (16u << 16), s.K_k, 8192, s.K_k, 8192, 0, I_GR);
+        mma_commit(s.bars + 8 * BAR_A);
+    } else if (op == OP_OUT) {
+        mma_k8_kmaj_mn<0>(s.tm_y, s.H_k, 16384, s.X_mn, I_Y1);
+        mma_k4_mn_mn(s.tm_y, s.V_mn, s.P_mn, I_Y2);
+        mma_commit(s.bars + 8 * BAR_A);
+        mma_k4_mn_mn(tm_U, s.V_mn, s.Kw_mn, I_ADV);
+        mma_commit(s.bars + 8 * BAR_B);
+    }
+}
+
+// Everything a slot thread needs to know about itself.
 struct SlotCtx {
-    int slot, t, warp_q;          // slot index, thread in warpgroup (= TMEM lane), warp within warpgroup
-    uint32_t sbase;               // shared address of the slot's buffers
-    unsigned char *sptr;          // generic pointer to the same
+    int slot, t;                  // slot index, thread in slot (0..255)
+    int lane, half, warp_q;       // TMEM lane (0..127), column / token half (0..1), warp % 4
+    unsigned char *sptr;          // the slot's shared buffers
     SlotScalars *sc;
     uint32_t bars;                // shared address of the slot's mbarriers
-    uint32_t tmem;                // TMEM base
-    uint32_t tm_y, tm_s, tm_kh;   // accumulator addresses (lane offset included for tm_s)
+    uint32_t tm_y, tm_s, tm_q;    // accumulator addresses (tm_s includes the slot's lane offset), q tile columns
+    uint32_t tm_H, tm_U;          // masters
     uint32_t lane_addr;           // (32 * warp_q) << 16
     uint32_t ph[BAR_COUNT];       // phase parity of each mbarrier
     volatile int *abort_flag;
     int *device_status;
 };
 
-__device__ __forceinline__ void slot_wait(SlotCtx &cx, int which) {
-    if (*cx.abort_flag == 0) {
-        if (!mbar_wait_bounded(cx.bars + 8 * which, cx.ph[which])) {
+// Wait for an mbarrier phase: one warp of the slot polls (bounded), the others sleep in the slot's
+// named barrier, so waiting warps do not take issue slots from the other slot's working warps.
+__device__ __forceinline__ void slot_wait_addr(SlotCtx &cx, uint32_t bar, uint32_t parity) {
+    if ((cx.t >> 5) == cx.slot && *cx.abort_flag == 0) {   // the polling warp of slot s sits on scheduler s
+        if (!mbar_wait_bounded(bar, parity)) {
             *cx.abort_flag = 1;
             if (cx.device_status) atomicExch(cx.device_status, (int)GKA_ERR_TIMEOUT);
         }
     }
+    slot_sync(cx.slot);
+}
+__device__ __forceinline__ void slot_wait(SlotCtx &cx, int which) {
+    slot_wait_addr(cx, cx.bars + 8 * which, cx.ph[which]);
     cx.ph[which] ^= 1u;
 }
+// Ask the issuer warp for a batch of MMAs.  Call after slot_sync: every thread's writes and fences are done.
+// The issuing thread can stall while the tensor pipe works through earlier batches, which is why it is not
+// one of the slot's own threads.
+__device__ __forceinline__ void slot_post(SlotCtx &cx, int op) {
+    if (cx.t == 0) {
+        *reinterpret_cast<volatile int *>(&cx.sc->req_op) = op;
+        mbar_arrive(cx.bars + 8 * BAR_REQ);
+    }
+}
 
-// Masked score epilogue: S^T (TMEM, M = 64 layout) -> P operand in shared memory.
+// Masked score epilogue: S^T (TMEM, M = 64 layout, 16 lanes per quadrant) -> P operand in shared memory.
+// Every thread of the slot takes part: warp quadrant q covers keys 16 q .. 16 q + 15, column half `half`.
 __device__ __forceinline__ void p_epilogue(SlotCtx &cx) {
-    const int l = cx.t & 31;
-    const bool valid = (l >> 4) == cx.slot;
-    const int j = 16 * cx.warp_q + (l & 15);
+    const int l = cx.lane & 31;
     const SlotScalars *sc = cx.sc;
-    const float bj = -sc->G2[j];
-    const float invz = exp2f(fminf(bj, 126.f));
     const bool clamped = sc->clamped != 0;
-    unsigned char *prow = cx.sptr + OFF_P + j * 128;
+    uint32_t r[16];
+    TMEM_LD_16x256b_x4(cx.tm_s + cx.lane_addr + 32 * cx.half, r);
+    tmem_wait_ld();
 #pragma unroll
-    for (int piece = 0; piece < 2; ++piece) {
-        uint32_t r[32];
-        TMEM_LD32(cx.tm_s + cx.lane_addr + 32 * piece, r);
-        tmem_wait_ld();
-        if (valid) {
+    for (int h = 0; h < 2; ++h) {
+        const int j = 16 * cx.warp_q + (l >> 2) + 8 * h;
+        const float bj = -sc->G2[j];
+        const float invz = ex2_fast(fminf(bj, 126.f));
+        unsigned char *prow = cx.sptr + OFF_P + j * 128 + (l & 3) * 4;
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                uint32_t pk[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c0 = 32 * piece + 8 * ch + 2 * u;
-                    float f0, f1;
-                    if (!clamped) {
-                        f0 = invz; f1 = invz;
-                    } else {
-                        f0 = ex2_fast(sc->ac[c0] + bj);
-                        f1 = ex2_fast(sc->ac[c0 + 1] + bj);
-                    }
-                    const float p0 = (j <= c0) ? __uint_as_float(r[8 * ch + 2 * u]) * f0 : 0.f;
-                    const float p1 = (j <= c0 + 1) ? __uint_as_float(r[8 * ch + 2 * u + 1]) * f1 : 0.f;
-                    pk[u] = pack_bf16(p0, p1);
-                }
-                const int chunk = (4 * piece + ch) ^ (j & 7);
-                *reinterpret_cast<uint4 *>(prow + chunk * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        for (int i = 0; i < 4; ++i) {
+            const int c0 = 32 * cx.half + 8 * i + 2 * (l & 3);
+            float f0 = invz, f1 = invz;
+            if (clamped) {
+                f0 = ex2_fast(sc->ac[c0] + bj);
+                f1 = ex2_fast(sc->ac[c0 + 1] + bj);
             }
+            const float p0 = (j <= c0) ? __uint_as_float(r[4 * i + 2 * h]) * f0 : 0.f;
+            const float p1 = (j <= c0 + 1) ? __uint_as_float(r[4 * i + 2 * h + 1]) * f1 : 0.f;
+            const int chunk = (4 * cx.half + i) ^ (j & 7);
+            *reinterpret_cast<uint32_t *>(prow + chunk * 16) = pack_bf16(p0, p1);
         }
     }
 }
 
-template <int NSLOT>
-__global__ void __launch_bounds__(WG *NSLOT, 1)
+// One pass over a master (H or U) for this thread's row and column half: source is TMEM, or global memory
+// at the start of a run.  Writes the bf16 operand copy, optionally accumulates the sum of squares, scales
+// by zeta_C and stores the result back to TMEM.
+template <bool SUMSQ>
+__device__ __forceinline__ float master_pass(SlotCtx &cx, uint32_t tm_master, bool from_global, const float *grow,
+                                             float zetaC) {
+    float ss = 0.f;
+    unsigned char *hrow = cx.sptr + OFF_H + cx.half * 16384 + cx.lane * 128;
+#pragma unroll
+    for (int piece = 0; piece < 2; ++piece) {
+        uint32_t r[32];
+        const uint32_t taddr = tm_master + cx.lane_addr + 64 * cx.half + 32 * piece;
+        if (!from_global) {
+            TMEM_LD32(taddr, r);
+            tmem_wait_ld();
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float4 v4 = grow ? *reinterpret_cast<const float4 *>(grow + 64 * cx.half + 32 * piece + 4 * i)
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+                r[4 * i + 0] = __float_as_uint(v4.x); r[4 * i + 1] = __float_as_uint(v4.y);
+                r[4 * i + 2] = __float_as_uint(v4.z); r[4 * i + 3] = __float_as_uint(v4.w);
+            }
+        }
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float v0 = __uint_as_float(r[8 * ch + 2 * u]), v1 = __uint_as_float(r[8 * ch + 2 * u + 1]);
+                if (SUMSQ) ss = fmaf(v0, v0, fmaf(v1, v1, ss));
+                pk[u] = pack_bf16(v0, v1);
+            }
+            const int chunk = (4 * piece + ch) ^ (cx.lane & 7);
+            *reinterpret_cast<uint4 *>(hrow + chunk * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * zetaC);
+        TMEM_ST32(taddr, r);
+    }
+    tmem_wait_st();
+    return ss;
+}
+
+// Copy this thread's part of a master from TMEM to global memory (final state of a sequence).
+__device__ __forceinline__ void master_store(SlotCtx &cx, uint32_t tm_master, float *grow) {
+#pragma unroll
+    for (int piece = 0; piece < 2; ++piece) {
+        uint32_t r[32];
+        TMEM_LD32(tm_master + cx.lane_addr + 64 * cx.half + 32 * piece, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            *reinterpret_cast<float4 *>(grow + 64 * cx.half + 32 * piece + 4 * i) =
+                make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]),
+                            __uint_as_float(r[4 * i + 3]));
+    }
+}
+
+// The solve of one chunk: x_0, n_iter Chebyshev iterations, and the masked scores of the final iterate.
+// Kept out of line on purpose: the iterate (x, x_prev: 64 registers per thread) must stay in registers for
+// the whole loop, and a call boundary makes the compiler park the caller's chunk-level values once per
+// chunk instead of reloading spilled values inside the loop (local memory misses the small L1 here).
+// Returns the updated phase parities of the slot's barriers A and B (bit 0, bit 1).
+__device__ __forceinline__ uint32_t chunk_solve(SlotCtx cx, int n_iter) {
+    SlotScalars *sc = cx.sc;
+    const int slot = cx.slot, t = cx.t, lane = cx.lane, half = cx.half;
+    TRACE_DECL;
+    // ---- x_0 = 2 q / (L + mu), X' operand (this thread: channel `lane`, tokens 32 half .. 32 half + 31)
+    float xm[32], xp[32];
+    {
+        uint32_t qp[16];
+        TMEM_LD16(cx.tm_q + cx.lane_addr + 16 * half, qp);
+        tmem_wait_ld();
+        unsigned char *xrow = cx.sptr + OFF_X + lane * 128;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i0 = 8 * ch + 2 * u, c0 = 32 * half + i0;
+                // the iterate is kept scaled by zt_c (the recurrence is linear), as the operand needs it
+                const float x0 = sc->s0[c0] * sc->zt[c0] * bf16_lo(qp[i0 >> 1]);
+                const float x1 = sc->s0[c0 + 1] * sc->zt[c0 + 1] * bf16_hi(qp[i0 >> 1]);
+                xm[i0] = x0; xm[i0 + 1] = x1;
+                xp[i0] = 0.f; xp[i0 + 1] = 0.f;
+                pk[u] = pack_bf16(x0, x1);
+            }
+            *reinterpret_cast<uint4 *>(xrow + (((4 * half + ch) ^ (lane & 7)) * 16)) =
+                make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+    }
+    fence_async_smem();
+    fence_before();
+    slot_sync(slot);
+    TSTAMP(6);
+
+    // ---- Algorithm 1: n_iter iterations on the whole chunk (+ one extra score pass for the output)
+    for (int it = 0; it <= n_iter; ++it) {
+        const bool last = (it == n_iter);
+        slot_post(cx, last ? OP_ITER1_LAST : OP_ITER1);
+        TSTAMP(17);
+        if (!last && t < C) {   // weight schedule and per-token coefficients of this iteration
+            const float omega = 4.f / (4.f - sc->rho2[t] * sc->omega[t]);
+            sc->omega[t] = omega;
+            const float sigma = sc->s0[t] * omega, beta = omega - 1.f;
+            sc->coef[it & 1][t] = make_float4(sigma * sc->zt[t], beta, 1.f + beta - sigma * sc->lam[t], 0.f);
+        }
+        TSTAMP(15);
+        slot_wait(cx, BAR_A);
+        fence_after();
+        TSTAMP(7);
+        p_epilogue(cx);
+        fence_async_smem();
+        fence_before();
+        slot_sync(slot);
+        TSTAMP(8);
+        if (last) break;
+        slot_post(cx, OP_ITER2);
+        TSTAMP(16);
+        slot_wait(cx, BAR_B);
+        fence_after();
+        TSTAMP(9);
+        {
+            const float4 *coef = sc->coef[it & 1] + 32 * half;
+            unsigned char *xrow = cx.sptr + OFF_X + lane * 128;
+#pragma unroll
+            for (int piece = 0; piece < 8; ++piece) {     // 4 tokens at a time keeps the transient registers few
+                uint32_t r[4], qq[2];
+                TMEM_LD4(cx.tm_y + cx.lane_addr + 32 * half + 4 * piece, r);
+                TMEM_LD2(cx.tm_q + cx.lane_addr + 16 * half + 2 * piece, qq);
+                tmem_wait_ld();
+                uint32_t pk[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    float xo[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int i = 4 * piece + 2 * u + e;
+                        const float4 cf = coef[i];
+                        const float qv = e == 0 ? bf16_lo(qq[u]) : bf16_hi(qq[u]);
+                        const float acc = __uint_as_float(r[2 * u + e]);
+                        const float xn = fmaf(cf.x, qv - acc, fmaf(cf.z, xm[i], -cf.y * xp[i]));
+                        xp[i] = xm[i];
+                        xm[i] = xn;
+                        xo[e] = xn;
+                    }
+                    pk[u] = pack_bf16(xo[0], xo[1]);
+                }
+                const int chunk = (4 * half + (piece >> 1)) ^ (lane & 7);
+                *reinterpret_cast<uint2 *>(xrow + chunk * 16 + 8 * (piece & 1)) = make_uint2(pk[0], pk[1]);
+            }
+        }
+        fence_async_smem();
+        fence_before();
+        slot_sync(slot);
+        TSTAMP(10);
+    }
+
+    return cx.ph[BAR_A] | (cx.ph[BAR_B] << 1);
+}
+
+__global__ void __launch_bounds__(kThreadsTc, 1)
 fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, FwdArgs a) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t s_bars[NSLOT * BAR_COUNT + 2];
@@ -206,24 +506,6 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
     unsigned char *smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     const int tid = threadIdx.x;
-    const int slot = tid / WG;
-    SlotCtx cx;
-    cx.slot = slot;
-    cx.t = tid % WG;
-    cx.warp_q = cx.t >> 5;
-    cx.sptr = smem + (size_t)slot * SLOT_BYTES;
-    cx.sbase = smem_u32(cx.sptr);
-    cx.sc = reinterpret_cast<SlotScalars *>(cx.sptr + OFF_SC);
-    cx.bars = smem_u32(&s_bars[slot * BAR_COUNT]);
-    cx.lane_addr = (uint32_t)(32 * cx.warp_q) << 16;
-#pragma unroll
-    for (int i = 0; i < BAR_COUNT; ++i) cx.ph[i] = 0;
-    cx.abort_flag = &s_abort;
-    cx.device_status = a.device_status;
-    const uint32_t tokH = smem_u32(&s_bars[NSLOT * BAR_COUNT]);
-    const uint32_t tokU = tokH + 8;
-    SlotScalars *sc = cx.sc;
-    const int t = cx.t;
 
     if (tid == 0) {
         s_abort = 0;
@@ -239,465 +521,516 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     fence_before();
     __syncthreads();
     fence_after();
-    cx.tmem = s_tmem_base;
-    cx.tm_y = cx.tmem + (slot == 0 ? TM_Y0 : TM_Y1);
-    cx.tm_kh = cx.tmem + (slot == 0 ? TM_Y0 : TM_SPARE) + ((uint32_t)(16 * slot) << 16);
-    cx.tm_s = cx.tmem + TM_S + ((uint32_t)(16 * slot) << 16);
-    const uint32_t tm_H = cx.tmem + TM_H, tm_U = cx.tmem + TM_U;
-
-    // ---- descriptors (k-step 0); later k-steps add a constant to the low word
-    const uint64_t dK_k = make_desc(cx.sbase + OFF_K, 16, 1024, 2);      // K as K-major (rows = keys)
-    const uint64_t dK_mn = make_desc(cx.sbase + OFF_K, 8192, 1024, 2);   // K as MN-major (rows = channels)
-    const uint64_t dV_mn = make_desc(cx.sbase + OFF_V, 8192, 1024, 2);
-    const uint64_t dKw_mn = make_desc(cx.sbase + OFF_KW, 8192, 1024, 2);
-    const uint64_t dH_k = make_desc(cx.sbase + OFF_H, 16, 1024, 2);      // H_0 / U_0, K-major
-    const uint64_t dX_mn = make_desc(cx.sbase + OFF_X, 8192, 1024, 2);
-    const uint64_t dP_mn = make_desc(cx.sbase + OFF_P, 8192, 1024, 2);
-    constexpr uint32_t I_S = make_idesc(64, 64, 0, 1);
-    constexpr uint32_t I_Y1 = make_idesc(128, 64, 0, 1);
-    constexpr uint32_t I_Y2 = make_idesc(128, 64, 1, 1);
-    constexpr uint32_t I_ADV = make_idesc(128, 128, 1, 1);
-    constexpr uint32_t I_KH = make_idesc(64, 128, 0, 0);
-    constexpr uint32_t I_GR = make_idesc(64, 64, 0, 0);
-    // K-major operand with two 64-column boxes: k-step ks -> box ks/4 (stride `box` bytes), +32 B per step inside
-    auto kmaj_step = [](uint64_t d0, int ks, uint32_t box_bytes) {
-        return d0 + (uint64_t)(((ks >> 2) * box_bytes + (ks & 3) * 32) >> 4);
-    };
-    auto mn_step = [](uint64_t d0, int ks) { return d0 + (uint64_t)((ks * 2048) >> 4); };
+    const uint32_t tmem = s_tmem_base;
+    const uint32_t tm_H = tmem + TM_H, tm_U = tmem + TM_U;
+    const uint32_t tokH = smem_u32(&s_bars[NSLOT * BAR_COUNT]);
+    const uint32_t tokU = tokH + 8;
+    TRACE_DECL;
 
     const WorkPlan &P = a.plan;
     const int item = blockIdx.x;
     const long long f_lo = P.lo(item), f_hi = P.lo(item + 1);
-    const __nv_bfloat16 *gq = reinterpret_cast<const __nv_bfloat16 *>(a.q);
-    __nv_bfloat16 *gout = reinterpret_cast<__nv_bfloat16 *>(a.out);
-    const size_t st = state_floats(D, D);
-    const bool adaptive = (a.flags & GKA_FLAG_ADAPTIVE_LAMBDA) != 0;
 
-    auto issue_tma = [&](long long f) {   // thread 0 of the warpgroup: K and V tiles of flat chunk f
-        const int seq = (int)(f / P.N), n = (int)(f % P.N);
-        const int b = seq / a.heads, h = seq % a.heads;
+    if (tid >= NSLOT * ST) {
+        // ================================ MMA issuer warpgroup ================================
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssuer));
+        const int s = ((tid - NSLOT * ST) >> 5) - 2;    // warps 2, 3 of the warpgroup (schedulers 2, 3) serve slots 0, 1
+        if ((tid & 31) == 0 && s >= 0 && f_lo + s < f_hi) {
+            const SlotScalars *isc = reinterpret_cast<const SlotScalars *>(smem + (size_t)s * SLOT_BYTES + OFF_SC);
+            const uint32_t sb = smem_u32(smem + (size_t)s * SLOT_BYTES);
+            IssueCtx ic;
+            ic.K_k = desc_lo(sb + OFF_K, 16);        // K as K-major (rows = keys)
+            ic.K_mn = desc_lo(sb + OFF_K, 8192);     // K as MN-major (rows = channels; 8192 bytes to the next 64)
+            ic.V_mn = desc_lo(sb + OFF_V, 8192);
+            ic.Kw_mn = desc_lo(sb + OFF_KW, 8192);
+            ic.H_k = desc_lo(sb + OFF_H, 16);        // H_0 / U_0, K-major
+            ic.X_mn = desc_lo(sb + OFF_X, 8192);
+            ic.P_mn = desc_lo(sb + OFF_P, 8192);
+            ic.tm_y = tmem + (s == 0 ? TM_Y0 : TM_Y1);
+            ic.tm_s = tmem + TM_S + ((uint32_t)(16 * s) << 16);
+            ic.bars = smem_u32(&s_bars[s * BAR_COUNT]);
+            uint32_t reqph = 0;
+            for (;;) {
+                // a request normally arrives within microseconds; give up after seconds of silence
+                bool got = false;
+                for (int tries = 0; tries < 4 && !got; ++tries) got = mbar_wait_bounded(ic.bars + 8 * BAR_REQ, reqph);
+                if (!got || s_abort != 0) {
+                    s_abort = 1;
+                    break;
+                }
+                reqph ^= 1u;
+                const int op = *reinterpret_cast<const volatile int *>(&isc->req_op);
+                TRACE(2 + s, 32 + op);
+                if (op == OP_EXIT) break;
+                fence_after();
+                issuer_run(ic, op, tm_H, tm_U);
+                TRACE(2 + s, 48 + op);
+            }
+        }
+    } else {
+        // ================================= slot threads =================================
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSlot));
+        SlotCtx cx;
+        cx.slot = tid / ST;
+        cx.t = tid % ST;
+        cx.lane = cx.t & 127;
+        cx.half = cx.t >> 7;
+        cx.warp_q = (cx.t >> 5) & 3;
+        cx.sptr = smem + (size_t)cx.slot * SLOT_BYTES;
+        cx.sc = reinterpret_cast<SlotScalars *>(cx.sptr + OFF_SC);
+        cx.bars = smem_u32(&s_bars[cx.slot * BAR_COUNT]);
+        cx.lane_addr = (uint32_t)(32 * cx.warp_q) << 16;
+#pragma unroll
+        for (int i = 0; i < BAR_COUNT; ++i) cx.ph[i] = 0;
+        cx.abort_flag = &s_abort;
+        cx.device_status = a.device_status;
+        cx.tm_y = tmem + (cx.slot == 0 ? TM_Y0 : TM_Y1);
+        cx.tm_q = tmem + TM_Q + 32 * cx.slot;
+        cx.tm_s = tmem + TM_S + ((uint32_t)(16 * cx.slot) << 16);
+        cx.tm_H = tm_H;
+        cx.tm_U = tm_U;
+        SlotScalars *sc = cx.sc;
+        const int slot = cx.slot, t = cx.t, lane = cx.lane, half = cx.half;
+        const uint32_t sbase = smem_u32(cx.sptr);
+
+        const __nv_bfloat16 *gq = reinterpret_cast<const __nv_bfloat16 *>(a.q);
+        __nv_bfloat16 *gout = reinterpret_cast<__nv_bfloat16 *>(a.out);
+        const size_t st = state_floats(D, D);
+        const bool adaptive = (a.flags & GKA_FLAG_ADAPTIVE_LAMBDA) != 0;
+
+        auto issue_tma = [&](long long f) {   // thread 0 of the slot: K and V tiles of flat chunk f
+            const int seq = (int)(f / P.N), n = (int)(f % P.N);
+            const int b = seq / a.heads, h = seq % a.heads;
+            const int y = b * a.T + n * C;
+            const uint32_t bar = cx.bars + 8 * BAR_TMA;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(32768u) : "memory");
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                const int x = h * D + 64 * hf;
+                asm volatile(
+                    "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
+                        "r"(sbase + OFF_K + 8192 * hf), "l"(reinterpret_cast<uint64_t>(&tmK)), "r"(x), "r"(y), "r"(bar)
+                    : "memory");
+                asm volatile(
+                    "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
+                        "r"(sbase + OFF_V + 8192 * hf), "l"(reinterpret_cast<uint64_t>(&tmV)), "r"(x), "r"(y), "r"(bar)
+                    : "memory");
+            }
+        };
+
+        if (t == 0 && f_lo + slot < f_hi) issue_tma(f_lo + slot);
+        slot_sync(slot);
+
+        for (long long f = f_lo + slot; f < f_hi; f += NSLOT) {
+            const long long m = f - f_lo;              // index of this chunk inside the block's range
+            const int seq = (int)(f / P.N), n = (int)(f % P.N);
+            const int b = seq / a.heads, h = seq % a.heads;
+            const size_t tok0 = ((size_t)b * a.T + (size_t)n * C) * a.heads + h;
+            const bool run_start = (m == 0) || (n == 0);
+            const bool seq_end = (n == P.N - 1);
+            const float *init_src = nullptr;           // where a run's start state comes from (nullptr = zero)
+            if (run_start) init_src = (n == 0) ? (a.state_in ? a.state_in + (size_t)seq * st : nullptr)
+                                               : a.ws.start + (size_t)item * st;
+
+            // ---- q for this thread's channel and its 32 tokens, packed bf16 pairs (issued early)
+            {
+                uint32_t qp[16];
+                const unsigned short *qs = reinterpret_cast<const unsigned short *>(gq) +
+                                           (tok0 + (size_t)32 * half * a.heads) * D + lane;
+                const size_t rs = (size_t)a.heads * D;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const uint32_t lo = qs[(size_t)(2 * i) * rs], hi = qs[(size_t)(2 * i + 1) * rs];
+                    qp[i] = lo | (hi << 16);
+                }
+                // parked in TMEM for the whole chunk (exact: q is bf16); this slot's previous chunk is done with it
+                TMEM_ST16(cx.tm_q + cx.lane_addr + 16 * half, qp);
+                tmem_wait_st();
+            }
+
+            // ---- gates (threads 0..63 own token c = t for scalar bookkeeping)
+            if (t < C) {
+                const float g = a.gate[tok0 + (size_t)t * a.heads];
+                sc->w[t] = fmaxf(log2f(g), -115.f);     // temporary: log2 gamma
+                sc->lam[t] = a.lam[tok0 + (size_t)t * a.heads];
+            }
+            slot_sync(slot);
+            float G2c = 0.f;
+            if (t < C) {
+                for (int i = 0; i <= t; ++i) G2c += sc->w[i];
+            }
+            slot_sync(slot);
+            if (t < C) {
+                sc->G2[t] = G2c;
+                const float mc = fmaxf(G2c, -60.f);
+                sc->zt[t] = exp2f(mc);
+                sc->ac[t] = G2c - mc;
+                if (t == C - 1) sc->clamped = (G2c < -60.f) ? 1 : 0;
+            }
+            slot_sync(slot);
+            if (t < C) sc->w[t] = exp2f(sc->G2[C - 1] - sc->G2[t]);
+            const float zetaC = exp2f(sc->G2[C - 1]);
+            slot_sync(slot);
+            TSTAMP(0);
+
+            // ---- K, V tiles have landed
+            slot_wait(cx, BAR_TMA);
+            TSTAMP(1);
+
+            // ---- w o K (same swizzled positions as K)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int qi = t + ST * i;                 // 16-byte chunk index in the 16 KB tile
+                const int j = (qi & 511) >> 3;             // key row of this chunk
+                uint4 v = *reinterpret_cast<const uint4 *>(cx.sptr + OFF_K + qi * 16);
+                const float wj = sc->w[j];
+                uint32_t *pv = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) pv[u] = pack_bf16(bf16_lo(pv[u]) * wj, bf16_hi(pv[u]) * wj);
+                *reinterpret_cast<uint4 *>(cx.sptr + OFF_KW + qi * 16) = v;
+            }
+            TSTAMP(2);
+
+            // ---- H master: wait for the previous chunk's advance, then one pass: ||H_0||^2, bf16 copy, scale
+            if (m > 0) slot_wait_addr(cx, tokH, (uint32_t)((m - 1) & 1));   // chunk m - 1 finished its H work
+            fence_after();
+            {
+                float hh = master_pass<true>(cx, tm_H, run_start,
+                                             init_src ? init_src + (size_t)lane * D : nullptr, zetaC);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) hh += __shfl_xor_sync(0xffffffffu, hh, o);
+                if ((t & 31) == 0) sc->red[t >> 5] = hh;
+            }
+            fence_async_smem();
+            fence_before();
+            slot_sync(slot);
+            slot_post(cx, OP_FROB);
+            if (t == 0) {
+                float s = 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) s += sc->red[i];
+                sc->hh = s;
+            }
+            TSTAMP(3);
+            slot_wait(cx, BAR_A);
+            fence_after();
+            TSTAMP(4);
+
+            // ---- chunk-wise Frobenius norms: partial sums per key from K H_0 and the Gram matrix.
+            // 32x32b loads address whole 32-lane quadrants; an M = 64 accumulator placed at lane offset 0 / 16
+            // has its rows on lanes 0..15 / 16..31 of every quadrant.  Each thread takes 32 of the 64 columns.
+            {
+                const int l = lane & 31;
+                const int j = 16 * cx.warp_q + (l & 15);
+                const uint32_t y_cols = cx.tm_y + cx.lane_addr + 32 * half;
+                const uint32_t s_cols = tmem + TM_S + cx.lane_addr + 32 * half;
+                float a0 = 0.f, a1 = 0.f, bjs = 0.f;
+#pragma unroll
+                for (int src = 0; src < 2; ++src) {     // (K H_0) columns 0..63 (Y region) and 64..127 (S region)
+                    uint32_t r[32];
+                    TMEM_LD32(src == 0 ? y_cols : s_cols, r);
+                    tmem_wait_ld();
+                    const unsigned char *krow = cx.sptr + OFF_K + src * 8192 + j * 128;
+                    float acc = 0.f;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        const int chunk = (4 * half + ch) ^ (j & 7);
+                        const uint4 kv = *reinterpret_cast<const uint4 *>(krow + chunk * 16);
+                        const uint32_t *pk = reinterpret_cast<const uint32_t *>(&kv);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            acc = fmaf(__uint_as_float(r[8 * ch + 2 * u]), bf16_lo(pk[u]), acc);
+                            acc = fmaf(__uint_as_float(r[8 * ch + 2 * u + 1]), bf16_hi(pk[u]), acc);
+                        }
+                    }
+                    if (src == 0) a0 = acc; else a1 = acc;
+                }
+                const float G2j = sc->G2[j];
+                {
+                    uint32_t r[32];
+                    TMEM_LD32(y_cols, r);                // Gram rows sit on lanes 16..31 of the Y columns
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int ii = 32 * half + i;
+                        const float g = __uint_as_float(r[i]);
+                        const float g2 = g * g;
+                        if (ii < j) bjs = fmaf(2.f * ex2_fast(G2j - sc->G2[ii]), g2, bjs);
+                        else if (ii == j) bjs += g2;
+                    }
+                }
+                if ((l >> 4) == 0) sc->part[0][half][j] = a0;
+                if ((l >> 4) == slot) sc->part[1][half][j] = a1;
+                if ((l >> 4) == 1) sc->part[2][half][j] = bjs;
+            }
+            fence_before();
+            slot_sync(slot);
+            // H master is final for this chunk, the Frobenius temporaries are consumed
+            if (seq_end && a.state_out) {
+                fence_after();
+                master_store(cx, tm_H, a.state_out + (size_t)seq * st + (size_t)lane * D);
+                fence_before();
+                slot_sync(slot);
+            }
+            if (t == 0) mbar_arrive(tokH);
+            TSTAMP(5);
+
+            // ---- f_c, Chebyshev initialisation (threads 0..63: token c = t)
+            if (t < C) {
+                sc->dj[t] = fmaf(2.f * exp2f(sc->G2[t]),
+                                 (sc->part[0][0][t] + sc->part[0][1][t]) + (sc->part[1][0][t] + sc->part[1][1][t]),
+                                 sc->part[2][0][t] + sc->part[2][1][t]);
+            }
+            slot_sync(slot);
+            if (t < C) {
+                const float G2t = sc->G2[t];
+                float s = exp2f(2.f * G2t) * sc->hh;
+                for (int j = 0; j <= t; ++j) s = fmaf(ex2_fast(2.f * (G2t - sc->G2[j])), sc->dj[j], s);
+                const float fc = sqrtf(fmaxf(s, 0.f));
+                float lamc = sc->lam[t];
+                if (adaptive) lamc *= fc;
+                const float Lpm = fc + 2.f * lamc;
+                const float rho = fc / Lpm;
+                sc->lam[t] = lamc;
+                sc->rho2[t] = rho * rho;
+                sc->omega[t] = 2.f;
+                sc->s0[t] = 2.f / Lpm;
+                if (a.fro_out) a.fro_out[tok0 + (size_t)t * a.heads] = fc;
+            }
+            slot_sync(slot);
+
+            // ---- x_0, Chebyshev iterations, final masked scores
+            {
+                const uint32_t phab = chunk_solve(cx, a.n_iter);
+                cx.ph[BAR_A] = phab & 1u;
+                cx.ph[BAR_B] = phab >> 1;
+            }
+
+            // ---- output: U master pass (bf16 copy into the H buffer, scale), O^T = U_0 X'^T + V^T P^T, U advance
+            if (m > 0) slot_wait_addr(cx, tokU, (uint32_t)((m - 1) & 1));   // chunk m - 1 wrote its output, advanced U
+            fence_after();
+            master_pass<false>(cx, tm_U, run_start,
+                               init_src ? init_src + (size_t)D * D + (size_t)lane * D : nullptr, zetaC);
+            fence_async_smem();
+            fence_before();
+            slot_sync(slot);
+            slot_post(cx, OP_OUT);
+            TSTAMP(11);
+            slot_wait(cx, BAR_A);
+            fence_after();
+            TSTAMP(12);
+            {
+                unsigned short *orow = reinterpret_cast<unsigned short *>(gout) +
+                                       (tok0 + (size_t)32 * half * a.heads) * D + lane;
+                const size_t rs = (size_t)a.heads * D;
+#pragma unroll
+                for (int piece = 0; piece < 2; ++piece) {
+                    uint32_t r[16];
+                    TMEM_LD16(cx.tm_y + cx.lane_addr + 32 * half + 16 * piece, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const __nv_bfloat16 ob = __float2bfloat16_rn(__uint_as_float(r[i]));
+                        orow[(size_t)(16 * piece + i) * rs] = *reinterpret_cast<const unsigned short *>(&ob);
+                    }
+                }
+            }
+            TSTAMP(13);
+            slot_wait(cx, BAR_B);     // U advance done: every tensor-core read of this chunk's tiles is done
+            fence_after();
+            if (seq_end && a.state_out)
+                master_store(cx, tm_U, a.state_out + (size_t)seq * st + (size_t)D * D + (size_t)lane * D);
+            fence_before();
+            slot_sync(slot);
+            if (t == 0) {
+                mbar_arrive(tokU);
+                if (f + NSLOT < f_hi && *cx.abort_flag == 0) issue_tma(f + NSLOT);
+            }
+            TSTAMP(14);
+            if (*cx.abort_flag != 0) break;
+        }
+        if (f_lo + slot < f_hi) slot_post(cx, OP_EXIT);
+    }
+
+#ifdef GKA_TC_TIMING
+    if (blockIdx.x == 0) {
+        if (tid == 0) g_trace_n[0] = trace_n;
+        if (tid == ST) g_trace_n[1] = trace_n;
+        if (tid == NSLOT * ST + 64) g_trace_n[2] = trace_n;
+        if (tid == NSLOT * ST + 96) g_trace_n[3] = trace_n;
+    }
+#endif
+    fence_before();
+    __syncthreads();
+    if (tid < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+}
+
+// ---------------------------------------------------------------------------------------------
+// Segment summaries on the tensor cores: for every work item whose range ends inside a sequence, the decay
+// product and (delta-H, delta-U) of its last run, i.e. the run's final state for a zero start state:
+//     dH <- zeta_C dH + K^T (w o K),   dU <- zeta_C dU + V^T (w o K)      chunk by chunk,
+// with the accumulators in TMEM.  One block of 128 threads per item; K and V tiles are double-buffered.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t SUM_STAGE = 32768;            // K tile + V tile
+constexpr uint32_t SUM_OFF_KW = 2 * SUM_STAGE;   // w o K
+constexpr uint32_t SUM_SMEM = SUM_OFF_KW + 16384 + 1024;
+
+__global__ void __launch_bounds__(128, 1)
+fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, FwdArgs a) {
+    const WorkPlan &P = a.plan;
+    const int item = blockIdx.x;
+    if (!P.cut_out(item)) return;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t s_bars[3];      // TMA stage 0, TMA stage 1, MMA
+    __shared__ uint32_t s_tmem_base;
+    __shared__ float s_lg[C], s_w[C], s_G2[C];
+    unsigned char *smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+    const uint32_t sb = smem_u32(smem);
+    const int t = threadIdx.x, warp_q = t >> 5;
+    const uint32_t lane_addr = (uint32_t)(32 * warp_q) << 16;
+
+    if (t == 0) {
+        for (int i = 0; i < 3; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_bars[i])));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (t < 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(&s_tmem_base))
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem = s_tmem_base, tm_H = tmem, tm_U = tmem + 128;
+    const uint32_t bar_mma = smem_u32(&s_bars[2]);
+
+    const long long f0 = P.last_run_start(item), f1 = P.lo(item + 1);
+    const int seq = (int)(f0 / P.N), b = seq / a.heads, h = seq % a.heads;
+    auto issue_tma = [&](long long f, int stage) {
+        const int n = (int)(f % P.N);
         const int y = b * a.T + n * C;
-        const uint32_t bar = cx.bars + 8 * BAR_TMA;
+        const uint32_t bar = smem_u32(&s_bars[stage]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(32768u) : "memory");
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int x = h * D + 64 * half;
+        for (int hf = 0; hf < 2; ++hf) {
+            const int x = h * D + 64 * hf;
             asm volatile(
                 "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
-                    "r"(cx.sbase + OFF_K + 8192 * half), "l"(reinterpret_cast<uint64_t>(&tmK)), "r"(x), "r"(y), "r"(bar)
+                    "r"(sb + stage * SUM_STAGE + 8192 * hf), "l"(reinterpret_cast<uint64_t>(&tmK)), "r"(x), "r"(y), "r"(bar)
                 : "memory");
             asm volatile(
                 "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
-                    "r"(cx.sbase + OFF_V + 8192 * half), "l"(reinterpret_cast<uint64_t>(&tmV)), "r"(x), "r"(y), "r"(bar)
+                    "r"(sb + stage * SUM_STAGE + 16384 + 8192 * hf), "l"(reinterpret_cast<uint64_t>(&tmV)), "r"(x), "r"(y),
+                "r"(bar)
                 : "memory");
         }
     };
+    auto load_gate = [&](long long f) -> float {
+        const int n = (int)(f % P.N);
+        return (t < C) ? a.gate[((size_t)b * a.T + (size_t)n * C + t) * a.heads + h] : 1.f;
+    };
 
-    // first chunk of this slot
-    if (t == 0 && f_lo + slot < f_hi) issue_tma(f_lo + slot);
-
-    for (long long f = f_lo + slot; f < f_hi; f += NSLOT) {
-        const long long m = f - f_lo;              // index of this chunk inside the block's range
-        const int seq = (int)(f / P.N), n = (int)(f % P.N);
-        const int b = seq / a.heads, h = seq % a.heads;
-        const size_t tok0 = ((size_t)b * a.T + (size_t)n * C) * a.heads + h;
-        const bool run_start = (m == 0) || (n == 0);
-        const bool seq_end = (n == P.N - 1);
-        const float *init_src = nullptr;           // where a run's start state comes from (nullptr = zero)
-        if (run_start) init_src = (n == 0) ? (a.state_in ? a.state_in + (size_t)seq * st : nullptr)
-                                           : a.ws.start + (size_t)item * st;
-
-        // ---- q for this thread's channel, all 64 tokens, packed bf16 pairs (issued early)
-        uint32_t qp[32];
-        {
-            const unsigned short *qs = reinterpret_cast<const unsigned short *>(gq) + tok0 * D + t;
-            const size_t rs = (size_t)a.heads * D;
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const uint32_t lo = qs[(size_t)(2 * i) * rs], hi = qs[(size_t)(2 * i + 1) * rs];
-                qp[i] = lo | (hi << 16);
-            }
+    if (t == 0) issue_tma(f0, 0);
+    float g_cur = load_gate(f0);
+    float decay_log2 = 0.f;
+    bool failed = false;
+    uint32_t ph_mma = 0;
+    constexpr uint32_t I_ADV = make_idesc(128, 128, 1, 1);
+    for (long long f = f0; f < f1 && !failed; ++f) {
+        const int stage = (int)((f - f0) & 1);
+        const uint32_t ph_tma = (uint32_t)(((f - f0) >> 1) & 1);
+        // prefetch the next chunk (its stage was last read by the MMAs of chunk f - 1, which have completed)
+        float g_next = 1.f;
+        if (f + 1 < f1) {
+            if (t == 0) issue_tma(f + 1, stage ^ 1);
+            g_next = load_gate(f + 1);
         }
-
-        // ---- gates (threads 0..63 own token c = t for scalar bookkeeping)
+        if (t < C) s_lg[t] = fmaxf(log2f(g_cur), -115.f);
+        __syncthreads();
         if (t < C) {
-            const float g = a.gate[tok0 + (size_t)t * a.heads];
-            sc->w[t] = fmaxf(log2f(g), -115.f);     // temporary: log2 gamma
-            sc->lam[t] = a.lam[tok0 + (size_t)t * a.heads];
+            float G2c = 0.f;
+            for (int i = 0; i <= t; ++i) G2c += s_lg[i];
+            s_G2[t] = G2c;
         }
-        wg_sync(slot);
-        float G2c = 0.f;
-        if (t < C) {
-            for (int i = 0; i <= t; ++i) G2c += sc->w[i];
-        }
-        wg_sync(slot);
-        if (t < C) {
-            sc->G2[t] = G2c;
-            const float mc = fmaxf(G2c, -60.f);
-            sc->zt[t] = exp2f(mc);
-            sc->ac[t] = G2c - mc;
-            if (t == C - 1) sc->clamped = (G2c < -60.f) ? 1 : 0;
-        }
-        wg_sync(slot);
-        if (t < C) sc->w[t] = exp2f(sc->G2[C - 1] - sc->G2[t]);
-        const float zetaC = exp2f(sc->G2[C - 1]);
-
-        // ---- K, V tiles have landed
-        slot_wait(cx, BAR_TMA);
-
-        // ---- w o K (same swizzled positions as K)
+        __syncthreads();
+        if (t < C) s_w[t] = exp2f(s_G2[C - 1] - s_G2[t]);
+        const float zetaC = exp2f(s_G2[C - 1]);
+        decay_log2 += s_G2[C - 1];
+        __syncthreads();
+        if (!mbar_wait_bounded(smem_u32(&s_bars[stage]), ph_tma)) failed = true;
+        // w o K
+        const unsigned char *kt = smem + stage * SUM_STAGE;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const int qi = t + WG * i;                 // 16-byte chunk index in the 16 KB tile
-            const int j = (qi & 511) >> 3;             // key row of this chunk
-            uint4 v = *reinterpret_cast<const uint4 *>(cx.sptr + OFF_K + qi * 16);
-            const float wj = sc->w[j];
+            const int qi = t + 128 * i;
+            const int j = (qi & 511) >> 3;
+            uint4 v = *reinterpret_cast<const uint4 *>(kt + qi * 16);
+            const float wj = s_w[j];
             uint32_t *pv = reinterpret_cast<uint32_t *>(&v);
 #pragma unroll
             for (int u = 0; u < 4; ++u) pv[u] = pack_bf16(bf16_lo(pv[u]) * wj, bf16_hi(pv[u]) * wj);
-            *reinterpret_cast<uint4 *>(cx.sptr + OFF_KW + qi * 16) = v;
+            *reinterpret_cast<uint4 *>(smem + SUM_OFF_KW + qi * 16) = v;
         }
-
-        // ---- H master: wait for the previous chunk's advance, then one pass: ||H_0||^2, bf16 copy, scale
-        if (NSLOT == 2 && m > 0) {   // chunk m - 1 (the other slot's) has finished its H work
-            if (*cx.abort_flag == 0 && !mbar_wait_bounded(tokH, (uint32_t)((m - 1) & 1))) *cx.abort_flag = 1;
-        }
-        fence_after();
-        {
-            float hh = 0.f;
-            const float *src = (run_start && init_src) ? init_src + (size_t)t * D : nullptr;
+        // decay the accumulators (not needed for the first chunk: its products overwrite)
+        if (f > f0) {
 #pragma unroll
-            for (int piece = 0; piece < 4; ++piece) {
+            for (int piece = 0; piece < 8; ++piece) {
                 uint32_t r[32];
-                if (!run_start) {
-                    TMEM_LD32(tm_H + cx.lane_addr + 32 * piece, r);
-                    tmem_wait_ld();
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        float4 v4 = src ? *reinterpret_cast<const float4 *>(src + 32 * piece + 4 * i)
-                                        : make_float4(0.f, 0.f, 0.f, 0.f);
-                        r[4 * i + 0] = __float_as_uint(v4.x); r[4 * i + 1] = __float_as_uint(v4.y);
-                        r[4 * i + 2] = __float_as_uint(v4.z); r[4 * i + 3] = __float_as_uint(v4.w);
-                    }
-                }
-                unsigned char *hrow = cx.sptr + OFF_H + (piece >> 1) * 16384 + t * 128;
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const float v0 = __uint_as_float(r[8 * ch + 2 * u]), v1 = __uint_as_float(r[8 * ch + 2 * u + 1]);
-                        hh = fmaf(v0, v0, fmaf(v1, v1, hh));
-                        pk[u] = pack_bf16(v0, v1);
-                    }
-                    const int chunk = (4 * (piece & 1) + ch) ^ (t & 7);
-                    *reinterpret_cast<uint4 *>(hrow + chunk * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                }
+                TMEM_LD32(tmem + lane_addr + 32 * piece, r);
+                tmem_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * zetaC);
-                TMEM_ST32(tm_H + cx.lane_addr + 32 * piece, r);
-            }
-            tmem_wait_st();
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) hh += __shfl_xor_sync(0xffffffffu, hh, o);
-            if ((t & 31) == 0) sc->red[cx.warp_q] = hh;
-        }
-        fence_async_smem();
-        fence_before();
-        wg_sync(slot);
-        if (t == 0) {
-            fence_after();
-            // H advance: Hm += K^T (w o K);  K H_0 (M = 64 keys, N = 128);  Gram K K^T
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) mma_ss(tm_H, mn_step(dK_mn, ks), mn_step(dKw_mn, ks), I_ADV, 1);
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-                mma_ss(cx.tm_kh, kmaj_step(dK_k, ks, 8192), kmaj_step(dH_k, ks, 16384), I_KH, ks > 0);
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-                mma_ss(cx.tm_s, kmaj_step(dK_k, ks, 8192), kmaj_step(dK_k, ks, 8192), I_GR, ks > 0);
-            mma_commit(cx.bars + 8 * BAR_A);
-        }
-        if (t == 0) sc->hh = sc->red[0] + sc->red[1] + sc->red[2] + sc->red[3];
-        slot_wait(cx, BAR_A);
-        fence_after();
-
-        // ---- chunk-wise Frobenius norms: d_j, then f_c
-        {
-            const int l = t & 31;
-            const bool valid = (l >> 4) == slot;
-            const int j = 16 * cx.warp_q + (l & 15);
-            float aj = 0.f;
-#pragma unroll
-            for (int piece = 0; piece < 4; ++piece) {
-                uint32_t r[32];
-                TMEM_LD32(cx.tm_kh + cx.lane_addr + 32 * piece, r);
-                tmem_wait_ld();
-                const unsigned char *krow = cx.sptr + OFF_K + (piece >> 1) * 8192 + j * 128;
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    const int chunk = (4 * (piece & 1) + ch) ^ (j & 7);
-                    const uint4 kv = *reinterpret_cast<const uint4 *>(krow + chunk * 16);
-                    const uint32_t *pk = reinterpret_cast<const uint32_t *>(&kv);
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        aj = fmaf(__uint_as_float(r[8 * ch + 2 * u]), bf16_lo(pk[u]), aj);
-                        aj = fmaf(__uint_as_float(r[8 * ch + 2 * u + 1]), bf16_hi(pk[u]), aj);
-                    }
-                }
-            }
-            float bjs = 0.f;
-            const float G2j = sc->G2[j];
-#pragma unroll
-            for (int piece = 0; piece < 2; ++piece) {
-                uint32_t r[32];
-                TMEM_LD32(cx.tm_s + cx.lane_addr + 32 * piece, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int ii = 32 * piece + i;
-                    const float g = __uint_as_float(r[i]);
-                    const float g2 = g * g;
-                    if (ii < j) bjs = fmaf(2.f * ex2_fast(G2j - sc->G2[ii]), g2, bjs);
-                    else if (ii == j) bjs += g2;
-                }
-            }
-            if (valid) sc->dj[j] = fmaf(2.f * exp2f(G2j) , aj, bjs);
-        }
-        fence_before();
-        wg_sync(slot);
-        // H master is final for this chunk, the Frobenius temporaries are consumed
-        if (seq_end && a.state_out) {
-            fence_after();
-            float *dst = a.state_out + (size_t)seq * st + (size_t)t * D;
-#pragma unroll
-            for (int piece = 0; piece < 4; ++piece) {
-                uint32_t r[32];
-                TMEM_LD32(tm_H + cx.lane_addr + 32 * piece, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    *reinterpret_cast<float4 *>(dst + 32 * piece + 4 * i) =
-                        make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
-                                    __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
-            }
-            fence_before();
-            wg_sync(slot);
-        }
-        if (NSLOT == 2 && t == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tokH) : "memory");
-
-        // ---- f_c, Chebyshev initialisation (threads 0..63: token c = t)
-        float omega = 2.f, rho2 = 0.f, s0c = 0.f, lamc = 0.f;
-        if (t < C) {
-            const float G2t = sc->G2[t];
-            float s = exp2f(2.f * G2t) * sc->hh;
-            for (int j = 0; j <= t; ++j) s = fmaf(ex2_fast(2.f * (G2t - sc->G2[j])), sc->dj[j], s);
-            const float fc = sqrtf(fmaxf(s, 0.f));
-            lamc = sc->lam[t];
-            if (adaptive) lamc *= fc;
-            const float Lpm = fc + 2.f * lamc;
-            const float rho = fc / Lpm;
-            rho2 = rho * rho;
-            s0c = 2.f / Lpm;
-            sc->s0[t] = s0c;
-            if (a.fro_out) a.fro_out[tok0 + (size_t)t * a.heads] = fc;
-        }
-        wg_sync(slot);
-
-        // ---- x_0 = 2 q / (L + mu), X' operand
-        float xm[C], xp[C];
-        {
-            unsigned char *xrow = cx.sptr + OFF_X + t * 128;
-#pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {
-                uint32_t pk[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c0 = 8 * ch + 2 * u;
-                    const float x0 = sc->s0[c0] * bf16_lo(qp[c0 >> 1]);
-                    const float x1 = sc->s0[c0 + 1] * bf16_hi(qp[c0 >> 1]);
-                    xm[c0] = x0; xm[c0 + 1] = x1;
-                    xp[c0] = 0.f; xp[c0 + 1] = 0.f;
-                    pk[u] = pack_bf16(x0 * sc->zt[c0], x1 * sc->zt[c0 + 1]);
-                }
-                *reinterpret_cast<uint4 *>(xrow + ((ch ^ (t & 7)) * 16)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            }
-        }
-        fence_async_smem();
-        fence_before();
-        wg_sync(slot);
-
-        // ---- Algorithm 1: n_iter iterations on the whole chunk (+ one extra score pass for the output)
-        for (int it = 0; it <= a.n_iter; ++it) {
-            const bool last = (it == a.n_iter);
-            if (t == 0) {
-                fence_after();
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    mma_ss(cx.tm_s, kmaj_step(dK_k, ks, 8192), mn_step(dX_mn, ks), I_S, ks > 0);
-                mma_commit(cx.bars + 8 * BAR_A);
-                if (!last) {
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        mma_ss(cx.tm_y, kmaj_step(dH_k, ks, 16384), mn_step(dX_mn, ks), I_Y1, ks > 0);
-                }
-            }
-            if (!last && t < C) {   // weight schedule and per-token coefficients of this iteration
-                omega = 4.f / (4.f - rho2 * omega);
-                const float sigma = s0c * omega, beta = omega - 1.f;
-                sc->coef[it & 1][t] = make_float4(sigma, beta, 1.f + beta - sigma * lamc, sc->zt[t]);
-            }
-            slot_wait(cx, BAR_A);
-            fence_after();
-            p_epilogue(cx);
-            fence_async_smem();
-            fence_before();
-            wg_sync(slot);
-            if (last) break;
-            if (t == 0) {
-                fence_after();
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) mma_ss(cx.tm_y, mn_step(dK_mn, ks), mn_step(dP_mn, ks), I_Y2, 1);
-                mma_commit(cx.bars + 8 * BAR_B);
-            }
-            slot_wait(cx, BAR_B);
-            fence_after();
-            {
-                const float4 *coef = sc->coef[it & 1];
-                unsigned char *xrow = cx.sptr + OFF_X + t * 128;
-#pragma unroll
-                for (int piece = 0; piece < 4; ++piece) {
-                    uint32_t r[16];
-                    TMEM_LD16(cx.tm_y + cx.lane_addr + 16 * piece, r);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int ch = 0; ch < 2; ++ch) {
-                        uint32_t pk[4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            float xo[2];
-#pragma unroll
-                            for (int e = 0; e < 2; ++e) {
-                                const int c = 16 * piece + 8 * ch + 2 * u + e;
-                                const float4 cf = coef[c];
-                                const float qv = e == 0 ? bf16_lo(qp[c >> 1]) : bf16_hi(qp[c >> 1]);
-                                const float acc = __uint_as_float(r[8 * ch + 2 * u + e]);
-                                const float xn = fmaf(cf.x, qv - acc, fmaf(cf.z, xm[c], -cf.y * xp[c]));
-                                xp[c] = xm[c];
-                                xm[c] = xn;
-                                xo[e] = xn * cf.w;
-                            }
-                            pk[u] = pack_bf16(xo[0], xo[1]);
-                        }
-                        const int chunk = (2 * piece + ch) ^ (t & 7);
-                        *reinterpret_cast<uint4 *>(xrow + chunk * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    }
-                }
-            }
-            fence_async_smem();
-            fence_before();
-            wg_sync(slot);
-        }
-
-        // ---- output: U master pass (bf16 copy into the H buffer, scale), O^T = U_0 X'^T + V^T P^T, U advance
-        if (NSLOT == 2 && m > 0) {   // chunk m - 1 has written its output and advanced U
-            if (*cx.abort_flag == 0 && !mbar_wait_bounded(tokU, (uint32_t)((m - 1) & 1))) *cx.abort_flag = 1;
-        }
-        fence_after();
-        {
-            const float *src = (run_start && init_src) ? init_src + (size_t)D * D + (size_t)t * D : nullptr;
-#pragma unroll
-            for (int piece = 0; piece < 4; ++piece) {
-                uint32_t r[32];
-                if (!run_start) {
-                    TMEM_LD32(tm_U + cx.lane_addr + 32 * piece, r);
-                    tmem_wait_ld();
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        float4 v4 = src ? *reinterpret_cast<const float4 *>(src + 32 * piece + 4 * i)
-                                        : make_float4(0.f, 0.f, 0.f, 0.f);
-                        r[4 * i + 0] = __float_as_uint(v4.x); r[4 * i + 1] = __float_as_uint(v4.y);
-                        r[4 * i + 2] = __float_as_uint(v4.z); r[4 * i + 3] = __float_as_uint(v4.w);
-                    }
-                }
-                unsigned char *hrow = cx.sptr + OFF_H + (piece >> 1) * 16384 + t * 128;
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        pk[u] = pack_bf16(__uint_as_float(r[8 * ch + 2 * u]), __uint_as_float(r[8 * ch + 2 * u + 1]));
-                    const int chunk = (4 * (piece & 1) + ch) ^ (t & 7);
-                    *reinterpret_cast<uint4 *>(hrow + chunk * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                }
-#pragma unroll
-                for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * zetaC);
-                TMEM_ST32(tm_U + cx.lane_addr + 32 * piece, r);
+                TMEM_ST32(tmem + lane_addr + 32 * piece, r);
             }
             tmem_wait_st();
         }
         fence_async_smem();
         fence_before();
-        wg_sync(slot);
+        __syncthreads();
         if (t == 0) {
             fence_after();
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-                mma_ss(cx.tm_y, kmaj_step(dH_k, ks, 16384), mn_step(dX_mn, ks), I_Y1, ks > 0);
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) mma_ss(cx.tm_y, mn_step(dV_mn, ks), mn_step(dP_mn, ks), I_Y2, 1);
-            mma_commit(cx.bars + 8 * BAR_A);
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) mma_ss(tm_U, mn_step(dV_mn, ks), mn_step(dKw_mn, ks), I_ADV, 1);
-            mma_commit(cx.bars + 8 * BAR_B);
-        }
-        slot_wait(cx, BAR_A);
-        fence_after();
-        {
-            unsigned short *orow = reinterpret_cast<unsigned short *>(gout) + tok0 * D + t;
-            const size_t rs = (size_t)a.heads * D;
-#pragma unroll
-            for (int piece = 0; piece < 4; ++piece) {
-                uint32_t r[16];
-                TMEM_LD16(cx.tm_y + cx.lane_addr + 16 * piece, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const __nv_bfloat16 ob = __float2bfloat16_rn(__uint_as_float(r[i]));
-                    orow[(size_t)(16 * piece + i) * rs] = *reinterpret_cast<const unsigned short *>(&ob);
-                }
+            const uint32_t k_mn = desc_lo(sb + stage * SUM_STAGE, 8192), v_mn = desc_lo(sb + stage * SUM_STAGE + 16384, 8192);
+            const uint32_t kw_mn = desc_lo(sb + SUM_OFF_KW, 8192);
+            if (f == f0) {
+                mma_ss<0>(tm_H, k_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
+                mma_ss<0>(tm_U, v_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
+            } else {
+                mma_ss<1>(tm_H, k_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
+                mma_ss<1>(tm_U, v_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
             }
-        }
-        slot_wait(cx, BAR_B);     // U advance done: every tensor-core read of this chunk's tiles is done
-        fence_after();
-        if (seq_end && a.state_out) {
-            float *dst = a.state_out + (size_t)seq * st + (size_t)D * D + (size_t)t * D;
 #pragma unroll
-            for (int piece = 0; piece < 4; ++piece) {
-                uint32_t r[32];
-                TMEM_LD32(tm_U + cx.lane_addr + 32 * piece, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    *reinterpret_cast<float4 *>(dst + 32 * piece + 4 * i) =
-                        make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
-                                    __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+            for (int ks = 1; ks < 4; ++ks) {
+                mma_ss<1>(tm_H, k_mn, mnstep(ks), kw_mn, mnstep(ks), I_ADV);
+                mma_ss<1>(tm_U, v_mn, mnstep(ks), kw_mn, mnstep(ks), I_ADV);
             }
+            mma_commit(bar_mma);
         }
-        fence_before();
-        wg_sync(slot);
-        if (t == 0) {
-            if (NSLOT == 2) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tokU) : "memory");
-            if (f + NSLOT < f_hi && *cx.abort_flag == 0) issue_tma(f + NSLOT);
-        }
-        if (*cx.abort_flag != 0) break;
+        if (!mbar_wait_bounded(bar_mma, ph_mma)) failed = true;
+        ph_mma ^= 1u;
+        fence_after();
+        g_cur = g_next;
     }
-
+    if (failed) {
+        if (t == 0 && a.device_status) atomicExch(a.device_status, (int)GKA_ERR_TIMEOUT);
+    } else {
+        const size_t st = state_floats(D, D);
+        float *dst = a.ws.delta + (size_t)item * st + (size_t)t * D;     // row t of dH, then row t of dU
+#pragma unroll
+        for (int piece = 0; piece < 8; ++piece) {
+            uint32_t r[32];
+            TMEM_LD32(tmem + lane_addr + 32 * piece, r);
+            tmem_wait_ld();
+            float *p = dst + (piece >> 2) * (size_t)D * D + 32 * (piece & 3);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                *reinterpret_cast<float4 *>(p + 4 * i) = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
+                                                                     __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+        }
+        if (t == 0) a.ws.decay[item] = exp2f(decay_log2);
+    }
     fence_before();
     __syncthreads();
-    if (tid < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(cx.tmem) : "memory");
+    if (t < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -729,8 +1062,6 @@ bool make_tile_map(CUtensorMap *map, const void *base, int rows, int cols) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr int kSlots = 1;
-
 }  // namespace
 
 bool fwd_tc_available() { return get_encode_fn() != nullptr; }
@@ -740,15 +1071,31 @@ cudaError_t launch_fwd_tc(const FwdArgs &a, cudaStream_t stream) {
     const int rows = a.B * a.T, cols = a.heads * D;
     if (!make_tile_map(&tmK, a.k, rows, cols) || !make_tile_map(&tmV, a.v, rows, cols))
         return cudaErrorInvalidValue;
-    cudaError_t err = launch_fwd_summary_scan_bf16_d128(a, stream);
-    if (err != cudaSuccess) return err;
-    const size_t smem = (size_t)kSlots * SLOT_BYTES + 1024;
-    err = cudaFuncSetAttribute(fwd_tc_kernel<kSlots>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t err = cudaSuccess;
+    bool any_cut = false;
+    for (int i = 0; i + 1 < a.plan.G; ++i) any_cut |= a.plan.cut_out(i);
+    if (any_cut) {
+        err = cudaFuncSetAttribute(fwd_tc_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM);
+        if (err != cudaSuccess) return err;
+        fwd_tc_summary_kernel<<<a.plan.G, 128, SUM_SMEM, stream>>>(tmK, tmV, a);
+        err = launch_fwd_scan(a, (int)state_floats(D, D), stream);
+        if (err != cudaSuccess) return err;
+    }
+    const size_t smem = (size_t)NSLOT * SLOT_BYTES + 1024;
+    err = cudaFuncSetAttribute(fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     if (a.ev_start) cudaEventRecord(a.ev_start, stream);
-    fwd_tc_kernel<kSlots><<<a.plan.G, WG * kSlots, smem, stream>>>(tmK, tmV, a);
+    fwd_tc_kernel<<<a.plan.G, kThreadsTc, smem, stream>>>(tmK, tmV, a);
     if (a.ev_stop) cudaEventRecord(a.ev_stop, stream);
     return cudaGetLastError();
 }
+
+#ifdef GKA_TC_TIMING
+extern "C" int gka_debug_tc_trace(long long *out /* 4 x 8192 */, int *counts /* 4 */) {
+    if (cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * 4 * 8192) != cudaSuccess) return 1;
+    if (cudaMemcpyFromSymbol(counts, g_trace_n, sizeof(int) * 4) != cudaSuccess) return 1;
+    return 0;
+}
+#endif
 
 }  // namespace gka

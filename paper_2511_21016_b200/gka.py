@@ -22,7 +22,7 @@ GKA_FLAG_ADAPTIVE_LAMBDA = 1
 GKA_ERR_TIMEOUT = 8
 
 EXPORTS = ("gka_fwd_workspace_bytes", "gka_fwd_chunked", "gka_decode_step", "gka_status_string",
-           "gka_fwd_num_work_items", "gka_fwd_work_range")
+           "gka_fwd_num_work_items", "gka_fwd_work_range", "gka_last_error_detail")
 
 
 class GkaDesc(ctypes.Structure):
@@ -40,7 +40,10 @@ class GkaDesc(ctypes.Structure):
 class GkaError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: {status_string(status)}")
+        detail = ""
+        if status == 7:
+            detail = " [" + load_library().gka_last_error_detail().decode() + "]"
+        super().__init__(f"{where}: {status_string(status)}{detail}")
 
 
 _lib = None
@@ -68,6 +71,8 @@ def load_library():
         llp, ip = ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int)
         lib.gka_fwd_work_range.argtypes = [dp, ci, ci, ci, llp, llp, ip, ip]
         lib.gka_fwd_work_range.restype = ci
+        lib.gka_last_error_detail.argtypes = []
+        lib.gka_last_error_detail.restype = ctypes.c_char_p
         lib.gka_status_string.argtypes = [ci]
         lib.gka_status_string.restype = ctypes.c_char_p
         _lib = lib
