@@ -136,6 +136,27 @@ gka_status gka_fwd_work_range(const gka_desc *desc, int chunk, int num_items, in
                               long long *first_chunk, long long *end_chunk, int *cut_in,
                               int *cut_out);
 
+/*
+ * Chunked forward without a caller workspace (the paper has no counterpart: this is a packaging
+ * variant of gka_fwd_chunked for callers that cannot allocate).  Same arguments, same results and
+ * same kernels as gka_fwd_chunked, but desc->workspace / workspace_bytes are ignored: the scratch of
+ * the cross-chunk state scan is a fixed array of GKA_NOALLOC_SCRATCH_BYTES inside the library image
+ * (resident in every CUDA context that loads the library until the context ends).
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - Problems whose scan needs more than the array (gka_fwd_workspace_bytes(desc, chunk) >
+ *     gka_noalloc_scratch_bytes()) are rejected with GKA_ERR_WORKSPACE before anything is launched:
+ *     d_k = 64 fits up to 170 chunks in total (B * heads * T / chunk), d_k = 128 up to 42 chunks.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) with
+ *     that device current; make that first call before any stream capture.
+ *   - All calls on one device share the array.  Calls that overlap on the GPU race, whatever their
+ *     streams; serialise them.  No part of the array has to be cleared between calls.
+ */
+#define GKA_NOALLOC_SCRATCH_BYTES (16u << 20)
+gka_status gka_fwd_chunked_noalloc(const gka_desc *desc, const void *q, const void *k, const void *v,
+                                   const float *gate, const float *lam, int n_iter, int chunk,
+                                   void *out, float *state_out);
+size_t gka_noalloc_scratch_bytes(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,8 @@ GKA_FLAG_ADAPTIVE_LAMBDA = 1
 GKA_ERR_TIMEOUT = 8
 
 EXPORTS = ("gka_fwd_workspace_bytes", "gka_fwd_chunked", "gka_decode_step", "gka_status_string",
-           "gka_fwd_num_work_items", "gka_fwd_work_range", "gka_last_error_detail")
+           "gka_fwd_num_work_items", "gka_fwd_work_range", "gka_last_error_detail",
+           "gka_fwd_chunked_noalloc", "gka_noalloc_scratch_bytes")
 
 
 class GkaDesc(ctypes.Structure):
@@ -66,6 +67,10 @@ def load_library():
         lib.gka_fwd_num_work_items.restype = ci
         lib.gka_fwd_chunked.argtypes = [dp, vp, vp, vp, vp, vp, ci, ci, vp, vp]
         lib.gka_fwd_chunked.restype = ci
+        lib.gka_fwd_chunked_noalloc.argtypes = [dp, vp, vp, vp, vp, vp, ci, ci, vp, vp]
+        lib.gka_fwd_chunked_noalloc.restype = ci
+        lib.gka_noalloc_scratch_bytes.argtypes = []
+        lib.gka_noalloc_scratch_bytes.restype = ctypes.c_size_t
         lib.gka_decode_step.argtypes = [dp, vp, vp, vp, vp, vp, vp, ci, vp]
         lib.gka_decode_step.restype = ci
         llp, ip = ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int)
@@ -175,6 +180,29 @@ def gka_fwd_chunked(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=No
                                         out.data_ptr(), _ptr(state_out))
     if rc != GKA_OK:
         raise GkaError(rc, "gka_fwd_chunked")
+    return out, state_out
+
+
+def gka_fwd_chunked_noalloc(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=None, *,
+                            state_in=None, precision=GKA_PREC_NATIVE, flags=0, stream=None):
+    """Chunk-wise forward for callers that cannot provide scratch memory: the library's built-in
+    scratch array is used instead of a workspace.  ``out`` and ``state_out`` must be given by such
+    callers; they are only created here (with torch) when omitted, for convenience in tests."""
+    _check_cuda(q, k, v, gate, lam, out, state_out, state_in)
+    B, T, heads, d = q.shape
+    if out is None:
+        out = torch.empty_like(v)
+    if state_out is None:
+        state_out = torch.empty(B, heads, 2 * d * d, dtype=torch.float32, device=q.device)
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    desc = make_desc(B, T, heads, d, v.shape[-1], _io_code(q), precision, flags, stream, None, state_in)
+    rc = load_library().gka_fwd_chunked_noalloc(ctypes.byref(desc), q.data_ptr(), k.data_ptr(),
+                                                v.data_ptr(), gate.data_ptr(), lam.data_ptr(),
+                                                int(n_iter), int(chunk), out.data_ptr(),
+                                                _ptr(state_out))
+    if rc != GKA_OK:
+        raise GkaError(rc, "gka_fwd_chunked_noalloc")
     return out, state_out
 
 
