@@ -109,6 +109,20 @@ gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, co
                            const void *v, const float *gate, const float *lam, int n_iter,
                            void *out);
 
+/*
+ * Host-buffer form of the chunked forward (same operation, eq. (CH) chunk-wise): q, k, v, gate, lam,
+ * out and state_out (nullable) are HOST pointers, preferably page-locked so that the copies are truly
+ * asynchronous.  `staging` is caller-owned DEVICE memory of at least gka_fwd_host_staging_bytes()
+ * bytes, 256-byte aligned; desc->workspace is required as for gka_fwd_chunked, desc->state_in (if
+ * any) stays a device pointer.  The call enqueues on desc->stream: host-to-device copies of the five
+ * inputs, the forward kernels, device-to-host copies of out (and state_out); it does not synchronise.
+ * The host buffers must stay valid and unmodified until the stream has passed the call.
+ */
+size_t gka_fwd_host_staging_bytes(const gka_desc *desc);
+gka_status gka_fwd_chunked_host(const gka_desc *desc, void *staging, const void *q, const void *k,
+                                const void *v, const float *gate, const float *lam, int n_iter,
+                                int chunk, void *out, float *state_out);
+
 /* Static, human-readable name of a status code. */
 const char *gka_status_string(int status);
 

@@ -179,4 +179,48 @@ gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, co
 
 const char *gka_last_error_detail(void) { return g_detail; }
 
+static size_t align256(size_t n) { return (n + 255) / 256 * 256; }
+
+size_t gka_fwd_host_staging_bytes(const gka_desc *desc) {
+    if (check_desc_common(desc) != GKA_OK || desc->T <= 0) return 0;
+    const size_t es = desc->io_dtype == GKA_BF16 ? 2 : 4;
+    const size_t tok = (size_t)desc->B * desc->T * desc->heads;
+    const size_t st = (size_t)desc->B * desc->heads * state_floats(desc->d_k, desc->d_v) * sizeof(float);
+    return 2 * align256(tok * desc->d_k * es) + 2 * align256(tok * desc->d_v * es) + 2 * align256(tok * 4) +
+           align256(st);
+}
+
+gka_status gka_fwd_chunked_host(const gka_desc *desc, void *staging, const void *q, const void *k,
+                                const void *v, const float *gate, const float *lam, int n_iter,
+                                int chunk, void *out, float *state_out) {
+    gka_status s = check_fwd_shape(desc, chunk);
+    if (s != GKA_OK) return s;
+    if (!staging || !q || !k || !v || !gate || !lam || !out) return GKA_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(staging) & 255u) != 0) return GKA_ERR_ALIGN;
+    const size_t es = desc->io_dtype == GKA_BF16 ? 2 : 4;
+    const size_t tok = (size_t)desc->B * desc->T * desc->heads;
+    const size_t nqk = tok * desc->d_k * es, nv = tok * desc->d_v * es, ng = tok * 4;
+    const size_t nst = (size_t)desc->B * desc->heads * state_floats(desc->d_k, desc->d_v) * sizeof(float);
+    unsigned char *p = reinterpret_cast<unsigned char *>(staging);
+    void *dq = p; p += align256(nqk);
+    void *dk = p; p += align256(nqk);
+    void *dv = p; p += align256(nv);
+    void *dout = p; p += align256(nv);
+    float *dgate = reinterpret_cast<float *>(p); p += align256(ng);
+    float *dlam = reinterpret_cast<float *>(p); p += align256(ng);
+    float *dstate = reinterpret_cast<float *>(p);
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(desc->stream);
+    cudaError_t err = cudaMemcpyAsync(dq, q, nqk, cudaMemcpyHostToDevice, stream);
+    if (err == cudaSuccess) err = cudaMemcpyAsync(dk, k, nqk, cudaMemcpyHostToDevice, stream);
+    if (err == cudaSuccess) err = cudaMemcpyAsync(dv, v, nv, cudaMemcpyHostToDevice, stream);
+    if (err == cudaSuccess) err = cudaMemcpyAsync(dgate, gate, ng, cudaMemcpyHostToDevice, stream);
+    if (err == cudaSuccess) err = cudaMemcpyAsync(dlam, lam, ng, cudaMemcpyHostToDevice, stream);
+    if (err != cudaSuccess) return cuda_result(err, "gka_fwd_chunked_host (host-to-device copies)");
+    s = gka_fwd_chunked(desc, dq, dk, dv, dgate, dlam, n_iter, chunk, dout, state_out ? dstate : nullptr);
+    if (s != GKA_OK) return s;
+    err = cudaMemcpyAsync(out, dout, nv, cudaMemcpyDeviceToHost, stream);
+    if (err == cudaSuccess && state_out) err = cudaMemcpyAsync(state_out, dstate, nst, cudaMemcpyDeviceToHost, stream);
+    return cuda_result(err, "gka_fwd_chunked_host (device-to-host copies)");
+}
+
 }  // extern "C"

@@ -217,12 +217,21 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_summary(FwdArgs a) {
 __global__ void fwd_scan(FwdArgs a, int st) {
     const WorkPlan &P = a.plan;
     const int i = blockIdx.y + 1;
-    if (!P.cut_in(i)) return;
+    __shared__ int s_j0, s_seq;           // the chain is found once per block (64-bit divisions are slow)
+    if (threadIdx.x == 0) {
+        int j0 = -1;
+        if (P.cut_in(i)) {
+            j0 = i - 1;                   // first item of the chain: the one that holds the sequence start
+            while (P.cut_in(j0)) --j0;
+        }
+        s_j0 = j0;
+        s_seq = (int)(P.lo(i) / P.N);
+    }
+    __syncthreads();
+    const int j0 = s_j0, seq = s_seq;
+    if (j0 < 0) return;
     const int e = 4 * (blockIdx.x * blockDim.x + threadIdx.x);
     if (e >= st) return;
-    int j0 = i - 1;                       // first item of the chain: the one that holds the sequence start
-    while (P.cut_in(j0)) --j0;
-    const int seq = (int)(P.lo(i) / P.N);
     float4 carry = a.state_in ? ld4(a.state_in + (size_t)seq * st + e) : make_float4(0.f, 0.f, 0.f, 0.f);
     for (int j = j0; j < i; ++j) {
         const float dcy = a.ws.decay[j];

@@ -23,7 +23,8 @@ GKA_ERR_TIMEOUT = 8
 
 EXPORTS = ("gka_fwd_workspace_bytes", "gka_fwd_chunked", "gka_decode_step", "gka_status_string",
            "gka_fwd_num_work_items", "gka_fwd_work_range", "gka_last_error_detail",
-           "gka_fwd_chunked_noalloc", "gka_noalloc_scratch_bytes")
+           "gka_fwd_chunked_noalloc", "gka_noalloc_scratch_bytes",
+           "gka_fwd_chunked_host", "gka_fwd_host_staging_bytes")
 
 
 class GkaDesc(ctypes.Structure):
@@ -71,6 +72,10 @@ def load_library():
         lib.gka_fwd_chunked_noalloc.restype = ci
         lib.gka_noalloc_scratch_bytes.argtypes = []
         lib.gka_noalloc_scratch_bytes.restype = ctypes.c_size_t
+        lib.gka_fwd_host_staging_bytes.argtypes = [dp]
+        lib.gka_fwd_host_staging_bytes.restype = ctypes.c_size_t
+        lib.gka_fwd_chunked_host.argtypes = [dp, vp, vp, vp, vp, vp, vp, ci, ci, vp, vp]
+        lib.gka_fwd_chunked_host.restype = ci
         lib.gka_decode_step.argtypes = [dp, vp, vp, vp, vp, vp, vp, ci, vp]
         lib.gka_decode_step.restype = ci
         llp, ip = ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int)
@@ -180,6 +185,32 @@ def gka_fwd_chunked(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=No
                                         out.data_ptr(), _ptr(state_out))
     if rc != GKA_OK:
         raise GkaError(rc, "gka_fwd_chunked")
+    return out, state_out
+
+
+def gka_fwd_host_staging_bytes(B, T, heads, d, io_dtype) -> int:
+    desc = make_desc(B, T, heads, d, d, io_dtype)
+    return int(load_library().gka_fwd_host_staging_bytes(ctypes.byref(desc)))
+
+
+def gka_fwd_chunked_host(q, k, v, gate, lam, n_iter, chunk, out, state_out, *, staging, workspace,
+                         precision=GKA_PREC_NATIVE, flags=0, stream=None, device_status=None):
+    """Host-buffer forward: q, k, v, gate, lam, out, state_out are (pinned) CPU tensors; staging and
+    workspace are CUDA byte tensors.  Copies and kernels are enqueued on the stream; no synchronisation."""
+    for t in (q, k, v, gate, lam, out, state_out):
+        if t is not None and (t.is_cuda or not t.is_contiguous()):
+            raise ValueError("host-buffer call takes contiguous CPU tensors")
+    _check_cuda(staging, workspace, device_status)
+    B, T, heads, d = q.shape
+    if stream is None:
+        stream = torch.cuda.current_stream(staging.device).cuda_stream
+    desc = make_desc(B, T, heads, d, v.shape[-1], _io_code(q), precision, flags, stream, workspace,
+                     device_status=device_status)
+    rc = load_library().gka_fwd_chunked_host(ctypes.byref(desc), staging.data_ptr(), q.data_ptr(),
+                                             k.data_ptr(), v.data_ptr(), gate.data_ptr(), lam.data_ptr(),
+                                             int(n_iter), int(chunk), out.data_ptr(), _ptr(state_out))
+    if rc != GKA_OK:
+        raise GkaError(rc, "gka_fwd_chunked_host")
     return out, state_out
 
 
