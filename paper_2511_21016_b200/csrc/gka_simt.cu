@@ -221,8 +221,11 @@ __global__ void fwd_scan(FwdArgs a, int st) {
     if (threadIdx.x == 0) {
         int j0 = -1;
         if (P.cut_in(i)) {
-            j0 = i - 1;                   // first item of the chain: the one that holds the sequence start
-            while (P.cut_in(j0)) --j0;
+            // first item of the chain: the one whose range holds the start of this sequence (its last run
+            // begins there, whatever sequence the item itself started in)
+            const long long seq_start = (P.lo(i) / P.N) * P.N;
+            j0 = i - 1;
+            while (P.lo(j0) > seq_start) --j0;
         }
         s_j0 = j0;
         s_seq = (int)(P.lo(i) / P.N);

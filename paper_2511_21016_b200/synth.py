@@ -66,12 +66,14 @@ def shrink(cfg: GkaConfig, **kw) -> GkaConfig:
 
 
 def round_bf16(x: np.ndarray) -> np.ndarray:
-    """Round float32 values to the nearest bf16 (ties to even); result stays float32."""
-    a = np.ascontiguousarray(x, dtype=np.float32)
-    u = a.view(np.uint32).astype(np.uint64)
-    lsb = (u >> 16) & 1
-    u = (u + 0x7FFF + lsb) & 0xFFFF0000
-    return u.astype(np.uint32).view(np.float32).reshape(a.shape)
+    """Round float32 values to the nearest bf16 (ties to even); result stays float32.  Finite inputs."""
+    a = np.array(x, dtype=np.float32, order="C", copy=True)
+    u = a.view(np.uint32)
+    lsb = (u >> np.uint32(16)) & np.uint32(1)
+    u += np.uint32(0x7FFF)
+    u += lsb
+    u &= np.uint32(0xFFFF0000)
+    return a
 
 
 def to_bf16_bits(x: np.ndarray) -> np.ndarray:

@@ -86,6 +86,16 @@ def test_fwd_f32_items_cut_sequences():
     check_fwd(cfg)
 
 
+@pytest.mark.parametrize("io,d", [("f32", 64), ("f32", 128), ("bf16", 128)])
+def test_fwd_slow_fading_state_crosses_many_items(io, d):
+    """Gates close to 1 (sigmoid(N(6,1))): the state of a sequence start is still alive many work items
+    later, so a wrong start state of any item shows (fast-fading gates would hide it).  Several sequences
+    whose boundaries fall inside items."""
+    cfg = synth.GkaConfig("slow", B=2, heads=3, T=64 * 70, d=d, chunk=64, n_iter=2, io_dtype=io, seed=21,
+                          gate_mean=6.0)
+    check_fwd(cfg)
+
+
 def test_fwd_f32_long_runs_d128():
     cfg = synth.shrink(SMALL, B=1, heads=2, d=128, T=64 * 160, n_iter=3)
     check_fwd(cfg)
