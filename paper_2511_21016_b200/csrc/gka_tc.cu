@@ -275,17 +275,20 @@ struct SlotCtx {
     uint32_t tm_H, tm_U;          // masters
     uint32_t lane_addr;           // (32 * warp_q) << 16
     uint32_t ph[BAR_COUNT];       // phase parity of each mbarrier
-    volatile int *abort_flag;
-    int *device_status;
+    uint32_t abort_addr;          // shared address of the block's abort flag
 };
 
+__device__ __forceinline__ bool slot_aborted(const SlotCtx &cx) {
+    int v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(cx.abort_addr) : "memory");
+    return v != 0;
+}
 // Wait for an mbarrier phase: one warp of the slot polls (bounded), the others sleep in the slot's
 // named barrier, so waiting warps do not take issue slots from the other slot's working warps.
 __device__ __forceinline__ void slot_wait_addr(SlotCtx &cx, uint32_t bar, uint32_t parity) {
-    if ((cx.t >> 5) == cx.slot && *cx.abort_flag == 0) {   // the polling warp of slot s sits on scheduler s
-        if (!mbar_wait_bounded(bar, parity)) {
-            *cx.abort_flag = 1;
-            if (cx.device_status) atomicExch(cx.device_status, (int)GKA_ERR_TIMEOUT);
+    if ((cx.t >> 5) == cx.slot && !slot_aborted(cx)) {   // the polling warp of slot s sits on scheduler s
+        if (!mbar_wait_bounded(bar, parity)) {             // the block reports GKA_ERR_TIMEOUT when it ends
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(cx.abort_addr), "r"(1) : "memory");
         }
     }
     slot_sync(cx.slot);
@@ -530,6 +533,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     const WorkPlan &P = a.plan;
     const int item = blockIdx.x;
     const long long f_lo = P.lo(item), f_hi = P.lo(item + 1);
+    const int n_mine = (int)(f_hi - f_lo);          // chunks of this block
 
     if (tid >= NSLOT * ST) {
         // ================================ MMA issuer warpgroup ================================
@@ -582,8 +586,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         cx.lane_addr = (uint32_t)(32 * cx.warp_q) << 16;
 #pragma unroll
         for (int i = 0; i < BAR_COUNT; ++i) cx.ph[i] = 0;
-        cx.abort_flag = &s_abort;
-        cx.device_status = a.device_status;
+        cx.abort_addr = smem_u32(&s_abort);
         cx.tm_y = tmem + (cx.slot == 0 ? TM_Y0 : TM_Y1);
         cx.tm_q = tmem + TM_Q + 32 * cx.slot;
         cx.tm_s = tmem + TM_S + ((uint32_t)(16 * cx.slot) << 16);
@@ -621,8 +624,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         if (t == 0 && f_lo + slot < f_hi) issue_tma(f_lo + slot);
         slot_sync(slot);
 
-        for (long long f = f_lo + slot; f < f_hi; f += NSLOT) {
-            const long long m = f - f_lo;              // index of this chunk inside the block's range
+        for (int m = slot; m < n_mine; m += NSLOT) {       // m: index of this chunk inside the block's range
+            const long long f = f_lo + m;
             const int seq = (int)(f / P.N), n = (int)(f % P.N);
             const int b = seq / a.heads, h = seq % a.heads;
             const size_t tok0 = ((size_t)b * a.T + (size_t)n * C) * a.heads + h;
@@ -844,10 +847,10 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             slot_sync(slot);
             if (t == 0) {
                 mbar_arrive(tokU);
-                if (f + NSLOT < f_hi && *cx.abort_flag == 0) issue_tma(f + NSLOT);
+                if (f + NSLOT < f_hi && !slot_aborted(cx)) issue_tma(f + NSLOT);
             }
             TSTAMP(14);
-            if (*cx.abort_flag != 0) break;
+            if (slot_aborted(cx)) break;
         }
         if (f_lo + slot < f_hi) slot_post(cx, OP_EXIT);
     }
@@ -862,6 +865,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #endif
     fence_before();
     __syncthreads();
+    if (tid == 0 && s_abort != 0 && a.device_status) atomicExch(a.device_status, (int)GKA_ERR_TIMEOUT);
     if (tid < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
 }
 
