@@ -872,12 +872,15 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 // ---------------------------------------------------------------------------------------------
 // Segment summaries on the tensor cores: for every work item whose range ends inside a sequence, the decay
 // product and (delta-H, delta-U) of its last run, i.e. the run's final state for a zero start state:
-//     dH <- zeta_C dH + K^T (w o K),   dU <- zeta_C dU + V^T (w o K)      chunk by chunk,
-// with the accumulators in TMEM.  One block of 128 threads per item; K and V tiles are double-buffered.
+//     dH = sum_j w_j k_j k_j^T,   dU = sum_j w_j v_j k_j^T,   w_j = prod of the gates after token j in the run.
+// The weights are formed in log2 space from the run's total log-decay (one pre-pass over the gates) and a
+// running prefix, so every chunk is a pure accumulation K^T (w o K), V^T (w o K) into TMEM: no rescaling pass
+// and no wait between chunks.  One block of 128 threads per item; K/V tiles in 4 stages, w o K in 2.
 // ---------------------------------------------------------------------------------------------
-constexpr uint32_t SUM_STAGE = 32768;            // K tile + V tile
-constexpr uint32_t SUM_OFF_KW = 2 * SUM_STAGE;   // w o K
-constexpr uint32_t SUM_SMEM = SUM_OFF_KW + 16384 + 1024;
+constexpr int SUM_NS = 4;
+constexpr uint32_t SUM_STAGE = 32768;                   // K tile + V tile
+constexpr uint32_t SUM_OFF_KW = SUM_NS * SUM_STAGE;     // 2 x (w o K)
+constexpr uint32_t SUM_SMEM = SUM_OFF_KW + 2 * 16384 + 1024;
 
 __global__ void __launch_bounds__(128, 1)
 fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, FwdArgs a) {
@@ -885,16 +888,16 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
     const int item = blockIdx.x;
     if (!P.cut_out(item)) return;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    __shared__ __align__(8) uint64_t s_bars[3];      // TMA stage 0, TMA stage 1, MMA
+    __shared__ __align__(8) uint64_t s_bars[SUM_NS + 2];      // TMA stages, MMA parity 0 / 1
     __shared__ uint32_t s_tmem_base;
-    __shared__ float s_lg[C], s_w[C], s_G2[C];
+    __shared__ float s_w[C], s_red[4];
     unsigned char *smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     const uint32_t sb = smem_u32(smem);
-    const int t = threadIdx.x, warp_q = t >> 5;
+    const int t = threadIdx.x, warp_q = t >> 5, l = t & 31;
     const uint32_t lane_addr = (uint32_t)(32 * warp_q) << 16;
 
     if (t == 0) {
-        for (int i = 0; i < 3; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_bars[i])));
+        for (int i = 0; i < SUM_NS + 2; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_bars[i])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (t < 32) {
@@ -906,13 +909,15 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
     __syncthreads();
     fence_after();
     const uint32_t tmem = s_tmem_base, tm_H = tmem, tm_U = tmem + 128;
-    const uint32_t bar_mma = smem_u32(&s_bars[2]);
 
     const long long f0 = P.last_run_start(item), f1 = P.lo(item + 1);
+    const int nch = (int)(f1 - f0);
     const int seq = (int)(f0 / P.N), b = seq / a.heads, h = seq % a.heads;
-    auto issue_tma = [&](long long f, int stage) {
-        const int n = (int)(f % P.N);
-        const int y = b * a.T + n * C;
+    const int n0 = (int)(f0 % P.N);                        // first chunk of the run inside its sequence
+    const float *grun = a.gate + ((size_t)b * a.T + (size_t)n0 * C) * a.heads + h;   // token stride: heads
+    auto issue_tma = [&](int n) {
+        const int stage = n % SUM_NS;
+        const int y = b * a.T + (n0 + n) * C;
         const uint32_t bar = smem_u32(&s_bars[stage]);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(32768u) : "memory");
 #pragma unroll
@@ -929,41 +934,56 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                 : "memory");
         }
     };
-    auto load_gate = [&](long long f) -> float {
-        const int n = (int)(f % P.N);
-        return (t < C) ? a.gate[((size_t)b * a.T + (size_t)n * C + t) * a.heads + h] : 1.f;
-    };
+    if (t == 0)
+        for (int n = 0; n < nch && n < SUM_NS; ++n) issue_tma(n);
 
-    if (t == 0) issue_tma(f0, 0);
-    float g_cur = load_gate(f0);
-    float decay_log2 = 0.f;
+    // ---- pre-pass: total log2 decay of the run
+    float total = 0.f;
+    {
+        float s = 0.f;
+        for (int i = t; i < nch * C; i += 128) s += fmaxf(log2f(grun[(size_t)i * a.heads]), -115.f);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (l == 0) s_red[warp_q] = s;
+        __syncthreads();
+        total = s_red[0] + s_red[1] + s_red[2] + s_red[3];
+        __syncthreads();
+    }
+
+    auto load_lg = [&](int n) -> float {   // threads 0..63: log2 gate of token t of chunk n
+        return (t < C && n < nch) ? fmaxf(log2f(grun[((size_t)n * C + t) * a.heads]), -115.f) : 0.f;
+    };
+    float lg_cur = load_lg(0);
+    float prefix = 0.f;                    // log2 decay of the chunks before the current one
     bool failed = false;
-    uint32_t ph_mma = 0;
     constexpr uint32_t I_ADV = make_idesc(128, 128, 1, 1);
-    for (long long f = f0; f < f1 && !failed; ++f) {
-        const int stage = (int)((f - f0) & 1);
-        const uint32_t ph_tma = (uint32_t)(((f - f0) >> 1) & 1);
-        // prefetch the next chunk (its stage was last read by the MMAs of chunk f - 1, which have completed)
-        float g_next = 1.f;
-        if (f + 1 < f1) {
-            if (t == 0) issue_tma(f + 1, stage ^ 1);
-            g_next = load_gate(f + 1);
+    for (int n = 0; n < nch && !failed; ++n) {
+        const int stage = n % SUM_NS, par = n & 1;
+        const float lg_next = load_lg(n + 1);
+        if (n >= 2) {   // the MMAs of chunk n - 2 are done: its w o K buffer and its tile stage are free
+            if (!mbar_wait_bounded(smem_u32(&s_bars[SUM_NS + par]), (uint32_t)(((n - 2) >> 1) & 1))) failed = true;
+            if (t == 0 && n + 2 < nch) issue_tma(n + 2);
         }
-        if (t < C) s_lg[t] = fmaxf(log2f(g_cur), -115.f);
-        __syncthreads();
-        if (t < C) {
-            float G2c = 0.f;
-            for (int i = 0; i <= t; ++i) G2c += s_lg[i];
-            s_G2[t] = G2c;
+        // inclusive prefix of the chunk's log2 gates over 64 tokens (two warps), chunk total
+        float incl = lg_cur;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (l >= o) incl += up;
         }
+        if (t == 31) s_red[0] = incl;
         __syncthreads();
-        if (t < C) s_w[t] = exp2f(s_G2[C - 1] - s_G2[t]);
-        const float zetaC = exp2f(s_G2[C - 1]);
-        decay_log2 += s_G2[C - 1];
+        if (t >= 32 && t < C) incl += s_red[0];
+        if (t == C - 1) s_red[1] = incl;
         __syncthreads();
-        if (!mbar_wait_bounded(smem_u32(&s_bars[stage]), ph_tma)) failed = true;
-        // w o K
+        const float chunk_total = s_red[1];
+        // w_j = 2^(decay from token j to the end of the run) = 2^((total - prefix) - incl_j)
+        if (t < C) s_w[t] = exp2f((total - prefix) - incl);
+        prefix += chunk_total;
+        __syncthreads();
+        if (!mbar_wait_bounded(smem_u32(&s_bars[stage]), (uint32_t)((n / SUM_NS) & 1))) failed = true;
         const unsigned char *kt = smem + stage * SUM_STAGE;
+        unsigned char *kw = smem + SUM_OFF_KW + par * 16384;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int qi = t + 128 * i;
@@ -973,29 +993,15 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             uint32_t *pv = reinterpret_cast<uint32_t *>(&v);
 #pragma unroll
             for (int u = 0; u < 4; ++u) pv[u] = pack_bf16(bf16_lo(pv[u]) * wj, bf16_hi(pv[u]) * wj);
-            *reinterpret_cast<uint4 *>(smem + SUM_OFF_KW + qi * 16) = v;
-        }
-        // decay the accumulators (not needed for the first chunk: its products overwrite)
-        if (f > f0) {
-#pragma unroll
-            for (int piece = 0; piece < 8; ++piece) {
-                uint32_t r[32];
-                TMEM_LD32(tmem + lane_addr + 32 * piece, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * zetaC);
-                TMEM_ST32(tmem + lane_addr + 32 * piece, r);
-            }
-            tmem_wait_st();
+            *reinterpret_cast<uint4 *>(kw + qi * 16) = v;
         }
         fence_async_smem();
-        fence_before();
         __syncthreads();
         if (t == 0) {
             fence_after();
             const uint32_t k_mn = desc_lo(sb + stage * SUM_STAGE, 8192), v_mn = desc_lo(sb + stage * SUM_STAGE + 16384, 8192);
-            const uint32_t kw_mn = desc_lo(sb + SUM_OFF_KW, 8192);
-            if (f == f0) {
+            const uint32_t kw_mn = desc_lo(sb + SUM_OFF_KW + par * 16384, 8192);
+            if (n == 0) {
                 mma_ss<0>(tm_H, k_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
                 mma_ss<0>(tm_U, v_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
             } else {
@@ -1007,13 +1013,14 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                 mma_ss<1>(tm_H, k_mn, mnstep(ks), kw_mn, mnstep(ks), I_ADV);
                 mma_ss<1>(tm_U, v_mn, mnstep(ks), kw_mn, mnstep(ks), I_ADV);
             }
-            mma_commit(bar_mma);
+            mma_commit(smem_u32(&s_bars[SUM_NS + par]));
         }
-        if (!mbar_wait_bounded(bar_mma, ph_mma)) failed = true;
-        ph_mma ^= 1u;
-        fence_after();
-        g_cur = g_next;
+        lg_cur = lg_next;
     }
+    // the last two chunks' MMAs
+    for (int n = (nch >= 2 ? nch - 2 : 0); n < nch && !failed; ++n)
+        if (!mbar_wait_bounded(smem_u32(&s_bars[SUM_NS + (n & 1)]), (uint32_t)((n >> 1) & 1))) failed = true;
+    fence_after();
     if (failed) {
         if (t == 0 && a.device_status) atomicExch(a.device_status, (int)GKA_ERR_TIMEOUT);
     } else {
@@ -1030,7 +1037,7 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                 *reinterpret_cast<float4 *>(p + 4 * i) = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
                                                                      __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
         }
-        if (t == 0) a.ws.decay[item] = exp2f(decay_log2);
+        if (t == 0) a.ws.decay[item] = exp2f(total);
     }
     fence_before();
     __syncthreads();
