@@ -36,9 +36,11 @@ METRIC = "gka_layer_fwd_tokens_per_s"
 UNIT = "tokens/s"
 L2_FLUSH_BYTES = 256 << 20
 
-# DRAM traffic per launch of the dominant kernels (dram__bytes_read.sum + dram__bytes_write.sum
-# from the ncu captures summarised under profiles/); None until a capture exists.
-NCU_TRAFFIC_BYTES = {"fwd_main": None, "decode": None}
+# DRAM traffic per launch of the dominant kernels (dram__bytes_read.sum + dram__bytes_write.sum from the
+# ncu captures summarised under profiles/).  Both captures ran a quarter/half-size case of the same kernel
+# (forward: 2048 of 4096 chunks, 136.61 MB; decode: 2048 of 8192 (sequence, head) pairs, 480.67 MB) and
+# are scaled by the units per launch; traffic is proportional to the units in both kernels.
+NCU_TRAFFIC_BYTES = {"fwd_main": 2 * 136_612_608, "decode": 4 * 480_674_816}
 
 
 def fwd_flops(n_chunks: int, n_iter: int, C: int = 64, D: int = 128) -> float:

@@ -3,8 +3,9 @@
 // One persistent thread block per SM walks its range of chunks (gka_common.cuh explains the work
 // decomposition).  The block has two "slots"; a slot is a group of 256 threads that owns one chunk of
 // C = 64 tokens at a time, so the tensor pipe works on one chunk while the CUDA cores run the
-// element-wise part of the other.  Slots take chunks alternately.  One extra warp issues every
-// tcgen05.mma: the slots post requests to it through mbarriers, it answers with tcgen05.commit.
+// element-wise part of the other.  Slots take chunks alternately.  An extra warpgroup (kept at 32
+// registers by setmaxnreg) holds one issuing thread per slot: every tcgen05.mma of a slot is issued
+// there; the slot posts requests to it through an mbarrier and it answers with tcgen05.commit.
 //
 // Orientation: every product is computed transposed, so that TMEM lanes are channels and TMEM
 // columns are tokens (Section 4.2.1 in row form; Algorithm 1 on the whole chunk):
