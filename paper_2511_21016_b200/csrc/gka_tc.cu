@@ -85,11 +85,24 @@ constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
 __device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
     return ((saddr >> 4) & 0x3FFF) | (((lbo_bytes >> 4) & 0x3FFF) << 16);
 }
-// a_step / b_step are added to the low words inside the asm block (as immediates), so that the compiler does
-// not keep one register per k-step alive in the issuer, which runs on a small register budget.
+// Every operand of a slot lives at a compile-time offset from the slot's base, and a shared-memory address
+// fits the 14-bit address field without carry, so a descriptor's low word is (slot base >> 4) plus a constant
+// (tile offset, k-step, leading-byte-offset field).  The constants are immediates of the asm block: the
+// issuing thread keeps one register per slot instead of one per operand, and runs on a small register budget.
+template <int ACC, uint32_t A_CONST, uint32_t B_CONST>
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t base14, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t.reg .b32 la, lb;\n\t"
+        "add.u32 la, %1, %4;\n\tadd.u32 lb, %1, %5;\n\t"
+        "mov.b64 da, {la, %3};\n\tmov.b64 db, {lb, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %2, %6;\n\t}" ::"r"(d_tmem), "r"(base14), "r"(idesc),
+        "r"(kDescHi), "n"(A_CONST), "n"(B_CONST), "n"(ACC)
+        : "memory");
+}
+// the same with run-time low words and k-steps (summary kernel: operand stages rotate)
 template <int ACC>
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, int a_step, uint32_t b_lo, int b_step,
-                                       uint32_t idesc) {
+__device__ __forceinline__ void mma_ss_r(uint32_t d_tmem, uint32_t a_lo, uint32_t a_step, uint32_t b_lo, uint32_t b_step,
+                                         uint32_t idesc) {
     asm volatile(
         "{\n\t.reg .b64 da, db;\n\t.reg .b32 la, lb;\n\t"
         "add.u32 la, %1, %5;\n\tadd.u32 lb, %2, %6;\n\t"
@@ -100,6 +113,20 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, int a_ste
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// Low-latency bounded wait for the issuing thread: polls without suspending (a suspended try_wait wakes
+// hundreds of cycles late).  About a second per call before it gives up.
+__device__ __forceinline__ bool mbar_spin_bounded(uint32_t bar, uint32_t parity) {
+    for (int tries = 0; tries < (1 << 25); ++tries) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
 }
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -176,6 +203,25 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 __device__ __forceinline__ float bf16_lo(uint32_t p) { return __uint_as_float(p << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t p) { return __uint_as_float(p & 0xFFFF0000u); }
+// Streaming global loads that leave the small L1 (what 228 KB of shared memory leave of it) to the
+// thread-local spill slots.
+__device__ __forceinline__ uint32_t ldg_stream_u16(const unsigned short *p) {
+    unsigned short v;
+    asm volatile("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float ldg_stream_f32(const float *p) {
+    float v;
+    asm volatile("ld.global.nc.L1::no_allocate.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float4 ldg_stream_f32x4(const float *p) {
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "l"(p));
+    return v;
+}
 __device__ __forceinline__ float ex2_fast(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -186,10 +232,12 @@ __device__ __forceinline__ float ex2_fast(float x) {
 // Debug build only: event trace of block 0 (thread 0 of each slot and the two issuer threads).
 __device__ long long g_trace[4][8192];
 __device__ int g_trace_n[4];
-#define TRACE_DECL int trace_n = 0
+__shared__ int s_trace_n[4];
+#define TRACE_DECL
 #define TRACE(role, id)                                                                                        \
     do {                                                                                                       \
-        if (blockIdx.x == 0 && trace_n < 8192) g_trace[role][trace_n++] = (clock64() << 8) | (long long)(id);  \
+        if (blockIdx.x == 0 && s_trace_n[role] < 8192)                                                         \
+            g_trace[role][s_trace_n[role]++] = (clock64() << 8) | (long long)(id);                             \
     } while (0)
 #define TSTAMP(k)                   \
     do {                            \
@@ -208,31 +256,40 @@ __device__ int g_trace_n[4];
 //   MN-major tiles: 16 k-rows = 2048 bytes per step.
 // ---------------------------------------------------------------------------------------------
 struct IssueCtx {
-    uint32_t K_k, K_mn, V_mn, Kw_mn, H_k, X_mn, P_mn;   // descriptor low words at k-step 0
+    uint32_t base14;              // (shared address of the slot's buffers) >> 4
     uint32_t tm_y, tm_s, bars;
 };
-__host__ __device__ constexpr int kstep(int ks, int box_bytes) { return ((ks >> 2) * box_bytes + (ks & 3) * 32) >> 4; }
-__host__ __device__ constexpr int mnstep(int ks) { return (ks * 2048) >> 4; }
-
-// acc = A(K-major, 2 boxes `abox` apart) x B(MN-major) over 8 k-steps; first step overwrites when !ACC0
-template <int ACC0>
-__device__ __forceinline__ void mma_k8_kmaj_mn(uint32_t d, uint32_t a_lo, int abox, uint32_t b_lo, uint32_t idesc) {
-    mma_ss<ACC0>(d, a_lo, kstep(0, abox), b_lo, mnstep(0), idesc);
-#pragma unroll
-    for (int ks = 1; ks < 8; ++ks) mma_ss<1>(d, a_lo, kstep(ks, abox), b_lo, mnstep(ks), idesc);
+// descriptor constants: tile offset and leading-byte-offset field, then the k-step
+__host__ __device__ constexpr uint32_t op_kmaj(uint32_t off) { return (off >> 4) | ((16u >> 4) << 16); }
+__host__ __device__ constexpr uint32_t op_mn(uint32_t off) { return (off >> 4) | ((8192u >> 4) << 16); }
+__host__ __device__ constexpr uint32_t kstep(int ks, int box_bytes) {
+    return (uint32_t)(((ks >> 2) * box_bytes + (ks & 3) * 32) >> 4);
 }
-// both operands K-major (8 k-steps); b_off is an extra row offset of B in 16-byte units
-template <int ACC0>
-__device__ __forceinline__ void mma_k8_kmaj_kmaj(uint32_t d, uint32_t a_lo, int abox, uint32_t b_lo, int bbox, int b_off,
-                                                 uint32_t idesc) {
-    mma_ss<ACC0>(d, a_lo, kstep(0, abox), b_lo, kstep(0, bbox) + b_off, idesc);
-#pragma unroll
-    for (int ks = 1; ks < 8; ++ks) mma_ss<1>(d, a_lo, kstep(ks, abox), b_lo, kstep(ks, bbox) + b_off, idesc);
+__host__ __device__ constexpr uint32_t mnstep(int ks) { return (uint32_t)((ks * 2048) >> 4); }
+
+// acc = A(K-major, 2 boxes ABOX apart) x B(MN-major) over 8 k-steps; first step overwrites when !ACC0
+template <int ACC0, uint32_t A, int ABOX, uint32_t B, int KS = 0>
+__device__ __forceinline__ void mma_k8_kmaj_mn(uint32_t d, uint32_t base14, uint32_t idesc) {
+    if constexpr (KS < 8) {
+        mma_ss<(KS == 0 ? ACC0 : 1), A + kstep(KS, ABOX), B + mnstep(KS)>(d, base14, idesc);
+        mma_k8_kmaj_mn<ACC0, A, ABOX, B, KS + 1>(d, base14, idesc);
+    }
+}
+// both operands K-major (8 k-steps); B_OFF is an extra row offset of B in 16-byte units
+template <int ACC0, uint32_t A, int ABOX, uint32_t B, int BBOX, uint32_t B_OFF, int KS = 0>
+__device__ __forceinline__ void mma_k8_kmaj_kmaj(uint32_t d, uint32_t base14, uint32_t idesc) {
+    if constexpr (KS < 8) {
+        mma_ss<(KS == 0 ? ACC0 : 1), A + kstep(KS, ABOX), B + kstep(KS, BBOX) + B_OFF>(d, base14, idesc);
+        mma_k8_kmaj_kmaj<ACC0, A, ABOX, B, BBOX, B_OFF, KS + 1>(d, base14, idesc);
+    }
 }
 // both operands MN-major over 4 k-steps (64 keys), accumulating
-__device__ __forceinline__ void mma_k4_mn_mn(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
-#pragma unroll
-    for (int ks = 0; ks < 4; ++ks) mma_ss<1>(d, a_lo, mnstep(ks), b_lo, mnstep(ks), idesc);
+template <uint32_t A, uint32_t B, int KS = 0>
+__device__ __forceinline__ void mma_k4_mn_mn(uint32_t d, uint32_t base14, uint32_t idesc) {
+    if constexpr (KS < 4) {
+        mma_ss<1, A + mnstep(KS), B + mnstep(KS)>(d, base14, idesc);
+        mma_k4_mn_mn<A, B, KS + 1>(d, base14, idesc);
+    }
 }
 
 __device__ __forceinline__ void issuer_run(const IssueCtx &s, int op, uint32_t tm_H, uint32_t tm_U) {
@@ -241,26 +298,29 @@ __device__ __forceinline__ void issuer_run(const IssueCtx &s, int op, uint32_t t
     constexpr uint32_t I_Y2 = make_idesc(128, 64, 1, 1);
     constexpr uint32_t I_ADV = make_idesc(128, 128, 1, 1);
     constexpr uint32_t I_GR = make_idesc(64, 64, 0, 0);
+    constexpr uint32_t K_k = op_kmaj(OFF_K), K_mn = op_mn(OFF_K), V_mn = op_mn(OFF_V), Kw_mn = op_mn(OFF_KW);
+    constexpr uint32_t H_k = op_kmaj(OFF_H), X_mn = op_mn(OFF_X), P_mn = op_mn(OFF_P);
+    const uint32_t b = s.base14;
     if (op == OP_ITER1 || op == OP_ITER1_LAST) {
-        mma_k8_kmaj_mn<0>(s.tm_s, s.K_k, 8192, s.X_mn, I_S);
+        mma_k8_kmaj_mn<0, K_k, 8192, X_mn>(s.tm_s, b, I_S);
         mma_commit(s.bars + 8 * BAR_A);
-        if (op == OP_ITER1) mma_k8_kmaj_mn<0>(s.tm_y, s.H_k, 16384, s.X_mn, I_Y1);
+        if (op == OP_ITER1) mma_k8_kmaj_mn<0, H_k, 16384, X_mn>(s.tm_y, b, I_Y1);
     } else if (op == OP_ITER2) {
-        mma_k4_mn_mn(s.tm_y, s.K_mn, s.P_mn, I_Y2);
+        mma_k4_mn_mn<K_mn, P_mn>(s.tm_y, b, I_Y2);
         mma_commit(s.bars + 8 * BAR_B);
     } else if (op == OP_FROB) {
         // H advance: Hm += K^T (w o K)
-        mma_k4_mn_mn(tm_H, s.K_mn, s.Kw_mn, I_ADV);
+        mma_k4_mn_mn<K_mn, Kw_mn>(tm_H, b, I_ADV);
         // (K H_0)[:, 0:64] -> Y columns, lanes +0;  (K H_0)[:, 64:128] -> the slot's S region;  Gram -> Y columns, lanes +16
-        mma_k8_kmaj_kmaj<0>(s.tm_y, s.K_k, 8192, s.H_k, 16384, 0, I_GR);
-        mma_k8_kmaj_kmaj<0>(s.tm_s, s.K_k, 8192, s.H_k, 16384, 8192 >> 4, I_GR);
-        mma_k8_kmaj_kmaj<0>(s.tm_y + (16u << 16), s.K_k, 8192, s.K_k, 8192, 0, I_GR);
+        mma_k8_kmaj_kmaj<0, K_k, 8192, H_k, 16384, 0>(s.tm_y, b, I_GR);
+        mma_k8_kmaj_kmaj<0, K_k, 8192, H_k, 16384, (8192u >> 4)>(s.tm_s, b, I_GR);
+        mma_k8_kmaj_kmaj<0, K_k, 8192, K_k, 8192, 0>(s.tm_y + (16u << 16), b, I_GR);
         mma_commit(s.bars + 8 * BAR_A);
     } else if (op == OP_OUT) {
-        mma_k8_kmaj_mn<0>(s.tm_y, s.H_k, 16384, s.X_mn, I_Y1);
-        mma_k4_mn_mn(s.tm_y, s.V_mn, s.P_mn, I_Y2);
+        mma_k8_kmaj_mn<0, H_k, 16384, X_mn>(s.tm_y, b, I_Y1);
+        mma_k4_mn_mn<V_mn, P_mn>(s.tm_y, b, I_Y2);
         mma_commit(s.bars + 8 * BAR_A);
-        mma_k4_mn_mn(tm_U, s.V_mn, s.Kw_mn, I_ADV);
+        mma_k4_mn_mn<V_mn, Kw_mn>(tm_U, b, I_ADV);
         mma_commit(s.bars + 8 * BAR_B);
     }
 }
@@ -357,7 +417,7 @@ __device__ __forceinline__ float master_pass(SlotCtx &cx, uint32_t tm_master, bo
         } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                float4 v4 = grow ? *reinterpret_cast<const float4 *>(grow + 64 * cx.half + 32 * piece + 4 * i)
+                float4 v4 = grow ? ldg_stream_f32x4(grow + 64 * cx.half + 32 * piece + 4 * i)
                                  : make_float4(0.f, 0.f, 0.f, 0.f);
                 r[4 * i + 0] = __float_as_uint(v4.x); r[4 * i + 1] = __float_as_uint(v4.y);
                 r[4 * i + 2] = __float_as_uint(v4.z); r[4 * i + 3] = __float_as_uint(v4.w);
@@ -408,7 +468,8 @@ __device__ __forceinline__ uint32_t chunk_solve(SlotCtx cx, int n_iter) {
     const int slot = cx.slot, t = cx.t, lane = cx.lane, half = cx.half;
     TRACE_DECL;
     // ---- x_0 = 2 q / (L + mu), X' operand (this thread: channel `lane`, tokens 32 half .. 32 half + 31)
-    float xm[32], xp[32];
+    float xm[32];
+    uint32_t dl[16];      // x_i - x_{i-1} as packed bf16 pairs: the momentum term shrinks as the iteration converges
     {
         uint32_t qp[16];
         TMEM_LD16(cx.tm_q + cx.lane_addr + 16 * half, qp);
@@ -424,8 +485,8 @@ __device__ __forceinline__ uint32_t chunk_solve(SlotCtx cx, int n_iter) {
                 const float x0 = sc->s0[c0] * sc->zt[c0] * bf16_lo(qp[i0 >> 1]);
                 const float x1 = sc->s0[c0 + 1] * sc->zt[c0 + 1] * bf16_hi(qp[i0 >> 1]);
                 xm[i0] = x0; xm[i0 + 1] = x1;
-                xp[i0] = 0.f; xp[i0 + 1] = 0.f;
-                pk[u] = pack_bf16(x0, x1);
+                dl[i0 >> 1] = pack_bf16(x0, x1);     // x_{-1} = 0 (Algorithm 1), so the first difference is x_0
+                pk[u] = dl[i0 >> 1];
             }
             *reinterpret_cast<uint4 *>(xrow + (((4 * half + ch) ^ (lane & 7)) * 16)) =
                 make_uint4(pk[0], pk[1], pk[2], pk[3]);
@@ -445,7 +506,7 @@ __device__ __forceinline__ uint32_t chunk_solve(SlotCtx cx, int n_iter) {
             const float omega = 4.f / (4.f - sc->rho2[t] * sc->omega[t]);
             sc->omega[t] = omega;
             const float sigma = sc->s0[t] * omega, beta = omega - 1.f;
-            sc->coef[it & 1][t] = make_float4(sigma * sc->zt[t], beta, 1.f + beta - sigma * sc->lam[t], 0.f);
+            sc->coef[it & 1][t] = make_float4(sigma * sc->zt[t], beta, sigma * sc->lam[t], 0.f);
         }
         TSTAMP(15);
         slot_wait(cx, BAR_A);
@@ -474,19 +535,20 @@ __device__ __forceinline__ uint32_t chunk_solve(SlotCtx cx, int n_iter) {
                 uint32_t pk[2];
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    float xo[2];
+                    float dn[2];
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
                         const int i = 4 * piece + 2 * u + e;
                         const float4 cf = coef[i];
                         const float qv = e == 0 ? bf16_lo(qq[u]) : bf16_hi(qq[u]);
+                        const float dv = e == 0 ? bf16_lo(dl[i >> 1]) : bf16_hi(dl[i >> 1]);
                         const float acc = __uint_as_float(r[2 * u + e]);
-                        const float xn = fmaf(cf.x, qv - acc, fmaf(cf.z, xm[i], -cf.y * xp[i]));
-                        xp[i] = xm[i];
-                        xm[i] = xn;
-                        xo[e] = xn;
+                        // x_{i+1} - x_i = beta (x_i - x_{i-1}) + sigma (q - A x_i), with the lambda part of A explicit
+                        dn[e] = fmaf(cf.x, qv - acc, fmaf(cf.y, dv, -cf.z * xm[i]));
+                        xm[i] += dn[e];
                     }
-                    pk[u] = pack_bf16(xo[0], xo[1]);
+                    dl[(4 * piece + 2 * u) >> 1] = pack_bf16(dn[0], dn[1]);
+                    pk[u] = pack_bf16(xm[4 * piece + 2 * u], xm[4 * piece + 2 * u + 1]);
                 }
                 const int chunk = (4 * half + (piece >> 1)) ^ (lane & 7);
                 *reinterpret_cast<uint2 *>(xrow + chunk * 16 + 8 * (piece & 1)) = make_uint2(pk[0], pk[1]);
@@ -513,6 +575,9 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
     if (tid == 0) {
         s_abort = 0;
+#ifdef GKA_TC_TIMING
+        for (int i = 0; i < 4; ++i) s_trace_n[i] = 0;
+#endif
         for (int i = 0; i < NSLOT * BAR_COUNT + 2; ++i)
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_bars[i])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -544,13 +609,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             const SlotScalars *isc = reinterpret_cast<const SlotScalars *>(smem + (size_t)s * SLOT_BYTES + OFF_SC);
             const uint32_t sb = smem_u32(smem + (size_t)s * SLOT_BYTES);
             IssueCtx ic;
-            ic.K_k = desc_lo(sb + OFF_K, 16);        // K as K-major (rows = keys)
-            ic.K_mn = desc_lo(sb + OFF_K, 8192);     // K as MN-major (rows = channels; 8192 bytes to the next 64)
-            ic.V_mn = desc_lo(sb + OFF_V, 8192);
-            ic.Kw_mn = desc_lo(sb + OFF_KW, 8192);
-            ic.H_k = desc_lo(sb + OFF_H, 16);        // H_0 / U_0, K-major
-            ic.X_mn = desc_lo(sb + OFF_X, 8192);
-            ic.P_mn = desc_lo(sb + OFF_P, 8192);
+            ic.base14 = (sb >> 4) & 0x3FFF;   // K, H_0 / U_0 are used K-major; K, V, w o K, X', P MN-major (8192 bytes
+                                              // from one group of 64 channels or tokens to the next)
             ic.tm_y = tmem + (s == 0 ? TM_Y0 : TM_Y1);
             ic.tm_s = tmem + TM_S + ((uint32_t)(16 * s) << 16);
             ic.bars = smem_u32(&s_bars[s * BAR_COUNT]);
@@ -558,7 +618,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             for (;;) {
                 // a request normally arrives within microseconds; give up after seconds of silence
                 bool got = false;
-                for (int tries = 0; tries < 4 && !got; ++tries) got = mbar_wait_bounded(ic.bars + 8 * BAR_REQ, reqph);
+                for (int tries = 0; tries < 4 && !got; ++tries) got = mbar_spin_bounded(ic.bars + 8 * BAR_REQ, reqph);
                 if (!got || s_abort != 0) {
                     s_abort = 1;
                     break;
@@ -644,7 +704,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
                 const size_t rs = (size_t)a.heads * D;
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const uint32_t lo = qs[(size_t)(2 * i) * rs], hi = qs[(size_t)(2 * i + 1) * rs];
+                    const uint32_t lo = ldg_stream_u16(qs + (size_t)(2 * i) * rs), hi = ldg_stream_u16(qs + (size_t)(2 * i + 1) * rs);
                     qp[i] = lo | (hi << 16);
                 }
                 // parked in TMEM for the whole chunk (exact: q is bf16); this slot's previous chunk is done with it
@@ -654,9 +714,9 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
             // ---- gates (threads 0..63 own token c = t for scalar bookkeeping)
             if (t < C) {
-                const float g = a.gate[tok0 + (size_t)t * a.heads];
+                const float g = ldg_stream_f32(a.gate + tok0 + (size_t)t * a.heads);
                 sc->w[t] = fmaxf(log2f(g), -115.f);     // temporary: log2 gamma
-                sc->lam[t] = a.lam[tok0 + (size_t)t * a.heads];
+                sc->lam[t] = ldg_stream_f32(a.lam + tok0 + (size_t)t * a.heads);
             }
             slot_sync(slot);
             float G2c = 0.f;
@@ -857,12 +917,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     }
 
 #ifdef GKA_TC_TIMING
-    if (blockIdx.x == 0) {
-        if (tid == 0) g_trace_n[0] = trace_n;
-        if (tid == ST) g_trace_n[1] = trace_n;
-        if (tid == NSLOT * ST + 64) g_trace_n[2] = trace_n;
-        if (tid == NSLOT * ST + 96) g_trace_n[3] = trace_n;
-    }
+    __syncthreads();
+    if (blockIdx.x == 0 && tid < 4) g_trace_n[tid] = s_trace_n[tid];
 #endif
     fence_before();
     __syncthreads();
@@ -1003,16 +1059,16 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             const uint32_t k_mn = desc_lo(sb + stage * SUM_STAGE, 8192), v_mn = desc_lo(sb + stage * SUM_STAGE + 16384, 8192);
             const uint32_t kw_mn = desc_lo(sb + SUM_OFF_KW + par * 16384, 8192);
             if (n == 0) {
-                mma_ss<0>(tm_H, k_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
-                mma_ss<0>(tm_U, v_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
+                mma_ss_r<0>(tm_H, k_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
+                mma_ss_r<0>(tm_U, v_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
             } else {
-                mma_ss<1>(tm_H, k_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
-                mma_ss<1>(tm_U, v_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
+                mma_ss_r<1>(tm_H, k_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
+                mma_ss_r<1>(tm_U, v_mn, mnstep(0), kw_mn, mnstep(0), I_ADV);
             }
 #pragma unroll
             for (int ks = 1; ks < 4; ++ks) {
-                mma_ss<1>(tm_H, k_mn, mnstep(ks), kw_mn, mnstep(ks), I_ADV);
-                mma_ss<1>(tm_U, v_mn, mnstep(ks), kw_mn, mnstep(ks), I_ADV);
+                mma_ss_r<1>(tm_H, k_mn, mnstep(ks), kw_mn, mnstep(ks), I_ADV);
+                mma_ss_r<1>(tm_U, v_mn, mnstep(ks), kw_mn, mnstep(ks), I_ADV);
             }
             mma_commit(smem_u32(&s_bars[SUM_NS + par]));
         }
