@@ -1,0 +1,793 @@
+// tcgen05 / TMEM chunk-wise GKA forward (bf16 operands, fp32 accumulation) for sm_100a, token-major tiles.
+//
+// One persistent thread block per SM walks its range of chunks (gka_common.cuh explains the work
+// decomposition) in tiles of up to two chunks = 128 tokens.  A tile puts one token on each TMEM lane, so
+// every product of the chunk-wise form (Section 4.2.1; Algorithm 1 on the whole tile) is an M = 128 tile:
+//     S[c][j]  = sum_e X'[c][e] K[j][e]                        scores      (A = X', B = K, both K-major)
+//     P[c][j]  = S[c][j] * Gamma[c][j] / zt_c  for j <= c        masked, as packed bf16 back into TMEM
+//     Y[c][d]  = sum_e X'[c][e] H_0[d][e] + sum_j P[c][j] Kw[j][d]   (second product: A = P from TMEM)
+//     x_c     <- x_c + beta (x_c - x_c^prev) + sigma (q_c - Y_c - lambda_c x_c)          Algorithm 1
+//     O[c][i]  = sum_e X'[c][e] U_0[i][e] + sum_j P[c][j] V[j][i]
+// with X' = zt_c x_c in bf16, zt_c = max(zeta_c, 2^-60).  16 compute warps: warp quadrant q owns tokens
+// 32 q .. 32 q + 31 (its TMEM lanes), column quarter cq owns 32 of the 128 columns; a thread therefore
+// holds one token's 32 channels of x, x - x^prev and q in registers, and every per-token coefficient of
+// Algorithm 1 (sigma_c, beta_c, lambda_c, zt_c) is a per-thread scalar.
+//
+// Decay factors.  Gamma[c][j] / zt_c = 2^(G_c - G_j) / zt_c (G the cumulative log2 gate in the tile).  When
+// the whole tile decays by less than 2^-60 this is 2^-G_last * w_j with w_j = 2^(G_last - G_j) <= 1, the
+// weight the state update needs anyway: the B operand of the second product is Kw = w o K and P needs one
+// tile-wide constant factor.  Tiles that decay more (and the last score pass, whose P multiplies the
+// unweighted V) compute the factor per element and pair P with the unweighted operand.
+//
+// State: fp32 masters of H and U live in TMEM (2 x 128 columns) for a whole run; per tile each is read once
+// (bf16 operand copy to shared memory, ||H_0||_F^2), scaled by the tile's decay and advanced by tensor-core
+// products K^T Kw, V^T Kw.  The Frobenius norms of Section 4.2.1 come from K H_0 and the Gram matrix K K^T
+// (two more tensor-core products per tile) and an affine scan over the tile's tokens.
+//
+// One thread of an extra warpgroup (kept at 32 registers by setmaxnreg) issues every tcgen05.mma; the
+// compute warps post requests through an mbarrier and wait for tcgen05.commit.  K tiles are double
+// buffered (the next tile's K is fetched by TMA during the solve), V arrives during the solve as well.
+#include <cuda.h>
+
+#include "gka_common.cuh"
+#include "gka_tc_util.cuh"
+
+namespace gka {
+namespace {
+
+using namespace tcu;
+
+constexpr int D = 128;
+constexpr int NT = 128;                    // tokens per tile: one per TMEM lane
+constexpr int CT = 512;                    // compute threads
+constexpr int kThreadsTile = CT + 128;     // + the warpgroup that holds the MMA-issuing thread
+constexpr int kRegsCompute = 112, kRegsIssuer = 32;   // register split after setmaxnreg (launch: 96 each)
+
+// ---- shared memory map (bytes; every operand buffer is 1024-byte aligned).  A [128 rows][128 columns] bf16
+// operand is two boxes of [128 rows][64 columns] with the 128-byte swizzle, 16384 bytes apart.
+constexpr uint32_t OFF_K0 = 0;           // K tile, stage 0 (rows = keys)
+constexpr uint32_t OFF_K1 = 32768;       // K tile, stage 1
+constexpr uint32_t OFF_V = 65536;        // V tile
+constexpr uint32_t OFF_KW = 98304;       // w o K
+constexpr uint32_t OFF_H = 131072;       // bf16 H_0 (later U_0), rows = state rows
+constexpr uint32_t OFF_X = 163840;       // X' (rows = tokens)
+constexpr uint32_t OFF_SC = 196608;      // scalars
+struct TileScalars {
+    float lg[NT];          // log2 gamma_c
+    float G2[NT];          // cumulative log2 gate
+    float ac[NT];          // G2_c - max(G2_c, -60): exponent correction of clamped tokens
+    float zt[NT];          // clamped zeta_c
+    float lam[NT];         // lambda_c (after the adaptive rule, if any)
+    float s0[NT];          // 2 / (L + mu)
+    float rho2[NT];
+    float part[2][4][NT];  // Frobenius partial sums: [k H_0 k | Gram part][column quarter][key]
+    float carry[2][2][4];  // per-warp totals (a, b) of the two scans
+    float red[16];         // per-warp sums of squares of H_0
+    int req_op;            // request to the MMA issuer
+    int stop;              // block-wide copy of the abort flag, taken between tiles
+};
+constexpr uint32_t SC_BYTES = 8192;
+static_assert(sizeof(TileScalars) <= SC_BYTES, "scalar block too large");
+constexpr uint32_t TILE_SMEM = OFF_SC + SC_BYTES + 1024;   // + slack for the 1024-byte alignment of the base
+
+// ---- TMEM columns: fp32 masters H, U; score accumulator S (P overwrites it in place); Y / O accumulator
+constexpr uint32_t TM_H = 0, TM_U = 128, TM_S = 256, TM_Y = 384;
+
+enum { BAR_K0 = 0, BAR_K1, BAR_V, BAR_A, BAR_B, BAR_REQ, BAR_COUNT };
+enum { OP_FROB = 1, OP_ITER1, OP_ITER1_LAST, OP_ITER2, OP_OUT, OP_EXIT };
+constexpr int OPF_STAGE = 1 << 8, OPF_PLAIN_K = 1 << 9;   // request flags: K stage; pair P with K instead of w o K
+
+// ---- operand descriptor constants relative to (shared base >> 4); k-steps of 16
+__host__ __device__ constexpr uint32_t t_kmaj(uint32_t off) { return (off >> 4) | ((16u >> 4) << 16); }
+__host__ __device__ constexpr uint32_t t_mn(uint32_t off) { return (off >> 4) | ((16384u >> 4) << 16); }
+__host__ __device__ constexpr uint32_t t_kstep(int ks) { return (uint32_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4); }
+__host__ __device__ constexpr uint32_t t_mnstep(int ks) { return (uint32_t)((ks * 2048) >> 4); }
+
+// D (+)= A x B, both operands in shared memory: low words are a base register plus an immediate
+template <int ACC, uint32_t A_CONST, uint32_t B_CONST>
+__device__ __forceinline__ void mma_ss2(uint32_t d_tmem, uint32_t a_base, uint32_t b_base, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t.reg .b32 la, lb;\n\t"
+        "add.u32 la, %1, %5;\n\tadd.u32 lb, %2, %6;\n\t"
+        "mov.b64 da, {la, %4};\n\tmov.b64 db, {lb, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, %7;\n\t}" ::"r"(d_tmem), "r"(a_base), "r"(b_base), "r"(idesc),
+        "r"(kDescHi), "n"(A_CONST), "n"(B_CONST), "n"(ACC)
+        : "memory");
+}
+// D += A x B with A (packed bf16 pairs) in TMEM
+template <uint32_t B_CONST>
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_base, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .b64 db;\n\t.reg .b32 lb;\n\t.reg .pred p;\n\t"
+        "add.u32 lb, %2, %5;\n\tmov.b64 db, {lb, %4};\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}" ::"r"(d_tmem), "r"(a_tmem), "r"(b_base), "r"(idesc),
+        "r"(kDescHi), "n"(B_CONST)
+        : "memory");
+}
+template <int ACC0, uint32_t A, uint32_t B, int KS = 0>   // both K-major, 8 k-steps over the 128 channels
+__device__ __forceinline__ void mma8_kk(uint32_t d, uint32_t a_base, uint32_t b_base, uint32_t idesc) {
+    if constexpr (KS < 8) {
+        mma_ss2<(KS == 0 ? ACC0 : 1), A + t_kstep(KS), B + t_kstep(KS)>(d, a_base, b_base, idesc);
+        mma8_kk<ACC0, A, B, KS + 1>(d, a_base, b_base, idesc);
+    }
+}
+template <uint32_t A, uint32_t B, int KS = 0>   // both MN-major, 8 k-steps over the 128 tokens, accumulating
+__device__ __forceinline__ void mma8_mm(uint32_t d, uint32_t a_base, uint32_t b_base, uint32_t idesc) {
+    if constexpr (KS < 8) {
+        mma_ss2<1, A + t_mnstep(KS), B + t_mnstep(KS)>(d, a_base, b_base, idesc);
+        mma8_mm<A, B, KS + 1>(d, a_base, b_base, idesc);
+    }
+}
+template <uint32_t B, int KS = 0>   // A = P in TMEM (a thread's 16 packed columns per column quarter), B MN-major
+__device__ __forceinline__ void mma8_pm(uint32_t d, uint32_t p_tmem, uint32_t b_base, uint32_t idesc) {
+    if constexpr (KS < 8) {
+        mma_ts<B + t_mnstep(KS)>(d, p_tmem + 32 * (KS >> 1) + 8 * (KS & 1), b_base, idesc);
+        mma8_pm<B, KS + 1>(d, p_tmem, b_base, idesc);
+    }
+}
+
+__device__ __forceinline__ void issuer_run(int req, uint32_t base14, uint32_t tmem, uint32_t bars) {
+    constexpr uint32_t I_KK = make_idesc(128, 128, 0, 0);   // both operands K-major
+    constexpr uint32_t I_PM = make_idesc(128, 128, 0, 1);   // A from TMEM, B MN-major
+    constexpr uint32_t I_MM = make_idesc(128, 128, 1, 1);   // both MN-major
+    constexpr uint32_t K_k = t_kmaj(0), K_mn = t_mn(0);     // relative to the K stage
+    constexpr uint32_t V_mn = t_mn(OFF_V), Kw_mn = t_mn(OFF_KW), H_k = t_kmaj(OFF_H), X_k = t_kmaj(OFF_X);
+    const int op = req & 0xFF;
+    const uint32_t kb = base14 + ((req & OPF_STAGE) ? (OFF_K1 >> 4) : (OFF_K0 >> 4));
+    const uint32_t tm_H = tmem + TM_H, tm_U = tmem + TM_U, tm_S = tmem + TM_S, tm_Y = tmem + TM_Y;
+    if (op == OP_ITER1 || op == OP_ITER1_LAST) {
+        mma8_kk<0, X_k, K_k>(tm_S, base14, kb, I_KK);
+        mma_commit(bars + 8 * BAR_A);
+        if (op == OP_ITER1) mma8_kk<0, X_k, H_k>(tm_Y, base14, base14, I_KK);
+    } else if (op == OP_ITER2) {
+        if (req & OPF_PLAIN_K) mma8_pm<K_mn>(tm_Y, tm_S, kb, I_PM);
+        else mma8_pm<Kw_mn>(tm_Y, tm_S, base14, I_PM);
+        mma_commit(bars + 8 * BAR_B);
+    } else if (op == OP_FROB) {
+        mma8_mm<K_mn, Kw_mn>(tm_H, kb, base14, I_MM);        // H += K^T (w o K)
+        mma8_kk<0, K_k, H_k>(tm_Y, kb, base14, I_KK);        // K H_0
+        mma8_kk<0, K_k, K_k>(tm_S, kb, kb, I_KK);            // Gram matrix K K^T
+        mma_commit(bars + 8 * BAR_A);
+    } else if (op == OP_OUT) {
+        mma8_kk<0, X_k, H_k>(tm_Y, base14, base14, I_KK);    // X' U_0^T (the H buffer holds U_0 now)
+        mma8_pm<V_mn>(tm_Y, tm_S, base14, I_PM);             // + P V
+        mma_commit(bars + 8 * BAR_A);
+        mma8_mm<V_mn, Kw_mn>(tm_U, base14, base14, I_MM);    // U += V^T (w o K)
+        mma_commit(bars + 8 * BAR_B);
+    }
+}
+
+#ifdef GKA_TC_TIMING
+// Debug build only: event trace of block 0 (compute thread 0 and the issuing thread).
+__device__ long long g_ttrace[2][8192];
+__device__ int g_ttrace_n[2];
+__shared__ int s_ttrace_n[2];
+#define TRACE(role, id)                                                                                        \
+    do {                                                                                                       \
+        if (blockIdx.x == 0 && s_ttrace_n[role] < 8192)                                                        \
+            g_ttrace[role][s_ttrace_n[role]++] = (clock64() << 8) | (long long)(id);                           \
+    } while (0)
+#define TSTAMP(k)               \
+    do {                        \
+        if (tid == 0) TRACE(0, k); \
+    } while (0)
+#else
+#define TRACE(role, id)
+#define TSTAMP(k)
+#endif
+
+#define TMEM_ST8(taddr, r)                                                                                       \
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]), \
+                 "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])                     \
+                 : "memory")
+
+__device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 1, 512;" ::: "memory"); }
+
+// Everything a compute thread needs to know about itself.
+struct Ctx {
+    int tid, l, q, cq;            // thread, lane in warp, TMEM lane quadrant, column quarter
+    int c;                        // token / TMEM lane / state row: 32 q + l
+    uint32_t lane_addr;           // (32 q) << 16
+    unsigned char *smem;
+    TileScalars *sc;
+    uint32_t bars, tmem, abort_addr;
+};
+
+__device__ __forceinline__ bool aborted(const Ctx &cx) {
+    int v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(cx.abort_addr) : "memory");
+    return v != 0;
+}
+// Wait for an mbarrier phase: warp 0 polls (bounded), the others sleep in the named barrier.
+__device__ __forceinline__ void wait_bar(const Ctx &cx, int which, uint32_t parity) {
+    if (cx.tid < 32 && !aborted(cx)) {
+        if (!mbar_spin_bounded(cx.bars + 8 * which, parity)) {   // the block reports GKA_ERR_TIMEOUT when it ends
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(cx.abort_addr), "r"(1) : "memory");
+        }
+#ifdef GKA_TC_TIMING
+        if (cx.tid == 0) TRACE(0, 20);
+#endif
+    }
+    cta_sync();
+}
+// Ask the issuer for a batch of MMAs.  Call after cta_sync: every thread's writes and fences are done.
+__device__ __forceinline__ void post(const Ctx &cx, int req) {
+    if (cx.tid == 0) {
+        *reinterpret_cast<volatile int *>(&cx.sc->req_op) = req;
+        mbar_arrive(cx.bars + 8 * BAR_REQ);
+    }
+}
+// byte offset of the 16-byte group holding columns 8 g .. 8 g + 7 (g = 0..15) of row r in a 128 x 128 operand
+__device__ __forceinline__ uint32_t tile_off(int r, int g) {
+    return (uint32_t)((g >> 3) * 16384 + r * 128 + (((g & 7) ^ (r & 7)) << 4));
+}
+
+// One pass over a master (H or U) for this thread's row and 32 columns: source is TMEM, or global memory at
+// the start of a run.  Writes the bf16 operand copy, optionally accumulates the sum of squares, scales by the
+// tile's decay and stores the result back to TMEM.
+template <bool SUMSQ>
+__device__ __forceinline__ float master_pass(const Ctx &cx, uint32_t tm_master, bool from_global, const float *grow,
+                                             float decay) {
+    float ss = 0.f;
+    uint32_t r[32];
+    const uint32_t taddr = tm_master + cx.lane_addr + 32 * cx.cq;
+    if (!from_global) {
+        TMEM_LD32(taddr, r);
+        tmem_wait_ld();
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float4 v4 = grow ? ldg_stream_f32x4(grow + 32 * cx.cq + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            r[4 * i + 0] = __float_as_uint(v4.x); r[4 * i + 1] = __float_as_uint(v4.y);
+            r[4 * i + 2] = __float_as_uint(v4.z); r[4 * i + 3] = __float_as_uint(v4.w);
+        }
+    }
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float v0 = __uint_as_float(r[8 * ch + 2 * u]), v1 = __uint_as_float(r[8 * ch + 2 * u + 1]);
+            if (SUMSQ) ss = fmaf(v0, v0, fmaf(v1, v1, ss));
+            pk[u] = pack_bf16(v0, v1);
+        }
+        *reinterpret_cast<uint4 *>(cx.smem + OFF_H + tile_off(cx.c, 4 * cx.cq + ch)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * decay);
+    TMEM_ST32(taddr, r);
+    tmem_wait_st();
+    return ss;
+}
+
+// Copy this thread's part of a master from TMEM to global memory (final state of a sequence).
+__device__ __forceinline__ void master_store(const Ctx &cx, uint32_t tm_master, float *grow) {
+    uint32_t r[32];
+    TMEM_LD32(tm_master + cx.lane_addr + 32 * cx.cq, r);
+    tmem_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        *reinterpret_cast<float4 *>(grow + 32 * cx.cq + 4 * i) =
+            make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]),
+                        __uint_as_float(r[4 * i + 3]));
+}
+
+// Masked score epilogue: S (TMEM, fp32) -> P (packed bf16 pairs, written over the first 16 of this thread's own
+// 32 score columns).  Keys j = 32 cq + i, token c = 32 q + l: blocks above the diagonal are zero, blocks below
+// it need no mask.  GENERAL: per-element factor 2^(ac_c - G_j) (strongly decaying tiles, and the pass whose P
+// multiplies the unweighted V); otherwise the tile-wide constant pf.
+template <bool GENERAL, bool DIAG>
+__device__ __forceinline__ void p_block(const Ctx &cx, uint32_t taddr, float pf, float ac_c) {
+    const uint64_t pf2 = f2_pack(pf, pf);
+#pragma unroll
+    for (int piece = 0; piece < 2; ++piece) {
+        uint32_t r[16], pk[8];
+        TMEM_LD16(taddr + 16 * piece, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i0 = 16 * piece + 2 * u;
+            uint64_t f2 = pf2;
+            if (GENERAL)
+                f2 = f2_pack(ex2_fast(fminf(ac_c - cx.sc->G2[32 * cx.cq + i0], 126.f)),
+                             ex2_fast(fminf(ac_c - cx.sc->G2[32 * cx.cq + i0 + 1], 126.f)));
+            float p0, p1;
+            f2_unpack(f2_mul(f2_pack(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1])), f2), p0, p1);
+            if (DIAG) {                     // keys i <= l are visible
+                p0 = (i0 <= cx.l) ? p0 : 0.f;
+                p1 = (i0 + 1 <= cx.l) ? p1 : 0.f;
+            }
+            pk[u] = pack_bf16(p0, p1);
+        }
+        TMEM_ST8(taddr + 8 * piece, pk);
+    }
+}
+__device__ __forceinline__ void p_epilogue(const Ctx &cx, bool general, float pf, float ac_c) {
+    const uint32_t taddr = cx.tmem + TM_S + cx.lane_addr + 32 * cx.cq;
+    if (cx.cq > cx.q) {
+        uint32_t z[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) z[i] = 0u;
+        TMEM_ST8(taddr, z);
+        TMEM_ST8(taddr + 8, z);
+    } else if (cx.cq == cx.q) {
+        if (general) p_block<true, true>(cx, taddr, pf, ac_c);
+        else p_block<false, true>(cx, taddr, pf, ac_c);
+    } else {
+        if (general) p_block<true, false>(cx, taddr, pf, ac_c);
+        else p_block<false, false>(cx, taddr, pf, ac_c);
+    }
+    tmem_wait_st();
+}
+
+// Inclusive scan over the tile's 128 tokens (threads 0..127 = warps 0..3, one token each) of the affine maps
+// s -> a s + b, composed in token order; returns the map's value at `seed`.  `slot` selects the carry row.
+__device__ __forceinline__ float affine_scan(const Ctx &cx, float a, float b, float seed, int slot) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float pa = __shfl_up_sync(0xffffffffu, a, o), pb = __shfl_up_sync(0xffffffffu, b, o);
+        if (cx.l >= o) {
+            b = fmaf(a, pb, b);
+            a *= pa;
+        }
+    }
+    // carries of whole warps go through shared memory
+    float *ca = cx.sc->carry[slot][0], *cb = cx.sc->carry[slot][1];
+    if (cx.l == 31) {
+        ca[cx.q] = a;
+        cb[cx.q] = b;
+    }
+    asm volatile("bar.sync 2, 128;" ::: "memory");
+    float s = seed;
+    for (int w = 0; w < cx.q; ++w) s = fmaf(ca[w], s, cb[w]);
+    return fmaf(a, s, b);
+}
+
+// What a phase needs to know about a tile; recomputed from the tile's first chunk index at the start of every
+// phase instead of being carried in registers through the solve loop.
+struct TileInfo {
+    int seq, n, ntok, m_next;
+    bool run_start, seq_end;
+    size_t tok0;
+    long long f;
+    const float *init_src;     // where a run's start state comes from (nullptr = zero)
+};
+__device__ __forceinline__ TileInfo tile_info(const FwdArgs &a, int item, long long f_lo, int n_mine, int m) {
+    const WorkPlan &P = a.plan;
+    TileInfo t;
+    t.f = f_lo + m;
+    t.seq = (int)(t.f / P.N);
+    t.n = (int)(t.f % P.N);
+    const int b = t.seq / a.heads, h = t.seq % a.heads;
+    const bool two = (t.n + 1 < P.N) && (m + 1 < n_mine);
+    t.ntok = two ? 2 * kChunk : kChunk;
+    t.m_next = m + (two ? 2 : 1);
+    t.tok0 = ((size_t)b * a.T + (size_t)t.n * kChunk) * a.heads + h;
+    t.run_start = (m == 0) || (t.n == 0);
+    t.seq_end = (t.n + (two ? 2 : 1) == P.N);
+    t.init_src = nullptr;
+    const size_t st = state_floats(D, D);
+    if (t.run_start) t.init_src = (t.n == 0) ? (a.state_in ? a.state_in + (size_t)t.seq * st : nullptr)
+                                             : a.ws.start + (size_t)item * st;
+    return t;
+}
+
+__global__ void __launch_bounds__(kThreadsTile, 1)
+fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                const __grid_constant__ CUtensorMap tmQ, FwdArgs a) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t s_bars[BAR_COUNT];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    unsigned char *smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+    const int tid = threadIdx.x;
+
+    if (tid == 0) {
+        s_abort = 0;
+#ifdef GKA_TC_TIMING
+        s_ttrace_n[0] = s_ttrace_n[1] = 0;
+#endif
+        for (int i = 0; i < BAR_COUNT; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&s_bars[i])));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (tid < 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&s_tmem_base))
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem = s_tmem_base;
+    const uint32_t bars = smem_u32(&s_bars[0]);
+    TileScalars *sc = reinterpret_cast<TileScalars *>(smem + OFF_SC);
+
+    const WorkPlan &P = a.plan;
+    const int item = blockIdx.x;
+    const long long f_lo = P.lo(item), f_hi = P.lo(item + 1);
+    const int n_mine = (int)(f_hi - f_lo);          // chunks of this block
+
+    if (tid >= CT) {
+        // ================================ MMA issuing thread ================================
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssuer));
+        if (tid == CT + 64 && n_mine > 0) {
+            const uint32_t base14 = (smem_u32(smem) >> 4) & 0x3FFF;
+            uint32_t reqph = 0;
+            for (;;) {
+                // a request normally arrives within microseconds; give up after seconds of silence
+                bool got = false;
+                for (int tries = 0; tries < 4 && !got; ++tries) got = mbar_spin_bounded(bars + 8 * BAR_REQ, reqph);
+                if (!got || s_abort != 0) {
+                    s_abort = 1;
+                    break;
+                }
+                reqph ^= 1u;
+                const int req = *reinterpret_cast<const volatile int *>(&sc->req_op);
+                TRACE(1, 32 + (req & 0xFF));
+                if ((req & 0xFF) == OP_EXIT) break;
+                fence_after();
+                issuer_run(req, base14, tmem, bars);
+                TRACE(1, 48 + (req & 0xFF));
+            }
+        }
+    } else {
+        // ================================= compute threads =================================
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsCompute));
+        Ctx cx;
+        cx.tid = tid;
+        cx.l = tid & 31;
+        cx.q = (tid >> 5) & 3;
+        cx.cq = tid >> 7;
+        cx.c = 32 * cx.q + cx.l;
+        cx.lane_addr = (uint32_t)(32 * cx.q) << 16;
+        cx.smem = smem;
+        cx.sc = sc;
+        cx.bars = bars;
+        cx.tmem = tmem;
+        cx.abort_addr = smem_u32(&s_abort);
+        const int c = cx.c, cq = cx.cq, l = cx.l;
+        const uint32_t sbase = smem_u32(smem);
+        __nv_bfloat16 *gout = reinterpret_cast<__nv_bfloat16 *>(a.out);
+        const size_t st = state_floats(D, D);
+        const bool adaptive = (a.flags & GKA_FLAG_ADAPTIVE_LAMBDA) != 0;
+        uint32_t ph_a = 0, ph_b = 0;
+
+        // K (or V) tile of flat chunk f: 128 rows starting at the chunk's first token; rows past the tile's
+        // tokens belong to later tokens (or are zero-filled past the tensor) and are never used
+        auto issue_tma = [&](const CUtensorMap *map, long long f, uint32_t dst, int bar_idx) {
+            const int seq = (int)(f / P.N), n = (int)(f % P.N);
+            const int b = seq / a.heads, h = seq % a.heads;
+            const int y = b * a.T + n * kChunk;
+            const uint32_t bar = bars + 8 * bar_idx;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(32768u) : "memory");
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                const int x = h * D + 64 * hf;
+                asm volatile(
+                    "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
+                        "r"(sbase + dst + 16384 * hf), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+                    : "memory");
+            }
+        };
+
+        if (tid == 0 && n_mine > 0) issue_tma(&tmK, f_lo, OFF_K0, BAR_K0);
+
+        int tile = 0;
+        for (int m = 0; m < n_mine; ++tile) {       // m: index of the tile's first chunk inside the block's range
+            const int stage = tile & 1;
+            const uint32_t off_k = stage ? OFF_K1 : OFF_K0;
+            bool valid, clamped;
+            float pf;
+
+            // ======================= phase 1: operands, state pass, Frobenius norms =======================
+            {
+                const TileInfo ti = tile_info(a, item, f_lo, n_mine, m);
+                const int ntok = ti.ntok;
+                valid = c < ntok;
+                // the previous tile is finished: the q / V buffer and the other K stage are free
+                if (tid == 0) {
+                    issue_tma(&tmQ, ti.f, OFF_V, BAR_V);
+                    if (ti.m_next < n_mine)
+                        issue_tma(&tmK, f_lo + ti.m_next, stage ? OFF_K0 : OFF_K1, stage ? BAR_K0 : BAR_K1);
+                }
+
+                // ---- gates: cumulative log2 decay by a scan over the tile (threads 0..127 own token c = tid)
+                if (tid < NT) {
+                    const float g = valid ? ldg_stream_f32(a.gate + ti.tok0 + (size_t)c * a.heads) : 1.f;
+                    const float lamv = valid ? ldg_stream_f32(a.lam + ti.tok0 + (size_t)c * a.heads) : 1.f;
+                    const float lgc = fmaxf(log2f(g), -115.f);
+                    const float G2c = affine_scan(cx, 1.f, lgc, 0.f, 0);
+                    const float mc = fmaxf(G2c, -60.f);
+                    sc->lg[c] = lgc;
+                    sc->G2[c] = G2c;
+                    sc->ac[c] = G2c - mc;
+                    sc->zt[c] = exp2f(mc);
+                    sc->lam[c] = lamv;
+                }
+                cta_sync();
+                TSTAMP(0);
+                const float Glast = sc->G2[ntok - 1];
+                clamped = Glast < -60.f;                      // the tile decays below 2^-60: per-element factors
+                pf = exp2f(-fmaxf(Glast, -60.f));             // Gamma[c][j] / zt_c = pf * w_j otherwise
+                const float decay = exp2f(Glast);             // zeta of the whole tile
+
+                // ---- K tile has landed; w o K (same swizzled positions as K), rows past the tile weigh nothing
+                wait_bar(cx, stage ? BAR_K1 : BAR_K0, (uint32_t)((tile >> 1) & 1));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int qi = tid + CT * i;               // 16-byte group index in the 32 KB tile
+                    const int j = (qi & 1023) >> 3;            // key row of this group
+                    uint4 v = *reinterpret_cast<const uint4 *>(smem + off_k + qi * 16);
+                    const float wj = (j < ntok) ? exp2f(Glast - sc->G2[j]) : 0.f;
+                    uint32_t *pv = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) pv[u] = pack_bf16(bf16_lo(pv[u]) * wj, bf16_hi(pv[u]) * wj);
+                    *reinterpret_cast<uint4 *>(smem + OFF_KW + qi * 16) = v;
+                }
+                TSTAMP(2);
+
+                // ---- H master, one pass: ||H_0||^2, bf16 copy, scale by the tile's decay
+                {
+                    float hs = master_pass<true>(cx, tmem + TM_H, ti.run_start,
+                                                 ti.init_src ? ti.init_src + (size_t)c * D : nullptr, decay);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) hs += __shfl_xor_sync(0xffffffffu, hs, o);
+                    if (l == 0) sc->red[tid >> 5] = hs;
+                }
+                fence_async_smem();
+                fence_before();
+                cta_sync();
+                post(cx, OP_FROB | (stage ? OPF_STAGE : 0));
+                TSTAMP(3);
+                wait_bar(cx, BAR_A, ph_a);
+                ph_a ^= 1u;
+                fence_after();
+                TSTAMP(4);
+
+                // ---- chunk-wise Frobenius norms: per key, k_j^T H_0 k_j and the decayed squared Gram entries of
+                // the earlier keys.  Thread = (key j = c, 32 columns).
+                {
+                    float kh = 0.f, gs = 0.f;
+#pragma unroll
+                    for (int piece = 0; piece < 2; ++piece) {
+                        uint32_t r[16];
+                        TMEM_LD16(tmem + TM_Y + cx.lane_addr + 32 * cq + 16 * piece, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int ch = 0; ch < 2; ++ch) {
+                            const uint4 kv =
+                                *reinterpret_cast<const uint4 *>(smem + off_k + tile_off(c, 4 * cq + 2 * piece + ch));
+                            const uint32_t *pk = reinterpret_cast<const uint32_t *>(&kv);
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                kh = fmaf(__uint_as_float(r[8 * ch + 2 * u]), bf16_lo(pk[u]), kh);
+                                kh = fmaf(__uint_as_float(r[8 * ch + 2 * u + 1]), bf16_hi(pk[u]), kh);
+                            }
+                        }
+                    }
+                    if (cq <= cx.q) {
+                        const float G2j = sc->G2[c];
+                        const int lim = (cq == cx.q) ? l : 32;   // keys i < lim come earlier, i == lim is the key itself
+#pragma unroll
+                        for (int piece = 0; piece < 2; ++piece) {
+                            uint32_t r[16];
+                            TMEM_LD16(tmem + TM_S + cx.lane_addr + 32 * cq + 16 * piece, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const int ii = 16 * piece + i;
+                                const float g = __uint_as_float(r[i]);
+                                const float g2 = g * g;
+                                if (ii < lim) gs = fmaf(2.f * ex2_fast(G2j - sc->G2[32 * cq + ii]), g2, gs);
+                                else if (ii == lim) gs += g2;
+                            }
+                        }
+                    }
+                    sc->part[0][cq][c] = kh;
+                    sc->part[1][cq][c] = gs;
+                }
+                fence_before();
+                cta_sync();
+                // the H master is final for this tile
+                if (ti.seq_end && a.state_out)
+                    master_store(cx, tmem + TM_H, a.state_out + (size_t)ti.seq * st + (size_t)c * D);
+                TSTAMP(5);
+
+                // ---- f_c by an affine scan (s_c = gamma_c^2 s_{c-1} + d_c, s_{-1} = ||H_0||^2), Chebyshev set-up
+                if (tid < NT) {
+                    float hh = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) hh += sc->red[i];
+                    const float kh = (sc->part[0][0][c] + sc->part[0][1][c]) + (sc->part[0][2][c] + sc->part[0][3][c]);
+                    const float gs = (sc->part[1][0][c] + sc->part[1][1][c]) + (sc->part[1][2][c] + sc->part[1][3][c]);
+                    const float dc = fmaf(2.f * exp2f(sc->G2[c]), kh, gs);
+                    const float s = affine_scan(cx, exp2f(2.f * sc->lg[c]), dc, hh, 1);
+                    const float fc = sqrtf(fmaxf(s, 0.f));
+                    float lamc = sc->lam[c];
+                    if (adaptive) lamc *= fc;
+                    const float Lpm = fc + 2.f * lamc;
+                    const float rho = fc / Lpm;
+                    sc->lam[c] = lamc;
+                    sc->rho2[c] = rho * rho;
+                    sc->s0[c] = 2.f / Lpm;
+                    if (a.fro_out && valid) a.fro_out[ti.tok0 + (size_t)c * a.heads] = fc;
+                }
+                wait_bar(cx, BAR_V, 0u);       // q tile has landed (the wait also publishes the set-up values)
+            }
+
+            // ======================= phase 2: Algorithm 1 on the whole tile =======================
+            {
+                // per-token scalars (this thread's token), x_0 = 2 q / (L + mu)
+                const float s0 = sc->s0[c], rho2 = sc->rho2[c], lamc = sc->lam[c], ztc = sc->zt[c], acc_c = sc->ac[c];
+                const unsigned char *qrow = smem + OFF_V;      // q tile: this thread reads row c, its 4 groups of 8 channels
+                uint64_t x2[16];   // the iterate (fp32 pairs), scaled by zt_c (the recurrence is linear), as the operand needs it
+                uint64_t d2[16];   // x_i - x_{i-1} (fp32 pairs)
+                {
+                    const float x0s = valid ? s0 * ztc : 0.f;  // tokens past the tile stay zero
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        const uint4 qv = *reinterpret_cast<const uint4 *>(qrow + tile_off(c, 4 * cq + ch));
+                        const uint32_t *qq = reinterpret_cast<const uint32_t *>(&qv);
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const float xa = x0s * bf16_lo(qq[u]), xb = x0s * bf16_hi(qq[u]);
+                            x2[4 * ch + u] = f2_pack(xa, xb);
+                            d2[4 * ch + u] = x2[4 * ch + u];     // x_{-1} = 0 (Algorithm 1): the first difference is x_0
+                            pk[u] = pack_bf16(xa, xb);
+                        }
+                        *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + ch)) =
+                            make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                }
+                fence_async_smem();
+                fence_before();
+                cta_sync();
+                TSTAMP(6);
+
+                const int rq = (stage ? OPF_STAGE : 0) | (clamped ? OPF_PLAIN_K : 0);
+                float omega = 2.f;
+                for (int it = 0; it <= a.n_iter; ++it) {       // + one extra score pass for the output
+                    const bool last = (it == a.n_iter);
+                    if (last && tid == 0) {                     // q is no longer needed: its buffer takes the V tile
+                        int mm = m;
+                        asm volatile("" : "+r"(mm));
+                        issue_tma(&tmV, f_lo + mm, OFF_V, BAR_V);
+                    }
+                    post(cx, (last ? OP_ITER1_LAST : OP_ITER1) | rq);
+                    // weight schedule and this token's coefficients, while the scores are computed
+                    omega = 4.f / (4.f - rho2 * omega);
+                    const float sigma = s0 * omega, beta = omega - 1.f;
+                    const float cfx = valid ? sigma * ztc : 0.f, cfz = sigma * lamc;
+                    const uint64_t cfx2 = f2_pack(cfx, cfx), ncfz2 = f2_pack(-cfz, -cfz), beta2 = f2_pack(beta, beta);
+                    wait_bar(cx, BAR_A, ph_a);
+                    ph_a ^= 1u;
+                    fence_after();
+                    TSTAMP(7);
+                    p_epilogue(cx, clamped || last, pf, acc_c);
+                    fence_before();
+                    cta_sync();
+                    TSTAMP(8);
+                    if (last) break;
+                    post(cx, OP_ITER2 | rq);
+                    wait_bar(cx, BAR_B, ph_b);
+                    ph_b ^= 1u;
+                    fence_after();
+                    TSTAMP(9);
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {        // 8 channels at a time keeps the transient registers few
+                        uint32_t r[8];
+                        TMEM_LD8(tmem + TM_Y + cx.lane_addr + 32 * cq + 8 * ch, r);
+                        const uint4 qv = *reinterpret_cast<const uint4 *>(qrow + tile_off(c, 4 * cq + ch));
+                        const uint32_t *qq = reinterpret_cast<const uint32_t *>(&qv);
+                        tmem_wait_ld();
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int i = 4 * ch + u;
+                            // x_{i+1} - x_i = beta (x_i - x_{i-1}) + sigma (q - A x_i), with the lambda part of A explicit
+                            const uint64_t t2 = f2_sub(f2_pack(bf16_lo(qq[u]), bf16_hi(qq[u])),
+                                                       f2_pack(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1])));
+                            const uint64_t dn = f2_fma(cfx2, t2, f2_fma(beta2, d2[i], f2_mul(ncfz2, x2[i])));
+                            d2[i] = dn;
+                            x2[i] = f2_add(x2[i], dn);
+                            float xa, xb;
+                            f2_unpack(x2[i], xa, xb);
+                            pk[u] = pack_bf16(xa, xb);
+                        }
+                        *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + ch)) =
+                            make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                    fence_async_smem();
+                    fence_before();
+                    cta_sync();
+                    TSTAMP(10);
+                }
+            }
+
+            // ======================= phase 3: output, U advance =======================
+            {
+                int mm = m;
+                asm volatile("" : "+r"(mm));                   // recompute the tile's description
+                const TileInfo ti = tile_info(a, item, f_lo, n_mine, mm);
+                const float decay = exp2f(sc->G2[ti.ntok - 1]);
+                // U master pass (bf16 copy into the H buffer, scale), O = X' U_0^T + P V, U advance
+                master_pass<false>(cx, tmem + TM_U, ti.run_start,
+                                   ti.init_src ? ti.init_src + (size_t)D * D + (size_t)c * D : nullptr, decay);
+                fence_async_smem();
+                fence_before();
+                wait_bar(cx, BAR_V, 1u);                       // V tile has landed
+                post(cx, OP_OUT | (stage ? OPF_STAGE : 0));
+                TSTAMP(11);
+                wait_bar(cx, BAR_A, ph_a);
+                ph_a ^= 1u;
+                fence_after();
+                TSTAMP(12);
+                if (c < ti.ntok) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(gout + (ti.tok0 + (size_t)c * a.heads) * D + 32 * cq);
+#pragma unroll
+                    for (int piece = 0; piece < 2; ++piece) {
+                        uint32_t r[16];
+                        TMEM_LD16(tmem + TM_Y + cx.lane_addr + 32 * cq + 16 * piece, r);
+                        tmem_wait_ld();
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            pk[u] = pack_bf16(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1]));
+                        dst[2 * piece] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        dst[2 * piece + 1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    }
+                }
+                TSTAMP(13);
+                wait_bar(cx, BAR_B, ph_b);     // U advance done: every tensor-core read of this tile's buffers is done
+                ph_b ^= 1u;
+                fence_after();
+                if (ti.seq_end && a.state_out)
+                    master_store(cx, tmem + TM_U, a.state_out + (size_t)ti.seq * st + (size_t)D * D + (size_t)c * D);
+                fence_before();
+                if (tid == 0) sc->stop = aborted(cx) ? 1 : 0;
+                cta_sync();
+                TSTAMP(14);
+                if (sc->stop) break;          // the same decision in every thread
+                m = ti.m_next;
+            }
+        }
+        if (n_mine > 0) post(cx, OP_EXIT);
+    }
+
+#ifdef GKA_TC_TIMING
+    __syncthreads();
+    if (blockIdx.x == 0 && tid < 2) g_ttrace_n[tid] = s_ttrace_n[tid];
+#endif
+    fence_before();
+    __syncthreads();
+    if (tid == 0 && s_abort != 0 && a.device_status) atomicExch(a.device_status, (int)GKA_ERR_TIMEOUT);
+    if (tid < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+}
+
+}  // namespace
+
+cudaError_t launch_fwd_tile(const FwdArgs &a, cudaStream_t stream) {
+    alignas(64) CUtensorMap tmK, tmV, tmQ;
+    const int rows = a.B * a.T, cols = a.heads * D;
+    if (!make_tile_map(&tmK, a.k, rows, cols, NT) || !make_tile_map(&tmV, a.v, rows, cols, NT) ||
+        !make_tile_map(&tmQ, a.q, rows, cols, NT))
+        return cudaErrorInvalidValue;
+    cudaError_t err = cudaFuncSetAttribute(fwd_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TILE_SMEM);
+    if (err != cudaSuccess) return err;
+    if (a.ev_start) cudaEventRecord(a.ev_start, stream);
+    fwd_tile_kernel<<<a.plan.G, kThreadsTile, TILE_SMEM, stream>>>(tmK, tmV, tmQ, a);
+    if (a.ev_stop) cudaEventRecord(a.ev_stop, stream);
+    return cudaGetLastError();
+}
+
+#ifdef GKA_TC_TIMING
+extern "C" int gka_debug_tile_trace(long long *out /* 2 x 8192 */, int *counts /* 2 */) {
+    if (cudaMemcpyFromSymbol(out, g_ttrace, sizeof(long long) * 2 * 8192) != cudaSuccess) return 1;
+    if (cudaMemcpyFromSymbol(counts, g_ttrace_n, sizeof(int) * 2) != cudaSuccess) return 1;
+    return 0;
+}
+#endif
+
+}  // namespace gka
