@@ -73,7 +73,7 @@ constexpr uint32_t TILE_SMEM = OFF_SC + SC_BYTES + 1024;   // + slack for the 10
 // ---- TMEM columns: fp32 masters H, U; score accumulator S (P overwrites it in place); Y / O accumulator
 constexpr uint32_t TM_H = 0, TM_U = 128, TM_S = 256, TM_Y = 384;
 
-enum { BAR_K0 = 0, BAR_K1, BAR_V, BAR_A, BAR_B, BAR_REQ, BAR_COUNT };
+enum { BAR_K0 = 0, BAR_K1, BAR_V, BAR_A, BAR_B, BAR_COUNT };
 enum { OP_FROB = 1, OP_ITER1, OP_ITER1_LAST, OP_ITER2, OP_OUT, OP_EXIT };
 constexpr int OPF_STAGE = 1 << 8, OPF_PLAIN_K = 1 << 9;   // request flags: K stage; pair P with K instead of w o K
 
@@ -198,24 +198,21 @@ __device__ __forceinline__ bool aborted(const Ctx &cx) {
     asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(cx.abort_addr) : "memory");
     return v != 0;
 }
-// Wait for an mbarrier phase: warp 0 polls (bounded), the others sleep in the named barrier.
+// Wait for an mbarrier phase (TMA arrival or tcgen05.commit): every warp polls for itself, bounded; the block
+// reports GKA_ERR_TIMEOUT when it ends if a wait gave up.
 __device__ __forceinline__ void wait_bar(const Ctx &cx, int which, uint32_t parity) {
-    if (cx.tid < 32 && !aborted(cx)) {
-        if (!mbar_spin_bounded(cx.bars + 8 * which, parity)) {   // the block reports GKA_ERR_TIMEOUT when it ends
-            asm volatile("st.shared.b32 [%0], %1;" ::"r"(cx.abort_addr), "r"(1) : "memory");
-        }
+    if (!mbar_spin_bounded(cx.bars + 8 * which, parity))
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(cx.abort_addr), "r"(1) : "memory");
 #ifdef GKA_TC_TIMING
-        if (cx.tid == 0) TRACE(0, 20);
+    if (cx.tid == 0) TRACE(0, 20);
 #endif
-    }
-    cta_sync();
 }
-// Ask the issuer for a batch of MMAs.  Call after cta_sync: every thread's writes and fences are done.
-__device__ __forceinline__ void post(const Ctx &cx, int req) {
-    if (cx.tid == 0) {
-        *reinterpret_cast<volatile int *>(&cx.sc->req_op) = req;
-        mbar_arrive(cx.bars + 8 * BAR_REQ);
-    }
+// Block-wide barrier of the compute threads that also hands a batch of MMAs to the issuing warp: the issuer
+// sits in the same hardware barrier, so it wakes with the last arriving compute warp.  Every thread's
+// writes and fences for the batch come before the call.
+__device__ __forceinline__ void sync_post(const Ctx &cx, int req) {
+    if (cx.tid == 0) *reinterpret_cast<volatile int *>(&cx.sc->req_op) = req;
+    asm volatile("bar.sync 3, 544;" ::: "memory");
 }
 // byte offset of the 16-byte group holding columns 8 g .. 8 g + 7 (g = 0..15) of row r in a 128 x 128 operand
 __device__ __forceinline__ uint32_t tile_off(int r, int g) {
@@ -411,24 +408,19 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     if (tid >= CT) {
         // ================================ MMA issuing thread ================================
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssuer));
-        if (tid == CT + 64 && n_mine > 0) {
+        if ((tid >> 5) == (CT >> 5) + 2 && n_mine > 0) {     // one warp takes the requests; its lane 0 issues
             const uint32_t base14 = (smem_u32(smem) >> 4) & 0x3FFF;
-            uint32_t reqph = 0;
             for (;;) {
-                // a request normally arrives within microseconds; give up after seconds of silence
-                bool got = false;
-                for (int tries = 0; tries < 4 && !got; ++tries) got = mbar_spin_bounded(bars + 8 * BAR_REQ, reqph);
-                if (!got || s_abort != 0) {
-                    s_abort = 1;
-                    break;
-                }
-                reqph ^= 1u;
+                asm volatile("bar.sync 3, 544;" ::: "memory");   // the compute threads' sync_post
                 const int req = *reinterpret_cast<const volatile int *>(&sc->req_op);
-                TRACE(1, 32 + (req & 0xFF));
                 if ((req & 0xFF) == OP_EXIT) break;
-                fence_after();
-                issuer_run(req, base14, tmem, bars);
-                TRACE(1, 48 + (req & 0xFF));
+                if ((tid & 31) == 0) {
+                    TRACE(1, 32 + (req & 0xFF));
+                    fence_after();
+                    issuer_run(req, base14, tmem, bars);
+                    TRACE(1, 48 + (req & 0xFF));
+                }
+                __syncwarp();
             }
         }
     } else {
@@ -537,8 +529,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 }
                 fence_async_smem();
                 fence_before();
-                cta_sync();
-                post(cx, OP_FROB | (stage ? OPF_STAGE : 0));
+                sync_post(cx, OP_FROB | (stage ? OPF_STAGE : 0));
                 TSTAMP(3);
                 wait_bar(cx, BAR_A, ph_a);
                 ph_a ^= 1u;
@@ -613,7 +604,8 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     sc->s0[c] = 2.f / Lpm;
                     if (a.fro_out && valid) a.fro_out[ti.tok0 + (size_t)c * a.heads] = fc;
                 }
-                wait_bar(cx, BAR_V, 0u);       // q tile has landed (the wait also publishes the set-up values)
+                wait_bar(cx, BAR_V, 0u);       // q tile has landed
+                cta_sync();                    // the set-up values are published
             }
 
             // ======================= phase 2: Algorithm 1 on the whole tile =======================
@@ -641,12 +633,12 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                             make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
                 }
+                const int rq = (stage ? OPF_STAGE : 0) | (clamped ? OPF_PLAIN_K : 0);
                 fence_async_smem();
                 fence_before();
-                cta_sync();
+                sync_post(cx, (a.n_iter == 0 ? OP_ITER1_LAST : OP_ITER1) | rq);
                 TSTAMP(6);
 
-                const int rq = (stage ? OPF_STAGE : 0) | (clamped ? OPF_PLAIN_K : 0);
                 float omega = 2.f;
                 for (int it = 0; it <= a.n_iter; ++it) {       // + one extra score pass for the output
                     const bool last = (it == a.n_iter);
@@ -655,7 +647,6 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         asm volatile("" : "+r"(mm));
                         issue_tma(&tmV, f_lo + mm, OFF_V, BAR_V);
                     }
-                    post(cx, (last ? OP_ITER1_LAST : OP_ITER1) | rq);
                     // weight schedule and this token's coefficients, while the scores are computed
                     omega = 4.f / (4.f - rho2 * omega);
                     const float sigma = s0 * omega, beta = omega - 1.f;
@@ -667,10 +658,9 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     TSTAMP(7);
                     p_epilogue(cx, clamped || last, pf, acc_c);
                     fence_before();
-                    cta_sync();
+                    if (last) break;                            // the output stage's barrier covers P
+                    sync_post(cx, OP_ITER2 | rq);
                     TSTAMP(8);
-                    if (last) break;
-                    post(cx, OP_ITER2 | rq);
                     wait_bar(cx, BAR_B, ph_b);
                     ph_b ^= 1u;
                     fence_after();
@@ -701,7 +691,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     }
                     fence_async_smem();
                     fence_before();
-                    cta_sync();
+                    sync_post(cx, (it + 1 == a.n_iter ? OP_ITER1_LAST : OP_ITER1) | rq);
                     TSTAMP(10);
                 }
             }
@@ -718,7 +708,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 fence_async_smem();
                 fence_before();
                 wait_bar(cx, BAR_V, 1u);                       // V tile has landed
-                post(cx, OP_OUT | (stage ? OPF_STAGE : 0));
+                sync_post(cx, OP_OUT | (stage ? OPF_STAGE : 0));
                 TSTAMP(11);
                 wait_bar(cx, BAR_A, ph_a);
                 ph_a ^= 1u;
@@ -753,7 +743,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 m = ti.m_next;
             }
         }
-        if (n_mine > 0) post(cx, OP_EXIT);
+        if (n_mine > 0) sync_post(cx, OP_EXIT);
     }
 
 #ifdef GKA_TC_TIMING
