@@ -614,7 +614,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const float s0 = sc->s0[c], rho2 = sc->rho2[c], lamc = sc->lam[c], ztc = sc->zt[c], acc_c = sc->ac[c];
                 const unsigned char *qrow = smem + OFF_V;      // q tile: this thread reads row c, its 4 groups of 8 channels
                 uint64_t x2[16];   // the iterate (fp32 pairs), scaled by zt_c (the recurrence is linear), as the operand needs it
-                uint64_t d2[16];   // x_i - x_{i-1} (fp32 pairs)
+                uint64_t xp2[16];  // the previous iterate (the arrays swap roles every iteration)
                 {
                     const float x0s = valid ? s0 * ztc : 0.f;  // tokens past the tile stay zero
 #pragma unroll
@@ -626,7 +626,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         for (int u = 0; u < 4; ++u) {
                             const float xa = x0s * bf16_lo(qq[u]), xb = x0s * bf16_hi(qq[u]);
                             x2[4 * ch + u] = f2_pack(xa, xb);
-                            d2[4 * ch + u] = x2[4 * ch + u];     // x_{-1} = 0 (Algorithm 1): the first difference is x_0
+                            xp2[4 * ch + u] = 0ull;              // x_{-1} = 0 (Algorithm 1)
                             pk[u] = pack_bf16(xa, xb);
                         }
                         *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + ch)) =
@@ -651,7 +651,8 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     omega = 4.f / (4.f - rho2 * omega);
                     const float sigma = s0 * omega, beta = omega - 1.f;
                     const float cfx = valid ? sigma * ztc : 0.f, cfz = sigma * lamc;
-                    const uint64_t cfx2 = f2_pack(cfx, cfx), ncfz2 = f2_pack(-cfz, -cfz), beta2 = f2_pack(beta, beta);
+                    const float cfa = 1.f + beta - cfz;     // x_{i+1} = cfa x_i - beta x_{i-1} + cfx (q - H_c x_i)
+                    const uint64_t cfx2 = f2_pack(cfx, cfx), cfa2 = f2_pack(cfa, cfa), nbeta2 = f2_pack(-beta, -beta);
                     wait_bar(cx, BAR_A, ph_a);
                     ph_a ^= 1u;
                     fence_after();
@@ -665,30 +666,33 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     ph_b ^= 1u;
                     fence_after();
                     TSTAMP(9);
+                    // x_{i+1} = cfa x_i - beta x_{i-1} + cfx (q - H_c x_i) overwrites x_{i-1}: the two register arrays
+                    // swap roles every iteration (two copies of the code instead of 32 register moves)
+                    auto x_epilogue = [&](uint64_t(&cur)[16], uint64_t(&prv)[16]) {
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {        // 8 channels at a time keeps the transient registers few
-                        uint32_t r[8];
-                        TMEM_LD8(tmem + TM_Y + cx.lane_addr + 32 * cq + 8 * ch, r);
-                        const uint4 qv = *reinterpret_cast<const uint4 *>(qrow + tile_off(c, 4 * cq + ch));
-                        const uint32_t *qq = reinterpret_cast<const uint32_t *>(&qv);
-                        tmem_wait_ld();
-                        uint32_t pk[4];
+                        for (int ch = 0; ch < 4; ++ch) {    // 8 channels at a time keeps the transient registers few
+                            uint32_t r[8];
+                            TMEM_LD8(tmem + TM_Y + cx.lane_addr + 32 * cq + 8 * ch, r);
+                            const uint4 qv = *reinterpret_cast<const uint4 *>(qrow + tile_off(c, 4 * cq + ch));
+                            const uint32_t *qq = reinterpret_cast<const uint32_t *>(&qv);
+                            tmem_wait_ld();
+                            uint32_t pk[4];
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int i = 4 * ch + u;
-                            // x_{i+1} - x_i = beta (x_i - x_{i-1}) + sigma (q - A x_i), with the lambda part of A explicit
-                            const uint64_t t2 = f2_sub(f2_pack(bf16_lo(qq[u]), bf16_hi(qq[u])),
-                                                       f2_pack(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1])));
-                            const uint64_t dn = f2_fma(cfx2, t2, f2_fma(beta2, d2[i], f2_mul(ncfz2, x2[i])));
-                            d2[i] = dn;
-                            x2[i] = f2_add(x2[i], dn);
-                            float xa, xb;
-                            f2_unpack(x2[i], xa, xb);
-                            pk[u] = pack_bf16(xa, xb);
+                            for (int u = 0; u < 4; ++u) {
+                                const int i = 4 * ch + u;
+                                const uint64_t t2 = f2_sub(f2_pack(bf16_lo(qq[u]), bf16_hi(qq[u])),
+                                                           f2_pack(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1])));
+                                prv[i] = f2_fma(cfx2, t2, f2_fma(cfa2, cur[i], f2_mul(nbeta2, prv[i])));
+                                float xa, xb;
+                                f2_unpack(prv[i], xa, xb);
+                                pk[u] = pack_bf16(xa, xb);
+                            }
+                            *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + ch)) =
+                                make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
-                        *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + ch)) =
-                            make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    }
+                    };
+                    if (it & 1) x_epilogue(xp2, x2);
+                    else x_epilogue(x2, xp2);
                     fence_async_smem();
                     fence_before();
                     sync_post(cx, (it + 1 == a.n_iter ? OP_ITER1_LAST : OP_ITER1) | rq);
