@@ -60,13 +60,14 @@ struct TileScalars {
     float lam[NT];         // lambda_c (after the adaptive rule, if any)
     float s0[NT];          // 2 / (L + mu)
     float rho2[NT];
+    __align__(16) float iz[NT];   // 2^-G2_c (tiles that are not clamped)
     float part[2][4][NT];  // Frobenius partial sums: [k H_0 k | Gram part][column quarter][key]
     float carry[2][2][4];  // per-warp totals (a, b) of the two scans
     float red[16];         // per-warp sums of squares of H_0
     int req_op;            // request to the MMA issuer
     int stop;              // block-wide copy of the abort flag, taken between tiles
 };
-constexpr uint32_t SC_BYTES = 8192;
+constexpr uint32_t SC_BYTES = 9216;
 static_assert(sizeof(TileScalars) <= SC_BYTES, "scalar block too large");
 constexpr uint32_t TILE_SMEM = OFF_SC + SC_BYTES + 1024;   // + slack for the 1024-byte alignment of the base
 
@@ -271,9 +272,10 @@ __device__ __forceinline__ void master_store(const Ctx &cx, uint32_t tm_master, 
 
 // Masked score epilogue: S (TMEM, fp32) -> P (packed bf16 pairs, written over the first 16 of this thread's own
 // 32 score columns).  Keys j = 32 cq + i, token c = 32 q + l: blocks above the diagonal are zero, blocks below
-// it need no mask.  GENERAL: per-element factor 2^(ac_c - G_j) (strongly decaying tiles, and the pass whose P
-// multiplies the unweighted V); otherwise the tile-wide constant pf.
-template <bool GENERAL, bool DIAG>
+// it need no mask.  The factor is the tile-wide constant pf, or per key (strongly decaying tiles, and the pass
+// whose P multiplies the unweighted V).
+enum { PF_CONST = 0, PF_TABLE = 1, PF_EXACT = 2 };   // tile-wide constant | 2^-G_j from the table | 2^(ac_c - G_j) per element
+template <int MODE, bool DIAG>
 __device__ __forceinline__ void p_block(const Ctx &cx, uint32_t taddr, float pf, float ac_c) {
     const uint64_t pf2 = f2_pack(pf, pf);
 #pragma unroll
@@ -285,9 +287,13 @@ __device__ __forceinline__ void p_block(const Ctx &cx, uint32_t taddr, float pf,
         for (int u = 0; u < 8; ++u) {
             const int i0 = 16 * piece + 2 * u;
             uint64_t f2 = pf2;
-            if (GENERAL)
+            if (MODE == PF_TABLE) {
+                const float2 z = *reinterpret_cast<const float2 *>(&cx.sc->iz[32 * cx.cq + i0]);
+                f2 = f2_pack(z.x, z.y);
+            } else if (MODE == PF_EXACT) {
                 f2 = f2_pack(ex2_fast(fminf(ac_c - cx.sc->G2[32 * cx.cq + i0], 126.f)),
                              ex2_fast(fminf(ac_c - cx.sc->G2[32 * cx.cq + i0 + 1], 126.f)));
+            }
             float p0, p1;
             f2_unpack(f2_mul(f2_pack(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1])), f2), p0, p1);
             if (DIAG) {                     // keys i <= l are visible
@@ -299,7 +305,7 @@ __device__ __forceinline__ void p_block(const Ctx &cx, uint32_t taddr, float pf,
         TMEM_ST8(taddr + 8 * piece, pk);
     }
 }
-__device__ __forceinline__ void p_epilogue(const Ctx &cx, bool general, float pf, float ac_c) {
+__device__ __forceinline__ void p_epilogue(const Ctx &cx, int mode, float pf, float ac_c) {
     const uint32_t taddr = cx.tmem + TM_S + cx.lane_addr + 32 * cx.cq;
     if (cx.cq > cx.q) {
         uint32_t z[8];
@@ -308,11 +314,13 @@ __device__ __forceinline__ void p_epilogue(const Ctx &cx, bool general, float pf
         TMEM_ST8(taddr, z);
         TMEM_ST8(taddr + 8, z);
     } else if (cx.cq == cx.q) {
-        if (general) p_block<true, true>(cx, taddr, pf, ac_c);
-        else p_block<false, true>(cx, taddr, pf, ac_c);
+        if (mode == PF_CONST) p_block<PF_CONST, true>(cx, taddr, pf, ac_c);
+        else if (mode == PF_TABLE) p_block<PF_TABLE, true>(cx, taddr, pf, ac_c);
+        else p_block<PF_EXACT, true>(cx, taddr, pf, ac_c);
     } else {
-        if (general) p_block<true, false>(cx, taddr, pf, ac_c);
-        else p_block<false, false>(cx, taddr, pf, ac_c);
+        if (mode == PF_CONST) p_block<PF_CONST, false>(cx, taddr, pf, ac_c);
+        else if (mode == PF_TABLE) p_block<PF_TABLE, false>(cx, taddr, pf, ac_c);
+        else p_block<PF_EXACT, false>(cx, taddr, pf, ac_c);
     }
     tmem_wait_st();
 }
@@ -495,6 +503,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     sc->G2[c] = G2c;
                     sc->ac[c] = G2c - mc;
                     sc->zt[c] = exp2f(mc);
+                    sc->iz[c] = exp2f(-mc);
                     sc->lam[c] = lamv;
                 }
                 cta_sync();
@@ -560,20 +569,38 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     if (cq <= cx.q) {
                         const float G2j = sc->G2[c];
                         const int lim = (cq == cx.q) ? l : 32;   // keys i < lim come earlier, i == lim is the key itself
+                        float gd = 0.f;                          // the key's own squared norm
+                        uint64_t acc2 = 0ull;
 #pragma unroll
                         for (int piece = 0; piece < 2; ++piece) {
                             uint32_t r[16];
                             TMEM_LD16(tmem + TM_S + cx.lane_addr + 32 * cq + 16 * piece, r);
                             tmem_wait_ld();
+                            if (!clamped) {         // sum_i g_i^2 2^-G_i over the earlier keys, times 2 2^G_j afterwards
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const int ii = 16 * piece + i;
-                                const float g = __uint_as_float(r[i]);
-                                const float g2 = g * g;
-                                if (ii < lim) gs = fmaf(2.f * ex2_fast(G2j - sc->G2[32 * cq + ii]), g2, gs);
-                                else if (ii == lim) gs += g2;
+                                for (int u = 0; u < 8; ++u) {
+                                    const int ii = 16 * piece + 2 * u;
+                                    const float g0 = __uint_as_float(r[2 * u]), g1 = __uint_as_float(r[2 * u + 1]);
+                                    if (ii == lim) gd = g0 * g0;
+                                    if (ii + 1 == lim) gd = g1 * g1;
+                                    const uint64_t gg = f2_pack(ii < lim ? g0 : 0.f, ii + 1 < lim ? g1 : 0.f);
+                                    const float2 z = *reinterpret_cast<const float2 *>(&sc->iz[32 * cq + ii]);
+                                    acc2 = f2_fma(f2_mul(gg, gg), f2_pack(z.x, z.y), acc2);
+                                }
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) {
+                                    const int ii = 16 * piece + i;
+                                    const float g = __uint_as_float(r[i]);
+                                    const float g2 = g * g;
+                                    if (ii < lim) gs = fmaf(2.f * ex2_fast(G2j - sc->G2[32 * cq + ii]), g2, gs);
+                                    else if (ii == lim) gd = g2;
+                                }
                             }
                         }
+                        float a0, a1;
+                        f2_unpack(acc2, a0, a1);
+                        gs = fmaf(2.f * ex2_fast(G2j), a0 + a1, gs) + gd;
                     }
                     sc->part[0][cq][c] = kh;
                     sc->part[1][cq][c] = gs;
@@ -640,13 +667,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 TSTAMP(6);
 
                 float omega = 2.f;
-                for (int it = 0; it <= a.n_iter; ++it) {       // + one extra score pass for the output
-                    const bool last = (it == a.n_iter);
-                    if (last && tid == 0) {                     // q is no longer needed: its buffer takes the V tile
-                        int mm = m;
-                        asm volatile("" : "+r"(mm));
-                        issue_tma(&tmV, f_lo + mm, OFF_V, BAR_V);
-                    }
+                for (int it = 0; it < a.n_iter; ++it) {
                     // weight schedule and this token's coefficients, while the scores are computed
                     omega = 4.f / (4.f - rho2 * omega);
                     const float sigma = s0 * omega, beta = omega - 1.f;
@@ -657,9 +678,8 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     ph_a ^= 1u;
                     fence_after();
                     TSTAMP(7);
-                    p_epilogue(cx, clamped || last, pf, acc_c);
+                    p_epilogue(cx, clamped ? PF_EXACT : PF_CONST, pf, acc_c);
                     fence_before();
-                    if (last) break;                            // the output stage's barrier covers P
                     sync_post(cx, OP_ITER2 | rq);
                     TSTAMP(8);
                     wait_bar(cx, BAR_B, ph_b);
@@ -700,17 +720,25 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 }
             }
 
-            // ======================= phase 3: output, U advance =======================
+            // ======================= phase 3: last score pass, output, U advance =======================
             {
                 int mm = m;
                 asm volatile("" : "+r"(mm));                   // recompute the tile's description
                 const TileInfo ti = tile_info(a, item, f_lo, n_mine, mm);
-                const float decay = exp2f(sc->G2[ti.ntok - 1]);
-                // U master pass (bf16 copy into the H buffer, scale), O = X' U_0^T + P V, U advance
+                // q is no longer needed: its buffer takes the V tile
+                if (tid == 0) issue_tma(&tmV, ti.f, OFF_V, BAR_V);
+                // while the scores of the final iterate are computed: U master pass (bf16 copy into the H buffer, which
+                // no pending product reads; scale by the tile's decay)
                 master_pass<false>(cx, tmem + TM_U, ti.run_start,
-                                   ti.init_src ? ti.init_src + (size_t)D * D + (size_t)c * D : nullptr, decay);
+                                   ti.init_src ? ti.init_src + (size_t)D * D + (size_t)c * D : nullptr,
+                                   exp2f(sc->G2[ti.ntok - 1]));
                 fence_async_smem();
+                wait_bar(cx, BAR_A, ph_a);
+                ph_a ^= 1u;
+                fence_after();
+                p_epilogue(cx, clamped ? PF_EXACT : PF_TABLE, pf, sc->ac[c]);   // this P multiplies the unweighted V
                 fence_before();
+                // O = X' U_0^T + P V (the H buffer holds U_0 since the last score pass), U advance
                 wait_bar(cx, BAR_V, 1u);                       // V tile has landed
                 sync_post(cx, OP_OUT | (stage ? OPF_STAGE : 0));
                 TSTAMP(11);
