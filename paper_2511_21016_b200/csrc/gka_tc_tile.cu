@@ -75,7 +75,7 @@ constexpr uint32_t TILE_SMEM = OFF_SC + SC_BYTES + 1024;   // + slack for the 10
 constexpr uint32_t TM_H = 0, TM_U = 128, TM_S = 256, TM_Y = 384;
 
 enum { BAR_K0 = 0, BAR_K1, BAR_V, BAR_A, BAR_B, BAR_COUNT };
-enum { OP_FROB = 1, OP_ITER1, OP_ITER1_LAST, OP_ITER2, OP_OUT, OP_EXIT };
+enum { OP_FROB = 1, OP_ITER1, OP_ITER1_LAST, OP_ITER2, OP_OUT, OP_EXIT, OP_GRAM };
 constexpr int OPF_STAGE = 1 << 8, OPF_PLAIN_K = 1 << 9;   // request flags: K stage; pair P with K instead of w o K
 
 // ---- operand descriptor constants relative to (shared base >> 4); k-steps of 16
@@ -144,10 +144,11 @@ __device__ __forceinline__ void issuer_run(int req, uint32_t base14, uint32_t tm
         if (req & OPF_PLAIN_K) mma8_pm<K_mn>(tm_Y, tm_S, kb, I_PM);
         else mma8_pm<Kw_mn>(tm_Y, tm_S, base14, I_PM);
         mma_commit(bars + 8 * BAR_B);
+    } else if (op == OP_GRAM) {
+        mma8_kk<0, K_k, K_k>(tm_S, kb, kb, I_KK);            // Gram matrix K K^T (completion is covered by OP_FROB's commit)
     } else if (op == OP_FROB) {
         mma8_mm<K_mn, Kw_mn>(tm_H, kb, base14, I_MM);        // H += K^T (w o K)
         mma8_kk<0, K_k, H_k>(tm_Y, kb, base14, I_KK);        // K H_0
-        mma8_kk<0, K_k, K_k>(tm_S, kb, kb, I_KK);            // Gram matrix K K^T
         mma_commit(bars + 8 * BAR_A);
     } else if (op == OP_OUT) {
         mma8_kk<0, X_k, H_k>(tm_Y, base14, base14, I_KK);    // X' U_0^T (the H buffer holds U_0 now)
@@ -379,7 +380,7 @@ __device__ __forceinline__ TileInfo tile_info(const FwdArgs &a, int item, long l
 
 __global__ void __launch_bounds__(kThreadsTile, 1)
 fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                const __grid_constant__ CUtensorMap tmQ, FwdArgs a) {
+                const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO, FwdArgs a) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t s_bars[BAR_COUNT];
     __shared__ uint32_t s_tmem_base;
@@ -448,7 +449,6 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         cx.abort_addr = smem_u32(&s_abort);
         const int c = cx.c, cq = cx.cq, l = cx.l;
         const uint32_t sbase = smem_u32(smem);
-        __nv_bfloat16 *gout = reinterpret_cast<__nv_bfloat16 *>(a.out);
         const size_t st = state_floats(D, D);
         const bool adaptive = (a.flags & GKA_FLAG_ADAPTIVE_LAMBDA) != 0;
         uint32_t ph_a = 0, ph_b = 0;
@@ -472,6 +472,17 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         };
 
         if (tid == 0 && n_mine > 0) issue_tma(&tmK, f_lo, OFF_K0, BAR_K0);
+        // gate and lambda of this thread's token (threads 0..127), fetched one tile ahead
+        float g_next = 1.f, lam_next = 1.f;
+        auto prefetch_gates = [&](int m_of_tile) {
+            if (tid < NT && m_of_tile < n_mine) {
+                const TileInfo tn = tile_info(a, item, f_lo, n_mine, m_of_tile);
+                const bool v = c < tn.ntok;
+                g_next = v ? ldg_stream_f32(a.gate + tn.tok0 + (size_t)c * a.heads) : 1.f;
+                lam_next = v ? ldg_stream_f32(a.lam + tn.tok0 + (size_t)c * a.heads) : 1.f;
+            }
+        };
+        prefetch_gates(0);
 
         int tile = 0;
         for (int m = 0; m < n_mine; ++tile) {       // m: index of the tile's first chunk inside the block's range
@@ -491,11 +502,13 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     if (ti.m_next < n_mine)
                         issue_tma(&tmK, f_lo + ti.m_next, stage ? OFF_K0 : OFF_K1, stage ? BAR_K0 : BAR_K1);
                 }
+                // ---- K tile has landed (it was fetched during the previous tile): Gram matrix under the set-up
+                wait_bar(cx, stage ? BAR_K1 : BAR_K0, (uint32_t)((tile >> 1) & 1));
+                sync_post(cx, OP_GRAM | (stage ? OPF_STAGE : 0));
 
                 // ---- gates: cumulative log2 decay by a scan over the tile (threads 0..127 own token c = tid)
                 if (tid < NT) {
-                    const float g = valid ? ldg_stream_f32(a.gate + ti.tok0 + (size_t)c * a.heads) : 1.f;
-                    const float lamv = valid ? ldg_stream_f32(a.lam + ti.tok0 + (size_t)c * a.heads) : 1.f;
+                    const float g = g_next, lamv = lam_next;
                     const float lgc = fmaxf(log2f(g), -115.f);
                     const float G2c = affine_scan(cx, 1.f, lgc, 0.f, 0);
                     const float mc = fmaxf(G2c, -60.f);
@@ -513,8 +526,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 pf = exp2f(-fmaxf(Glast, -60.f));             // Gamma[c][j] / zt_c = pf * w_j otherwise
                 const float decay = exp2f(Glast);             // zeta of the whole tile
 
-                // ---- K tile has landed; w o K (same swizzled positions as K), rows past the tile weigh nothing
-                wait_bar(cx, stage ? BAR_K1 : BAR_K0, (uint32_t)((tile >> 1) & 1));
+                // ---- w o K (same swizzled positions as K), rows past the tile weigh nothing
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int qi = tid + CT * i;               // 16-byte group index in the 32 KB tile
@@ -632,6 +644,8 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     if (a.fro_out && valid) a.fro_out[ti.tok0 + (size_t)c * a.heads] = fc;
                 }
                 wait_bar(cx, BAR_V, 0u);       // q tile has landed
+                // the previous tile's output stores have read the X' buffer, which x_0 is about to overwrite
+                if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 cta_sync();                    // the set-up values are published
             }
 
@@ -727,6 +741,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const TileInfo ti = tile_info(a, item, f_lo, n_mine, mm);
                 // q is no longer needed: its buffer takes the V tile
                 if (tid == 0) issue_tma(&tmV, ti.f, OFF_V, BAR_V);
+                prefetch_gates(ti.m_next);
                 // while the scores of the final iterate are computed: U master pass (bf16 copy into the H buffer, which
                 // no pending product reads; scale by the tile's decay)
                 master_pass<false>(cx, tmem + TM_U, ti.run_start,
@@ -746,21 +761,22 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 ph_a ^= 1u;
                 fence_after();
                 TSTAMP(12);
-                if (c < ti.ntok) {
-                    uint4 *dst = reinterpret_cast<uint4 *>(gout + (ti.tok0 + (size_t)c * a.heads) * D + 32 * cq);
+                // O as bf16 into the X' buffer (no product reads it any more), stored by TMA after the tile's last barrier
 #pragma unroll
-                    for (int piece = 0; piece < 2; ++piece) {
-                        uint32_t r[16];
-                        TMEM_LD16(tmem + TM_Y + cx.lane_addr + 32 * cq + 16 * piece, r);
-                        tmem_wait_ld();
-                        uint32_t pk[8];
+                for (int piece = 0; piece < 2; ++piece) {
+                    uint32_t r[16];
+                    TMEM_LD16(tmem + TM_Y + cx.lane_addr + 32 * cq + 16 * piece, r);
+                    tmem_wait_ld();
+                    uint32_t pk[8];
 #pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            pk[u] = pack_bf16(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1]));
-                        dst[2 * piece] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                        dst[2 * piece + 1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-                    }
+                    for (int u = 0; u < 8; ++u)
+                        pk[u] = pack_bf16(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1]));
+                    *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + 2 * piece)) =
+                        make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + 2 * piece + 1)) =
+                        make_uint4(pk[4], pk[5], pk[6], pk[7]);
                 }
+                fence_async_smem();
                 TSTAMP(13);
                 wait_bar(cx, BAR_B, ph_b);     // U advance done: every tensor-core read of this tile's buffers is done
                 ph_b ^= 1u;
@@ -771,11 +787,22 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (tid == 0) sc->stop = aborted(cx) ? 1 : 0;
                 cta_sync();
                 TSTAMP(14);
+                if (tid == 0) {               // one box of 64 tokens x 64 channels per chunk and channel half
+                    const int b = ti.seq / a.heads, h = ti.seq % a.heads;
+                    for (int hh = 0; hh < ti.ntok / kChunk; ++hh)
+                        for (int hf = 0; hf < 2; ++hf)
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::
+                                             "l"(reinterpret_cast<uint64_t>(&tmO)), "r"(h * D + 64 * hf),
+                                         "r"(b * a.T + (ti.n + hh) * kChunk), "r"(sbase + OFF_X + 16384 * hf + 8192 * hh)
+                                         : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
                 if (sc->stop) break;          // the same decision in every thread
                 m = ti.m_next;
             }
         }
         if (n_mine > 0) sync_post(cx, OP_EXIT);
+        if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");    // output stores are complete
     }
 
 #ifdef GKA_TC_TIMING
@@ -791,15 +818,15 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 }  // namespace
 
 cudaError_t launch_fwd_tile(const FwdArgs &a, cudaStream_t stream) {
-    alignas(64) CUtensorMap tmK, tmV, tmQ;
+    alignas(64) CUtensorMap tmK, tmV, tmQ, tmO;     // the output is stored chunk by chunk: boxes of 64 rows
     const int rows = a.B * a.T, cols = a.heads * D;
     if (!make_tile_map(&tmK, a.k, rows, cols, NT) || !make_tile_map(&tmV, a.v, rows, cols, NT) ||
-        !make_tile_map(&tmQ, a.q, rows, cols, NT))
+        !make_tile_map(&tmQ, a.q, rows, cols, NT) || !make_tile_map(&tmO, a.out, rows, cols, kChunk))
         return cudaErrorInvalidValue;
     cudaError_t err = cudaFuncSetAttribute(fwd_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TILE_SMEM);
     if (err != cudaSuccess) return err;
     if (a.ev_start) cudaEventRecord(a.ev_start, stream);
-    fwd_tile_kernel<<<a.plan.G, kThreadsTile, TILE_SMEM, stream>>>(tmK, tmV, tmQ, a);
+    fwd_tile_kernel<<<a.plan.G, kThreadsTile, TILE_SMEM, stream>>>(tmK, tmV, tmQ, tmO, a);
     if (a.ev_stop) cudaEventRecord(a.ev_stop, stream);
     return cudaGetLastError();
 }
