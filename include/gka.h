@@ -142,9 +142,11 @@ int gka_fwd_num_work_items(const gka_desc *desc, int chunk);
 /*
  * Introspection of the work decomposition (pure host arithmetic, no CUDA call): the flat list of
  * B*heads*(T/chunk) chunks is split into num_items contiguous ranges; item `item` owns chunks
- * [*first_chunk, *end_chunk).  *cut_in / *cut_out tell whether the range starts / ends inside a
- * sequence (then its start state comes from the cross-item scan / its last run is summarised).
- * Returns GKA_OK or an argument error.
+ * [*first_chunk, *end_chunk).  Range sizes differ by at most one chunk; when T/chunk is even and
+ * there are at least two chunks per item the boundaries are kept at even chunk offsets (the
+ * tensor-core kernel works on pairs of chunks) and sizes differ by at most two.  *cut_in / *cut_out
+ * tell whether the range starts / ends inside a sequence (then its start state comes from the
+ * cross-item scan / its last run is summarised).  Returns GKA_OK or an argument error.
  */
 gka_status gka_fwd_work_range(const gka_desc *desc, int chunk, int num_items, int item,
                               long long *first_chunk, long long *end_chunk, int *cut_in,

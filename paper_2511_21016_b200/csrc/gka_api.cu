@@ -102,11 +102,8 @@ gka_status gka_fwd_work_range(const gka_desc *desc, int chunk, int num_items, in
     if (s != GKA_OK) return s;
     if (!first_chunk || !end_chunk || !cut_in || !cut_out) return GKA_ERR_NULL;
     WorkPlan p;
-    p.BH = desc->B * desc->heads;
-    p.N = desc->T / chunk;
-    p.NC = (long long)p.BH * p.N;
+    p.set(desc->B * desc->heads, desc->T / chunk, num_items > 0 ? num_items : 1);
     if (num_items <= 0 || num_items > p.NC || item < 0 || item >= num_items) return GKA_ERR_SHAPE;
-    p.G = num_items;
     *first_chunk = p.lo(item);
     *end_chunk = p.lo(item + 1);
     *cut_in = p.cut_in(item) ? 1 : 0;
@@ -141,10 +138,7 @@ gka_status gka_fwd_chunked(const gka_desc *desc, const void *q, const void *k, c
     a.B = desc->B; a.T = desc->T; a.heads = desc->heads;
     a.n_iter = n_iter;
     a.flags = desc->flags;
-    a.plan.BH = desc->B * desc->heads;
-    a.plan.N = desc->T / chunk;
-    a.plan.NC = (long long)a.plan.BH * a.plan.N;
-    a.plan.G = G;
+    a.plan.set(desc->B * desc->heads, desc->T / chunk, G);
     a.ws = carve_workspace(desc->workspace, G, desc->d_k, desc->d_v);
     a.ev_start = reinterpret_cast<cudaEvent_t>(desc->profile_start);
     a.ev_stop = reinterpret_cast<cudaEvent_t>(desc->profile_stop);

@@ -20,13 +20,24 @@ constexpr int kMaxWorkItems = 296;    // upper bound on persistent work items (2
 // inside a sequence the item's last run is summarised (decay product, delta-H, delta-U) by the
 // summary kernel, a scan turns summaries into the start state of the next item, and the main
 // kernel then processes all items independently, carrying (H, U) on chip inside each run.
+// Range boundaries are multiples of `unit` chunks: 2 when every sequence has an even number of chunks
+// and there are at least two chunks per item (the tensor-core kernel pairs chunks into 128-token tiles;
+// even boundaries keep every run an even number of chunks long), else 1.
 // ---------------------------------------------------------------------------------------------
 struct WorkPlan {
     int BH;        // B * heads
     int N;         // chunks per sequence
     long long NC;  // total chunks
     int G;         // work items
-    __host__ __device__ long long lo(int i) const { return ((long long)i * NC) / G; }
+    int unit;      // granularity of the range boundaries in chunks (1 or 2)
+    __host__ __device__ long long lo(int i) const { return unit * (((long long)i * (NC / unit)) / G); }
+    __host__ __device__ void set(int bh, int n, int g) {
+        BH = bh;
+        N = n;
+        NC = (long long)bh * n;
+        G = g;
+        unit = (n % 2 == 0 && 2LL * g <= NC) ? 2 : 1;
+    }
     // start of the last run of item i (flat chunk index)
     __host__ __device__ long long last_run_start(int i) const {
         long long l = lo(i), h = lo(i + 1);
