@@ -49,6 +49,7 @@ gka_status check_fwd_shape(const gka_desc *d, int chunk) {
     if (s != GKA_OK) return s;
     if (chunk != kChunk) return chunk <= 0 ? GKA_ERR_SHAPE : GKA_ERR_UNSUPPORTED;
     if (d->T <= 0 || d->T % chunk != 0) return GKA_ERR_SHAPE;
+    if ((long long)d->B * d->heads * (d->T / chunk) >= (1LL << 31)) return GKA_ERR_UNSUPPORTED;   // 32-bit chunk indices
     return GKA_OK;
 }
 

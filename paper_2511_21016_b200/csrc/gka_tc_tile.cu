@@ -64,10 +64,11 @@ struct TileScalars {
     float part[2][4][NT];  // Frobenius partial sums: [k H_0 k | Gram part][column quarter][key]
     float carry[2][2][4];  // per-warp totals (a, b) of the two scans
     float red[16];         // per-warp sums of squares of H_0
+    float gpre[NT], lpre[NT];   // gate and lambda of the next tile, copied asynchronously a tile ahead
     int req_op;            // request to the MMA issuer
     int stop;              // block-wide copy of the abort flag, taken between tiles
 };
-constexpr uint32_t SC_BYTES = 9216;
+constexpr uint32_t SC_BYTES = 10240;
 static_assert(sizeof(TileScalars) <= SC_BYTES, "scalar block too large");
 constexpr uint32_t TILE_SMEM = OFF_SC + SC_BYTES + 1024;   // + slack for the 1024-byte alignment of the base
 
@@ -169,11 +170,21 @@ __shared__ int s_ttrace_n[2];
         if (blockIdx.x == 0 && s_ttrace_n[role] < 8192)                                                        \
             g_ttrace[role][s_ttrace_n[role]++] = (clock64() << 8) | (long long)(id);                           \
     } while (0)
+#if GKA_TC_TIMING == 2   /* light mode: no stamps inside the solve loop, none in waits or in the issuer */
+#define TSTAMP(k)                                                         \
+    do {                                                                  \
+        if (tid == 0 && (k) != 7 && (k) != 8 && (k) != 9 && (k) != 10) TRACE(0, k); \
+    } while (0)
+#define TRACE_HEAVY(role, id)
+#else
 #define TSTAMP(k)               \
     do {                        \
         if (tid == 0) TRACE(0, k); \
     } while (0)
+#define TRACE_HEAVY(role, id) TRACE(role, id)
+#endif
 #else
+#define TRACE_HEAVY(role, id)
 #define TRACE(role, id)
 #define TSTAMP(k)
 #endif
@@ -206,7 +217,7 @@ __device__ __forceinline__ void wait_bar(const Ctx &cx, int which, uint32_t pari
     if (!mbar_spin_bounded(cx.bars + 8 * which, parity))
         asm volatile("st.shared.b32 [%0], %1;" ::"r"(cx.abort_addr), "r"(1) : "memory");
 #ifdef GKA_TC_TIMING
-    if (cx.tid == 0) TRACE(0, 20);
+    if (cx.tid == 0) TRACE_HEAVY(0, 20);
 #endif
 }
 // Block-wide barrier of the compute threads that also hands a batch of MMAs to the issuing warp: the issuer
@@ -228,33 +239,37 @@ template <bool SUMSQ>
 __device__ __forceinline__ float master_pass(const Ctx &cx, uint32_t tm_master, bool from_global, const float *grow,
                                              float decay) {
     float ss = 0.f;
-    uint32_t r[32];
-    const uint32_t taddr = tm_master + cx.lane_addr + 32 * cx.cq;
-    if (!from_global) {
-        TMEM_LD32(taddr, r);
-        tmem_wait_ld();
-    } else {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            float4 v4 = grow ? ldg_stream_f32x4(grow + 32 * cx.cq + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
-            r[4 * i + 0] = __float_as_uint(v4.x); r[4 * i + 1] = __float_as_uint(v4.y);
-            r[4 * i + 2] = __float_as_uint(v4.z); r[4 * i + 3] = __float_as_uint(v4.w);
+    for (int piece = 0; piece < 2; ++piece) {       // 16 columns at a time keeps the transient registers few
+        uint32_t r[16];
+        const uint32_t taddr = tm_master + cx.lane_addr + 32 * cx.cq + 16 * piece;
+        if (!from_global) {
+            TMEM_LD16(taddr, r);
+            tmem_wait_ld();
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float4 v4 = grow ? ldg_stream_f32x4(grow + 32 * cx.cq + 16 * piece + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                r[4 * i + 0] = __float_as_uint(v4.x); r[4 * i + 1] = __float_as_uint(v4.y);
+                r[4 * i + 2] = __float_as_uint(v4.z); r[4 * i + 3] = __float_as_uint(v4.w);
+            }
         }
-    }
 #pragma unroll
-    for (int ch = 0; ch < 4; ++ch) {
-        uint32_t pk[4];
+        for (int ch = 0; ch < 2; ++ch) {
+            uint32_t pk[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const float v0 = __uint_as_float(r[8 * ch + 2 * u]), v1 = __uint_as_float(r[8 * ch + 2 * u + 1]);
-            if (SUMSQ) ss = fmaf(v0, v0, fmaf(v1, v1, ss));
-            pk[u] = pack_bf16(v0, v1);
+            for (int u = 0; u < 4; ++u) {
+                const float v0 = __uint_as_float(r[8 * ch + 2 * u]), v1 = __uint_as_float(r[8 * ch + 2 * u + 1]);
+                if (SUMSQ) ss = fmaf(v0, v0, fmaf(v1, v1, ss));
+                pk[u] = pack_bf16(v0, v1);
+            }
+            *reinterpret_cast<uint4 *>(cx.smem + OFF_H + tile_off(cx.c, 4 * cx.cq + 2 * piece + ch)) =
+                make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
-        *reinterpret_cast<uint4 *>(cx.smem + OFF_H + tile_off(cx.c, 4 * cx.cq + ch)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-    }
 #pragma unroll
-    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * decay);
-    TMEM_ST32(taddr, r);
+        for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * decay);
+        TMEM_ST16(taddr, r);
+    }
     tmem_wait_st();
     return ss;
 }
@@ -343,7 +358,13 @@ __device__ __forceinline__ float affine_scan(const Ctx &cx, float a, float b, fl
         ca[cx.q] = a;
         cb[cx.q] = b;
     }
+#ifdef GKA_TC_TIMING
+    if (cx.tid == 0) TRACE(0, 25);
+#endif
     asm volatile("bar.sync 2, 128;" ::: "memory");
+#ifdef GKA_TC_TIMING
+    if (cx.tid == 0) TRACE(0, 26);
+#endif
     float s = seed;
     for (int w = 0; w < cx.q; ++w) s = fmaf(ca[w], s, cb[w]);
     return fmaf(a, s, b);
@@ -362,8 +383,9 @@ __device__ __forceinline__ TileInfo tile_info(const FwdArgs &a, int item, long l
     const WorkPlan &P = a.plan;
     TileInfo t;
     t.f = f_lo + m;
-    t.seq = (int)(t.f / P.N);
-    t.n = (int)(t.f % P.N);
+    const unsigned fu = (unsigned)t.f;         // the chunk list is shorter than 2^31 (checked on the host)
+    t.seq = (int)(fu / (unsigned)P.N);
+    t.n = (int)(fu - (unsigned)t.seq * (unsigned)P.N);
     const int b = t.seq / a.heads, h = t.seq % a.heads;
     const bool two = (t.n + 1 < P.N) && (m + 1 < n_mine);
     t.ntok = two ? 2 * kChunk : kChunk;
@@ -424,10 +446,10 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const int req = *reinterpret_cast<const volatile int *>(&sc->req_op);
                 if ((req & 0xFF) == OP_EXIT) break;
                 if ((tid & 31) == 0) {
-                    TRACE(1, 32 + (req & 0xFF));
+                    TRACE_HEAVY(1, 32 + (req & 0xFF));
                     fence_after();
                     issuer_run(req, base14, tmem, bars);
-                    TRACE(1, 48 + (req & 0xFF));
+                    TRACE_HEAVY(1, 48 + (req & 0xFF));
                 }
                 __syncwarp();
             }
@@ -456,7 +478,8 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         // K (or V) tile of flat chunk f: 128 rows starting at the chunk's first token; rows past the tile's
         // tokens belong to later tokens (or are zero-filled past the tensor) and are never used
         auto issue_tma = [&](const CUtensorMap *map, long long f, uint32_t dst, int bar_idx) {
-            const int seq = (int)(f / P.N), n = (int)(f % P.N);
+            const unsigned fu = (unsigned)f;
+            const int seq = (int)(fu / (unsigned)P.N), n = (int)(fu - (unsigned)seq * (unsigned)P.N);
             const int b = seq / a.heads, h = seq % a.heads;
             const int y = b * a.T + n * kChunk;
             const uint32_t bar = bars + 8 * bar_idx;
@@ -473,13 +496,19 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
         if (tid == 0 && n_mine > 0) issue_tma(&tmK, f_lo, OFF_K0, BAR_K0);
         // gate and lambda of this thread's token (threads 0..127), fetched one tile ahead
-        float g_next = 1.f, lam_next = 1.f;
+        // gate and lambda of this thread's token (threads 0..127) travel global -> shared one tile ahead
         auto prefetch_gates = [&](int m_of_tile) {
             if (tid < NT && m_of_tile < n_mine) {
                 const TileInfo tn = tile_info(a, item, f_lo, n_mine, m_of_tile);
-                const bool v = c < tn.ntok;
-                g_next = v ? ldg_stream_f32(a.gate + tn.tok0 + (size_t)c * a.heads) : 1.f;
-                lam_next = v ? ldg_stream_f32(a.lam + tn.tok0 + (size_t)c * a.heads) : 1.f;
+                if (c < tn.ntok) {
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->gpre[c])),
+                                 "l"(a.gate + tn.tok0 + (size_t)c * a.heads) : "memory");
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->lpre[c])),
+                                 "l"(a.lam + tn.tok0 + (size_t)c * a.heads) : "memory");
+                } else {
+                    sc->gpre[c] = 1.f;
+                    sc->lpre[c] = 1.f;
+                }
             }
         };
         prefetch_gates(0);
@@ -502,15 +531,14 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     if (ti.m_next < n_mine)
                         issue_tma(&tmK, f_lo + ti.m_next, stage ? OFF_K0 : OFF_K1, stage ? BAR_K0 : BAR_K1);
                 }
-                // ---- K tile has landed (it was fetched during the previous tile): Gram matrix under the set-up
-                wait_bar(cx, stage ? BAR_K1 : BAR_K0, (uint32_t)((tile >> 1) & 1));
-                sync_post(cx, OP_GRAM | (stage ? OPF_STAGE : 0));
-
                 // ---- gates: cumulative log2 decay by a scan over the tile (threads 0..127 own token c = tid)
                 if (tid < NT) {
-                    const float g = g_next, lamv = lam_next;
+                    asm volatile("cp.async.wait_all;" ::: "memory");
+                    const float g = sc->gpre[c], lamv = sc->lpre[c];
+                    TSTAMP(21);
                     const float lgc = fmaxf(log2f(g), -115.f);
                     const float G2c = affine_scan(cx, 1.f, lgc, 0.f, 0);
+                    TSTAMP(22);
                     const float mc = fmaxf(G2c, -60.f);
                     sc->lg[c] = lgc;
                     sc->G2[c] = G2c;
@@ -518,8 +546,11 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     sc->zt[c] = exp2f(mc);
                     sc->iz[c] = exp2f(-mc);
                     sc->lam[c] = lamv;
+                    TSTAMP(23);
                 }
-                cta_sync();
+                // ---- K tile has landed (it was fetched during the previous tile): Gram matrix under the set-up
+                wait_bar(cx, stage ? BAR_K1 : BAR_K0, (uint32_t)((tile >> 1) & 1));
+                sync_post(cx, OP_GRAM | (stage ? OPF_STAGE : 0));     // also publishes the gate scalars
                 TSTAMP(0);
                 const float Glast = sc->G2[ntok - 1];
                 clamped = Glast < -60.f;                      // the tile decays below 2^-60: per-element factors
@@ -645,7 +676,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 }
                 wait_bar(cx, BAR_V, 0u);       // q tile has landed
                 // the previous tile's output stores have read the X' buffer, which x_0 is about to overwrite
-                if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                if (tid == 32) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 cta_sync();                    // the set-up values are published
             }
 
@@ -696,6 +727,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     fence_before();
                     sync_post(cx, OP_ITER2 | rq);
                     TSTAMP(8);
+
                     wait_bar(cx, BAR_B, ph_b);
                     ph_b ^= 1u;
                     fence_after();
@@ -735,6 +767,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
 
             // ======================= phase 3: last score pass, output, U advance =======================
+            TSTAMP(17);
             {
                 int mm = m;
                 asm volatile("" : "+r"(mm));                   // recompute the tile's description
@@ -751,8 +784,10 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 wait_bar(cx, BAR_A, ph_a);
                 ph_a ^= 1u;
                 fence_after();
+                TSTAMP(15);
                 p_epilogue(cx, clamped ? PF_EXACT : PF_TABLE, pf, sc->ac[c]);   // this P multiplies the unweighted V
                 fence_before();
+                TSTAMP(16);
                 // O = X' U_0^T + P V (the H buffer holds U_0 since the last score pass), U advance
                 wait_bar(cx, BAR_V, 1u);                       // V tile has landed
                 sync_post(cx, OP_OUT | (stage ? OPF_STAGE : 0));
@@ -787,7 +822,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (tid == 0) sc->stop = aborted(cx) ? 1 : 0;
                 cta_sync();
                 TSTAMP(14);
-                if (tid == 0) {               // one box of 64 tokens x 64 channels per chunk and channel half
+                if (tid == 32) {              // one box of 64 tokens x 64 channels per chunk and channel half
                     const int b = ti.seq / a.heads, h = ti.seq % a.heads;
                     for (int hh = 0; hh < ti.ntok / kChunk; ++hh)
                         for (int hf = 0; hf < 2; ++hf)
@@ -802,7 +837,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
         }
         if (n_mine > 0) sync_post(cx, OP_EXIT);
-        if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");    // output stores are complete
+        if (tid == 32) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // output stores are complete
     }
 
 #ifdef GKA_TC_TIMING
