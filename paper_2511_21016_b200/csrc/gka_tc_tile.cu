@@ -235,8 +235,18 @@ __device__ __forceinline__ uint32_t tile_off(int r, int g) {
 // One pass over a master (H or U) for this thread's row and 32 columns: source is TMEM, or global memory at
 // the start of a run.  Writes the bf16 operand copy, optionally accumulates the sum of squares, scales by the
 // tile's decay and stores the result back to TMEM.
+// Where a run's start state comes from: the caller's initial state of the sequence (or zero), carried through
+// the segment summaries (decay product, delta) of the work items j0 .. j1 - 1 that hold the earlier part of the
+// sequence: state <- decay_j * state + delta_j.  `off` selects the master (H or U) and this thread's row.
+struct StartSrc {
+    const float *state;      // caller's state of the sequence, or nullptr (zero)
+    const float *delta;      // summaries [item][st]
+    const float *decay;      // [item]
+    int j0, j1;
+    size_t st, off;
+};
 template <bool SUMSQ>
-__device__ __forceinline__ float master_pass(const Ctx &cx, uint32_t tm_master, bool from_global, const float *grow,
+__device__ __forceinline__ float master_pass(const Ctx &cx, uint32_t tm_master, bool from_global, const StartSrc &src,
                                              float decay) {
     float ss = 0.f;
 #pragma unroll
@@ -247,11 +257,26 @@ __device__ __forceinline__ float master_pass(const Ctx &cx, uint32_t tm_master, 
             TMEM_LD16(taddr, r);
             tmem_wait_ld();
         } else {
+            const size_t e = src.off + 32 * cx.cq + 16 * piece;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                float4 v4 = grow ? ldg_stream_f32x4(grow + 32 * cx.cq + 16 * piece + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 v4 = src.state ? ldg_stream_f32x4(src.state + e + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
                 r[4 * i + 0] = __float_as_uint(v4.x); r[4 * i + 1] = __float_as_uint(v4.y);
                 r[4 * i + 2] = __float_as_uint(v4.z); r[4 * i + 3] = __float_as_uint(v4.w);
+            }
+            for (int j = src.j0; j < src.j1; ++j) {
+                const float dj = __ldg(src.decay + j);
+                float4 dd[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) dd[i] = __ldg(reinterpret_cast<const float4 *>(src.delta + (size_t)j * src.st + e) + i);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float4 d4 = dd[i];
+                    r[4 * i + 0] = __float_as_uint(fmaf(dj, __uint_as_float(r[4 * i + 0]), d4.x));
+                    r[4 * i + 1] = __float_as_uint(fmaf(dj, __uint_as_float(r[4 * i + 1]), d4.y));
+                    r[4 * i + 2] = __float_as_uint(fmaf(dj, __uint_as_float(r[4 * i + 2]), d4.z));
+                    r[4 * i + 3] = __float_as_uint(fmaf(dj, __uint_as_float(r[4 * i + 3]), d4.w));
+                }
             }
         }
 #pragma unroll
@@ -377,7 +402,8 @@ struct TileInfo {
     bool run_start, seq_end;
     size_t tok0;
     long long f;
-    const float *init_src;     // where a run's start state comes from (nullptr = zero)
+    const float *seq_state;    // caller's initial state of the tile's sequence, or nullptr
+    bool chained;              // the run starts inside a sequence: its start state comes through the summaries
 };
 __device__ __forceinline__ TileInfo tile_info(const FwdArgs &a, int item, long long f_lo, int n_mine, int m) {
     const WorkPlan &P = a.plan;
@@ -393,10 +419,8 @@ __device__ __forceinline__ TileInfo tile_info(const FwdArgs &a, int item, long l
     t.tok0 = ((size_t)b * a.T + (size_t)t.n * kChunk) * a.heads + h;
     t.run_start = (m == 0) || (t.n == 0);
     t.seq_end = (t.n + (two ? 2 : 1) == P.N);
-    t.init_src = nullptr;
-    const size_t st = state_floats(D, D);
-    if (t.run_start) t.init_src = (t.n == 0) ? (a.state_in ? a.state_in + (size_t)t.seq * st : nullptr)
-                                             : a.ws.start + (size_t)item * st;
+    t.seq_state = a.state_in ? a.state_in + (size_t)t.seq * state_floats(D, D) : nullptr;
+    t.chained = t.run_start && t.n != 0;
     return t;
 }
 
@@ -474,6 +498,14 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const size_t st = state_floats(D, D);
         const bool adaptive = (a.flags & GKA_FLAG_ADAPTIVE_LAMBDA) != 0;
         uint32_t ph_a = 0, ph_b = 0;
+        // first item of the chain of summaries behind this block's start state: the one whose range holds the
+        // start of the sequence (its last run begins there, whatever sequence the item itself started in)
+        int chain_j0 = item;
+        if (n_mine > 0 && P.cut_in(item)) {
+            const long long seq_start = (f_lo / P.N) * P.N;
+            chain_j0 = item - 1;
+            while (P.lo(chain_j0) > seq_start) --chain_j0;
+        }
 
         // K (or V) tile of flat chunk f: 128 rows starting at the chunk's first token; rows past the tile's
         // tokens belong to later tokens (or are zero-filled past the tensor) and are never used
@@ -573,8 +605,9 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
                 // ---- H master, one pass: ||H_0||^2, bf16 copy, scale by the tile's decay
                 {
-                    float hs = master_pass<true>(cx, tmem + TM_H, ti.run_start,
-                                                 ti.init_src ? ti.init_src + (size_t)c * D : nullptr, decay);
+                    const StartSrc src = {ti.seq_state, a.ws.delta, a.ws.decay, ti.chained ? chain_j0 : 0,
+                                          ti.chained ? item : 0, st, (size_t)c * D};
+                    float hs = master_pass<true>(cx, tmem + TM_H, ti.run_start, src, decay);
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) hs += __shfl_xor_sync(0xffffffffu, hs, o);
                     if (l == 0) sc->red[tid >> 5] = hs;
@@ -777,9 +810,9 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 prefetch_gates(ti.m_next);
                 // while the scores of the final iterate are computed: U master pass (bf16 copy into the H buffer, which
                 // no pending product reads; scale by the tile's decay)
-                master_pass<false>(cx, tmem + TM_U, ti.run_start,
-                                   ti.init_src ? ti.init_src + (size_t)D * D + (size_t)c * D : nullptr,
-                                   exp2f(sc->G2[ti.ntok - 1]));
+                const StartSrc src = {ti.seq_state, a.ws.delta, a.ws.decay, ti.chained ? chain_j0 : 0,
+                                      ti.chained ? item : 0, st, (size_t)D * D + (size_t)c * D};
+                master_pass<false>(cx, tmem + TM_U, ti.run_start, src, exp2f(sc->G2[ti.ntok - 1]));
                 fence_async_smem();
                 wait_bar(cx, BAR_A, ph_a);
                 ph_a ^= 1u;
