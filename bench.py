@@ -38,9 +38,9 @@ L2_FLUSH_BYTES = 256 << 20
 
 # DRAM traffic per launch of the dominant kernels (dram__bytes_read.sum + dram__bytes_write.sum from the
 # ncu captures summarised under profiles/).  Both captures ran a quarter/half-size case of the same kernel
-# (forward: 2048 of 4096 chunks, 136.61 MB; decode: 2048 of 8192 (sequence, head) pairs, 480.67 MB) and
+# (forward: 2048 of 4096 chunks, 134.20 MB; decode: 2048 of 8192 (sequence, head) pairs, 480.67 MB) and
 # are scaled by the units per launch; traffic is proportional to the units in both kernels.
-NCU_TRAFFIC_BYTES = {"fwd_main": 2 * 136_612_608, "decode": 4 * 480_674_816}
+NCU_TRAFFIC_BYTES = {"fwd_main": 2 * 134_204_672, "decode": 4 * 480_674_816}
 
 
 def fwd_flops(n_chunks: int, n_iter: int, C: int = 64, D: int = 128) -> float:
@@ -315,7 +315,7 @@ def run_ours(args):
     work_items = gka.gka_fwd_num_work_items(cfg.B, cfg.T, cfg.heads, cfg.d)
     any_cut = any(gka.gka_fwd_work_range(cfg.B, cfg.T, cfg.heads, cfg.d, work_items, i)[3]
                   for i in range(work_items))
-    launches_per_step = 3 if any_cut else 1     # segment summaries + scan + main kernel, or the main kernel alone
+    launches_per_step = 2 if any_cut else 1     # segment summaries + main kernel, or the main kernel alone
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
