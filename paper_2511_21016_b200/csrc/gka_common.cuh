@@ -18,8 +18,10 @@ constexpr int kMaxWorkItems = 296;    // upper bound on persistent work items (2
 // NC = B*heads*N chunks; work item i of G owns the contiguous range [lo(i), lo(i+1)).  A range
 // may cover several sequences and may cut a sequence in the middle.  Where an item's range ends
 // inside a sequence the item's last run is summarised (decay product, delta-H, delta-U) by the
-// summary kernel, a scan turns summaries into the start state of the next item, and the main
-// kernel then processes all items independently, carrying (H, U) on chip inside each run.
+// summary kernel, the summaries of the items that hold the earlier part of a sequence are folded into
+// the start state of the next item (by a scan kernel on the fp32 path, by the main kernel itself on the
+// tensor-core path), and the main kernel then processes all items independently, carrying (H, U) on
+// chip inside each run.
 // Range boundaries are multiples of `unit` chunks: 2 when every sequence has an even number of chunks
 // and there are at least two chunks per item (the tensor-core kernel pairs chunks into 128-token tiles;
 // even boundaries keep every run an even number of chunks long), else 1.
