@@ -100,6 +100,19 @@ gka_status gka_fwd_chunked(const gka_desc *desc, const void *q, const void *k, c
                            void *out, float *state_out);
 
 /*
+ * The solve alone, chunk-wise: x_out[b,t,h,:] = CH(H_t + lambda_t I, rhs_t, n_iter) with H_t, lambda_t and the
+ * bounds L, mu as in gka_fwd_chunked (Algorithm 1; H_t from k and gate only).  With rhs = q it returns the
+ * iterate x_t that gka_fwd_chunked multiplies by U_t; with rhs = dL/dx_t it returns dL/dq_t, the first
+ * step of the backward pass: the fixed-iteration Chebyshev map is linear in its right-hand side and
+ * self-adjoint, so the gradient is the same solve with a different right-hand side (Section 4.3,
+ * implicit differentiation, Lemma 2).  rhs, k, x_out : [B, T, heads, d_k] (d_v is ignored and must
+ * equal d_k in the descriptor); gate, lam : [B, T, heads].  Same dtype rules, workspace, state_in (H part
+ * used), flags and error behaviour as gka_fwd_chunked; no state is written.
+ */
+gka_status gka_solve_chunked(const gka_desc *desc, const void *rhs, const void *k, const float *gate,
+                             const float *lam, int n_iter, int chunk, void *x_out);
+
+/*
  * Recurrent single-token step (eq. (CH) applied once): state is read, decayed by gate, updated
  * with k k^T / v k^T and written back in place; out[B,heads,d_v] = U_t CH(H_t + lambda_t I, q_t).
  * q, k : [B, heads, d_k]; v, out : [B, heads, d_v]; gate, lam : [B, heads].  Needs no workspace.

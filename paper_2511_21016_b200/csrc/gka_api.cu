@@ -112,9 +112,9 @@ gka_status gka_fwd_work_range(const gka_desc *desc, int chunk, int num_items, in
     return GKA_OK;
 }
 
-gka_status gka_fwd_chunked(const gka_desc *desc, const void *q, const void *k, const void *v,
+static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, const void *v,
                            const float *gate, const float *lam, int n_iter, int chunk, void *out,
-                           float *state_out) {
+                           float *state_out, bool solve_only) {
     gka_status s = check_fwd_shape(desc, chunk);
     if (s != GKA_OK) return s;
     if (!q || !k || !v || !gate || !lam || !out) return GKA_ERR_NULL;
@@ -139,6 +139,7 @@ gka_status gka_fwd_chunked(const gka_desc *desc, const void *q, const void *k, c
     a.B = desc->B; a.T = desc->T; a.heads = desc->heads;
     a.n_iter = n_iter;
     a.flags = desc->flags;
+    a.solve_only = solve_only ? 1 : 0;
     a.plan.set(desc->B * desc->heads, desc->T / chunk, G);
     a.ws = carve_workspace(desc->workspace, G, desc->d_k, desc->d_v);
     a.ev_start = reinterpret_cast<cudaEvent_t>(desc->profile_start);
@@ -153,6 +154,19 @@ gka_status gka_fwd_chunked(const gka_desc *desc, const void *q, const void *k, c
     else
         err = launch_fwd_simt(a, desc->d_k, desc->io_dtype, stream);
     return cuda_result(err, tensor_path ? "gka_fwd_chunked (tensor-core path)" : "gka_fwd_chunked (fp32 path)");
+}
+
+gka_status gka_fwd_chunked(const gka_desc *desc, const void *q, const void *k, const void *v,
+                           const float *gate, const float *lam, int n_iter, int chunk, void *out,
+                           float *state_out) {
+    return fwd_impl(desc, q, k, v, gate, lam, n_iter, chunk, out, state_out, false);
+}
+
+gka_status gka_solve_chunked(const gka_desc *desc, const void *rhs, const void *k, const float *gate,
+                             const float *lam, int n_iter, int chunk, void *x_out) {
+    if (desc && desc->d_k != desc->d_v) return GKA_ERR_SHAPE;
+    // the value stream plays no part in the solve: the key tensor stands in for it
+    return fwd_impl(desc, rhs, k, k, gate, lam, n_iter, chunk, x_out, nullptr, true);
 }
 
 gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, const void *k,

@@ -154,6 +154,7 @@ struct FwdArgs {
     int B, T, heads;
     int n_iter;
     unsigned flags;
+    int solve_only;        // write the solve x_t = CH(H_t + lambda_t I, q_t, r) itself instead of U_t x_t (v unused)
     WorkPlan plan;
     Workspace ws;
     cudaEvent_t ev_start, ev_stop;   // optional, recorded around the main kernel (host side only)

@@ -438,6 +438,16 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
             __syncthreads();
         }
 
+        if (a.solve_only) {      // the solve itself is the result (Section 4.3: the same solve gives dq from dx)
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int c = 4 * tc + t;
+#pragma unroll
+                for (int g = 0; g < DG; ++g)
+                    Io<IoT>::store4(gout + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td,
+                                    make_float4(xm[t][4 * g + 0], xm[t][4 * g + 1], xm[t][4 * g + 2], xm[t][4 * g + 3]));
+            }
+        }
         // ---- output O = zeta o (X U_0^T) + P V
         masked_scores();
         for (int idx = tid; idx < D * (D / 4); idx += kThreads) {   // sH <- U_0^T
@@ -462,7 +472,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
                 for (int u = 0; u < NCH; ++u) acc[t][u] *= zet[t];
             gemm_tok_mat<D>(acc, sPt, sV, kChunk, tc, td);
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
+            for (int t = 0; t < 4 && !a.solve_only; ++t) {
                 const int c = 4 * tc + t;
 #pragma unroll
                 for (int g = 0; g < DG; ++g)

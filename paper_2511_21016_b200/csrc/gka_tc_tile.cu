@@ -76,7 +76,7 @@ constexpr uint32_t TILE_SMEM = OFF_SC + SC_BYTES + 1024;   // + slack for the 10
 constexpr uint32_t TM_H = 0, TM_U = 128, TM_S = 256, TM_Y = 384;
 
 enum { BAR_K0 = 0, BAR_K1, BAR_V, BAR_A, BAR_B, BAR_COUNT };
-enum { OP_FROB = 1, OP_ITER1, OP_ITER1_LAST, OP_ITER2, OP_OUT, OP_EXIT, OP_GRAM };
+enum { OP_FROB = 1, OP_ITER1, OP_ITER1_LAST, OP_ITER2, OP_OUT, OP_EXIT, OP_GRAM, OP_NONE };
 constexpr int OPF_STAGE = 1 << 8, OPF_PLAIN_K = 1 << 9;   // request flags: K stage; pair P with K instead of w o K
 
 // ---- operand descriptor constants relative to (shared base >> 4); k-steps of 16
@@ -497,6 +497,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const uint32_t sbase = smem_u32(smem);
         const size_t st = state_floats(D, D);
         const bool adaptive = (a.flags & GKA_FLAG_ADAPTIVE_LAMBDA) != 0;
+        const bool solve_only = a.solve_only != 0;      // the result is the solve itself: no V, no U, no output product
         uint32_t ph_a = 0, ph_b = 0;
         // first item of the chain of summaries behind this block's start state: the one whose range holds the
         // start of the sequence (its last run begins there, whatever sequence the item itself started in)
@@ -707,7 +708,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     sc->s0[c] = 2.f / Lpm;
                     if (a.fro_out && valid) a.fro_out[ti.tok0 + (size_t)c * a.heads] = fc;
                 }
-                wait_bar(cx, BAR_V, 0u);       // q tile has landed
+                wait_bar(cx, BAR_V, solve_only ? (uint32_t)(tile & 1) : 0u);   // q tile has landed (V shares the barrier)
                 // the previous tile's output stores have read the X' buffer, which x_0 is about to overwrite
                 if (tid == 32) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 cta_sync();                    // the set-up values are published
@@ -741,7 +742,8 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const int rq = (stage ? OPF_STAGE : 0) | (clamped ? OPF_PLAIN_K : 0);
                 fence_async_smem();
                 fence_before();
-                sync_post(cx, (a.n_iter == 0 ? OP_ITER1_LAST : OP_ITER1) | rq);
+                const int op_last = solve_only ? OP_NONE : OP_ITER1_LAST;   // after the last update: scores for the output
+                sync_post(cx, (a.n_iter == 0 ? op_last : OP_ITER1) | rq);
                 TSTAMP(6);
 
                 float omega = 2.f;
@@ -794,8 +796,30 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     else x_epilogue(x2, xp2);
                     fence_async_smem();
                     fence_before();
-                    sync_post(cx, (it + 1 == a.n_iter ? OP_ITER1_LAST : OP_ITER1) | rq);
+                    sync_post(cx, (it + 1 == a.n_iter ? op_last : OP_ITER1) | rq);
                     TSTAMP(10);
+                }
+                if (solve_only) {
+                    // the solve is the result: x_c = x'_c / zt_c as bf16 into the X' buffer (no product reads it any
+                    // more), stored by TMA after the tile's last barrier
+                    const float inv = sc->iz[c];
+                    auto stage_x = [&](const uint64_t(&x)[16]) {
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                float xa, xb;
+                                f2_unpack(x[4 * ch + u], xa, xb);
+                                pk[u] = pack_bf16(xa * inv, xb * inv);
+                            }
+                            *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + ch)) =
+                                make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
+                    };
+                    if (a.n_iter & 1) stage_x(xp2);
+                    else stage_x(x2);
+                    fence_async_smem();
                 }
             }
 
@@ -805,52 +829,54 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 int mm = m;
                 asm volatile("" : "+r"(mm));                   // recompute the tile's description
                 const TileInfo ti = tile_info(a, item, f_lo, n_mine, mm);
-                // q is no longer needed: its buffer takes the V tile
-                if (tid == 0) issue_tma(&tmV, ti.f, OFF_V, BAR_V);
                 prefetch_gates(ti.m_next);
-                // while the scores of the final iterate are computed: U master pass (bf16 copy into the H buffer, which
-                // no pending product reads; scale by the tile's decay)
-                const StartSrc src = {ti.seq_state, a.ws.delta, a.ws.decay, ti.chained ? chain_j0 : 0,
-                                      ti.chained ? item : 0, st, (size_t)D * D + (size_t)c * D};
-                master_pass<false>(cx, tmem + TM_U, ti.run_start, src, exp2f(sc->G2[ti.ntok - 1]));
-                fence_async_smem();
-                wait_bar(cx, BAR_A, ph_a);
-                ph_a ^= 1u;
-                fence_after();
-                TSTAMP(15);
-                p_epilogue(cx, clamped ? PF_EXACT : PF_TABLE, pf, sc->ac[c]);   // this P multiplies the unweighted V
-                fence_before();
-                TSTAMP(16);
-                // O = X' U_0^T + P V (the H buffer holds U_0 since the last score pass), U advance
-                wait_bar(cx, BAR_V, 1u);                       // V tile has landed
-                sync_post(cx, OP_OUT | (stage ? OPF_STAGE : 0));
-                TSTAMP(11);
-                wait_bar(cx, BAR_A, ph_a);
-                ph_a ^= 1u;
-                fence_after();
-                TSTAMP(12);
-                // O as bf16 into the X' buffer (no product reads it any more), stored by TMA after the tile's last barrier
+                if (!solve_only) {
+                    // q is no longer needed: its buffer takes the V tile
+                    if (tid == 0) issue_tma(&tmV, ti.f, OFF_V, BAR_V);
+                    // while the scores of the final iterate are computed: U master pass (bf16 copy into the H buffer, which
+                    // no pending product reads; scale by the tile's decay)
+                    const StartSrc src = {ti.seq_state, a.ws.delta, a.ws.decay, ti.chained ? chain_j0 : 0,
+                                          ti.chained ? item : 0, st, (size_t)D * D + (size_t)c * D};
+                    master_pass<false>(cx, tmem + TM_U, ti.run_start, src, exp2f(sc->G2[ti.ntok - 1]));
+                    fence_async_smem();
+                    wait_bar(cx, BAR_A, ph_a);
+                    ph_a ^= 1u;
+                    fence_after();
+                    TSTAMP(15);
+                    p_epilogue(cx, clamped ? PF_EXACT : PF_TABLE, pf, sc->ac[c]);   // this P multiplies the unweighted V
+                    fence_before();
+                    TSTAMP(16);
+                    // O = X' U_0^T + P V (the H buffer holds U_0 since the last score pass), U advance
+                    wait_bar(cx, BAR_V, 1u);                       // V tile has landed
+                    sync_post(cx, OP_OUT | (stage ? OPF_STAGE : 0));
+                    TSTAMP(11);
+                    wait_bar(cx, BAR_A, ph_a);
+                    ph_a ^= 1u;
+                    fence_after();
+                    TSTAMP(12);
+                    // O as bf16 into the X' buffer (no product reads it any more), stored by TMA after the tile's last barrier
 #pragma unroll
-                for (int piece = 0; piece < 2; ++piece) {
-                    uint32_t r[16];
-                    TMEM_LD16(tmem + TM_Y + cx.lane_addr + 32 * cq + 16 * piece, r);
-                    tmem_wait_ld();
-                    uint32_t pk[8];
+                    for (int piece = 0; piece < 2; ++piece) {
+                        uint32_t r[16];
+                        TMEM_LD16(tmem + TM_Y + cx.lane_addr + 32 * cq + 16 * piece, r);
+                        tmem_wait_ld();
+                        uint32_t pk[8];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        pk[u] = pack_bf16(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1]));
-                    *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + 2 * piece)) =
-                        make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + 2 * piece + 1)) =
-                        make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                        for (int u = 0; u < 8; ++u)
+                            pk[u] = pack_bf16(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1]));
+                        *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + 2 * piece)) =
+                            make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + 2 * piece + 1)) =
+                            make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    }
+                    fence_async_smem();
+                    TSTAMP(13);
+                    wait_bar(cx, BAR_B, ph_b);     // U advance done: every tensor-core read of this tile's buffers is done
+                    ph_b ^= 1u;
+                    fence_after();
+                    if (ti.seq_end && a.state_out)
+                        master_store(cx, tmem + TM_U, a.state_out + (size_t)ti.seq * st + (size_t)D * D + (size_t)c * D);
                 }
-                fence_async_smem();
-                TSTAMP(13);
-                wait_bar(cx, BAR_B, ph_b);     // U advance done: every tensor-core read of this tile's buffers is done
-                ph_b ^= 1u;
-                fence_after();
-                if (ti.seq_end && a.state_out)
-                    master_store(cx, tmem + TM_U, a.state_out + (size_t)ti.seq * st + (size_t)D * D + (size_t)c * D);
                 fence_before();
                 if (tid == 0) sc->stop = aborted(cx) ? 1 : 0;
                 cta_sync();

@@ -24,7 +24,7 @@ GKA_ERR_TIMEOUT = 8
 EXPORTS = ("gka_fwd_workspace_bytes", "gka_fwd_chunked", "gka_decode_step", "gka_status_string",
            "gka_fwd_num_work_items", "gka_fwd_work_range", "gka_last_error_detail",
            "gka_fwd_chunked_noalloc", "gka_noalloc_scratch_bytes",
-           "gka_fwd_chunked_host", "gka_fwd_host_staging_bytes")
+           "gka_fwd_chunked_host", "gka_fwd_host_staging_bytes", "gka_solve_chunked")
 
 
 class GkaDesc(ctypes.Structure):
@@ -76,6 +76,8 @@ def load_library():
         lib.gka_fwd_host_staging_bytes.restype = ctypes.c_size_t
         lib.gka_fwd_chunked_host.argtypes = [dp, vp, vp, vp, vp, vp, vp, ci, ci, vp, vp]
         lib.gka_fwd_chunked_host.restype = ci
+        lib.gka_solve_chunked.argtypes = [dp, vp, vp, vp, vp, ci, ci, vp]
+        lib.gka_solve_chunked.restype = ci
         lib.gka_decode_step.argtypes = [dp, vp, vp, vp, vp, vp, vp, ci, vp]
         lib.gka_decode_step.restype = ci
         llp, ip = ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int)
@@ -186,6 +188,28 @@ def gka_fwd_chunked(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=No
     if rc != GKA_OK:
         raise GkaError(rc, "gka_fwd_chunked")
     return out, state_out
+
+
+def gka_solve_chunked(rhs, k, gate, lam, n_iter, chunk=64, out=None, *, state_in=None, workspace=None,
+                      precision=GKA_PREC_NATIVE, flags=0, device_status=None, stream=None):
+    """The solve alone: x_t = CH(H_t + lambda_t I, rhs_t, n_iter).  rhs, k: [B,T,heads,d]; gate, lam: [B,T,heads] f32.
+
+    With rhs = q this is the iterate the forward multiplies by U_t; with rhs = dL/dx it is dL/dq.
+    """
+    _check_cuda(rhs, k, gate, lam, out, state_in, workspace, device_status)
+    B, T, heads, d = rhs.shape
+    if out is None:
+        out = torch.empty_like(rhs)
+    if workspace is None:
+        workspace = alloc_workspace(B, T, heads, d, rhs.device, chunk)
+    if stream is None:
+        stream = torch.cuda.current_stream(rhs.device).cuda_stream
+    desc = make_desc(B, T, heads, d, d, _io_code(rhs), precision, flags, stream, workspace, state_in, device_status)
+    rc = load_library().gka_solve_chunked(ctypes.byref(desc), rhs.data_ptr(), k.data_ptr(), gate.data_ptr(),
+                                          lam.data_ptr(), int(n_iter), int(chunk), out.data_ptr())
+    if rc != GKA_OK:
+        raise GkaError(rc, "gka_solve_chunked")
+    return out
 
 
 def gka_fwd_host_staging_bytes(B, T, heads, d, io_dtype) -> int:

@@ -415,3 +415,45 @@ def test_adaptive_regularisation_gives_kappa_bound():
     ab = oracle.fwd(*as_bthd(q, k, v, gate, a * fro), n_iter=5)
     assert rel(ad["out"], ab["out"]) < 1e-14
     assert np.allclose((fro + a * fro) / (a * fro), 51.0)
+
+
+# --------------------------------------------------------------------------- backward solve for dq
+def test_fixed_iteration_solve_is_linear_and_self_adjoint():
+    """Section 4.3 (implicit differentiation), Lemma 2: with r fixed the Chebyshev map q -> x is x = p_r(A) q,
+    a polynomial in the symmetric matrix A = H_t + lambda_t I whose coefficients depend on (L, mu, r) only.
+    Hence it is linear in the right-hand side and self-adjoint, so dL/dq = CH(A, dL/dx, r): the same solve
+    with another right-hand side.  Checked on the oracle's per-token solves: <CH(u), w> = <u, CH(w)> and
+    CH(a u + b w) = a CH(u) + b CH(w), token by token, with H_t built by the recurrence."""
+    T, D, r = 24, 16, 7
+    _, k, v, gate, lam = draw(T, D, seed=31)
+    rng = np.random.default_rng(32)
+    u, w = rng.standard_normal((T, D)), rng.standard_normal((T, D))
+
+    def solve(rhs):
+        return oracle.fwd(*as_bthd(rhs, k, v, gate, lam), n_iter=r, want_x=True)["x"][0, :, 0]
+
+    xu, xw, xc = solve(u), solve(w), solve(0.3 * u - 1.7 * w)
+    lhs = np.einsum("td,td->t", xu, w)
+    rhs = np.einsum("td,td->t", u, xw)
+    assert np.allclose(lhs, rhs, rtol=1e-10, atol=1e-12)
+    assert rel(xc, 0.3 * xu - 1.7 * xw) < 1e-12
+
+
+def test_solve_gradient_matches_finite_differences():
+    """The same statement as a gradient check: for the loss sum_t <g_t, x_t(q)>, dL/dq_t = CH(A_t, g_t, r);
+    compared with central differences of the oracle's forward solve (the map is linear, so they agree to
+    rounding)."""
+    T, D, r = 6, 8, 5
+    q, k, v, gate, lam = draw(T, D, seed=41)
+    g = np.random.default_rng(42).standard_normal((T, D))
+
+    def solve(rhs):
+        return oracle.fwd(*as_bthd(rhs, k, v, gate, lam), n_iter=r, want_x=True)["x"][0, :, 0]
+
+    dq = solve(g)
+    eps = 1e-3
+    for (t, i) in [(0, 0), (2, 5), (5, 7)]:
+        e = np.zeros_like(q)
+        e[t, i] = eps
+        fd = (np.sum(g * solve(q + e)) - np.sum(g * solve(q - e))) / (2 * eps)
+        assert abs(fd - dq[t, i]) <= 1e-8 * max(1.0, abs(dq[t, i]))

@@ -253,3 +253,52 @@ def test_decode_adaptive_lambda():
                               to_dev(step["v"][:, 0]), to_dev(step["gate"][:, 0]), to_dev(a), 8,
                               flags=gka.GKA_FLAG_ADAPTIVE_LAMBDA)
     assert rel(out.cpu().numpy(), ref["out"]) < TOL_F32
+
+
+# --------------------------------------------------------------------------- the solve alone (backward solve for dq)
+def run_solve(inp, rhs, n_iter, bf16, precision=gka.GKA_PREC_NATIVE, flags=0):
+    r_, k = to_dev(rhs, bf16), to_dev(inp["k"], bf16)
+    gate, lam = to_dev(inp["gate"]), to_dev(inp["lam"])
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    x = gka.gka_solve_chunked(r_, k, gate, lam, n_iter, 64, precision=precision, flags=flags, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return x.float().cpu().numpy()
+
+
+@pytest.mark.parametrize("d,n_iter", [(64, 6), (128, 0), (128, 8)])
+def test_solve_f32_matches_the_oracle_iterates(d, n_iter):
+    """x_t = CH(H_t + lambda_t I, rhs_t, r) for an arbitrary right-hand side (not unit norm: a gradient)."""
+    cfg = synth.shrink(synth.CONFIGS[0], d=d, T=320, heads=3)
+    inp = synth.make_inputs(cfg)
+    rhs = np.random.default_rng(5).standard_normal(inp["q"].shape).astype(np.float32)
+    ref = oracle.fwd(rhs, inp["k"], inp["v"], inp["gate"], inp["lam"], n_iter, want_x=True)["x"]
+    x = run_solve(inp, rhs, n_iter, bf16=False)
+    assert rel(x, ref) <= TOL_F32
+
+
+@pytest.mark.parametrize("n_iter", [0, 1, 10])
+def test_solve_bf16_native_matches_the_oracle_iterates(n_iter):
+    """Tensor-core path; several work items cut the sequences so the start states come through the summaries."""
+    cfg = synth.shrink(synth.CONFIGS[1], B=2, heads=3, T=64 * 70)
+    inp = synth.make_inputs(cfg)
+    rng = np.random.default_rng(6)
+    rhs = synth.round_bf16(rng.standard_normal(inp["q"].shape).astype(np.float32))
+    ref = oracle.fwd(rhs, inp["k"], inp["v"], inp["gate"], inp["lam"], n_iter, want_x=True)["x"]
+    x = run_solve(inp, rhs, n_iter, bf16=True)
+    assert np.all(np.isfinite(x))
+    e = rel(x, ref)
+    print("solve bf16 n_iter %d rel L2 %.3e" % (n_iter, e))
+    assert e <= TOL_BF16
+
+
+def test_solve_with_q_gives_the_forward_output_through_u():
+    """Consistency of the two entry points: U_t x_t from the forward equals the oracle's U_t applied to the
+    iterate that gka_solve_chunked returns for rhs = q (fp32 path, where both are accurate to 1e-4)."""
+    cfg = synth.shrink(synth.CONFIGS[0], d=64, T=192, heads=2)
+    inp = synth.make_inputs(cfg)
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], cfg.n_iter, want_x=True)
+    x = run_solve(inp, inp["q"], cfg.n_iter, bf16=False)
+    assert rel(x, ref["x"]) <= TOL_F32
+    out, _, _ = run_fwd(inp, cfg.n_iter, bf16=False)
+    assert rel(out, ref["out"]) <= TOL_F32
