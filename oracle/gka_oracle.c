@@ -10,6 +10,9 @@
  *   - forward recurrence, eq. (CH), Section 4.1:
  *         H_t = gamma_t H_{t-1} + k_t k_t^T,   U_t = gamma_t U_{t-1} + v_t k_t^T,
  *         x_t = CH(H_t + lambda_t I, q_t, r),  y_t = U_t x_t
+ *   - beta_t-augmented write, Remark "canonical beta_t-augmented variant" (Section 4.1) and the
+ *     appendix's modified eq. (CH): H_t = gamma_t H_{t-1} + beta_t k_t k_t^T,
+ *     U_t = gamma_t U_{t-1} + beta_t v_t k_t^T (beta == NULL means beta_t = 1, the paper's experiments)
  *   - Chebyshev Iteration, Algorithm 1 (weight schedule, grad descent, momentum)
  *   - eigenvalue bounds, Section 4.1 "Adaptive Regularization":
  *         L = ||H_t||_F + lambda_t,   mu = lambda_t
@@ -115,16 +118,16 @@ int gka_oracle_cholesky_solve(int D, const double *A, const double *b, double *x
 /* One token of eq. (CH) on one head's state.  H: dk x dk, U: dv x dk, A: scratch dk x dk. */
 static int gka_token(int dk, int dv, double *H, double *U, double *A,
                      const double *q, const double *k, const double *v,
-                     double gamma, double lam_in, int lam_mode, int r,
+                     double gamma, double beta, double lam_in, int lam_mode, int r,
                      double *xi, double *y_ch, double *y_exact, double *fro_out, double *xi_exact)
 {
     /* state write: decay, then rank-one update */
     for (int i = 0; i < dk; ++i)
         for (int j = 0; j < dk; ++j)
-            H[(size_t)i * dk + j] = gamma * H[(size_t)i * dk + j] + k[i] * k[j];
+            H[(size_t)i * dk + j] = gamma * H[(size_t)i * dk + j] + beta * k[i] * k[j];
     for (int i = 0; i < dv; ++i)
         for (int j = 0; j < dk; ++j)
-            U[(size_t)i * dk + j] = gamma * U[(size_t)i * dk + j] + v[i] * k[j];
+            U[(size_t)i * dk + j] = gamma * U[(size_t)i * dk + j] + beta * v[i] * k[j];
     /* direct Frobenius norm */
     double ss = 0.0;
     for (size_t e = 0; e < (size_t)dk * dk; ++e) ss += H[e] * H[e];
@@ -154,13 +157,13 @@ static int gka_token(int dk, int dv, double *H, double *U, double *A,
 }
 
 /*
- * Forward recurrence over whole sequences.  Nullable: state_in (zero state), out_exact,
- * fro, x_ch (the Chebyshev iterates xi_r, [B,T,heads,d_k]), state_out.
+ * Forward recurrence over whole sequences.  Nullable: beta (write strength 1), state_in (zero state),
+ * out_exact, fro, x_ch (the Chebyshev iterates xi_r, [B,T,heads,d_k]), state_out.
  * threads <= 0 uses the OpenMP default.  Returns 0, or 1 if a Cholesky factorisation failed.
  */
 int gka_oracle_fwd(int B, int T, int heads, int dk, int dv,
                    const double *q, const double *k, const double *v,
-                   const double *gate, const double *lam, int lam_mode, int n_iter,
+                   const double *gate, const double *lam, const double *beta, int lam_mode, int n_iter,
                    const double *state_in,
                    double *out_ch, double *out_exact, double *fro, double *x_ch,
                    double *state_out, int threads)
@@ -184,7 +187,7 @@ int gka_oracle_fwd(int B, int T, int heads, int dk, int dv,
             size_t tok = ((size_t)b * T + t) * heads + h;
             double f;
             int rc = gka_token(dk, dv, H, U, A, q + tok * dk, k + tok * dk, v + tok * dv,
-                               gate[tok], lam[tok], lam_mode, n_iter, xi,
+                               gate[tok], beta ? beta[tok] : 1.0, lam[tok], lam_mode, n_iter, xi,
                                out_ch + tok * dv, out_exact ? ye : NULL, &f, xe);
             rc_all |= rc;
             if (out_exact) memcpy(out_exact + tok * dv, ye, (size_t)dv * sizeof(double));
@@ -204,7 +207,7 @@ int gka_oracle_fwd(int B, int T, int heads, int dk, int dv,
  */
 int gka_oracle_decode(int N, int heads, int dk, int dv, double *state,
                       const double *q, const double *k, const double *v,
-                      const double *gate, const double *lam, int lam_mode, int n_iter,
+                      const double *gate, const double *lam, const double *beta, int lam_mode, int n_iter,
                       double *out_ch, double *out_exact, int threads)
 {
     int rc_all = 0;
@@ -220,7 +223,7 @@ int gka_oracle_decode(int N, int heads, int dk, int dv, double *state,
         double *xi = (double *)malloc((size_t)dk * sizeof(double));
         double *xe = (double *)malloc((size_t)dk * sizeof(double));
         rc_all |= gka_token(dk, dv, H, U, A, q + (size_t)nh * dk, k + (size_t)nh * dk,
-                            v + (size_t)nh * dv, gate[nh], lam[nh], lam_mode, n_iter, xi,
+                            v + (size_t)nh * dv, gate[nh], beta ? beta[nh] : 1.0, lam[nh], lam_mode, n_iter, xi,
                             out_ch + (size_t)nh * dv,
                             out_exact ? out_exact + (size_t)nh * dv : NULL, NULL, xe);
         free(A); free(xi); free(xe);

@@ -457,3 +457,32 @@ def test_solve_gradient_matches_finite_differences():
         e[t, i] = eps
         fd = (np.sum(g * solve(q + e)) - np.sum(g * solve(q - e))) / (2 * eps)
         assert abs(fd - dq[t, i]) <= 1e-8 * max(1.0, abs(dq[t, i]))
+
+
+# --------------------------------------------------------------------------- beta-augmented write
+def test_beta_write_equals_rescaled_keys_and_values():
+    """Remark "canonical beta_t-augmented variant" (Section 4.1): H_t = gamma_t H_{t-1} + beta_t k k^T and
+    U_t = gamma_t U_{t-1} + beta_t v k^T.  Writing beta_t k k^T = (sqrt(beta_t) k)(sqrt(beta_t) k)^T and
+    beta_t v k^T = (sqrt(beta_t) v)(sqrt(beta_t) k)^T reduces it to the beta == 1 recurrence (pinned above) on
+    rescaled keys and values; queries are untouched, so outputs, norms and states must agree."""
+    T, D, r = 40, 12, 6
+    q, k, v, gate, lam = draw(T, D, seed=51)
+    beta = 1.0 / (1.0 + np.exp(-np.random.default_rng(52).standard_normal(T)))
+    a = oracle.fwd(*as_bthd(q, k, v, gate, lam), n_iter=r, beta=beta[None, :, None], exact=True)
+    sb = np.sqrt(beta)[:, None]
+    b = oracle.fwd(*as_bthd(q, sb * k, sb * v, gate, lam), n_iter=r, exact=True)
+    for name in ("out", "out_exact", "fro", "state"):
+        assert rel(a[name], b[name]) < 1e-12, name
+    # and it is not a no-op
+    c = oracle.fwd(*as_bthd(q, k, v, gate, lam), n_iter=r)
+    assert rel(a["out"], c["out"]) > 1e-2
+
+
+def test_beta_zero_tokens_write_nothing():
+    """A token with beta_t = 0 only decays the state: the next state is gamma_t times the previous one."""
+    T, D = 5, 6
+    q, k, v, gate, lam = draw(T, D, seed=53)
+    beta = np.array([1.0, 1.0, 0.0, 0.0, 1.0])
+    res = [oracle.fwd(*as_bthd(q[:n], k[:n], v[:n], gate[:n], lam[:n]), n_iter=2, beta=beta[None, :n, None])["state"]
+           for n in (2, 4)]
+    assert rel(res[1], gate[2] * gate[3] * res[0]) < 1e-13
