@@ -79,6 +79,10 @@ typedef struct {
     float *fro_out;      /* optional [B, T, heads] float32: ||H_t||_F per token (debug output) */
     void *profile_start; /* optional cudaEvent_t recorded on the stream right before the dominant  */
     void *profile_stop;  /* kernel (main forward kernel / decode kernel) and right after it        */
+    const float *beta;   /* optional write strengths beta_t (device pointer): [B, T, heads] for the chunked
+                            calls, [B, heads] for the decode step; H_t = gamma_t H_{t-1} + beta_t k_t k_t^T,
+                            U_t = gamma_t U_{t-1} + beta_t v_t k_t^T (Remark "canonical beta_t-augmented
+                            variant", Section 4.1).  NULL = 1, the recurrence of eq. (CH).  Must be >= 0. */
 } gka_desc;
 
 /*

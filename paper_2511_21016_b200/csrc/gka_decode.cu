@@ -23,7 +23,7 @@ __global__ void __launch_bounds__(kThreads, 2)
 decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *__restrict__ k,
               const IoT *__restrict__ v, const float *__restrict__ gate,
               const float *__restrict__ lam, int n_iter, IoT *__restrict__ out, unsigned flags,
-              int *__restrict__ device_status) {
+              const float *__restrict__ beta, int *__restrict__ device_status) {
     constexpr int RPT = D / 32;   // rows per thread
     constexpr int CG = D / 32;    // float4 column groups per thread
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -67,9 +67,12 @@ decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *_
                                                                 4 * (lane8 + 8 * n)));
 
     if (tid < D) {
+        // write strength beta (Remark on the beta-augmented variant, Section 4.1): beta k k^T and beta v k^T are
+        // the plain writes of sqrt(beta) k and sqrt(beta) v
+        const float sb = beta ? sqrtf(fmaxf(beta[head], 0.f)) : 1.f;
         sQ[tid] = Io<IoT>::load1(q + (size_t)head * D + tid);
-        sKv[tid] = Io<IoT>::load1(k + (size_t)head * D + tid);
-        sVv[tid] = Io<IoT>::load1(v + (size_t)head * D + tid);
+        sKv[tid] = sb * Io<IoT>::load1(k + (size_t)head * D + tid);
+        sVv[tid] = sb * Io<IoT>::load1(v + (size_t)head * D + tid);
     }
     const float gam = gate[head];
     float lamv = lam[head];
@@ -202,7 +205,7 @@ decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *_
 
 template <int D, typename IoT>
 cudaError_t launch_typed(float *state, const void *q, const void *k, const void *v, const float *gate,
-                         const float *lam, int n_iter, void *out, int nheads_total, unsigned flags,
+                         const float *lam, int n_iter, void *out, int nheads_total, unsigned flags, const float *beta,
                          int *device_status, cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream) {
     const size_t smem = (size_t)(D * D + 5 * D + 16) * sizeof(float) + 16;
     cudaError_t err = cudaFuncSetAttribute(decode_kernel<D, IoT>,
@@ -211,7 +214,7 @@ cudaError_t launch_typed(float *state, const void *q, const void *k, const void 
     if (ev_start) cudaEventRecord(ev_start, stream);
     decode_kernel<D, IoT><<<nheads_total, kThreads, smem, stream>>>(
         state, reinterpret_cast<const IoT *>(q), reinterpret_cast<const IoT *>(k),
-        reinterpret_cast<const IoT *>(v), gate, lam, n_iter, reinterpret_cast<IoT *>(out), flags,
+        reinterpret_cast<const IoT *>(v), gate, lam, n_iter, reinterpret_cast<IoT *>(out), flags, beta,
         device_status);
     if (ev_stop) cudaEventRecord(ev_stop, stream);
     return cudaGetLastError();
@@ -221,16 +224,16 @@ cudaError_t launch_typed(float *state, const void *q, const void *k, const void 
 
 cudaError_t launch_decode(float *state, const void *q, const void *k, const void *v, const float *gate,
                           const float *lam, int n_iter, void *out, int nseq, int heads, int d,
-                          int io_dtype, unsigned flags, int *device_status, cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream) {
+                          int io_dtype, unsigned flags, const float *beta, int *device_status, cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream) {
     const int total = nseq * heads;
     if (d == 128) {
         return io_dtype == GKA_BF16
-                   ? launch_typed<128, __nv_bfloat16>(state, q, k, v, gate, lam, n_iter, out, total, flags, device_status, ev_start, ev_stop, stream)
-                   : launch_typed<128, float>(state, q, k, v, gate, lam, n_iter, out, total, flags, device_status, ev_start, ev_stop, stream);
+                   ? launch_typed<128, __nv_bfloat16>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, device_status, ev_start, ev_stop, stream)
+                   : launch_typed<128, float>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, device_status, ev_start, ev_stop, stream);
     }
     return io_dtype == GKA_BF16
-               ? launch_typed<64, __nv_bfloat16>(state, q, k, v, gate, lam, n_iter, out, total, flags, device_status, ev_start, ev_stop, stream)
-               : launch_typed<64, float>(state, q, k, v, gate, lam, n_iter, out, total, flags, device_status, ev_start, ev_stop, stream);
+               ? launch_typed<64, __nv_bfloat16>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, device_status, ev_start, ev_stop, stream)
+               : launch_typed<64, float>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, device_status, ev_start, ev_stop, stream);
 }
 
 }  // namespace gka

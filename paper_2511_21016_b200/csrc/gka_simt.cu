@@ -119,14 +119,21 @@ __device__ __forceinline__ void state_update(float *M, const float *A, const flo
 }
 
 // Load one chunk's rows of a [B,T,heads,D] tensor into smem row-major (dst) and, optionally,
-// transposed with stride XS (dstT[d][token]).
+// transposed with stride XS (dstT[d][token]).  With write strengths (beta-augmented variant, Remark in
+// Section 4.1) key and value rows are scaled by sqrt(beta_t): beta k k^T and beta v k^T are the plain writes of
+// the scaled rows, and every later use of a key in the chunk-wise form carries exactly this factor.
 template <int D, typename IoT>
 __device__ __forceinline__ void load_rows(const IoT *src, size_t row0_elem, size_t row_stride_elem,
-                                          float *dst, float *dstT) {
+                                          float *dst, float *dstT, const float *beta = nullptr, size_t tok0 = 0,
+                                          int heads = 0) {
     constexpr int F4 = D / 4;
     for (int idx = threadIdx.x; idx < kChunk * F4; idx += kThreads) {
         const int row = idx / F4, c4 = idx % F4;
         float4 v = Io<IoT>::load4(src + row0_elem + (size_t)row * row_stride_elem + 4 * c4);
+        if (beta) {
+            const float sb = sqrtf(fmaxf(beta[tok0 + (size_t)row * heads], 0.f));
+            v.x *= sb; v.y *= sb; v.z *= sb; v.w *= sb;
+        }
         if (dst) st4(dst + row * D + 4 * c4, v);
         if (dstT) {
             dstT[(4 * c4 + 0) * XS + row] = v.x;
@@ -196,8 +203,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_summary(FwdArgs a) {
     for (long long f = f0; f < f1; ++f) {
         const int n = (int)(f % P.N);
         const size_t tok0 = ((size_t)b * a.T + (size_t)n * kChunk) * a.heads + h;
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, nullptr);
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, nullptr, a.beta, tok0, a.heads);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr, a.beta, tok0, a.heads);
         load_gates(a.gate, a.lam, tok0, a.heads, sG, sZeta, sLam, sW);
         const float zc = sZeta[kChunk - 1];
         decay_log += sG[kChunk - 1];
@@ -292,8 +299,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
         __syncthreads();
 
         // ---- stage the chunk
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, sKt);
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, sKt, a.beta, tok0, a.heads);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr, a.beta, tok0, a.heads);
         for (int e = 4 * tid; e < D * D; e += 4 * kThreads) st4(sH + e, ld4(mH + e));
         load_gates(a.gate, a.lam, tok0, a.heads, sG, sZeta, sLam, sW);  // ends with a barrier
 

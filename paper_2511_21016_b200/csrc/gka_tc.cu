@@ -96,6 +96,7 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         const int seq = (int)((unsigned)f0 / (unsigned)P.N), b = seq / a.heads, h = seq % a.heads;
         const int n0 = (int)((unsigned)f0 - (unsigned)seq * (unsigned)P.N);   // first chunk of the run in its sequence
         const float *grun = a.gate + ((size_t)b * a.T + (size_t)n0 * C) * a.heads + h;   // token stride: heads
+        const float *brun = a.beta ? a.beta + ((size_t)b * a.T + (size_t)n0 * C) * a.heads + h : nullptr;
         const int ntok_run = nch * C;
         auto issue_tma = [&](int n) {
             const uint32_t dst = sb + (uint32_t)(n % SUM_NS) * SUM_STAGE;
@@ -168,7 +169,9 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                 }
                 incl += before;
                 // w_j = 2^(decay from token j to the end of the run) = 2^((total - prefix) - incl_j); 0 past the run
-                s_w[t] = (n * NT + t < ntok_run) ? exp2f((total - prefix) - incl) : 0.f;
+                float wt = (n * NT + t < ntok_run) ? exp2f((total - prefix) - incl) : 0.f;
+                if (brun && n * NT + t < ntok_run) wt *= fmaxf(__ldg(brun + (size_t)(n * NT + t) * a.heads), 0.f);   // write strength
+                s_w[t] = wt;
                 prefix += tile_total;
             }
             // the previous tile's products are done: the w o K buffer and that tile's stage are free

@@ -64,11 +64,12 @@ struct TileScalars {
     float part[2][4][NT];  // Frobenius partial sums: [k H_0 k | Gram part][column quarter][key]
     float carry[2][2][4];  // per-warp totals (a, b) of the two scans
     float red[16];         // per-warp sums of squares of H_0
-    float gpre[NT], lpre[NT];   // gate and lambda of the next tile, copied asynchronously a tile ahead
+    float gpre[NT], lpre[NT], bpre[NT];   // gate, lambda, write strength of the next tile, copied asynchronously a tile ahead
+    float sb[NT];          // sqrt(beta_j) of the tile's keys (beta-augmented write)
     int req_op;            // request to the MMA issuer
     int stop;              // block-wide copy of the abort flag, taken between tiles
 };
-constexpr uint32_t SC_BYTES = 10240;
+constexpr uint32_t SC_BYTES = 11264;
 static_assert(sizeof(TileScalars) <= SC_BYTES, "scalar block too large");
 constexpr uint32_t TILE_SMEM = OFF_SC + SC_BYTES + 1024;   // + slack for the 1024-byte alignment of the base
 
@@ -366,6 +367,20 @@ __device__ __forceinline__ void p_epilogue(const Ctx &cx, int mode, float pf, fl
     tmem_wait_st();
 }
 
+// Scale the 128 rows of a bf16 operand tile in place by per-row factors (each thread takes four 16-byte groups).
+__device__ __forceinline__ void scale_rows(unsigned char *tile, const float *factor, int tid) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int qi = tid + CT * i;               // 16-byte group index in the 32 KB tile
+        const float f = factor[(qi & 1023) >> 3];  // row of this group
+        uint4 v = *reinterpret_cast<const uint4 *>(tile + qi * 16);
+        uint32_t *pv = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) pv[u] = pack_bf16(bf16_lo(pv[u]) * f, bf16_hi(pv[u]) * f);
+        *reinterpret_cast<uint4 *>(tile + qi * 16) = v;
+    }
+}
+
 // Inclusive scan over the tile's 128 tokens (threads 0..127 = warps 0..3, one token each) of the affine maps
 // s -> a s + b, composed in token order; returns the map's value at `seed`.  `slot` selects the carry row.
 __device__ __forceinline__ float affine_scan(const Ctx &cx, float a, float b, float seed, int slot) {
@@ -538,9 +553,13 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                  "l"(a.gate + tn.tok0 + (size_t)c * a.heads) : "memory");
                     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->lpre[c])),
                                  "l"(a.lam + tn.tok0 + (size_t)c * a.heads) : "memory");
+                    if (a.beta)
+                        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->bpre[c])),
+                                     "l"(a.beta + tn.tok0 + (size_t)c * a.heads) : "memory");
                 } else {
                     sc->gpre[c] = 1.f;
                     sc->lpre[c] = 1.f;
+                    sc->bpre[c] = 1.f;
                 }
             }
         };
@@ -579,10 +598,16 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     sc->zt[c] = exp2f(mc);
                     sc->iz[c] = exp2f(-mc);
                     sc->lam[c] = lamv;
+                    if (a.beta) sc->sb[c] = sqrtf(fmaxf(sc->bpre[c], 0.f));
                     TSTAMP(23);
                 }
                 // ---- K tile has landed (it was fetched during the previous tile): Gram matrix under the set-up
                 wait_bar(cx, stage ? BAR_K1 : BAR_K0, (uint32_t)((tile >> 1) & 1));
+                if (a.beta) {      // beta k k^T is the plain write of sqrt(beta) k: rescale the key rows in place
+                    cta_sync();
+                    scale_rows(smem + off_k, sc->sb, tid);
+                    fence_async_smem();
+                }
                 sync_post(cx, OP_GRAM | (stage ? OPF_STAGE : 0));     // also publishes the gate scalars
                 TSTAMP(0);
                 const float Glast = sc->G2[ntok - 1];
@@ -848,6 +873,10 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     TSTAMP(16);
                     // O = X' U_0^T + P V (the H buffer holds U_0 since the last score pass), U advance
                     wait_bar(cx, BAR_V, 1u);                       // V tile has landed
+                    if (a.beta) {  // beta v k^T with sqrt(beta) k already in place: the value rows take the other sqrt(beta)
+                        scale_rows(smem + OFF_V, sc->sb, tid);
+                        fence_async_smem();
+                    }
                     sync_post(cx, OP_OUT | (stage ? OPF_STAGE : 0));
                     TSTAMP(11);
                     wait_bar(cx, BAR_A, ph_a);

@@ -35,7 +35,7 @@ class GkaDesc(ctypes.Structure):
         ("stream", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t), ("state_in", ctypes.c_void_p),
         ("device_status", ctypes.c_void_p), ("fro_out", ctypes.c_void_p),
-        ("profile_start", ctypes.c_void_p), ("profile_stop", ctypes.c_void_p),
+        ("profile_start", ctypes.c_void_p), ("profile_stop", ctypes.c_void_p), ("beta", ctypes.c_void_p),
     ]
 
 
@@ -118,7 +118,7 @@ def _check_cuda(*ts):
 
 def make_desc(B, T, heads, d_k, d_v, io_dtype, precision=GKA_PREC_NATIVE, flags=0, stream=None,
               workspace=None, state_in=None, device_status=None, fro_out=None,
-              profile_events=None) -> GkaDesc:
+              profile_events=None, beta=None) -> GkaDesc:
     d = GkaDesc()
     d.B, d.T, d.heads, d.d_k, d.d_v = B, T, heads, d_k, d_v
     d.io_dtype, d.precision, d.flags = io_dtype, precision, flags
@@ -128,6 +128,7 @@ def make_desc(B, T, heads, d_k, d_v, io_dtype, precision=GKA_PREC_NATIVE, flags=
     d.state_in = _ptr(state_in)
     d.device_status = _ptr(device_status)
     d.fro_out = _ptr(fro_out)
+    d.beta = _ptr(beta)
     if profile_events is not None:
         d.profile_start, d.profile_stop = profile_events
     return d
@@ -165,12 +166,12 @@ def alloc_workspace(B, T, heads, d, device, chunk=64) -> torch.Tensor:
 
 def gka_fwd_chunked(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=None, *,
                     state_in=None, workspace=None, precision=GKA_PREC_NATIVE, flags=0,
-                    fro_out=None, device_status=None, stream=None, profile_events=None):
-    """Chunk-wise GKA forward.  q,k,v: [B,T,heads,d] (f32 or bf16); gate, lam: [B,T,heads] f32.
+                    fro_out=None, device_status=None, stream=None, profile_events=None, beta=None):
+    """Chunk-wise GKA forward.  q,k,v: [B,T,heads,d] (f32 or bf16); gate, lam, beta (optional): [B,T,heads] f32.
 
     Returns (out, state_out).  Work is enqueued on ``stream`` (default: torch's current stream).
     """
-    _check_cuda(q, k, v, gate, lam, out, state_out, state_in, workspace, fro_out, device_status)
+    _check_cuda(q, k, v, gate, lam, out, state_out, state_in, workspace, fro_out, device_status, beta)
     B, T, heads, d = q.shape
     if out is None:
         out = torch.empty_like(v)
@@ -181,7 +182,7 @@ def gka_fwd_chunked(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=No
     if stream is None:
         stream = torch.cuda.current_stream(q.device).cuda_stream
     desc = make_desc(B, T, heads, d, v.shape[-1], _io_code(q), precision, flags, stream, workspace,
-                     state_in, device_status, fro_out, profile_events)
+                     state_in, device_status, fro_out, profile_events, beta)
     rc = load_library().gka_fwd_chunked(ctypes.byref(desc), q.data_ptr(), k.data_ptr(), v.data_ptr(),
                                         gate.data_ptr(), lam.data_ptr(), int(n_iter), int(chunk),
                                         out.data_ptr(), _ptr(state_out))
@@ -191,7 +192,7 @@ def gka_fwd_chunked(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=No
 
 
 def gka_solve_chunked(rhs, k, gate, lam, n_iter, chunk=64, out=None, *, state_in=None, workspace=None,
-                      precision=GKA_PREC_NATIVE, flags=0, device_status=None, stream=None):
+                      precision=GKA_PREC_NATIVE, flags=0, device_status=None, stream=None, beta=None):
     """The solve alone: x_t = CH(H_t + lambda_t I, rhs_t, n_iter).  rhs, k: [B,T,heads,d]; gate, lam: [B,T,heads] f32.
 
     With rhs = q this is the iterate the forward multiplies by U_t; with rhs = dL/dx it is dL/dq.
@@ -204,7 +205,8 @@ def gka_solve_chunked(rhs, k, gate, lam, n_iter, chunk=64, out=None, *, state_in
         workspace = alloc_workspace(B, T, heads, d, rhs.device, chunk)
     if stream is None:
         stream = torch.cuda.current_stream(rhs.device).cuda_stream
-    desc = make_desc(B, T, heads, d, d, _io_code(rhs), precision, flags, stream, workspace, state_in, device_status)
+    desc = make_desc(B, T, heads, d, d, _io_code(rhs), precision, flags, stream, workspace, state_in, device_status,
+                     beta=beta)
     rc = load_library().gka_solve_chunked(ctypes.byref(desc), rhs.data_ptr(), k.data_ptr(), gate.data_ptr(),
                                           lam.data_ptr(), int(n_iter), int(chunk), out.data_ptr())
     if rc != GKA_OK:
@@ -262,7 +264,7 @@ def gka_fwd_chunked_noalloc(q, k, v, gate, lam, n_iter, chunk=64, out=None, stat
 
 
 def gka_decode_step(state, q, k, v, gate, lam, n_iter, out=None, *, flags=0, device_status=None,
-                    stream=None, profile_events=None):
+                    stream=None, profile_events=None, beta=None):
     """One recurrent step.  state: [N,heads,2*d*d] f32, updated in place; q,k,v: [N,heads,d]."""
     _check_cuda(state, q, k, v, gate, lam, out, device_status)
     N, heads, d = q.shape
@@ -271,7 +273,7 @@ def gka_decode_step(state, q, k, v, gate, lam, n_iter, out=None, *, flags=0, dev
     if stream is None:
         stream = torch.cuda.current_stream(q.device).cuda_stream
     desc = make_desc(N, 1, heads, d, v.shape[-1], _io_code(q), GKA_PREC_NATIVE, flags, stream,
-                     device_status=device_status, profile_events=profile_events)
+                     device_status=device_status, profile_events=profile_events, beta=beta)
     rc = load_library().gka_decode_step(ctypes.byref(desc), state.data_ptr(), q.data_ptr(),
                                         k.data_ptr(), v.data_ptr(), gate.data_ptr(), lam.data_ptr(),
                                         int(n_iter), out.data_ptr())

@@ -302,3 +302,69 @@ def test_solve_with_q_gives_the_forward_output_through_u():
     assert rel(x, ref["x"]) <= TOL_F32
     out, _, _ = run_fwd(inp, cfg.n_iter, bf16=False)
     assert rel(out, ref["out"]) <= TOL_F32
+
+
+# --------------------------------------------------------------------------- beta-augmented write
+def _beta_for(inp, seed):
+    rng = np.random.default_rng(seed)
+    return (1.0 / (1.0 + np.exp(-rng.standard_normal(inp["gate"].shape)))).astype(np.float32)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_fwd_beta_write_f32(d):
+    """H_t = gamma_t H_{t-1} + beta_t k k^T, U_t = gamma_t U_{t-1} + beta_t v k^T (Remark on the beta-augmented
+    variant, Section 4.1), fp32 path, sequences cut by work items."""
+    cfg = synth.shrink(synth.CONFIGS[0], d=d, T=384, heads=3)
+    inp = synth.make_inputs(cfg)
+    beta = _beta_for(inp, 7)
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], cfg.n_iter, beta=beta)
+    q, k, v = (to_dev(inp[n]) for n in ("q", "k", "v"))
+    out, st = gka.gka_fwd_chunked(q, k, v, to_dev(inp["gate"]), to_dev(inp["lam"]), cfg.n_iter, 64, beta=to_dev(beta))
+    torch.cuda.synchronize()
+    assert rel(out.cpu().numpy(), ref["out"]) <= TOL_F32
+    assert rel(st.cpu().numpy(), ref["state"]) <= 1e-5
+
+
+def test_fwd_beta_write_bf16_native():
+    """Tensor-core path with write strengths; the run crosses several work items."""
+    cfg = synth.shrink(synth.CONFIGS[1], B=2, heads=3, T=64 * 70)
+    inp = synth.make_inputs(cfg)
+    beta = _beta_for(inp, 8)
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], cfg.n_iter, beta=beta, want_x=True)
+    q, k, v = (to_dev(inp[n], True) for n in ("q", "k", "v"))
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out, st = gka.gka_fwd_chunked(q, k, v, to_dev(inp["gate"]), to_dev(inp["lam"]), cfg.n_iter, 64,
+                                  beta=to_dev(beta), device_status=status)
+    x = gka.gka_solve_chunked(q, k, to_dev(inp["gate"]), to_dev(inp["lam"]), cfg.n_iter, 64, beta=to_dev(beta))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    e, es, ex = rel(out.float().cpu().numpy(), ref["out"]), rel(st.cpu().numpy(), ref["state"]), \
+        rel(x.float().cpu().numpy(), ref["x"])
+    print("beta bf16 rel L2 out %.3e state %.3e solve %.3e" % (e, es, ex))
+    assert e <= TOL_BF16 and es <= 5e-3 and ex <= TOL_BF16
+
+
+def test_decode_beta_write():
+    cfg = synth.shrink(synth.CONFIGS[2], B=6, heads=4)
+    rng = np.random.default_rng(9)
+    N, Hh, d = cfg.B, cfg.heads, cfg.d
+    state = (0.05 * rng.standard_normal((N, Hh, 2 * d * d))).astype(np.float32)
+    # a valid H block: symmetric positive semi-definite
+    for n in range(N):
+        for h in range(Hh):
+            A = rng.standard_normal((d, 8)) * 0.2
+            state[n, h, :d * d] = (A @ A.T).astype(np.float32).ravel()
+    unit = lambda x: x / np.linalg.norm(x, axis=-1, keepdims=True)
+    q = synth.round_bf16(unit(rng.standard_normal((N, Hh, d))).astype(np.float32))
+    k = synth.round_bf16(unit(rng.standard_normal((N, Hh, d))).astype(np.float32))
+    v = synth.round_bf16(rng.standard_normal((N, Hh, d)).astype(np.float32))
+    gate = (1 / (1 + np.exp(-rng.normal(2, 1, (N, Hh))))).astype(np.float32)
+    lam = (np.log1p(np.exp(rng.standard_normal((N, Hh)))) + 1e-2).astype(np.float32)
+    beta = (1 / (1 + np.exp(-rng.standard_normal((N, Hh))))).astype(np.float32)
+    ref = oracle.decode(state, q, k, v, gate, lam, 10, beta=beta)
+    s_dev = to_dev(state)
+    out = gka.gka_decode_step(s_dev, to_dev(q, True), to_dev(k, True), to_dev(v, True), to_dev(gate), to_dev(lam), 10,
+                              beta=to_dev(beta))
+    torch.cuda.synchronize()
+    assert rel(out.float().cpu().numpy(), ref["out"]) <= TOL_BF16
+    assert rel(s_dev.cpu().numpy(), ref["state"]) <= 1e-5
