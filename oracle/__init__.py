@@ -44,9 +44,9 @@ def _load():
         lib.gka_oracle_chebyshev.restype = None
         lib.gka_oracle_cholesky_solve.argtypes = [ci, dp, dp, dp]
         lib.gka_oracle_cholesky_solve.restype = ci
-        lib.gka_oracle_fwd.argtypes = [ci] * 5 + [dp] * 6 + [ci, ci] + [dp] * 6 + [ci]
+        lib.gka_oracle_fwd.argtypes = [ci] * 5 + [dp] * 7 + [ci, ci] + [dp] * 6 + [ci]
         lib.gka_oracle_fwd.restype = ci
-        lib.gka_oracle_decode.argtypes = [ci] * 4 + [dp] * 7 + [ci, ci] + [dp, dp] + [ci]
+        lib.gka_oracle_decode.argtypes = [ci] * 4 + [dp] * 8 + [ci, ci] + [dp, dp] + [ci]
         lib.gka_oracle_decode.restype = ci
         lib.gka_oracle_max_threads.argtypes = []
         lib.gka_oracle_max_threads.restype = ci
@@ -97,10 +97,11 @@ def cholesky_solve(A, b) -> np.ndarray:
 
 
 def fwd(q, k, v, gate, lam, n_iter: int, state_in=None, lam_mode: int = 0, exact: bool = False,
-        want_x: bool = False, threads: int = 0, beta=None) -> dict:
+        want_x: bool = False, threads: int = 0, beta=None, alpha=None) -> dict:
     """Token-by-token forward recurrence.
 
-    q, k: [B,T,heads,d_k]; v: [B,T,heads,d_v]; gate, lam, beta (optional write strength): [B,T,heads].
+    q, k: [B,T,heads,d_k]; v: [B,T,heads,d_v]; gate, lam, beta (optional write strength), alpha (optional
+    alpha-connection: the read uses alpha x + (1 - alpha) q): [B,T,heads].
     Returns dict(out [B,T,heads,d_v], fro [B,T,heads], state [B,heads,d_k*d_k+d_v*d_k],
     and, on request, out_exact and x).
     """
@@ -118,7 +119,9 @@ def fwd(q, k, v, gate, lam, n_iter: int, state_in=None, lam_mode: int = 0, exact
     state = np.zeros((B, Hh, st))
     bt = None if beta is None else _f64(beta)
     assert bt is None or bt.shape == (B, T, Hh)
-    rc = _load().gka_oracle_fwd(B, T, Hh, dk, dv, _p(q), _p(k), _p(v), _p(gate), _p(lam), _p(bt),
+    al = None if alpha is None else _f64(alpha)
+    assert al is None or al.shape == (B, T, Hh)
+    rc = _load().gka_oracle_fwd(B, T, Hh, dk, dv, _p(q), _p(k), _p(v), _p(gate), _p(lam), _p(bt), _p(al),
                                 int(lam_mode), int(n_iter), _p(s_in), _p(out), _p(out_exact),
                                 _p(fro), _p(x), _p(state), int(threads))
     if rc:
@@ -132,7 +135,7 @@ def fwd(q, k, v, gate, lam, n_iter: int, state_in=None, lam_mode: int = 0, exact
 
 
 def decode(state, q, k, v, gate, lam, n_iter: int, lam_mode: int = 0, exact: bool = False,
-           threads: int = 0, beta=None) -> dict:
+           threads: int = 0, beta=None, alpha=None) -> dict:
     """One recurrent step.  state [N,heads,st] is copied, the new state is returned."""
     q, k, v, gate, lam = map(_f64, (q, k, v, gate, lam))
     N, Hh, dk = q.shape
@@ -142,8 +145,9 @@ def decode(state, q, k, v, gate, lam, n_iter: int, lam_mode: int = 0, exact: boo
     out = np.zeros((N, Hh, dv))
     out_exact = np.zeros((N, Hh, dv)) if exact else None
     bt = None if beta is None else _f64(beta)
+    al = None if alpha is None else _f64(alpha)
     rc = _load().gka_oracle_decode(N, Hh, dk, dv, _p(new_state), _p(q), _p(k), _p(v), _p(gate),
-                                   _p(lam), _p(bt), int(lam_mode), int(n_iter), _p(out), _p(out_exact),
+                                   _p(lam), _p(bt), _p(al), int(lam_mode), int(n_iter), _p(out), _p(out_exact),
                                    int(threads))
     if rc:
         raise np.linalg.LinAlgError("Cholesky failed in the exact branch")

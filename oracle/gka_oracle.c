@@ -13,6 +13,8 @@
  *   - beta_t-augmented write, Remark "canonical beta_t-augmented variant" (Section 4.1) and the
  *     appendix's modified eq. (CH): H_t = gamma_t H_{t-1} + beta_t k_t k_t^T,
  *     U_t = gamma_t U_{t-1} + beta_t v_t k_t^T (beta == NULL means beta_t = 1, the paper's experiments)
+ *   - alpha-connection, Section 4.4 "Architectural Consideration": the read uses the convex combination
+ *     alpha_t x_t + (1 - alpha_t) q_t in place of x_t (alpha == NULL means alpha_t = 1: y_t = U_t x_t)
  *   - Chebyshev Iteration, Algorithm 1 (weight schedule, grad descent, momentum)
  *   - eigenvalue bounds, Section 4.1 "Adaptive Regularization":
  *         L = ||H_t||_F + lambda_t,   mu = lambda_t
@@ -118,7 +120,7 @@ int gka_oracle_cholesky_solve(int D, const double *A, const double *b, double *x
 /* One token of eq. (CH) on one head's state.  H: dk x dk, U: dv x dk, A: scratch dk x dk. */
 static int gka_token(int dk, int dv, double *H, double *U, double *A,
                      const double *q, const double *k, const double *v,
-                     double gamma, double beta, double lam_in, int lam_mode, int r,
+                     double gamma, double beta, double alpha, double lam_in, int lam_mode, int r,
                      double *xi, double *y_ch, double *y_exact, double *fro_out, double *xi_exact)
 {
     /* state write: decay, then rank-one update */
@@ -141,7 +143,7 @@ static int gka_token(int dk, int dv, double *H, double *U, double *A,
     gka_oracle_chebyshev(dk, A, q, L, mu, r, xi);
     for (int i = 0; i < dv; ++i) {
         double s = 0.0;
-        for (int j = 0; j < dk; ++j) s += U[(size_t)i * dk + j] * xi[j];
+        for (int j = 0; j < dk; ++j) s += U[(size_t)i * dk + j] * (alpha * xi[j] + (1.0 - alpha) * q[j]);
         y_ch[i] = s;
     }
     int rc = 0;
@@ -149,7 +151,7 @@ static int gka_token(int dk, int dv, double *H, double *U, double *A,
         rc = gka_oracle_cholesky_solve(dk, A, q, xi_exact);
         for (int i = 0; i < dv; ++i) {
             double s = 0.0;
-            for (int j = 0; j < dk; ++j) s += U[(size_t)i * dk + j] * xi_exact[j];
+            for (int j = 0; j < dk; ++j) s += U[(size_t)i * dk + j] * (alpha * xi_exact[j] + (1.0 - alpha) * q[j]);
             y_exact[i] = s;
         }
     }
@@ -157,14 +159,14 @@ static int gka_token(int dk, int dv, double *H, double *U, double *A,
 }
 
 /*
- * Forward recurrence over whole sequences.  Nullable: beta (write strength 1), state_in (zero state),
+ * Forward recurrence over whole sequences.  Nullable: beta (write strength 1), alpha (1), state_in (zero state),
  * out_exact, fro, x_ch (the Chebyshev iterates xi_r, [B,T,heads,d_k]), state_out.
  * threads <= 0 uses the OpenMP default.  Returns 0, or 1 if a Cholesky factorisation failed.
  */
 int gka_oracle_fwd(int B, int T, int heads, int dk, int dv,
                    const double *q, const double *k, const double *v,
-                   const double *gate, const double *lam, const double *beta, int lam_mode, int n_iter,
-                   const double *state_in,
+                   const double *gate, const double *lam, const double *beta, const double *alpha,
+                   int lam_mode, int n_iter, const double *state_in,
                    double *out_ch, double *out_exact, double *fro, double *x_ch,
                    double *state_out, int threads)
 {
@@ -187,7 +189,8 @@ int gka_oracle_fwd(int B, int T, int heads, int dk, int dv,
             size_t tok = ((size_t)b * T + t) * heads + h;
             double f;
             int rc = gka_token(dk, dv, H, U, A, q + tok * dk, k + tok * dk, v + tok * dv,
-                               gate[tok], beta ? beta[tok] : 1.0, lam[tok], lam_mode, n_iter, xi,
+                               gate[tok], beta ? beta[tok] : 1.0, alpha ? alpha[tok] : 1.0, lam[tok], lam_mode,
+                               n_iter, xi,
                                out_ch + tok * dv, out_exact ? ye : NULL, &f, xe);
             rc_all |= rc;
             if (out_exact) memcpy(out_exact + tok * dv, ye, (size_t)dv * sizeof(double));
@@ -207,8 +210,8 @@ int gka_oracle_fwd(int B, int T, int heads, int dk, int dv,
  */
 int gka_oracle_decode(int N, int heads, int dk, int dv, double *state,
                       const double *q, const double *k, const double *v,
-                      const double *gate, const double *lam, const double *beta, int lam_mode, int n_iter,
-                      double *out_ch, double *out_exact, int threads)
+                      const double *gate, const double *lam, const double *beta, const double *alpha,
+                      int lam_mode, int n_iter, double *out_ch, double *out_exact, int threads)
 {
     int rc_all = 0;
     size_t st = (size_t)dk * dk + (size_t)dv * dk;
@@ -223,7 +226,8 @@ int gka_oracle_decode(int N, int heads, int dk, int dv, double *state,
         double *xi = (double *)malloc((size_t)dk * sizeof(double));
         double *xe = (double *)malloc((size_t)dk * sizeof(double));
         rc_all |= gka_token(dk, dv, H, U, A, q + (size_t)nh * dk, k + (size_t)nh * dk,
-                            v + (size_t)nh * dv, gate[nh], beta ? beta[nh] : 1.0, lam[nh], lam_mode, n_iter, xi,
+                            v + (size_t)nh * dv, gate[nh], beta ? beta[nh] : 1.0, alpha ? alpha[nh] : 1.0, lam[nh],
+                            lam_mode, n_iter, xi,
                             out_ch + (size_t)nh * dv,
                             out_exact ? out_exact + (size_t)nh * dv : NULL, NULL, xe);
         free(A); free(xi); free(xe);

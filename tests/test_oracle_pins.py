@@ -486,3 +486,20 @@ def test_beta_zero_tokens_write_nothing():
     res = [oracle.fwd(*as_bthd(q[:n], k[:n], v[:n], gate[:n], lam[:n]), n_iter=2, beta=beta[None, :n, None])["state"]
            for n in (2, 4)]
     assert rel(res[1], gate[2] * gate[3] * res[0]) < 1e-13
+
+
+# --------------------------------------------------------------------------- alpha-connection
+def test_alpha_connection_is_a_convex_combination_of_two_reads():
+    """Section 4.4: the read uses alpha_t x_t + (1 - alpha_t) q_t.  By linearity of the read,
+    y_t(alpha) = alpha_t U_t x_t + (1 - alpha_t) U_t q_t, where U_t x_t is the alpha == 1 output (pinned above) and
+    U_t q_t is gated linear attention, written out here by brute force from the definition of U_t."""
+    T, D, r = 30, 10, 5
+    q, k, v, gate, lam = draw(T, D, seed=61)
+    alpha = 1.0 / (1.0 + np.exp(-np.random.default_rng(62).standard_normal(T)))
+    y1 = oracle.fwd(*as_bthd(q, k, v, gate, lam), n_iter=r)["out"][0, :, 0]
+    ya = oracle.fwd(*as_bthd(q, k, v, gate, lam), n_iter=r, alpha=alpha[None, :, None])["out"][0, :, 0]
+    lin = np.zeros_like(y1)
+    for t in range(T):
+        for i in range(t + 1):
+            lin[t] += np.prod(gate[i + 1:t + 1]) * v[i] * (k[i] @ q[t])
+    assert rel(ya, alpha[:, None] * y1 + (1 - alpha[:, None]) * lin) < 1e-12
