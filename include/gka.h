@@ -83,6 +83,9 @@ typedef struct {
                             calls, [B, heads] for the decode step; H_t = gamma_t H_{t-1} + beta_t k_t k_t^T,
                             U_t = gamma_t U_{t-1} + beta_t v_t k_t^T (Remark "canonical beta_t-augmented
                             variant", Section 4.1).  NULL = 1, the recurrence of eq. (CH).  Must be >= 0. */
+    const float *alpha;  /* optional alpha-connection weights alpha_t (device pointer, same shapes as beta): the
+                            read becomes out_t = U_t (alpha_t x_t + (1 - alpha_t) q_t) (Section 4.4).  NULL = 1.
+                            Ignored by gka_solve_chunked.                                                     */
 } gka_desc;
 
 /*

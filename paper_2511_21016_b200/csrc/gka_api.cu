@@ -136,6 +136,7 @@ static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, c
     a.state_in = desc->state_in;
     a.fro_out = desc->fro_out;
     a.beta = desc->beta;
+    a.alpha = solve_only ? nullptr : desc->alpha;
     a.device_status = desc->device_status;
     a.B = desc->B; a.T = desc->T; a.heads = desc->heads;
     a.n_iter = n_iter;
@@ -180,7 +181,7 @@ gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, co
     if (!aligned16(state) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
         return GKA_ERR_ALIGN;
     cudaError_t err = launch_decode(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->heads,
-                                    desc->d_k, desc->io_dtype, desc->flags, desc->beta, desc->device_status,
+                                    desc->d_k, desc->io_dtype, desc->flags, desc->beta, desc->alpha, desc->device_status,
                                     reinterpret_cast<cudaEvent_t>(desc->profile_start),
                                     reinterpret_cast<cudaEvent_t>(desc->profile_stop),
                                     reinterpret_cast<cudaStream_t>(desc->stream));

@@ -151,6 +151,7 @@ struct FwdArgs {
     const float *state_in;
     float *fro_out;
     const float *beta;     // optional write strengths [B, T, heads]; nullptr = 1
+    const float *alpha;    // optional alpha-connection weights [B, T, heads]; nullptr = 1
     int *device_status;
     int B, T, heads;
     int n_iter;
@@ -166,7 +167,7 @@ cudaError_t launch_fwd_simt(const FwdArgs &a, int d, int io_dtype, cudaStream_t 
 cudaError_t launch_fwd_scan(const FwdArgs &a, int st, cudaStream_t stream);   // cross-item scan of the summaries
 cudaError_t launch_decode(float *state, const void *q, const void *k, const void *v,
                           const float *gate, const float *lam, int n_iter, void *out, int nseq,
-                          int heads, int d, int io_dtype, unsigned flags, const float *beta, int *device_status,
+                          int heads, int d, int io_dtype, unsigned flags, const float *beta, const float *alpha, int *device_status,
                           cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream);
 
 }  // namespace gka

@@ -23,7 +23,7 @@ __global__ void __launch_bounds__(kThreads, 2)
 decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *__restrict__ k,
               const IoT *__restrict__ v, const float *__restrict__ gate,
               const float *__restrict__ lam, int n_iter, IoT *__restrict__ out, unsigned flags,
-              const float *__restrict__ beta, int *__restrict__ device_status) {
+              const float *__restrict__ beta, const float *__restrict__ alpha, int *__restrict__ device_status) {
     constexpr int RPT = D / 32;   // rows per thread
     constexpr int CG = D / 32;    // float4 column groups per thread
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -166,11 +166,17 @@ decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *_
         }
     }
     const float *xs = sX + cur * D;
+    const float al = alpha ? alpha[head] : 1.f;     // alpha-connection (Section 4.4): the read uses alpha x + (1 - alpha) q
     float xc[CG][4];
     float kx = 0.f;
 #pragma unroll
     for (int n = 0; n < CG; ++n) {
         float4 t4 = *reinterpret_cast<const float4 *>(xs + 4 * (lane8 + 8 * n));
+        if (alpha) {
+            const float4 q4 = *reinterpret_cast<const float4 *>(sQ + 4 * (lane8 + 8 * n));
+            t4.x = fmaf(al, t4.x - q4.x, q4.x); t4.y = fmaf(al, t4.y - q4.y, q4.y);
+            t4.z = fmaf(al, t4.z - q4.z, q4.z); t4.w = fmaf(al, t4.w - q4.w, q4.w);
+        }
         xc[n][0] = t4.x; xc[n][1] = t4.y; xc[n][2] = t4.z; xc[n][3] = t4.w;
 #pragma unroll
         for (int u = 0; u < 4; ++u) kx = fmaf(kc[n][u], xc[n][u], kx);
@@ -205,7 +211,7 @@ decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *_
 
 template <int D, typename IoT>
 cudaError_t launch_typed(float *state, const void *q, const void *k, const void *v, const float *gate,
-                         const float *lam, int n_iter, void *out, int nheads_total, unsigned flags, const float *beta,
+                         const float *lam, int n_iter, void *out, int nheads_total, unsigned flags, const float *beta, const float *alpha,
                          int *device_status, cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream) {
     const size_t smem = (size_t)(D * D + 5 * D + 16) * sizeof(float) + 16;
     cudaError_t err = cudaFuncSetAttribute(decode_kernel<D, IoT>,
@@ -214,7 +220,7 @@ cudaError_t launch_typed(float *state, const void *q, const void *k, const void 
     if (ev_start) cudaEventRecord(ev_start, stream);
     decode_kernel<D, IoT><<<nheads_total, kThreads, smem, stream>>>(
         state, reinterpret_cast<const IoT *>(q), reinterpret_cast<const IoT *>(k),
-        reinterpret_cast<const IoT *>(v), gate, lam, n_iter, reinterpret_cast<IoT *>(out), flags, beta,
+        reinterpret_cast<const IoT *>(v), gate, lam, n_iter, reinterpret_cast<IoT *>(out), flags, beta, alpha,
         device_status);
     if (ev_stop) cudaEventRecord(ev_stop, stream);
     return cudaGetLastError();
@@ -224,16 +230,16 @@ cudaError_t launch_typed(float *state, const void *q, const void *k, const void 
 
 cudaError_t launch_decode(float *state, const void *q, const void *k, const void *v, const float *gate,
                           const float *lam, int n_iter, void *out, int nseq, int heads, int d,
-                          int io_dtype, unsigned flags, const float *beta, int *device_status, cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream) {
+                          int io_dtype, unsigned flags, const float *beta, const float *alpha, int *device_status, cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream) {
     const int total = nseq * heads;
     if (d == 128) {
         return io_dtype == GKA_BF16
-                   ? launch_typed<128, __nv_bfloat16>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, device_status, ev_start, ev_stop, stream)
-                   : launch_typed<128, float>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, device_status, ev_start, ev_stop, stream);
+                   ? launch_typed<128, __nv_bfloat16>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, alpha, device_status, ev_start, ev_stop, stream)
+                   : launch_typed<128, float>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, alpha, device_status, ev_start, ev_stop, stream);
     }
     return io_dtype == GKA_BF16
-               ? launch_typed<64, __nv_bfloat16>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, device_status, ev_start, ev_stop, stream)
-               : launch_typed<64, float>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, device_status, ev_start, ev_stop, stream);
+               ? launch_typed<64, __nv_bfloat16>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, alpha, device_status, ev_start, ev_stop, stream)
+               : launch_typed<64, float>(state, q, k, v, gate, lam, n_iter, out, total, flags, beta, alpha, device_status, ev_start, ev_stop, stream);
 }
 
 }  // namespace gka

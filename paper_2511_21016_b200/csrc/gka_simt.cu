@@ -455,6 +455,17 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
                                     make_float4(xm[t][4 * g + 0], xm[t][4 * g + 1], xm[t][4 * g + 2], xm[t][4 * g + 3]));
             }
         }
+        if (a.alpha && !a.solve_only) {    // alpha-connection (Section 4.4): the read uses alpha x + (1 - alpha) q
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const float al = a.alpha[tok0 + (size_t)(4 * tc + t) * a.heads];
+#pragma unroll
+                for (int u = 0; u < NCH; ++u) xm[t][u] = fmaf(al, xm[t][u] - qm[t][u], qm[t][u]);
+            }
+            __syncthreads();      // every read of the published iterate is done
+            publish_x();
+            __syncthreads();
+        }
         // ---- output O = zeta o (X U_0^T) + P V
         masked_scores();
         for (int idx = tid; idx < D * (D / 4); idx += kThreads) {   // sH <- U_0^T

@@ -64,12 +64,13 @@ struct TileScalars {
     float part[2][4][NT];  // Frobenius partial sums: [k H_0 k | Gram part][column quarter][key]
     float carry[2][2][4];  // per-warp totals (a, b) of the two scans
     float red[16];         // per-warp sums of squares of H_0
-    float gpre[NT], lpre[NT], bpre[NT];   // gate, lambda, write strength of the next tile, copied asynchronously a tile ahead
+    float gpre[NT], lpre[NT], bpre[NT], apre[NT];   // gate, lambda, write strength, alpha of the next tile, copied asynchronously a tile ahead
+    float al[NT];          // alpha_c of the tile's tokens (alpha-connection)
     float sb[NT];          // sqrt(beta_j) of the tile's keys (beta-augmented write)
     int req_op;            // request to the MMA issuer
     int stop;              // block-wide copy of the abort flag, taken between tiles
 };
-constexpr uint32_t SC_BYTES = 11264;
+constexpr uint32_t SC_BYTES = 12288;
 static_assert(sizeof(TileScalars) <= SC_BYTES, "scalar block too large");
 constexpr uint32_t TILE_SMEM = OFF_SC + SC_BYTES + 1024;   // + slack for the 1024-byte alignment of the base
 
@@ -513,6 +514,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const size_t st = state_floats(D, D);
         const bool adaptive = (a.flags & GKA_FLAG_ADAPTIVE_LAMBDA) != 0;
         const bool solve_only = a.solve_only != 0;      // the result is the solve itself: no V, no U, no output product
+        const bool mix = a.alpha != nullptr && !solve_only;   // alpha-connection: the read uses alpha x + (1 - alpha) q
         uint32_t ph_a = 0, ph_b = 0;
         // first item of the chain of summaries behind this block's start state: the one whose range holds the
         // start of the sequence (its last run begins there, whatever sequence the item itself started in)
@@ -556,10 +558,14 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     if (a.beta)
                         asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->bpre[c])),
                                      "l"(a.beta + tn.tok0 + (size_t)c * a.heads) : "memory");
+                    if (a.alpha)
+                        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->apre[c])),
+                                     "l"(a.alpha + tn.tok0 + (size_t)c * a.heads) : "memory");
                 } else {
                     sc->gpre[c] = 1.f;
                     sc->lpre[c] = 1.f;
                     sc->bpre[c] = 1.f;
+                    sc->apre[c] = 1.f;
                 }
             }
         };
@@ -599,6 +605,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     sc->iz[c] = exp2f(-mc);
                     sc->lam[c] = lamv;
                     if (a.beta) sc->sb[c] = sqrtf(fmaxf(sc->bpre[c], 0.f));
+                    if (a.alpha) sc->al[c] = sc->apre[c];
                     TSTAMP(23);
                 }
                 // ---- K tile has landed (it was fetched during the previous tile): Gram matrix under the set-up
@@ -767,7 +774,8 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const int rq = (stage ? OPF_STAGE : 0) | (clamped ? OPF_PLAIN_K : 0);
                 fence_async_smem();
                 fence_before();
-                const int op_last = solve_only ? OP_NONE : OP_ITER1_LAST;   // after the last update: scores for the output
+                // after the last update: scores for the output (posted later when the iterate is still to be mixed with q)
+                const int op_last = (solve_only || mix) ? OP_NONE : OP_ITER1_LAST;
                 sync_post(cx, (a.n_iter == 0 ? op_last : OP_ITER1) | rq);
                 TSTAMP(6);
 
@@ -845,6 +853,32 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     if (a.n_iter & 1) stage_x(xp2);
                     else stage_x(x2);
                     fence_async_smem();
+                }
+                if (mix) {
+                    // alpha-connection (Section 4.4): X' <- zt (alpha x + (1 - alpha) q) = alpha x' + (1 - alpha) zt q
+                    const float alc = sc->al[c];
+                    auto mix_x = [&](const uint64_t(&x)[16]) {
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            const uint4 qv = *reinterpret_cast<const uint4 *>(qrow + tile_off(c, 4 * cq + ch));
+                            const uint32_t *qq = reinterpret_cast<const uint32_t *>(&qv);
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                float xa, xb;
+                                f2_unpack(x[4 * ch + u], xa, xb);
+                                const float qa = valid ? ztc * bf16_lo(qq[u]) : 0.f, qb = valid ? ztc * bf16_hi(qq[u]) : 0.f;
+                                pk[u] = pack_bf16(fmaf(alc, xa - qa, qa), fmaf(alc, xb - qb, qb));
+                            }
+                            *reinterpret_cast<uint4 *>(smem + OFF_X + tile_off(c, 4 * cq + ch)) =
+                                make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
+                    };
+                    if (a.n_iter & 1) mix_x(xp2);
+                    else mix_x(x2);
+                    fence_async_smem();
+                    fence_before();
+                    sync_post(cx, OP_ITER1_LAST | rq);
                 }
             }
 

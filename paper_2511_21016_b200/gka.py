@@ -36,6 +36,7 @@ class GkaDesc(ctypes.Structure):
         ("workspace_bytes", ctypes.c_size_t), ("state_in", ctypes.c_void_p),
         ("device_status", ctypes.c_void_p), ("fro_out", ctypes.c_void_p),
         ("profile_start", ctypes.c_void_p), ("profile_stop", ctypes.c_void_p), ("beta", ctypes.c_void_p),
+        ("alpha", ctypes.c_void_p),
     ]
 
 
@@ -118,7 +119,7 @@ def _check_cuda(*ts):
 
 def make_desc(B, T, heads, d_k, d_v, io_dtype, precision=GKA_PREC_NATIVE, flags=0, stream=None,
               workspace=None, state_in=None, device_status=None, fro_out=None,
-              profile_events=None, beta=None) -> GkaDesc:
+              profile_events=None, beta=None, alpha=None) -> GkaDesc:
     d = GkaDesc()
     d.B, d.T, d.heads, d.d_k, d.d_v = B, T, heads, d_k, d_v
     d.io_dtype, d.precision, d.flags = io_dtype, precision, flags
@@ -129,6 +130,7 @@ def make_desc(B, T, heads, d_k, d_v, io_dtype, precision=GKA_PREC_NATIVE, flags=
     d.device_status = _ptr(device_status)
     d.fro_out = _ptr(fro_out)
     d.beta = _ptr(beta)
+    d.alpha = _ptr(alpha)
     if profile_events is not None:
         d.profile_start, d.profile_stop = profile_events
     return d
@@ -166,12 +168,12 @@ def alloc_workspace(B, T, heads, d, device, chunk=64) -> torch.Tensor:
 
 def gka_fwd_chunked(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=None, *,
                     state_in=None, workspace=None, precision=GKA_PREC_NATIVE, flags=0,
-                    fro_out=None, device_status=None, stream=None, profile_events=None, beta=None):
+                    fro_out=None, device_status=None, stream=None, profile_events=None, beta=None, alpha=None):
     """Chunk-wise GKA forward.  q,k,v: [B,T,heads,d] (f32 or bf16); gate, lam, beta (optional): [B,T,heads] f32.
 
     Returns (out, state_out).  Work is enqueued on ``stream`` (default: torch's current stream).
     """
-    _check_cuda(q, k, v, gate, lam, out, state_out, state_in, workspace, fro_out, device_status, beta)
+    _check_cuda(q, k, v, gate, lam, out, state_out, state_in, workspace, fro_out, device_status, beta, alpha)
     B, T, heads, d = q.shape
     if out is None:
         out = torch.empty_like(v)
@@ -182,7 +184,7 @@ def gka_fwd_chunked(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=No
     if stream is None:
         stream = torch.cuda.current_stream(q.device).cuda_stream
     desc = make_desc(B, T, heads, d, v.shape[-1], _io_code(q), precision, flags, stream, workspace,
-                     state_in, device_status, fro_out, profile_events, beta)
+                     state_in, device_status, fro_out, profile_events, beta, alpha)
     rc = load_library().gka_fwd_chunked(ctypes.byref(desc), q.data_ptr(), k.data_ptr(), v.data_ptr(),
                                         gate.data_ptr(), lam.data_ptr(), int(n_iter), int(chunk),
                                         out.data_ptr(), _ptr(state_out))
@@ -264,7 +266,7 @@ def gka_fwd_chunked_noalloc(q, k, v, gate, lam, n_iter, chunk=64, out=None, stat
 
 
 def gka_decode_step(state, q, k, v, gate, lam, n_iter, out=None, *, flags=0, device_status=None,
-                    stream=None, profile_events=None, beta=None):
+                    stream=None, profile_events=None, beta=None, alpha=None):
     """One recurrent step.  state: [N,heads,2*d*d] f32, updated in place; q,k,v: [N,heads,d]."""
     _check_cuda(state, q, k, v, gate, lam, out, device_status)
     N, heads, d = q.shape
@@ -273,7 +275,7 @@ def gka_decode_step(state, q, k, v, gate, lam, n_iter, out=None, *, flags=0, dev
     if stream is None:
         stream = torch.cuda.current_stream(q.device).cuda_stream
     desc = make_desc(N, 1, heads, d, v.shape[-1], _io_code(q), GKA_PREC_NATIVE, flags, stream,
-                     device_status=device_status, profile_events=profile_events, beta=beta)
+                     device_status=device_status, profile_events=profile_events, beta=beta, alpha=alpha)
     rc = load_library().gka_decode_step(ctypes.byref(desc), state.data_ptr(), q.data_ptr(),
                                         k.data_ptr(), v.data_ptr(), gate.data_ptr(), lam.data_ptr(),
                                         int(n_iter), out.data_ptr())

@@ -368,3 +368,48 @@ def test_decode_beta_write():
     torch.cuda.synchronize()
     assert rel(out.float().cpu().numpy(), ref["out"]) <= TOL_BF16
     assert rel(s_dev.cpu().numpy(), ref["state"]) <= 1e-5
+
+
+# --------------------------------------------------------------------------- alpha-connection
+@pytest.mark.parametrize("bf16,n_iter", [(False, 8), (True, 10), (True, 0), (True, 3)])
+def test_fwd_alpha_connection(bf16, n_iter):
+    """out_t = U_t (alpha_t x_t + (1 - alpha_t) q_t) (Section 4.4), both forward paths, with write strengths too."""
+    cfg = synth.shrink(synth.CONFIGS[1 if bf16 else 0], B=2, heads=3, T=64 * 9, d=128)
+    inp = synth.make_inputs(cfg)
+    alpha, beta = _beta_for(inp, 11), _beta_for(inp, 12)
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], n_iter, alpha=alpha, beta=beta)
+    q, k, v = (to_dev(inp[n], bf16) for n in ("q", "k", "v"))
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out, st = gka.gka_fwd_chunked(q, k, v, to_dev(inp["gate"]), to_dev(inp["lam"]), n_iter, 64,
+                                  alpha=to_dev(alpha), beta=to_dev(beta), device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    e = rel(out.float().cpu().numpy(), ref["out"])
+    print("alpha bf16=%s n_iter %d rel L2 %.3e" % (bf16, n_iter, e))
+    assert e <= (TOL_BF16 if bf16 else TOL_F32)
+    assert rel(st.cpu().numpy(), ref["state"]) <= (5e-3 if bf16 else 1e-5)
+
+
+def test_decode_alpha_connection():
+    cfg = synth.shrink(synth.CONFIGS[2], B=5, heads=3)
+    rng = np.random.default_rng(13)
+    N, Hh, d = cfg.B, cfg.heads, cfg.d
+    state = np.zeros((N, Hh, 2 * d * d), np.float32)
+    for n in range(N):
+        for h in range(Hh):
+            A = rng.standard_normal((d, 8)) * 0.2
+            state[n, h, :d * d] = (A @ A.T).astype(np.float32).ravel()
+            state[n, h, d * d:] = (0.05 * rng.standard_normal(d * d)).astype(np.float32)
+    unit = lambda x: x / np.linalg.norm(x, axis=-1, keepdims=True)
+    q = unit(rng.standard_normal((N, Hh, d))).astype(np.float32)
+    k = unit(rng.standard_normal((N, Hh, d))).astype(np.float32)
+    v = rng.standard_normal((N, Hh, d)).astype(np.float32)
+    gate = (1 / (1 + np.exp(-rng.normal(2, 1, (N, Hh))))).astype(np.float32)
+    lam = (np.log1p(np.exp(rng.standard_normal((N, Hh)))) + 1e-2).astype(np.float32)
+    alpha = (1 / (1 + np.exp(-rng.standard_normal((N, Hh))))).astype(np.float32)
+    ref = oracle.decode(state, q, k, v, gate, lam, 10, alpha=alpha)
+    s_dev = to_dev(state)
+    out = gka.gka_decode_step(s_dev, to_dev(q), to_dev(k), to_dev(v), to_dev(gate), to_dev(lam), 10, alpha=to_dev(alpha))
+    torch.cuda.synchronize()
+    assert rel(out.cpu().numpy(), ref["out"]) <= TOL_F32
+    assert rel(s_dev.cpu().numpy(), ref["state"]) <= 1e-5
