@@ -440,6 +440,9 @@ __device__ __forceinline__ TileInfo tile_info(const FwdArgs &a, int item, long l
     return t;
 }
 
+// EXTRA: the instantiation that also serves write strengths, the alpha-connection and the solve-only result; the
+// plain forward runs the other one, whose code those options do not touch.
+template <bool EXTRA>
 __global__ void __launch_bounds__(kThreadsTile, 1)
 fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO, FwdArgs a) {
@@ -513,8 +516,10 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const uint32_t sbase = smem_u32(smem);
         const size_t st = state_floats(D, D);
         const bool adaptive = (a.flags & GKA_FLAG_ADAPTIVE_LAMBDA) != 0;
-        const bool solve_only = a.solve_only != 0;      // the result is the solve itself: no V, no U, no output product
-        const bool mix = a.alpha != nullptr && !solve_only;   // alpha-connection: the read uses alpha x + (1 - alpha) q
+        const bool solve_only = EXTRA && a.solve_only != 0;   // the result is the solve itself: no V, no U, no output product
+        const float *const beta_p = EXTRA ? a.beta : nullptr;
+        const float *const alpha_p = EXTRA ? a.alpha : nullptr;
+        const bool mix = alpha_p != nullptr && !solve_only;   // alpha-connection: the read uses alpha x + (1 - alpha) q
         uint32_t ph_a = 0, ph_b = 0;
         // first item of the chain of summaries behind this block's start state: the one whose range holds the
         // start of the sequence (its last run begins there, whatever sequence the item itself started in)
@@ -555,12 +560,12 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                  "l"(a.gate + tn.tok0 + (size_t)c * a.heads) : "memory");
                     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->lpre[c])),
                                  "l"(a.lam + tn.tok0 + (size_t)c * a.heads) : "memory");
-                    if (a.beta)
+                    if (beta_p)
                         asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->bpre[c])),
-                                     "l"(a.beta + tn.tok0 + (size_t)c * a.heads) : "memory");
-                    if (a.alpha)
+                                     "l"(beta_p + tn.tok0 + (size_t)c * a.heads) : "memory");
+                    if (alpha_p)
                         asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->apre[c])),
-                                     "l"(a.alpha + tn.tok0 + (size_t)c * a.heads) : "memory");
+                                     "l"(alpha_p + tn.tok0 + (size_t)c * a.heads) : "memory");
                 } else {
                     sc->gpre[c] = 1.f;
                     sc->lpre[c] = 1.f;
@@ -604,13 +609,13 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     sc->zt[c] = exp2f(mc);
                     sc->iz[c] = exp2f(-mc);
                     sc->lam[c] = lamv;
-                    if (a.beta) sc->sb[c] = sqrtf(fmaxf(sc->bpre[c], 0.f));
-                    if (a.alpha) sc->al[c] = sc->apre[c];
+                    if (beta_p) sc->sb[c] = sqrtf(fmaxf(sc->bpre[c], 0.f));
+                    if (alpha_p) sc->al[c] = sc->apre[c];
                     TSTAMP(23);
                 }
                 // ---- K tile has landed (it was fetched during the previous tile): Gram matrix under the set-up
                 wait_bar(cx, stage ? BAR_K1 : BAR_K0, (uint32_t)((tile >> 1) & 1));
-                if (a.beta) {      // beta k k^T is the plain write of sqrt(beta) k: rescale the key rows in place
+                if (beta_p) {      // beta k k^T is the plain write of sqrt(beta) k: rescale the key rows in place
                     cta_sync();
                     scale_rows(smem + off_k, sc->sb, tid);
                     fence_async_smem();
@@ -907,7 +912,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     TSTAMP(16);
                     // O = X' U_0^T + P V (the H buffer holds U_0 since the last score pass), U advance
                     wait_bar(cx, BAR_V, 1u);                       // V tile has landed
-                    if (a.beta) {  // beta v k^T with sqrt(beta) k already in place: the value rows take the other sqrt(beta)
+                    if (beta_p) {  // beta v k^T with sqrt(beta) k already in place: the value rows take the other sqrt(beta)
                         scale_rows(smem + OFF_V, sc->sb, tid);
                         fence_async_smem();
                     }
@@ -980,10 +985,12 @@ cudaError_t launch_fwd_tile(const FwdArgs &a, cudaStream_t stream) {
     if (!make_tile_map(&tmK, a.k, rows, cols, NT) || !make_tile_map(&tmV, a.v, rows, cols, NT) ||
         !make_tile_map(&tmQ, a.q, rows, cols, NT) || !make_tile_map(&tmO, a.out, rows, cols, kChunk))
         return cudaErrorInvalidValue;
-    cudaError_t err = cudaFuncSetAttribute(fwd_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TILE_SMEM);
+    const bool extra = a.beta != nullptr || a.alpha != nullptr || a.solve_only != 0;
+    auto kernel = extra ? fwd_tile_kernel<true> : fwd_tile_kernel<false>;
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TILE_SMEM);
     if (err != cudaSuccess) return err;
     if (a.ev_start) cudaEventRecord(a.ev_start, stream);
-    fwd_tile_kernel<<<a.plan.G, kThreadsTile, TILE_SMEM, stream>>>(tmK, tmV, tmQ, tmO, a);
+    kernel<<<a.plan.G, kThreadsTile, TILE_SMEM, stream>>>(tmK, tmV, tmQ, tmO, a);
     if (a.ev_stop) cudaEventRecord(a.ev_stop, stream);
     return cudaGetLastError();
 }
