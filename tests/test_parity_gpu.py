@@ -413,3 +413,26 @@ def test_decode_alpha_connection():
     torch.cuda.synchronize()
     assert rel(out.cpu().numpy(), ref["out"]) <= TOL_F32
     assert rel(s_dev.cpu().numpy(), ref["state"]) <= 1e-5
+
+
+# --------------------------------------------------------------------------- tile shapes of the tensor-core path
+@pytest.mark.parametrize("B,heads,T", [(1, 1, 64), (1, 1, 64 * 5), (1, 2, 64 * 7), (3, 1, 64 * 3), (1, 1, 64 * 300)])
+def test_fwd_bf16_native_tile_shapes(B, heads, T):
+    """One-chunk sequences, odd chunk counts (half-filled 128-token tiles at run ends), one chunk per work item
+    (every start state comes through a chain of summaries), one long sequence over all work items; with a
+    caller-supplied initial state."""
+    cfg = synth.shrink(synth.CONFIGS[1], B=B, heads=heads, T=T, n_iter=3)
+    inp = synth.make_inputs(cfg)
+    rng = np.random.default_rng(21)
+    d = cfg.d
+    s_in = np.zeros((B, heads, 2 * d * d), np.float32)
+    for b in range(B):
+        for h in range(heads):
+            A = rng.standard_normal((d, 6)) * 0.3
+            s_in[b, h, :d * d] = (A @ A.T).astype(np.float32).ravel()
+            s_in[b, h, d * d:] = (0.1 * rng.standard_normal(d * d)).astype(np.float32)
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], 3, state_in=s_in)
+    out, st, _ = run_fwd(inp, 3, True, state_in=s_in, want_fro=False)
+    assert np.all(np.isfinite(out))
+    assert rel(out, ref["out"]) <= TOL_BF16
+    assert rel(st, ref["state"]) <= 5e-3
