@@ -134,9 +134,14 @@ gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, co
  * out and state_out (nullable) are HOST pointers, preferably page-locked so that the copies are truly
  * asynchronous.  `staging` is caller-owned DEVICE memory of at least gka_fwd_host_staging_bytes()
  * bytes, 256-byte aligned; desc->workspace is required as for gka_fwd_chunked, desc->state_in (if
- * any) stays a device pointer.  The call enqueues on desc->stream: host-to-device copies of the five
- * inputs, the forward kernels, device-to-host copies of out (and state_out); it does not synchronise.
- * The host buffers must stay valid and unmodified until the stream has passed the call.
+ * any, as well as beta / alpha) stays a device pointer.  The call enqueues host-to-device copies of the
+ * five inputs, the forward kernels and device-to-host copies of out (and state_out), and does not
+ * synchronise.  Sequences being independent, the batch is cut into up to 8 slices that pass through the
+ * three stages on three streams (copies in and out on two helper streams the library creates once per
+ * device, kernels on desc->stream), so both copy directions and the kernels overlap; work already on
+ * desc->stream is waited for, and desc->stream waits for the last copy, so stream order is as if
+ * everything ran on desc->stream.  The host buffers must stay valid and unmodified until the stream has
+ * passed the call.
  */
 size_t gka_fwd_host_staging_bytes(const gka_desc *desc);
 gka_status gka_fwd_chunked_host(const gka_desc *desc, void *staging, const void *q, const void *k,

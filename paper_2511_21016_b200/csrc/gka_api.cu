@@ -2,6 +2,9 @@
 // Every step of the path runs in the kernels of this library; nothing here computes.
 #include <stdio.h>
 
+#include <mutex>
+#include <vector>
+
 #include "gka_common.cuh"
 
 namespace gka {
@@ -201,6 +204,42 @@ size_t gka_fwd_host_staging_bytes(const gka_desc *desc) {
            align256(st);
 }
 
+namespace {
+// Helper streams and events of the host-buffer entry point, one set per device, created on first use and
+// kept for the life of the process.
+struct HostPipe {
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, done = nullptr;
+    std::vector<cudaEvent_t> copied, computed;
+};
+std::mutex g_pipe_mutex;
+HostPipe g_pipes[64];
+
+cudaError_t get_pipe(int slices, HostPipe **pipe) {
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipe &hp = g_pipes[dev];
+    if (!hp.in) {
+        if ((err = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking)) != cudaSuccess) return err;
+        if ((err = cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking)) != cudaSuccess) return err;
+        if ((err = cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming)) != cudaSuccess) return err;
+        if ((err = cudaEventCreateWithFlags(&hp.done, cudaEventDisableTiming)) != cudaSuccess) return err;
+    }
+    while ((int)hp.copied.size() < slices) {
+        cudaEvent_t e0, e1;
+        if ((err = cudaEventCreateWithFlags(&e0, cudaEventDisableTiming)) != cudaSuccess) return err;
+        if ((err = cudaEventCreateWithFlags(&e1, cudaEventDisableTiming)) != cudaSuccess) return err;
+        hp.copied.push_back(e0);
+        hp.computed.push_back(e1);
+    }
+    *pipe = &hp;
+    return cudaSuccess;
+}
+}  // namespace
+
 gka_status gka_fwd_chunked_host(const gka_desc *desc, void *staging, const void *q, const void *k,
                                 const void *v, const float *gate, const float *lam, int n_iter,
                                 int chunk, void *out, float *state_out) {
@@ -211,27 +250,69 @@ gka_status gka_fwd_chunked_host(const gka_desc *desc, void *staging, const void 
     const size_t es = desc->io_dtype == GKA_BF16 ? 2 : 4;
     const size_t tok = (size_t)desc->B * desc->T * desc->heads;
     const size_t nqk = tok * desc->d_k * es, nv = tok * desc->d_v * es, ng = tok * 4;
-    const size_t nst = (size_t)desc->B * desc->heads * state_floats(desc->d_k, desc->d_v) * sizeof(float);
+    const size_t st_floats = state_floats(desc->d_k, desc->d_v);
     unsigned char *p = reinterpret_cast<unsigned char *>(staging);
-    void *dq = p; p += align256(nqk);
-    void *dk = p; p += align256(nqk);
-    void *dv = p; p += align256(nv);
-    void *dout = p; p += align256(nv);
-    float *dgate = reinterpret_cast<float *>(p); p += align256(ng);
-    float *dlam = reinterpret_cast<float *>(p); p += align256(ng);
+    unsigned char *dq = p; p += align256(nqk);
+    unsigned char *dk = p; p += align256(nqk);
+    unsigned char *dv = p; p += align256(nv);
+    unsigned char *dout = p; p += align256(nv);
+    unsigned char *dgate = p; p += align256(ng);
+    unsigned char *dlam = p; p += align256(ng);
     float *dstate = reinterpret_cast<float *>(p);
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(desc->stream);
-    cudaError_t err = cudaMemcpyAsync(dq, q, nqk, cudaMemcpyHostToDevice, stream);
-    if (err == cudaSuccess) err = cudaMemcpyAsync(dk, k, nqk, cudaMemcpyHostToDevice, stream);
-    if (err == cudaSuccess) err = cudaMemcpyAsync(dv, v, nv, cudaMemcpyHostToDevice, stream);
-    if (err == cudaSuccess) err = cudaMemcpyAsync(dgate, gate, ng, cudaMemcpyHostToDevice, stream);
-    if (err == cudaSuccess) err = cudaMemcpyAsync(dlam, lam, ng, cudaMemcpyHostToDevice, stream);
-    if (err != cudaSuccess) return cuda_result(err, "gka_fwd_chunked_host (host-to-device copies)");
-    s = gka_fwd_chunked(desc, dq, dk, dv, dgate, dlam, n_iter, chunk, dout, state_out ? dstate : nullptr);
-    if (s != GKA_OK) return s;
-    err = cudaMemcpyAsync(out, dout, nv, cudaMemcpyDeviceToHost, stream);
-    if (err == cudaSuccess && state_out) err = cudaMemcpyAsync(state_out, dstate, nst, cudaMemcpyDeviceToHost, stream);
-    return cuda_result(err, "gka_fwd_chunked_host (device-to-host copies)");
+
+    // Sequences are independent, so the batch is cut into slices that move through three stages on three
+    // streams: copies in (helper stream), kernels (the caller's stream), copies out (second helper stream).
+    // The two copy directions and the kernels overlap; the caller's stream ends up waiting for everything.
+    const int per = (desc->B + 7) / 8;                       // at most 8 slices
+    const int slices = (desc->B + per - 1) / per;
+    HostPipe *hp = nullptr;
+    cudaError_t err = get_pipe(slices, &hp);
+    if (err != cudaSuccess) return cuda_result(err, "gka_fwd_chunked_host (helper streams)");
+    if ((err = cudaEventRecord(hp->start, stream)) != cudaSuccess ||
+        (err = cudaStreamWaitEvent(hp->in, hp->start, 0)) != cudaSuccess ||
+        (err = cudaStreamWaitEvent(hp->out, hp->start, 0)) != cudaSuccess)
+        return cuda_result(err, "gka_fwd_chunked_host (stream ordering)");
+    const size_t tok1 = (size_t)desc->T * desc->heads;       // tokens x heads of one batch element
+    for (int i = 0; i < slices; ++i) {
+        const int b0 = i * per, nb = (b0 + per <= desc->B) ? per : desc->B - b0;
+        const size_t oqk = (size_t)b0 * tok1 * desc->d_k * es, ov = (size_t)b0 * tok1 * desc->d_v * es, og = (size_t)b0 * tok1 * 4;
+        const size_t bqk = (size_t)nb * tok1 * desc->d_k * es, bv = (size_t)nb * tok1 * desc->d_v * es, bg = (size_t)nb * tok1 * 4;
+        err = cudaMemcpyAsync(dq + oqk, static_cast<const unsigned char *>(q) + oqk, bqk, cudaMemcpyHostToDevice, hp->in);
+        if (err == cudaSuccess) err = cudaMemcpyAsync(dk + oqk, static_cast<const unsigned char *>(k) + oqk, bqk, cudaMemcpyHostToDevice, hp->in);
+        if (err == cudaSuccess) err = cudaMemcpyAsync(dv + ov, static_cast<const unsigned char *>(v) + ov, bv, cudaMemcpyHostToDevice, hp->in);
+        if (err == cudaSuccess) err = cudaMemcpyAsync(dgate + og, reinterpret_cast<const unsigned char *>(gate) + og, bg, cudaMemcpyHostToDevice, hp->in);
+        if (err == cudaSuccess) err = cudaMemcpyAsync(dlam + og, reinterpret_cast<const unsigned char *>(lam) + og, bg, cudaMemcpyHostToDevice, hp->in);
+        if (err == cudaSuccess) err = cudaEventRecord(hp->copied[i], hp->in);
+        if (err != cudaSuccess) return cuda_result(err, "gka_fwd_chunked_host (host-to-device copies)");
+    }
+    for (int i = 0; i < slices; ++i) {
+        const int b0 = i * per, nb = (b0 + per <= desc->B) ? per : desc->B - b0;
+        const size_t oqk = (size_t)b0 * tok1 * desc->d_k * es, ov = (size_t)b0 * tok1 * desc->d_v * es, og = (size_t)b0 * tok1 * 4;
+        const size_t ost = (size_t)b0 * desc->heads * st_floats;
+        if ((err = cudaStreamWaitEvent(stream, hp->copied[i], 0)) != cudaSuccess)
+            return cuda_result(err, "gka_fwd_chunked_host (stream ordering)");
+        gka_desc sub = *desc;
+        sub.B = nb;
+        if (desc->state_in) sub.state_in = desc->state_in + ost;
+        if (desc->fro_out) sub.fro_out = desc->fro_out + (size_t)b0 * tok1;
+        if (desc->beta) sub.beta = desc->beta + (size_t)b0 * tok1;
+        if (desc->alpha) sub.alpha = desc->alpha + (size_t)b0 * tok1;
+        if (i > 0) sub.profile_start = sub.profile_stop = nullptr;
+        s = gka_fwd_chunked(&sub, dq + oqk, dk + oqk, dv + ov, reinterpret_cast<const float *>(dgate + og),
+                            reinterpret_cast<const float *>(dlam + og), n_iter, chunk, dout + ov,
+                            state_out ? dstate + ost : nullptr);
+        if (s != GKA_OK) return s;
+        const size_t bv = (size_t)nb * tok1 * desc->d_v * es, bst = (size_t)nb * desc->heads * st_floats * sizeof(float);
+        err = cudaEventRecord(hp->computed[i], stream);
+        if (err == cudaSuccess) err = cudaStreamWaitEvent(hp->out, hp->computed[i], 0);
+        if (err == cudaSuccess) err = cudaMemcpyAsync(static_cast<unsigned char *>(out) + ov, dout + ov, bv, cudaMemcpyDeviceToHost, hp->out);
+        if (err == cudaSuccess && state_out) err = cudaMemcpyAsync(state_out + ost, dstate + ost, bst, cudaMemcpyDeviceToHost, hp->out);
+        if (err != cudaSuccess) return cuda_result(err, "gka_fwd_chunked_host (device-to-host copies)");
+    }
+    err = cudaEventRecord(hp->done, hp->out);
+    if (err == cudaSuccess) err = cudaStreamWaitEvent(stream, hp->done, 0);
+    return cuda_result(err, "gka_fwd_chunked_host (stream ordering)");
 }
 
 }  // extern "C"

@@ -436,3 +436,33 @@ def test_fwd_bf16_native_tile_shapes(B, heads, T):
     assert np.all(np.isfinite(out))
     assert rel(out, ref["out"]) <= TOL_BF16
     assert rel(st, ref["state"]) <= 5e-3
+
+
+# --------------------------------------------------------------------------- host-buffer entry point
+@pytest.mark.parametrize("bf16,B", [(False, 3), (True, 5), (True, 11)])
+def test_fwd_host_buffers_match_device_call_and_oracle(bf16, B):
+    """gka_fwd_chunked_host (pinned host buffers in, pinned host buffers out; the batch moves through the copy
+    and kernel stages in slices) against the oracle and against the device-pointer call."""
+    cfg = synth.shrink(synth.CONFIGS[1 if bf16 else 0], B=B, heads=2, T=64 * 6, d=128, n_iter=4)
+    inp = synth.make_inputs(cfg)
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], cfg.n_iter)
+    tdt = torch.bfloat16 if bf16 else torch.float32
+    pin = {n: torch.from_numpy(np.ascontiguousarray(inp[n])).to(tdt if n in ("q", "k", "v") else torch.float32).pin_memory()
+           for n in ("q", "k", "v", "gate", "lam")}
+    out_pin = torch.empty_like(pin["v"]).pin_memory()
+    st_pin = torch.empty(B, cfg.heads, 2 * cfg.d * cfg.d, dtype=torch.float32).pin_memory()
+    staging = torch.empty(gka.gka_fwd_host_staging_bytes(B, cfg.T, cfg.heads, cfg.d, gka.GKA_BF16 if bf16 else gka.GKA_F32),
+                          dtype=torch.uint8, device=DEV)
+    ws = gka.alloc_workspace(B, cfg.T, cfg.heads, cfg.d, DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for _ in range(2):      # the second call reuses staging and helper streams while the first is still in flight
+        gka.gka_fwd_chunked_host(pin["q"], pin["k"], pin["v"], pin["gate"], pin["lam"], cfg.n_iter, 64, out_pin, st_pin,
+                                 staging=staging, workspace=ws, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    out, st = out_pin.float().numpy(), st_pin.numpy()
+    assert rel(out, ref["out"]) <= (TOL_BF16 if bf16 else TOL_F32)
+    assert rel(st, ref["state"]) <= (5e-3 if bf16 else 1e-5)
+    dev_out, dev_st, _ = run_fwd(inp, cfg.n_iter, bf16, want_fro=False)
+    assert rel(out, dev_out) <= (1e-2 if bf16 else 1e-5)
+    assert rel(st, dev_st) <= (5e-3 if bf16 else 1e-5)
