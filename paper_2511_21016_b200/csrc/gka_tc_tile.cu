@@ -757,7 +757,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const float s0 = sc->s0[c], rho2 = sc->rho2[c], lamc = sc->lam[c], ztc = sc->zt[c], acc_c = sc->ac[c];
                 const unsigned char *qrow = smem + OFF_V;      // q tile: this thread reads row c, its 4 groups of 8 channels
                 uint64_t x2[16];   // the iterate (fp32 pairs), scaled by zt_c (the recurrence is linear), as the operand needs it
-                uint64_t xp2[16];  // the previous iterate (the arrays swap roles every iteration)
+                uint64_t xp2[16];  // the previous iterate
                 {
                     const float x0s = valid ? s0 * ztc : 0.f;  // tokens past the tile stay zero
 #pragma unroll
@@ -805,8 +805,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     ph_b ^= 1u;
                     fence_after();
                     TSTAMP(9);
-                    // x_{i+1} = cfa x_i - beta x_{i-1} + cfx (q - H_c x_i) overwrites x_{i-1}: the two register arrays
-                    // swap roles every iteration (two copies of the code instead of 32 register moves)
+                    // x_{i+1} = cfa x_i - beta x_{i-1} + cfx (q - H_c x_i) overwrites x_{i-1}; the arrays are swapped after
                     auto x_epilogue = [&](uint64_t(&cur)[16], uint64_t(&prv)[16]) {
 #pragma unroll
                         for (int ch = 0; ch < 4; ++ch) {    // 8 channels at a time keeps the transient registers few
@@ -830,8 +829,13 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                 make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
                     };
-                    if (it & 1) x_epilogue(xp2, x2);
-                    else x_epilogue(x2, xp2);
+                    x_epilogue(x2, xp2);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {      // the new iterate becomes x2 again
+                        const uint64_t tmp = x2[i];
+                        x2[i] = xp2[i];
+                        xp2[i] = tmp;
+                    }
                     fence_async_smem();
                     fence_before();
                     sync_post(cx, (it + 1 == a.n_iter ? op_last : OP_ITER1) | rq);
@@ -855,8 +859,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                 make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
                     };
-                    if (a.n_iter & 1) stage_x(xp2);
-                    else stage_x(x2);
+                    stage_x(x2);
                     fence_async_smem();
                 }
                 if (mix) {
@@ -879,8 +882,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                 make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
                     };
-                    if (a.n_iter & 1) mix_x(xp2);
-                    else mix_x(x2);
+                    mix_x(x2);
                     fence_async_smem();
                     fence_before();
                     sync_post(cx, OP_ITER1_LAST | rq);
