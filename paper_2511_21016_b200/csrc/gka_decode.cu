@@ -18,7 +18,9 @@ namespace {
 constexpr int kThreads = 256;
 
 
-template <int D, typename IoT>
+// EXTRA: the instantiation that also serves write strengths and the alpha-connection; the plain step runs the
+// other one (the kernel sits at its register limit).
+template <int D, typename IoT, bool EXTRA>
 __global__ void __launch_bounds__(kThreads, 2)
 decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *__restrict__ k,
               const IoT *__restrict__ v, const float *__restrict__ gate,
@@ -69,7 +71,7 @@ decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *_
     if (tid < D) {
         // write strength beta (Remark on the beta-augmented variant, Section 4.1): beta k k^T and beta v k^T are
         // the plain writes of sqrt(beta) k and sqrt(beta) v
-        const float sb = beta ? sqrtf(fmaxf(beta[head], 0.f)) : 1.f;
+        const float sb = (EXTRA && beta) ? sqrtf(fmaxf(beta[head], 0.f)) : 1.f;
         sQ[tid] = Io<IoT>::load1(q + (size_t)head * D + tid);
         sKv[tid] = sb * Io<IoT>::load1(k + (size_t)head * D + tid);
         sVv[tid] = sb * Io<IoT>::load1(v + (size_t)head * D + tid);
@@ -166,13 +168,13 @@ decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *_
         }
     }
     const float *xs = sX + cur * D;
-    const float al = alpha ? alpha[head] : 1.f;     // alpha-connection (Section 4.4): the read uses alpha x + (1 - alpha) q
+    const float al = (EXTRA && alpha) ? alpha[head] : 1.f;   // alpha-connection (Section 4.4): the read uses alpha x + (1 - alpha) q
     float xc[CG][4];
     float kx = 0.f;
 #pragma unroll
     for (int n = 0; n < CG; ++n) {
         float4 t4 = *reinterpret_cast<const float4 *>(xs + 4 * (lane8 + 8 * n));
-        if (alpha) {
+        if (EXTRA && alpha) {
             const float4 q4 = *reinterpret_cast<const float4 *>(sQ + 4 * (lane8 + 8 * n));
             t4.x = fmaf(al, t4.x - q4.x, q4.x); t4.y = fmaf(al, t4.y - q4.y, q4.y);
             t4.z = fmaf(al, t4.z - q4.z, q4.z); t4.w = fmaf(al, t4.w - q4.w, q4.w);
@@ -214,11 +216,11 @@ cudaError_t launch_typed(float *state, const void *q, const void *k, const void 
                          const float *lam, int n_iter, void *out, int nheads_total, unsigned flags, const float *beta, const float *alpha,
                          int *device_status, cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream) {
     const size_t smem = (size_t)(D * D + 5 * D + 16) * sizeof(float) + 16;
-    cudaError_t err = cudaFuncSetAttribute(decode_kernel<D, IoT>,
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    auto kernel = (beta || alpha) ? decode_kernel<D, IoT, true> : decode_kernel<D, IoT, false>;
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     if (ev_start) cudaEventRecord(ev_start, stream);
-    decode_kernel<D, IoT><<<nheads_total, kThreads, smem, stream>>>(
+    kernel<<<nheads_total, kThreads, smem, stream>>>(
         state, reinterpret_cast<const IoT *>(q), reinterpret_cast<const IoT *>(k),
         reinterpret_cast<const IoT *>(v), gate, lam, n_iter, reinterpret_cast<IoT *>(out), flags, beta, alpha,
         device_status);
