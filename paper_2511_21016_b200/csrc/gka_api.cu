@@ -145,6 +145,7 @@ static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, c
     a.n_iter = n_iter;
     a.flags = desc->flags;
     a.solve_only = solve_only ? 1 : 0;
+    a.start_from_scan = 0;
     a.plan.set(desc->B * desc->heads, desc->T / chunk, G);
     a.ws = carve_workspace(desc->workspace, G, desc->d_k, desc->d_v);
     a.ev_start = reinterpret_cast<cudaEvent_t>(desc->profile_start);

@@ -156,6 +156,7 @@ struct FwdArgs {
     int B, T, heads;
     int n_iter;
     unsigned flags;
+    int start_from_scan;   // tensor path: start states were materialised by the scan kernel (long chains of summaries)
     int solve_only;        // write the solve x_t = CH(H_t + lambda_t I, q_t, r) itself instead of U_t x_t (v unused)
     WorkPlan plan;
     Workspace ws;

@@ -234,10 +234,20 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 
 bool fwd_tc_available() { return get_encode_fn() != nullptr; }
 
-cudaError_t launch_fwd_tc(const FwdArgs &a, cudaStream_t stream) {
+cudaError_t launch_fwd_tc(const FwdArgs &a_in, cudaStream_t stream) {
+    FwdArgs a = a_in;
     cudaError_t err = cudaSuccess;
     bool any_cut = false;
-    for (int i = 0; i + 1 < a.plan.G; ++i) any_cut |= a.plan.cut_out(i);
+    int chain = 0, longest = 0;        // number of summaries behind an item's start state
+    for (int i = 0; i + 1 < a.plan.G; ++i) {
+        any_cut |= a.plan.cut_out(i);
+        chain = a.plan.cut_out(i) ? (a.plan.cut_in(i) ? chain + 1 : 1) : 0;
+        longest = chain > longest ? chain : longest;
+    }
+    // Short chains are folded by the main kernel's blocks themselves; long ones (a sequence spread over many
+    // work items) would make every block re-read its whole chain, so the scan kernel materialises the start
+    // states once instead.
+    a.start_from_scan = longest > 2 ? 1 : 0;
     if (any_cut) {
         alignas(64) CUtensorMap tmK, tmV;      // boxes of 128 tokens x 64 channels
         const int rows = a.B * a.T, cols = a.heads * D;
@@ -245,8 +255,11 @@ cudaError_t launch_fwd_tc(const FwdArgs &a, cudaStream_t stream) {
             return cudaErrorInvalidValue;
         err = cudaFuncSetAttribute(fwd_tc_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM);
         if (err != cudaSuccess) return err;
-        // the main kernel folds the summaries into each block's start state itself
         fwd_tc_summary_kernel<<<a.plan.G, SUM_CT + 32, SUM_SMEM, stream>>>(tmK, tmV, a);
+        if (a.start_from_scan) {
+            err = launch_fwd_scan(a, (int)state_floats(D, D), stream);
+            if (err != cudaSuccess) return err;
+        }
     }
     return launch_fwd_tile(a, stream);
 }

@@ -643,8 +643,9 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
                 // ---- H master, one pass: ||H_0||^2, bf16 copy, scale by the tile's decay
                 {
-                    const StartSrc src = {ti.seq_state, a.ws.delta, a.ws.decay, ti.chained ? chain_j0 : 0,
-                                          ti.chained ? item : 0, st, (size_t)c * D};
+                    const StartSrc src = {(ti.chained && a.start_from_scan) ? a.ws.start + (size_t)item * st : ti.seq_state,
+                                          a.ws.delta, a.ws.decay, (ti.chained && !a.start_from_scan) ? chain_j0 : 0,
+                                          (ti.chained && !a.start_from_scan) ? item : 0, st, (size_t)c * D};
                     float hs = master_pass<true>(cx, tmem + TM_H, ti.run_start, src, decay);
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) hs += __shfl_xor_sync(0xffffffffu, hs, o);
@@ -901,8 +902,9 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     if (tid == 0) issue_tma(&tmV, ti.f, OFF_V, BAR_V);
                     // while the scores of the final iterate are computed: U master pass (bf16 copy into the H buffer, which
                     // no pending product reads; scale by the tile's decay)
-                    const StartSrc src = {ti.seq_state, a.ws.delta, a.ws.decay, ti.chained ? chain_j0 : 0,
-                                          ti.chained ? item : 0, st, (size_t)D * D + (size_t)c * D};
+                    const StartSrc src = {(ti.chained && a.start_from_scan) ? a.ws.start + (size_t)item * st : ti.seq_state,
+                                          a.ws.delta, a.ws.decay, (ti.chained && !a.start_from_scan) ? chain_j0 : 0,
+                                          (ti.chained && !a.start_from_scan) ? item : 0, st, (size_t)D * D + (size_t)c * D};
                     master_pass<false>(cx, tmem + TM_U, ti.run_start, src, exp2f(sc->G2[ti.ntok - 1]));
                     fence_async_smem();
                     wait_bar(cx, BAR_A, ph_a);
