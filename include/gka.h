@@ -12,6 +12,8 @@
  * L = ||H_t||_F + lambda_t, mu = lambda_t (Section 4.1, "Adaptive Regularization").
  * ||H_t||_F is evaluated per token inside each chunk from the chunk-initial state
  * (Section 4.2.1).  The spec name M_t is the paper's U_t; this header uses U.
+ * Optional per-token inputs in the descriptor: write strengths beta_t (beta_t k k^T, beta_t v k^T)
+ * and alpha-connection weights alpha_t (o_t = U_t (alpha_t x_t + (1 - alpha_t) q_t)).
  *
  * Conventions shared by every call
  *   - All data pointers are DEVICE pointers, 16-byte aligned, contiguous row-major.
@@ -22,8 +24,9 @@
  *   - state / state_in / state_out : [B, heads, d_k*d_k + d_v*d_k] float32; per head first
  *     H (d_k x d_k, row-major) then U (d_v x d_k, row-major, U[i][j] = sum v_i k_j).
  *   - The caller owns every buffer.  The library allocates no device memory, keeps no state
- *     between calls apart from cached device attributes, and never synchronises: work is
- *     enqueued on desc->stream and the call returns.
+ *     between calls apart from cached device attributes (and, for gka_fwd_chunked_host, two helper
+ *     streams and a few events per device), and never synchronises: work is enqueued on
+ *     desc->stream and the call returns.
  *   - Argument errors are reported by the return value before anything is launched.  Nothing
  *     throws or aborts.  Device-side waits are bounded; if one runs out the kernel stores
  *     GKA_ERR_TIMEOUT into *desc->device_status (when given) and returns cleanly.
