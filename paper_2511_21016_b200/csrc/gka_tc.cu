@@ -238,16 +238,19 @@ cudaError_t launch_fwd_tc(const FwdArgs &a_in, cudaStream_t stream) {
     FwdArgs a = a_in;
     cudaError_t err = cudaSuccess;
     bool any_cut = false;
-    int chain = 0, longest = 0;        // number of summaries behind an item's start state
-    for (int i = 0; i + 1 < a.plan.G; ++i) {
-        any_cut |= a.plan.cut_out(i);
-        chain = a.plan.cut_out(i) ? (a.plan.cut_in(i) ? chain + 1 : 1) : 0;
-        longest = chain > longest ? chain : longest;
+    int longest = 0;                   // most summaries behind any item's start state
+    for (int i = 0; i + 1 < a.plan.G; ++i) any_cut |= a.plan.cut_out(i);
+    for (int i = 1; i < a.plan.G && any_cut; ++i) {
+        if (!a.plan.cut_in(i)) continue;
+        const long long seq_start = (a.plan.lo(i) / a.plan.N) * a.plan.N;
+        int j0 = i - 1;
+        while (a.plan.lo(j0) > seq_start) --j0;
+        longest = (i - j0) > longest ? (i - j0) : longest;
     }
     // Short chains are folded by the main kernel's blocks themselves; long ones (a sequence spread over many
     // work items) would make every block re-read its whole chain, so the scan kernel materialises the start
     // states once instead.
-    a.start_from_scan = longest > 2 ? 1 : 0;
+    a.start_from_scan = longest > 4 ? 1 : 0;
     if (any_cut) {
         alignas(64) CUtensorMap tmK, tmV;      // boxes of 128 tokens x 64 channels
         const int rows = a.B * a.T, cols = a.heads * D;
