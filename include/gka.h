@@ -133,6 +133,18 @@ gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, co
                            void *out);
 
 /*
+ * The recurrent step over desc->T >= 1 consecutive tokens per sequence (multi-token / speculative decoding):
+ * token after token, exactly what desc->T calls of gka_decode_step compute (eq. (CH) per token), but the
+ * state is read from and written to device memory once per call instead of once per token.
+ * q, k : [B, T, heads, d_k]; v, out : [B, T, heads, d_v]; gate, lam (and desc->beta, desc->alpha when
+ * given) : [B, T, heads]; state : [B, heads, 2*d*d] fp32, updated in place to the state after the last
+ * token.  Needs no workspace.  Same dtype rules, flags and error behaviour as gka_decode_step.
+ */
+gka_status gka_decode_tokens(const gka_desc *desc, float *state, const void *q, const void *k,
+                             const void *v, const float *gate, const float *lam, int n_iter,
+                             void *out);
+
+/*
  * Host-buffer form of the chunked forward (same operation, eq. (CH) chunk-wise): q, k, v, gate, lam,
  * out and state_out (nullable) are HOST pointers, preferably page-locked so that the copies are truly
  * asynchronous.  `staging` is caller-owned DEVICE memory of at least gka_fwd_host_staging_bytes()

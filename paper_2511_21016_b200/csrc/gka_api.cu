@@ -192,6 +192,24 @@ gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, co
     return cuda_result(err, "gka_decode_step");
 }
 
+gka_status gka_decode_tokens(const gka_desc *desc, float *state, const void *q, const void *k,
+                             const void *v, const float *gate, const float *lam, int n_iter,
+                             void *out) {
+    gka_status s = check_desc_common(desc);
+    if (s != GKA_OK) return s;
+    if (!state || !q || !k || !v || !gate || !lam || !out) return GKA_ERR_NULL;
+    if (n_iter < 0 || desc->T < 1) return GKA_ERR_SHAPE;
+    if (!aligned16(state) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+        return GKA_ERR_ALIGN;
+    cudaError_t err = launch_decode_multi(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->T, desc->heads,
+                                          desc->d_k, desc->io_dtype, desc->flags, desc->beta, desc->alpha,
+                                          desc->device_status,
+                                          reinterpret_cast<cudaEvent_t>(desc->profile_start),
+                                          reinterpret_cast<cudaEvent_t>(desc->profile_stop),
+                                          reinterpret_cast<cudaStream_t>(desc->stream));
+    return cuda_result(err, "gka_decode_tokens");
+}
+
 const char *gka_last_error_detail(void) { return g_detail; }
 
 static size_t align256(size_t n) { return (n + 255) / 256 * 256; }

@@ -24,7 +24,7 @@ GKA_ERR_TIMEOUT = 8
 EXPORTS = ("gka_fwd_workspace_bytes", "gka_fwd_chunked", "gka_decode_step", "gka_status_string",
            "gka_fwd_num_work_items", "gka_fwd_work_range", "gka_last_error_detail",
            "gka_fwd_chunked_noalloc", "gka_noalloc_scratch_bytes",
-           "gka_fwd_chunked_host", "gka_fwd_host_staging_bytes", "gka_solve_chunked")
+           "gka_fwd_chunked_host", "gka_fwd_host_staging_bytes", "gka_solve_chunked", "gka_decode_tokens")
 
 
 class GkaDesc(ctypes.Structure):
@@ -81,6 +81,8 @@ def load_library():
         lib.gka_solve_chunked.restype = ci
         lib.gka_decode_step.argtypes = [dp, vp, vp, vp, vp, vp, vp, ci, vp]
         lib.gka_decode_step.restype = ci
+        lib.gka_decode_tokens.argtypes = [dp, vp, vp, vp, vp, vp, vp, ci, vp]
+        lib.gka_decode_tokens.restype = ci
         llp, ip = ctypes.POINTER(ctypes.c_longlong), ctypes.POINTER(ctypes.c_int)
         lib.gka_fwd_work_range.argtypes = [dp, ci, ci, ci, llp, llp, ip, ip]
         lib.gka_fwd_work_range.restype = ci
@@ -281,4 +283,24 @@ def gka_decode_step(state, q, k, v, gate, lam, n_iter, out=None, *, flags=0, dev
                                         int(n_iter), out.data_ptr())
     if rc != GKA_OK:
         raise GkaError(rc, "gka_decode_step")
+    return out
+
+
+def gka_decode_tokens(state, q, k, v, gate, lam, n_iter, out=None, *, flags=0, device_status=None,
+                      stream=None, profile_events=None, beta=None, alpha=None):
+    """The recurrent step over T consecutive tokens.  state: [N,heads,2*d*d] f32, updated in place;
+    q,k,v: [N,T,heads,d]; gate, lam (beta, alpha): [N,T,heads]."""
+    _check_cuda(state, q, k, v, gate, lam, out, device_status)
+    N, T, heads, d = q.shape
+    if out is None:
+        out = torch.empty_like(v)
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    desc = make_desc(N, T, heads, d, v.shape[-1], _io_code(q), GKA_PREC_NATIVE, flags, stream,
+                     device_status=device_status, profile_events=profile_events, beta=beta, alpha=alpha)
+    rc = load_library().gka_decode_tokens(ctypes.byref(desc), state.data_ptr(), q.data_ptr(),
+                                          k.data_ptr(), v.data_ptr(), gate.data_ptr(), lam.data_ptr(),
+                                          int(n_iter), out.data_ptr())
+    if rc != GKA_OK:
+        raise GkaError(rc, "gka_decode_tokens")
     return out

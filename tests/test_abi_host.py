@@ -83,6 +83,10 @@ def test_argument_errors_are_reported_before_any_launch(lib):
     assert rc == 9
     rc = lib.gka_decode_step(None, ok, ok, ok, ok, ok, ok, 3, ok)
     assert rc == 1
+    d0 = gka.make_desc(4, 0, 2, 128, 128, gka.GKA_BF16)
+    assert lib.gka_decode_tokens(ctypes.byref(d0), ok, ok, ok, ok, ok, ok, 3, ok) == 2   # no token
+    assert lib.gka_decode_tokens(ctypes.byref(dd), ok, None, ok, ok, ok, ok, 3, ok) == 1
+    assert lib.gka_decode_tokens(ctypes.byref(dd), ok + 4, ok, ok, ok, ok, ok, 3, ok) == 9
 
 
 @pytest.mark.parametrize("B,T,heads,G", [(4, 4096, 16, 148), (1, 131072, 32, 148), (1, 256, 2, 8),

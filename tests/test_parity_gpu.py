@@ -415,6 +415,49 @@ def test_decode_alpha_connection():
     assert rel(s_dev.cpu().numpy(), ref["state"]) <= 1e-5
 
 
+# --------------------------------------------------------------------------- multi-token decode
+@pytest.mark.parametrize("d,bf16,T,extras", [(128, False, 1, False), (128, False, 7, True), (128, True, 16, False),
+                                              (64, False, 5, True), (64, True, 3, False), (128, True, 4, True)])
+def test_decode_tokens_matches_the_token_recurrence(d, bf16, T, extras):
+    """T tokens in one call continue a prefix state exactly like the token-by-token recurrence (eq. (CH)):
+    outputs and final state against the oracle run on prefix + T tokens, and against T single-token calls."""
+    P = 64
+    cfg = synth.shrink(synth.CONFIGS[0], B=3, heads=2, T=P + T, d=d, n_iter=7)
+    inp = synth.make_inputs(cfg)
+    if bf16:
+        inp = {n: (synth.round_bf16(a) if n in ("q", "k", "v") else a) for n, a in inp.items()}
+    alpha = _beta_for(inp, 3) if extras else None
+    beta = _beta_for(inp, 4) if extras else None
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], 7, alpha=alpha, beta=beta)
+    pre = oracle.fwd(inp["q"][:, :P], inp["k"][:, :P], inp["v"][:, :P], inp["gate"][:, :P], inp["lam"][:, :P], 0,
+                     beta=None if beta is None else beta[:, :P])
+    state0 = pre["state"].astype(np.float32)
+    tail = lambda a, b16=False: to_dev(np.ascontiguousarray(a[:, P:]), b16)
+    opt = lambda a: None if a is None else tail(a)
+    st = to_dev(state0)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = gka.gka_decode_tokens(st, tail(inp["q"], bf16), tail(inp["k"], bf16), tail(inp["v"], bf16),
+                                tail(inp["gate"]), tail(inp["lam"]), 7, alpha=opt(alpha), beta=opt(beta),
+                                device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert rel(out.float().cpu().numpy(), ref["out"][:, P:]) <= (TOL_BF16 if bf16 else TOL_F32)
+    assert rel(st.cpu().numpy(), ref["state"]) <= 1e-5
+    # the same tokens one call at a time
+    st1 = to_dev(state0)
+    outs = []
+    for t in range(P, P + T):
+        one = lambda a, b16=False: to_dev(np.ascontiguousarray(a[:, t]), b16)
+        o = gka.gka_decode_step(st1, one(inp["q"], bf16), one(inp["k"], bf16), one(inp["v"], bf16),
+                                one(inp["gate"]), one(inp["lam"]), 7,
+                                alpha=None if alpha is None else one(alpha),
+                                beta=None if beta is None else one(beta))
+        outs.append(o.float().cpu().numpy())
+    torch.cuda.synchronize()
+    assert rel(out.float().cpu().numpy(), np.stack(outs, axis=1)) <= (1e-2 if bf16 else 1e-6)
+    assert rel(st.cpu().numpy(), st1.cpu().numpy()) <= 1e-6
+
+
 # --------------------------------------------------------------------------- tile shapes of the tensor-core path
 @pytest.mark.parametrize("B,heads,T", [(1, 1, 64), (1, 1, 64 * 5), (1, 2, 64 * 7), (3, 1, 64 * 3), (1, 1, 64 * 300)])
 def test_fwd_bf16_native_tile_shapes(B, heads, T):
