@@ -16,7 +16,8 @@
  * and alpha-connection weights alpha_t (o_t = U_t (alpha_t x_t + (1 - alpha_t) q_t)).
  *
  * Conventions shared by every call
- *   - All data pointers are DEVICE pointers, 16-byte aligned, contiguous row-major.
+ *   - All data pointers are DEVICE pointers, contiguous row-major; q, k, v, out and the states are 16-byte
+ *     aligned, the per-token scalars (gate, lam, fro_out, beta, alpha) 4-byte aligned.
  *     The descriptor itself is a host struct.
  *   - q, k : [B, T, heads, d_k];  v, out : [B, T, heads, d_v];  gate, lam : [B, T, heads] float32.
  *     gate holds gamma_t in (0, 1]; lam holds lambda_t > 0 (absolute), or, with
@@ -30,7 +31,8 @@
  *   - Argument errors are reported by the return value before anything is launched.  Nothing
  *     throws or aborts.  Device-side waits are bounded; if one runs out the kernel stores
  *     GKA_ERR_TIMEOUT into *desc->device_status (when given) and returns cleanly.
- *   - Supported: d_k == d_v in {64, 128}; chunk == 64; T a multiple of chunk; n_iter >= 0.
+ *   - Supported: d_k == d_v in {64, 128}; chunk == 64; any T >= 1 (a sequence is ceil(T / chunk) chunks, the
+ *     last one holds the remaining T mod chunk tokens); n_iter >= 0.
  */
 #ifndef GKA_H_
 #define GKA_H_
@@ -44,14 +46,14 @@ extern "C" {
 typedef enum {
     GKA_OK = 0,
     GKA_ERR_NULL = 1,        /* a required pointer is NULL                                   */
-    GKA_ERR_SHAPE = 2,       /* non-positive size, T not a multiple of chunk, d_k != d_v     */
+    GKA_ERR_SHAPE = 2,       /* non-positive size, d_k != d_v                                */
     GKA_ERR_DTYPE = 3,       /* unknown io_dtype / precision value                           */
     GKA_ERR_UNSUPPORTED = 4, /* a shape or mode outside the supported set                    */
     GKA_ERR_WORKSPACE = 5,   /* workspace missing, misaligned or smaller than required       */
     GKA_ERR_DOMAIN = 6,      /* reserved: input outside its domain                           */
     GKA_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed (launch, attribute, map) */
     GKA_ERR_TIMEOUT = 8,     /* written to *device_status by a kernel whose bounded wait ran out */
-    GKA_ERR_ALIGN = 9        /* a data pointer is not 16-byte aligned                        */
+    GKA_ERR_ALIGN = 9        /* a data pointer is not aligned as required                    */
 } gka_status;
 
 typedef enum { GKA_F32 = 0, GKA_BF16 = 1 } gka_dtype;
@@ -181,8 +183,8 @@ int gka_fwd_num_work_items(const gka_desc *desc, int chunk);
 
 /*
  * Introspection of the work decomposition (pure host arithmetic, no CUDA call): the flat list of
- * B*heads*(T/chunk) chunks is split into num_items contiguous ranges; item `item` owns chunks
- * [*first_chunk, *end_chunk).  Range sizes differ by at most one chunk; when T/chunk is even and
+ * B*heads*ceil(T/chunk) chunks is split into num_items contiguous ranges; item `item` owns chunks
+ * [*first_chunk, *end_chunk).  Range sizes differ by at most one chunk; when ceil(T/chunk) is even and
  * there are at least two chunks per item the boundaries are kept at even chunk offsets (the
  * tensor-core kernel works on pairs of chunks) and sizes differ by at most two.  *cut_in / *cut_out
  * tell whether the range starts / ends inside a sequence (then its start state comes from the

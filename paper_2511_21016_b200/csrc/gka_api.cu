@@ -35,6 +35,7 @@ int sm_count() {
 }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned4(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 
 gka_status check_desc_common(const gka_desc *d) {
     if (!d) return GKA_ERR_NULL;
@@ -51,14 +52,14 @@ gka_status check_fwd_shape(const gka_desc *d, int chunk) {
     gka_status s = check_desc_common(d);
     if (s != GKA_OK) return s;
     if (chunk != kChunk) return chunk <= 0 ? GKA_ERR_SHAPE : GKA_ERR_UNSUPPORTED;
-    if (d->T <= 0 || d->T % chunk != 0) return GKA_ERR_SHAPE;
-    if ((long long)d->B * d->heads * (d->T / chunk) >= (1LL << 31)) return GKA_ERR_UNSUPPORTED;   // 32-bit chunk indices
+    if (d->T <= 0) return GKA_ERR_SHAPE;
+    if ((long long)d->B * d->heads * chunks_of(d->T) >= (1LL << 31)) return GKA_ERR_UNSUPPORTED;   // 32-bit chunk indices
     return GKA_OK;
 }
 
 // Upper bound on work items used for sizing (independent of the device).
 int work_items_cap(const gka_desc *d, int chunk) {
-    long long nc = (long long)d->B * d->heads * (d->T / chunk);
+    long long nc = (long long)d->B * d->heads * chunks_of(d->T);
     return (int)(nc < kMaxWorkItems ? nc : kMaxWorkItems);
 }
 
@@ -73,14 +74,14 @@ const char *gka_status_string(int status) {
     switch (status) {
         case GKA_OK: return "GKA_OK";
         case GKA_ERR_NULL: return "GKA_ERR_NULL: a required pointer is NULL";
-        case GKA_ERR_SHAPE: return "GKA_ERR_SHAPE: bad size (non-positive, T not a multiple of chunk, or d_k != d_v)";
+        case GKA_ERR_SHAPE: return "GKA_ERR_SHAPE: bad size (non-positive, or d_k != d_v)";
         case GKA_ERR_DTYPE: return "GKA_ERR_DTYPE: unknown io_dtype or precision";
         case GKA_ERR_UNSUPPORTED: return "GKA_ERR_UNSUPPORTED: shape or mode outside the supported set";
         case GKA_ERR_WORKSPACE: return "GKA_ERR_WORKSPACE: workspace missing, misaligned or too small";
         case GKA_ERR_DOMAIN: return "GKA_ERR_DOMAIN: input outside its domain";
         case GKA_ERR_CUDA: return "GKA_ERR_CUDA: a CUDA call failed";
         case GKA_ERR_TIMEOUT: return "GKA_ERR_TIMEOUT: a bounded device-side wait ran out";
-        case GKA_ERR_ALIGN: return "GKA_ERR_ALIGN: a data pointer is not 16-byte aligned";
+        case GKA_ERR_ALIGN: return "GKA_ERR_ALIGN: a data pointer is not aligned as required (16 bytes for vectors and states, 4 for per-token scalars)";
         default: return "GKA_ERR_?: unknown status";
     }
 }
@@ -106,7 +107,7 @@ gka_status gka_fwd_work_range(const gka_desc *desc, int chunk, int num_items, in
     if (s != GKA_OK) return s;
     if (!first_chunk || !end_chunk || !cut_in || !cut_out) return GKA_ERR_NULL;
     WorkPlan p;
-    p.set(desc->B * desc->heads, desc->T / chunk, num_items > 0 ? num_items : 1);
+    p.set(desc->B * desc->heads, chunks_of(desc->T), num_items > 0 ? num_items : 1);
     if (num_items <= 0 || num_items > p.NC || item < 0 || item >= num_items) return GKA_ERR_SHAPE;
     *first_chunk = p.lo(item);
     *end_chunk = p.lo(item + 1);
@@ -122,9 +123,10 @@ static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, c
     if (s != GKA_OK) return s;
     if (!q || !k || !v || !gate || !lam || !out) return GKA_ERR_NULL;
     if (n_iter < 0) return GKA_ERR_SHAPE;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(gate) || !aligned16(lam) ||
-        !aligned16(out) || !aligned16(state_out) || !aligned16(desc->state_in) ||
-        !aligned16(desc->fro_out))
+    // vectors and states move in 16-byte pieces; the per-token scalars are read and written one float at a time
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(state_out) ||
+        !aligned16(desc->state_in) || !aligned4(gate) || !aligned4(lam) || !aligned4(desc->fro_out) ||
+        !aligned4(desc->beta) || !aligned4(desc->alpha))
         return GKA_ERR_ALIGN;
     const size_t need = gka_fwd_workspace_bytes(desc, chunk);
     if (!desc->workspace || desc->workspace_bytes < need ||
@@ -146,7 +148,7 @@ static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, c
     a.flags = desc->flags;
     a.solve_only = solve_only ? 1 : 0;
     a.start_from_scan = 0;
-    a.plan.set(desc->B * desc->heads, desc->T / chunk, G);
+    a.plan.set(desc->B * desc->heads, chunks_of(desc->T), G);
     a.ws = carve_workspace(desc->workspace, G, desc->d_k, desc->d_v);
     a.ev_start = reinterpret_cast<cudaEvent_t>(desc->profile_start);
     a.ev_stop = reinterpret_cast<cudaEvent_t>(desc->profile_stop);

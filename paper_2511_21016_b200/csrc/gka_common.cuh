@@ -12,9 +12,11 @@ namespace gka {
 
 constexpr int kChunk = 64;            // tokens per chunk (C)
 constexpr int kMaxWorkItems = 296;    // upper bound on persistent work items (2 per SM on 148 SMs)
+// chunks per sequence: the last one holds the T mod C remaining tokens when T is not a multiple of C
+__host__ __device__ constexpr int chunks_of(int T) { return (T + kChunk - 1) / kChunk; }
 
 // ---------------------------------------------------------------------------------------------
-// Work decomposition.  The B*heads sequences of N = T/C chunks each form one flat list of
+// Work decomposition.  The B*heads sequences of N = ceil(T/C) chunks each form one flat list of
 // NC = B*heads*N chunks; work item i of G owns the contiguous range [lo(i), lo(i+1)).  A range
 // may cover several sequences and may cut a sequence in the middle.  Where an item's range ends
 // inside a sequence the item's last run is summarised (decay product, delta-H, delta-U) by the

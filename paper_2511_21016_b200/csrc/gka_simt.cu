@@ -122,15 +122,18 @@ __device__ __forceinline__ void state_update(float *M, const float *A, const flo
 // transposed with stride XS (dstT[d][token]).  With write strengths (beta-augmented variant, Remark in
 // Section 4.1) key and value rows are scaled by sqrt(beta_t): beta k k^T and beta v k^T are the plain writes of
 // the scaled rows, and every later use of a key in the chunk-wise form carries exactly this factor.
+// Rows from nvalid on (the last chunk of a sequence whose length is not a multiple of C) are zero: a zero key
+// and value write nothing, a zero query solves to zero.
 template <int D, typename IoT>
 __device__ __forceinline__ void load_rows(const IoT *src, size_t row0_elem, size_t row_stride_elem,
-                                          float *dst, float *dstT, const float *beta = nullptr, size_t tok0 = 0,
-                                          int heads = 0) {
+                                          float *dst, float *dstT, int nvalid, const float *beta = nullptr,
+                                          size_t tok0 = 0, int heads = 0) {
     constexpr int F4 = D / 4;
     for (int idx = threadIdx.x; idx < kChunk * F4; idx += kThreads) {
         const int row = idx / F4, c4 = idx % F4;
-        float4 v = Io<IoT>::load4(src + row0_elem + (size_t)row * row_stride_elem + 4 * c4);
-        if (beta) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row < nvalid) v = Io<IoT>::load4(src + row0_elem + (size_t)row * row_stride_elem + 4 * c4);
+        if (beta && row < nvalid) {
             const float sb = sqrtf(fmaxf(beta[tok0 + (size_t)row * heads], 0.f));
             v.x *= sb; v.y *= sb; v.z *= sb; v.w *= sb;
         }
@@ -157,12 +160,12 @@ __device__ __forceinline__ float block_sum(float v, float *red) {
 }
 
 // Gates of one chunk: G[c] = sum_{i<=c} log gamma_i (clamped), zeta = exp(G), w[j] = exp(G[C-1]-G[j]).
-__device__ __forceinline__ void load_gates(const float *gate, const float *lam, size_t tok0, int heads,
+__device__ __forceinline__ void load_gates(const float *gate, const float *lam, size_t tok0, int heads, int nvalid,
                                            float *sG, float *sZeta, float *sLam, float *sW) {
     const int c = threadIdx.x;
-    if (c < kChunk) {
-        sW[c] = fmaxf(logf(gate[tok0 + (size_t)c * heads]), -80.f);  // temporary: log gamma
-        sLam[c] = lam[tok0 + (size_t)c * heads];
+    if (c < kChunk) {      // past the sequence: no decay, any positive lambda
+        sW[c] = c < nvalid ? fmaxf(logf(gate[tok0 + (size_t)c * heads]), -80.f) : 0.f;  // temporary: log gamma
+        sLam[c] = c < nvalid ? lam[tok0 + (size_t)c * heads] : 1.f;
     }
     __syncthreads();
     float g = 0.f;
@@ -203,9 +206,10 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_summary(FwdArgs a) {
     for (long long f = f0; f < f1; ++f) {
         const int n = (int)(f % P.N);
         const size_t tok0 = ((size_t)b * a.T + (size_t)n * kChunk) * a.heads + h;
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, nullptr, a.beta, tok0, a.heads);
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr, a.beta, tok0, a.heads);
-        load_gates(a.gate, a.lam, tok0, a.heads, sG, sZeta, sLam, sW);
+        const int nvalid = min(kChunk, a.T - n * kChunk);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, nullptr, nvalid, a.beta, tok0, a.heads);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr, nvalid, a.beta, tok0, a.heads);
+        load_gates(a.gate, a.lam, tok0, a.heads, nvalid, sG, sZeta, sLam, sW);
         const float zc = sZeta[kChunk - 1];
         decay_log += sG[kChunk - 1];
         state_update<D>(dH, sK, sK, sW, zc, f == f0);
@@ -288,6 +292,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
         const int seq = (int)(f / P.N), n = (int)(f % P.N);
         const int b = seq / a.heads, h = seq % a.heads;
         const size_t tok0 = ((size_t)b * a.T + (size_t)n * kChunk) * a.heads + h;
+        const int nvalid = min(kChunk, a.T - n * kChunk);     // tokens of this chunk that exist
 
         // ---- run start: fetch the start state into the running masters
         if (f == f_lo || n == 0) {
@@ -299,10 +304,10 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
         __syncthreads();
 
         // ---- stage the chunk
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, sKt, a.beta, tok0, a.heads);
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr, a.beta, tok0, a.heads);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, sKt, nvalid, a.beta, tok0, a.heads);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr, nvalid, a.beta, tok0, a.heads);
         for (int e = 4 * tid; e < D * D; e += 4 * kThreads) st4(sH + e, ld4(mH + e));
-        load_gates(a.gate, a.lam, tok0, a.heads, sG, sZeta, sLam, sW);  // ends with a barrier
+        load_gates(a.gate, a.lam, tok0, a.heads, nvalid, sG, sZeta, sLam, sW);  // ends with a barrier
 
         // ---- chunk-wise Frobenius norms (Section 4.2.1), O(C^2) form:
         //      f_c^2 = zeta_c^2 ||H_0||^2 + sum_{j<=c} Gamma[c][j]^2 d_j,
@@ -358,7 +363,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
             const float fc = sqrtf(fmaxf(s, 0.f));
             sF[c] = fc;
             if (adaptive) sLam[c] = sLam[c] * fc;
-            if (a.fro_out) a.fro_out[tok0 + (size_t)c * a.heads] = fc;
+            if (a.fro_out && c < nvalid) a.fro_out[tok0 + (size_t)c * a.heads] = fc;
         }
         __syncthreads();
 
@@ -378,7 +383,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
             omega[t] = 2.f;
 #pragma unroll
             for (int g = 0; g < DG; ++g) {
-                float4 qv = Io<IoT>::load4(gq + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td);
+                float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (c < nvalid) qv = Io<IoT>::load4(gq + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td);
                 qm[t][4 * g + 0] = qv.x; qm[t][4 * g + 1] = qv.y;
                 qm[t][4 * g + 2] = qv.z; qm[t][4 * g + 3] = qv.w;
             }
@@ -450,7 +456,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
             for (int t = 0; t < 4; ++t) {
                 const int c = 4 * tc + t;
 #pragma unroll
-                for (int g = 0; g < DG; ++g)
+                for (int g = 0; g < DG && c < nvalid; ++g)
                     Io<IoT>::store4(gout + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td,
                                     make_float4(xm[t][4 * g + 0], xm[t][4 * g + 1], xm[t][4 * g + 2], xm[t][4 * g + 3]));
             }
@@ -458,7 +464,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
         if (a.alpha && !a.solve_only) {    // alpha-connection (Section 4.4): the read uses alpha x + (1 - alpha) q
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
-                const float al = a.alpha[tok0 + (size_t)(4 * tc + t) * a.heads];
+                const float al = (4 * tc + t < nvalid) ? a.alpha[tok0 + (size_t)(4 * tc + t) * a.heads] : 1.f;
 #pragma unroll
                 for (int u = 0; u < NCH; ++u) xm[t][u] = fmaf(al, xm[t][u] - qm[t][u], qm[t][u]);
             }
@@ -493,7 +499,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
             for (int t = 0; t < 4 && !a.solve_only; ++t) {
                 const int c = 4 * tc + t;
 #pragma unroll
-                for (int g = 0; g < DG; ++g)
+                for (int g = 0; g < DG && c < nvalid; ++g)
                     Io<IoT>::store4(gout + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td,
                                     make_float4(acc[t][4 * g + 0], acc[t][4 * g + 1],
                                                 acc[t][4 * g + 2], acc[t][4 * g + 3]));

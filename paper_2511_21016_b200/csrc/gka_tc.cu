@@ -100,19 +100,19 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         const int ntok_run = nch * C;
         auto issue_tma = [&](int n) {
             const uint32_t dst = sb + (uint32_t)(n % SUM_NS) * SUM_STAGE;
-            const int y = b * a.T + (n0 + 2 * n) * C;
+            const int y = (n0 + 2 * n) * C;
             const uint32_t bar = bars + 8 * (SB_KV0 + n % SUM_NS);
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(65536u) : "memory");
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 const int x = h * D + 64 * hf;
                 asm volatile(
-                    "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
-                        "r"(dst + 16384 * hf), "l"(reinterpret_cast<uint64_t>(&tmK)), "r"(x), "r"(y), "r"(bar)
+                    "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::
+                        "r"(dst + 16384 * hf), "l"(reinterpret_cast<uint64_t>(&tmK)), "r"(x), "r"(y), "r"(b), "r"(bar)
                     : "memory");
                 asm volatile(
-                    "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
-                        "r"(dst + 32768 + 16384 * hf), "l"(reinterpret_cast<uint64_t>(&tmV)), "r"(x), "r"(y), "r"(bar)
+                    "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::
+                        "r"(dst + 32768 + 16384 * hf), "l"(reinterpret_cast<uint64_t>(&tmV)), "r"(x), "r"(y), "r"(b), "r"(bar)
                     : "memory");
             }
         };
@@ -253,8 +253,8 @@ cudaError_t launch_fwd_tc(const FwdArgs &a_in, cudaStream_t stream) {
     a.start_from_scan = longest > 4 ? 1 : 0;
     if (any_cut) {
         alignas(64) CUtensorMap tmK, tmV;      // boxes of 128 tokens x 64 channels
-        const int rows = a.B * a.T, cols = a.heads * D;
-        if (!make_tile_map(&tmK, a.k, rows, cols, NT) || !make_tile_map(&tmV, a.v, rows, cols, NT))
+        const int cols = a.heads * D;
+        if (!make_tile_map(&tmK, a.k, a.B, a.T, cols, NT) || !make_tile_map(&tmV, a.v, a.B, a.T, cols, NT))
             return cudaErrorInvalidValue;
         err = cudaFuncSetAttribute(fwd_tc_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SUM_SMEM);
         if (err != cudaSuccess) return err;

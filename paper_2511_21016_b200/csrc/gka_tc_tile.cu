@@ -430,7 +430,7 @@ __device__ __forceinline__ TileInfo tile_info(const FwdArgs &a, int item, long l
     t.n = (int)(fu - (unsigned)t.seq * (unsigned)P.N);
     const int b = t.seq / a.heads, h = t.seq % a.heads;
     const bool two = (t.n + 1 < P.N) && (m + 1 < n_mine);
-    t.ntok = two ? 2 * kChunk : kChunk;
+    t.ntok = min(two ? 2 * kChunk : kChunk, a.T - t.n * kChunk);   // the last chunk of a sequence may be short
     t.m_next = m + (two ? 2 : 1);
     t.tok0 = ((size_t)b * a.T + (size_t)t.n * kChunk) * a.heads + h;
     t.run_start = (m == 0) || (t.n == 0);
@@ -531,20 +531,20 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
 
         // K (or V) tile of flat chunk f: 128 rows starting at the chunk's first token; rows past the tile's
-        // tokens belong to later tokens (or are zero-filled past the tensor) and are never used
+        // tokens belong to later tokens (or are zero-filled past the end of the sequence) and are never used
         auto issue_tma = [&](const CUtensorMap *map, long long f, uint32_t dst, int bar_idx) {
             const unsigned fu = (unsigned)f;
             const int seq = (int)(fu / (unsigned)P.N), n = (int)(fu - (unsigned)seq * (unsigned)P.N);
             const int b = seq / a.heads, h = seq % a.heads;
-            const int y = b * a.T + n * kChunk;
+            const int y = n * kChunk;
             const uint32_t bar = bars + 8 * bar_idx;
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(32768u) : "memory");
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 const int x = h * D + 64 * hf;
                 asm volatile(
-                    "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
-                        "r"(sbase + dst + 16384 * hf), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+                    "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::
+                        "r"(sbase + dst + 16384 * hf), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(b), "r"(bar)
                     : "memory");
             }
         };
@@ -955,11 +955,11 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 TSTAMP(14);
                 if (tid == 32) {              // one box of 64 tokens x 64 channels per chunk and channel half
                     const int b = ti.seq / a.heads, h = ti.seq % a.heads;
-                    for (int hh = 0; hh < ti.ntok / kChunk; ++hh)
+                    for (int hh = 0; hh < (ti.ntok + kChunk - 1) / kChunk; ++hh)     // rows past the sequence are clipped
                         for (int hf = 0; hf < 2; ++hf)
-                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::
+                            asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::
                                              "l"(reinterpret_cast<uint64_t>(&tmO)), "r"(h * D + 64 * hf),
-                                         "r"(b * a.T + (ti.n + hh) * kChunk), "r"(sbase + OFF_X + 16384 * hf + 8192 * hh)
+                                         "r"((ti.n + hh) * kChunk), "r"(b), "r"(sbase + OFF_X + 16384 * hf + 8192 * hh)
                                          : "memory");
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
@@ -985,9 +985,9 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 
 cudaError_t launch_fwd_tile(const FwdArgs &a, cudaStream_t stream) {
     alignas(64) CUtensorMap tmK, tmV, tmQ, tmO;     // the output is stored chunk by chunk: boxes of 64 rows
-    const int rows = a.B * a.T, cols = a.heads * D;
-    if (!make_tile_map(&tmK, a.k, rows, cols, NT) || !make_tile_map(&tmV, a.v, rows, cols, NT) ||
-        !make_tile_map(&tmQ, a.q, rows, cols, NT) || !make_tile_map(&tmO, a.out, rows, cols, kChunk))
+    const int cols = a.heads * D;
+    if (!make_tile_map(&tmK, a.k, a.B, a.T, cols, NT) || !make_tile_map(&tmV, a.v, a.B, a.T, cols, NT) ||
+        !make_tile_map(&tmQ, a.q, a.B, a.T, cols, NT) || !make_tile_map(&tmO, a.out, a.B, a.T, cols, kChunk))
         return cudaErrorInvalidValue;
     const bool extra = a.beta != nullptr || a.alpha != nullptr || a.solve_only != 0;
     auto kernel = extra ? fwd_tile_kernel<true> : fwd_tile_kernel<false>;

@@ -214,15 +214,17 @@ inline EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// 2-D map over a [B*T rows][heads*D columns] bf16 tensor, box = 64 columns x box_rows rows, 128-byte swizzle.
-inline bool make_tile_map(CUtensorMap *map, const void *base, int rows, int cols, int box_rows) {
+// 3-D map over a [B][T][heads*D] bf16 tensor (coordinates: column, token, batch), box = 64 columns x box_rows
+// tokens of one batch entry, 128-byte swizzle.  Tokens past T read as zero and are not written: the last tile of
+// a sequence may reach past its end.
+inline bool make_tile_map(CUtensorMap *map, const void *base, int B, int T, int cols, int box_rows) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)T, (cuuint64_t)B};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * (cuuint64_t)T};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

@@ -47,7 +47,9 @@ def test_workspace_bytes_arithmetic(lib):
     # tiny problem: 2 sequences x 4 chunks = 8 items
     n = gka.gka_fwd_workspace_bytes(1, 256, 2, 64)
     assert n == ((3 * 8 * 2 * 64 * 64 + 8) * 4 + 255) // 256 * 256
-    assert gka.gka_fwd_workspace_bytes(1, 100, 2, 64) == 0       # T not a multiple of 64
+    # T need not be a multiple of the chunk: 100 tokens are two chunks, the second one short
+    assert gka.gka_fwd_workspace_bytes(1, 100, 2, 64) == gka.gka_fwd_workspace_bytes(1, 128, 2, 64)
+    assert gka.gka_fwd_workspace_bytes(1, 0, 2, 64) == 0
     assert gka.gka_fwd_workspace_bytes(1, 128, 2, 96) == 0       # unsupported head dim
 
 
@@ -68,8 +70,10 @@ def test_argument_errors_are_reported_before_any_launch(lib):
     assert _call_fwd(lib, d, ptrs) == 5                                    # no workspace
     d.workspace, d.workspace_bytes = 256, 16
     assert _call_fwd(lib, d, ptrs) == 5                                    # workspace too small
+    d2 = gka.make_desc(1, 0, 2, 64, 64, gka.GKA_F32)
+    assert _call_fwd(lib, d2, ptrs) == 2                                   # no token
     d2 = gka.make_desc(1, 100, 2, 64, 64, gka.GKA_F32)
-    assert _call_fwd(lib, d2, ptrs) == 2                                   # T % chunk != 0
+    assert _call_fwd(lib, d2, ptrs) == 5                                   # a ragged T passes the shape check
     d3 = gka.make_desc(1, 128, 2, 64, 128, gka.GKA_F32)
     assert _call_fwd(lib, d3, ptrs) == 2                                   # d_k != d_v
     d4 = gka.make_desc(1, 128, 2, 64, 64, 7)

@@ -179,9 +179,10 @@ def test_fwd_is_deterministic():
 
 def test_fwd_gpu_argument_errors():
     q = torch.zeros(1, 100, 1, 64, device=DEV)
+    v = torch.zeros(1, 100, 1, 128, device=DEV)
     g = torch.ones(1, 100, 1, device=DEV)
     with pytest.raises(gka.GkaError) as ei:
-        gka.gka_fwd_chunked(q, q, q, g, g, 1)
+        gka.gka_fwd_chunked(q, q, v, g, g, 1)          # d_k != d_v
     assert ei.value.status == 2
     q = torch.zeros(1, 128, 1, 64, device=DEV)
     g = torch.ones(1, 128, 1, device=DEV)
@@ -415,6 +416,73 @@ def test_decode_alpha_connection():
     assert rel(s_dev.cpu().numpy(), ref["state"]) <= 1e-5
 
 
+# --------------------------------------------------------------------------- sequence lengths that are not multiples of the chunk
+@pytest.mark.parametrize("bf16,d,B,heads,T", [
+    (True, 128, 2, 3, 1), (True, 128, 2, 3, 63), (True, 128, 1, 2, 65), (True, 128, 2, 2, 127), (True, 128, 2, 3, 129),
+    (True, 128, 3, 2, 64 * 5 + 17), (True, 128, 1, 3, 64 * 70 + 33), (True, 128, 1, 1, 64 * 301 + 1),
+    (False, 64, 2, 3, 1), (False, 64, 2, 2, 50), (False, 128, 2, 3, 100), (False, 128, 1, 5, 64 * 5 + 17),
+    (True, 64, 2, 2, 64 * 3 + 5)])
+def test_fwd_ragged_sequence_length(bf16, d, B, heads, T):
+    """The last chunk of every sequence holds T mod 64 tokens: outputs, norms and final state follow the token
+    recurrence (eq. (CH)) for exactly T tokens, and nothing past a sequence's last token is written."""
+    cfg = synth.shrink(synth.CONFIGS[1 if bf16 else 0], B=B, heads=heads, T=T, d=d, n_iter=5)
+    inp = synth.make_inputs(cfg)
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], 5, want_x=True)
+    q, k, v = (to_dev(inp[n], bf16) for n in ("q", "k", "v"))
+    pad = 3 * heads * d
+    big = torch.full((B * T * heads * d + pad,), 7.0, dtype=q.dtype, device=DEV)
+    out = big[:B * T * heads * d].view(B, T, heads, d)
+    fbig = torch.full((B * T * heads + 8,), -3.0, dtype=torch.float32, device=DEV)
+    fro = fbig[:B * T * heads].view(B, T, heads)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    _, st = gka.gka_fwd_chunked(q, k, v, to_dev(inp["gate"]), to_dev(inp["lam"]), 5, 64, out=out, fro_out=fro,
+                                device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert bool((big[B * T * heads * d:] == 7.0).all()) and bool((fbig[B * T * heads:] == -3.0).all())
+    tensor_path = bf16 and d == 128
+    o = out.float().cpu().numpy()
+    if tensor_path and T == 1:
+        # a single token per sequence: o = v (k . x) reads only the component of x along k, which bf16 operands
+        # resolve to eps * |x|, so the bound is the forward error of o = U x under a relative perturbation of x
+        U = ref["state"][..., d * d:].reshape(B, heads, d, d)
+        bound = TOL_BF16 * np.linalg.norm(U, axis=(-2, -1)) * np.linalg.norm(ref["x"][:, 0], axis=-1)
+        assert np.all(np.linalg.norm(o[:, 0] - ref["out"][:, 0], axis=-1) <= bound)
+    else:
+        assert rel(o, ref["out"]) <= (TOL_BF16 if bf16 else TOL_F32)
+    assert rel(fro.cpu().numpy(), ref["fro"]) <= (5e-3 if tensor_path else 1e-5)
+    assert rel(st.cpu().numpy(), ref["state"]) <= (5e-3 if tensor_path else 1e-5)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_ragged_length_with_every_option(bf16):
+    """Write strengths, alpha-connection, a caller's initial state and the solve alone on a ragged length."""
+    B, heads, T, d = 2, 3, 64 * 9 + 40, 128
+    cfg = synth.shrink(synth.CONFIGS[1 if bf16 else 0], B=B, heads=heads, T=T, d=d, n_iter=4)
+    inp = synth.make_inputs(cfg)
+    alpha, beta = _beta_for(inp, 5), _beta_for(inp, 6)
+    rng = np.random.default_rng(17)
+    s_in = np.zeros((B, heads, 2 * d * d), np.float32)
+    for b in range(B):
+        for h in range(heads):
+            A = rng.standard_normal((d, 6)) * 0.3
+            s_in[b, h, :d * d] = (A @ A.T).astype(np.float32).ravel()
+            s_in[b, h, d * d:] = (0.1 * rng.standard_normal(d * d)).astype(np.float32)
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], 4, state_in=s_in, alpha=alpha, beta=beta,
+                     want_x=True)
+    q, k, v = (to_dev(inp[n], bf16) for n in ("q", "k", "v"))
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out, st = gka.gka_fwd_chunked(q, k, v, to_dev(inp["gate"]), to_dev(inp["lam"]), 4, 64, state_in=to_dev(s_in),
+                                  alpha=to_dev(alpha), beta=to_dev(beta), device_status=status)
+    x = gka.gka_solve_chunked(q, k, to_dev(inp["gate"]), to_dev(inp["lam"]), 4, 64, state_in=to_dev(s_in),
+                              beta=to_dev(beta), device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert rel(out.float().cpu().numpy(), ref["out"]) <= (TOL_BF16 if bf16 else TOL_F32)
+    assert rel(x.float().cpu().numpy(), ref["x"]) <= (TOL_BF16 if bf16 else TOL_F32)
+    assert rel(st.cpu().numpy(), ref["state"]) <= (5e-3 if bf16 else 1e-5)
+
+
 # --------------------------------------------------------------------------- multi-token decode
 @pytest.mark.parametrize("d,bf16,T,extras", [(128, False, 1, False), (128, False, 7, True), (128, True, 16, False),
                                               (64, False, 5, True), (64, True, 3, False), (128, True, 4, True)])
@@ -482,11 +550,12 @@ def test_fwd_bf16_native_tile_shapes(B, heads, T):
 
 
 # --------------------------------------------------------------------------- host-buffer entry point
-@pytest.mark.parametrize("bf16,B", [(False, 3), (True, 5), (True, 11)])
-def test_fwd_host_buffers_match_device_call_and_oracle(bf16, B):
+@pytest.mark.parametrize("bf16,B,T", [(False, 3, 64 * 6), (True, 5, 64 * 6), (True, 11, 64 * 6), (True, 5, 64 * 6 + 21),
+                                      (False, 2, 64 + 9)])
+def test_fwd_host_buffers_match_device_call_and_oracle(bf16, B, T):
     """gka_fwd_chunked_host (pinned host buffers in, pinned host buffers out; the batch moves through the copy
     and kernel stages in slices) against the oracle and against the device-pointer call."""
-    cfg = synth.shrink(synth.CONFIGS[1 if bf16 else 0], B=B, heads=2, T=64 * 6, d=128, n_iter=4)
+    cfg = synth.shrink(synth.CONFIGS[1 if bf16 else 0], B=B, heads=2, T=T, d=128, n_iter=4)
     inp = synth.make_inputs(cfg)
     ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], cfg.n_iter)
     tdt = torch.bfloat16 if bf16 else torch.float32

@@ -67,6 +67,6 @@ def test_noalloc_rejects_problems_beyond_the_builtin_scratch():
         gka.gka_fwd_chunked_noalloc(q, q, q, g, g, 1)
     assert ei.value.status == 5                   # GKA_ERR_WORKSPACE, nothing was launched
     # argument errors are still named by their own status
-    desc = gka.make_desc(1, 100, 1, 64, 64, gka.GKA_F32)
+    desc = gka.make_desc(1, 0, 1, 64, 64, gka.GKA_F32)       # no token: rejected before any pointer is used
     rc = lib.gka_fwd_chunked_noalloc(ctypes.byref(desc), 256, 256, 256, 256, 256, 1, 64, 256, None)
     assert rc == 2
