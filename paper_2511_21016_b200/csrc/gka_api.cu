@@ -144,6 +144,7 @@ static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, c
     a.alpha = solve_only ? nullptr : desc->alpha;
     a.device_status = desc->device_status;
     a.B = desc->B; a.T = desc->T; a.heads = desc->heads;
+    a.divH.set((unsigned)desc->heads);
     a.n_iter = n_iter;
     a.flags = desc->flags;
     a.solve_only = solve_only ? 1 : 0;

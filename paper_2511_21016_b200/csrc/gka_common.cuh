@@ -12,6 +12,21 @@ namespace gka {
 
 constexpr int kChunk = 64;            // tokens per chunk (C)
 constexpr int kMaxWorkItems = 296;    // upper bound on persistent work items (2 per SM on 148 SMs)
+// Division of an index below 2^31 by a divisor fixed for a launch, as a multiplication: with l = ceil(log2 d),
+// k = 31 + l and M = floor(2^k / d) + 1, floor(n M / 2^k) = floor(n / d) for every n < 2^31 (the excess
+// M d - 2^k is at most d, so the error n (M d - 2^k) / (d 2^k) stays below 1 / d).
+struct FastDiv {
+    unsigned mul, shift, d;
+    __host__ __device__ void set(unsigned div) {
+        d = div;
+        unsigned l = 0;
+        while ((1ull << l) < div) ++l;
+        shift = 31 + l;
+        mul = (unsigned)((1ull << shift) / div + 1ull);
+    }
+    __host__ __device__ unsigned div(unsigned n) const { return (unsigned)(((unsigned long long)n * mul) >> shift); }
+};
+
 // chunks per sequence: the last one holds the T mod C remaining tokens when T is not a multiple of C
 __host__ __device__ constexpr int chunks_of(int T) { return (T + kChunk - 1) / kChunk; }
 
@@ -34,12 +49,14 @@ struct WorkPlan {
     long long NC;  // total chunks
     int G;         // work items
     int unit;      // granularity of the range boundaries in chunks (1 or 2)
+    FastDiv divN;  // flat chunk index -> sequence
     __host__ __device__ long long lo(int i) const { return unit * (((long long)i * (NC / unit)) / G); }
     __host__ __device__ void set(int bh, int n, int g) {
         BH = bh;
         N = n;
         NC = (long long)bh * n;
         G = g;
+        divN.set((unsigned)n);
         unit = (n % 2 == 0 && 2LL * g <= NC) ? 2 : 1;
     }
     // start of the last run of item i (flat chunk index)
@@ -156,6 +173,7 @@ struct FwdArgs {
     const float *alpha;    // optional alpha-connection weights [B, T, heads]; nullptr = 1
     int *device_status;
     int B, T, heads;
+    FastDiv divH;          // sequence index -> batch entry (divisor: heads)
     int n_iter;
     unsigned flags;
     int start_from_scan;   // tensor path: start states were materialised by the scan kernel (long chains of summaries)

@@ -414,7 +414,7 @@ __device__ __forceinline__ float affine_scan(const Ctx &cx, float a, float b, fl
 // What a phase needs to know about a tile; recomputed from the tile's first chunk index at the start of every
 // phase instead of being carried in registers through the solve loop.
 struct TileInfo {
-    int seq, n, ntok, m_next;
+    int seq, n, ntok, m_next, b, h;
     bool run_start, seq_end;
     size_t tok0;
     long long f;
@@ -426,9 +426,11 @@ __device__ __forceinline__ TileInfo tile_info(const FwdArgs &a, int item, long l
     TileInfo t;
     t.f = f_lo + m;
     const unsigned fu = (unsigned)t.f;         // the chunk list is shorter than 2^31 (checked on the host)
-    t.seq = (int)(fu / (unsigned)P.N);
+    t.seq = (int)P.divN.div(fu);
     t.n = (int)(fu - (unsigned)t.seq * (unsigned)P.N);
-    const int b = t.seq / a.heads, h = t.seq % a.heads;
+    const int b = (int)a.divH.div((unsigned)t.seq), h = t.seq - b * a.heads;
+    t.b = b;
+    t.h = h;
     const bool two = (t.n + 1 < P.N) && (m + 1 < n_mine);
     t.ntok = min(two ? 2 * kChunk : kChunk, a.T - t.n * kChunk);   // the last chunk of a sequence may be short
     t.m_next = m + (two ? 2 : 1);
@@ -534,8 +536,8 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         // tokens belong to later tokens (or are zero-filled past the end of the sequence) and are never used
         auto issue_tma = [&](const CUtensorMap *map, long long f, uint32_t dst, int bar_idx) {
             const unsigned fu = (unsigned)f;
-            const int seq = (int)(fu / (unsigned)P.N), n = (int)(fu - (unsigned)seq * (unsigned)P.N);
-            const int b = seq / a.heads, h = seq % a.heads;
+            const int seq = (int)P.divN.div(fu), n = (int)(fu - (unsigned)seq * (unsigned)P.N);
+            const int b = (int)a.divH.div((unsigned)seq), h = seq - b * a.heads;
             const int y = n * kChunk;
             const uint32_t bar = bars + 8 * bar_idx;
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(32768u) : "memory");
@@ -588,8 +590,9 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 const TileInfo ti = tile_info(a, item, f_lo, n_mine, m);
                 const int ntok = ti.ntok;
                 valid = c < ntok;
-                // the previous tile is finished: the q / V buffer and the other K stage are free
-                if (tid == 0) {
+                // the previous tile is finished: the q / V buffer and the other K stage are free (issued by a thread
+                // that has no part in the gate scan below, which every warp waits for)
+                if (tid == NT) {
                     issue_tma(&tmQ, ti.f, OFF_V, BAR_V);
                     if (ti.m_next < n_mine)
                         issue_tma(&tmK, f_lo + ti.m_next, stage ? OFF_K0 : OFF_K1, stage ? BAR_K0 : BAR_K1);
@@ -954,7 +957,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 cta_sync();
                 TSTAMP(14);
                 if (tid == 32) {              // one box of 64 tokens x 64 channels per chunk and channel half
-                    const int b = ti.seq / a.heads, h = ti.seq % a.heads;
+                    const int b = ti.b, h = ti.h;
                     for (int hh = 0; hh < (ti.ntok + kChunk - 1) / kChunk; ++hh)     // rows past the sequence are clipped
                         for (int hf = 0; hf < 2; ++hf)
                             asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::
