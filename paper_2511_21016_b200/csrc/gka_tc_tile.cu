@@ -42,6 +42,9 @@ constexpr int NT = 128;                    // tokens per tile: one per TMEM lane
 constexpr int CT = 512;                    // compute threads
 constexpr int kThreadsTile = CT + 128;     // + the warpgroup that holds the MMA-issuing thread
 constexpr int kRegsCompute = 112, kRegsIssuer = 32;   // register split after setmaxnreg (launch: 96 each)
+// setmaxnreg.inc waits, without a bound, for registers that the other warpgroup gives back: the split must fit
+// what the block was launched with
+static_assert(CT * kRegsCompute + 128 * kRegsIssuer <= kThreadsTile * 96, "register split exceeds the launch allocation");
 
 // ---- shared memory map (bytes; every operand buffer is 1024-byte aligned).  A [128 rows][128 columns] bf16
 // operand is two boxes of [128 rows][64 columns] with the 128-byte swizzle, 16384 bytes apart.
@@ -52,32 +55,38 @@ constexpr uint32_t OFF_KW = 98304;       // w o K
 constexpr uint32_t OFF_H = 131072;       // bf16 H_0 (later U_0), rows = state rows
 constexpr uint32_t OFF_X = 163840;       // X' (rows = tokens)
 constexpr uint32_t OFF_SC = 196608;      // scalars
-struct TileScalars {
+// Per-token scalars that depend on the gates and the other per-token inputs alone: a helper warp prepares them
+// one tile ahead, into the buffer the tile's parity selects.
+struct GateScalars {
     float lg[NT];          // log2 gamma_c
     float G2[NT];          // cumulative log2 gate
     float ac[NT];          // G2_c - max(G2_c, -60): exponent correction of clamped tokens
     float zt[NT];          // clamped zeta_c
+    float lam[NT];         // lambda_c as given
+    float al[NT];          // alpha_c of the tile's tokens (alpha-connection)
+    float sb[NT];          // sqrt(beta_j) of the tile's keys (beta-augmented write)
+    __align__(16) float iz[NT];   // 2^-G2_c (tiles that are not clamped)
+};
+struct TileScalars {
+    GateScalars g[2];
+    float G2cur[NT];       // copy of the current tile's cumulative log2 gates at a fixed place (read inside the solve loop)
     float lam[NT];         // lambda_c (after the adaptive rule, if any)
     float s0[NT];          // 2 / (L + mu)
     float rho2[NT];
-    __align__(16) float iz[NT];   // 2^-G2_c (tiles that are not clamped)
     float part[2][4][NT];  // Frobenius partial sums: [k H_0 k | Gram part][column quarter][key]
     float carry[2][2][4];  // per-warp totals (a, b) of the two scans
     float red[16];         // per-warp sums of squares of H_0
-    float gpre[NT], lpre[NT], bpre[NT], apre[NT];   // gate, lambda, write strength, alpha of the next tile, copied asynchronously a tile ahead
-    float al[NT];          // alpha_c of the tile's tokens (alpha-connection)
-    float sb[NT];          // sqrt(beta_j) of the tile's keys (beta-augmented write)
     int req_op;            // request to the MMA issuer
     int stop;              // block-wide copy of the abort flag, taken between tiles
 };
-constexpr uint32_t SC_BYTES = 12288;
+constexpr uint32_t SC_BYTES = 15360;
 static_assert(sizeof(TileScalars) <= SC_BYTES, "scalar block too large");
 constexpr uint32_t TILE_SMEM = OFF_SC + SC_BYTES + 1024;   // + slack for the 1024-byte alignment of the base
 
 // ---- TMEM columns: fp32 masters H, U; score accumulator S (P overwrites it in place); Y / O accumulator
 constexpr uint32_t TM_H = 0, TM_U = 128, TM_S = 256, TM_Y = 384;
 
-enum { BAR_K0 = 0, BAR_K1, BAR_V, BAR_A, BAR_B, BAR_COUNT };
+enum { BAR_K0 = 0, BAR_K1, BAR_V, BAR_A, BAR_B, BAR_G0, BAR_G1, BAR_COUNT };   // G: gate scalars of a buffer are ready
 enum { OP_FROB = 1, OP_ITER1, OP_ITER1_LAST, OP_ITER2, OP_OUT, OP_EXIT, OP_GRAM, OP_NONE };
 constexpr int OPF_STAGE = 1 << 8, OPF_PLAIN_K = 1 << 9;   // request flags: K stage; pair P with K instead of w o K
 
@@ -319,7 +328,7 @@ __device__ __forceinline__ void master_store(const Ctx &cx, uint32_t tm_master, 
 // whose P multiplies the unweighted V).
 enum { PF_CONST = 0, PF_TABLE = 1, PF_EXACT = 2 };   // tile-wide constant | 2^-G_j from the table | 2^(ac_c - G_j) per element
 template <int MODE, bool DIAG>
-__device__ __forceinline__ void p_block(const Ctx &cx, uint32_t taddr, float pf, float ac_c) {
+__device__ __forceinline__ void p_block(const Ctx &cx, const GateScalars *gs, uint32_t taddr, float pf, float ac_c) {
     const uint64_t pf2 = f2_pack(pf, pf);
 #pragma unroll
     for (int piece = 0; piece < 2; ++piece) {
@@ -331,11 +340,11 @@ __device__ __forceinline__ void p_block(const Ctx &cx, uint32_t taddr, float pf,
             const int i0 = 16 * piece + 2 * u;
             uint64_t f2 = pf2;
             if (MODE == PF_TABLE) {
-                const float2 z = *reinterpret_cast<const float2 *>(&cx.sc->iz[32 * cx.cq + i0]);
+                const float2 z = *reinterpret_cast<const float2 *>(&gs->iz[32 * cx.cq + i0]);
                 f2 = f2_pack(z.x, z.y);
             } else if (MODE == PF_EXACT) {
-                f2 = f2_pack(ex2_fast(fminf(ac_c - cx.sc->G2[32 * cx.cq + i0], 126.f)),
-                             ex2_fast(fminf(ac_c - cx.sc->G2[32 * cx.cq + i0 + 1], 126.f)));
+                f2 = f2_pack(ex2_fast(fminf(ac_c - cx.sc->G2cur[32 * cx.cq + i0], 126.f)),
+                             ex2_fast(fminf(ac_c - cx.sc->G2cur[32 * cx.cq + i0 + 1], 126.f)));
             }
             float p0, p1;
             f2_unpack(f2_mul(f2_pack(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1])), f2), p0, p1);
@@ -348,7 +357,7 @@ __device__ __forceinline__ void p_block(const Ctx &cx, uint32_t taddr, float pf,
         TMEM_ST8(taddr + 8 * piece, pk);
     }
 }
-__device__ __forceinline__ void p_epilogue(const Ctx &cx, int mode, float pf, float ac_c) {
+__device__ __forceinline__ void p_epilogue(const Ctx &cx, const GateScalars *gs, int mode, float pf, float ac_c) {
     const uint32_t taddr = cx.tmem + TM_S + cx.lane_addr + 32 * cx.cq;
     if (cx.cq > cx.q) {
         uint32_t z[8];
@@ -357,13 +366,13 @@ __device__ __forceinline__ void p_epilogue(const Ctx &cx, int mode, float pf, fl
         TMEM_ST8(taddr, z);
         TMEM_ST8(taddr + 8, z);
     } else if (cx.cq == cx.q) {
-        if (mode == PF_CONST) p_block<PF_CONST, true>(cx, taddr, pf, ac_c);
-        else if (mode == PF_TABLE) p_block<PF_TABLE, true>(cx, taddr, pf, ac_c);
-        else p_block<PF_EXACT, true>(cx, taddr, pf, ac_c);
+        if (mode == PF_CONST) p_block<PF_CONST, true>(cx, gs, taddr, pf, ac_c);
+        else if (mode == PF_TABLE) p_block<PF_TABLE, true>(cx, gs, taddr, pf, ac_c);
+        else p_block<PF_EXACT, true>(cx, gs, taddr, pf, ac_c);
     } else {
-        if (mode == PF_CONST) p_block<PF_CONST, false>(cx, taddr, pf, ac_c);
-        else if (mode == PF_TABLE) p_block<PF_TABLE, false>(cx, taddr, pf, ac_c);
-        else p_block<PF_EXACT, false>(cx, taddr, pf, ac_c);
+        if (mode == PF_CONST) p_block<PF_CONST, false>(cx, gs, taddr, pf, ac_c);
+        else if (mode == PF_TABLE) p_block<PF_TABLE, false>(cx, gs, taddr, pf, ac_c);
+        else p_block<PF_EXACT, false>(cx, gs, taddr, pf, ac_c);
     }
     tmem_wait_st();
 }
@@ -475,6 +484,8 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     const uint32_t tmem = s_tmem_base;
     const uint32_t bars = smem_u32(&s_bars[0]);
     TileScalars *sc = reinterpret_cast<TileScalars *>(smem + OFF_SC);
+    if (tid == 0) *reinterpret_cast<volatile int *>(&sc->stop) = 0;
+    __syncthreads();
 
     const WorkPlan &P = a.plan;
     const int item = blockIdx.x;
@@ -484,6 +495,56 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     if (tid >= CT) {
         // ================================ MMA issuing thread ================================
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssuer));
+        if ((tid >> 5) == (CT >> 5) && n_mine > 0) {
+            // ---- helper warp: the gate scalars of every tile, one tile ahead of the compute warps (cumulative log2
+            // decay by a scan over the tile's tokens, 32 at a time)
+            const int lane = tid & 31;
+            const float *const beta_h = EXTRA ? a.beta : nullptr;
+            const float *const alpha_h = EXTRA ? a.alpha : nullptr;
+            int t = 0;
+            for (int m = 0; m < n_mine; ++t) {
+                const TileInfo ti = tile_info(a, item, f_lo, n_mine, m);
+                // the buffer was last read by tile t - 2: wait for the compute warps to start tile t - 1 (they arrive on
+                // this barrier at the start of every tile that has a successor, and once more if they stop early)
+                if (t >= 2) {
+                    asm volatile("bar.sync 4, 544;" ::: "memory");
+                    if (*reinterpret_cast<const volatile int *>(&sc->stop)) break;
+                }
+                GateScalars *g = &sc->g[t & 1];
+                float run = 0.f;
+#pragma unroll 1
+                for (int grp = 0; grp < 4; ++grp) {
+                    const int cc = 32 * grp + lane;
+                    const bool in = cc < ti.ntok;       // tokens past the tile: no decay, unit lambda / strengths
+                    const size_t idx = ti.tok0 + (size_t)cc * a.heads;
+                    const float gv = in ? __ldg(a.gate + idx) : 1.f;
+                    const float lamv = in ? __ldg(a.lam + idx) : 1.f;
+                    const float bv = (beta_h && in) ? __ldg(beta_h + idx) : 1.f;
+                    const float av = (alpha_h && in) ? __ldg(alpha_h + idx) : 1.f;
+                    const float lgc = fmaxf(log2f(gv), -115.f);
+                    float incl = lgc;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const float up = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= o) incl += up;
+                    }
+                    const float G2c = run + incl;
+                    run += __shfl_sync(0xffffffffu, incl, 31);
+                    const float mc = fmaxf(G2c, -60.f);
+                    g->lg[cc] = lgc;
+                    g->G2[cc] = G2c;
+                    g->ac[cc] = G2c - mc;
+                    g->zt[cc] = exp2f(mc);
+                    g->iz[cc] = exp2f(-mc);
+                    g->lam[cc] = lamv;
+                    g->sb[cc] = sqrtf(fmaxf(bv, 0.f));
+                    g->al[cc] = av;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bars + 8 * (BAR_G0 + (t & 1)));
+                m = ti.m_next;
+            }
+        }
         if ((tid >> 5) == (CT >> 5) + 2 && n_mine > 0) {     // one warp takes the requests; its lane 0 issues
             const uint32_t base14 = (smem_u32(smem) >> 4) & 0x3FFF;
             for (;;) {
@@ -552,33 +613,9 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         };
 
         if (tid == 0 && n_mine > 0) issue_tma(&tmK, f_lo, OFF_K0, BAR_K0);
-        // gate and lambda of this thread's token (threads 0..127), fetched one tile ahead
-        // gate and lambda of this thread's token (threads 0..127) travel global -> shared one tile ahead
-        auto prefetch_gates = [&](int m_of_tile) {
-            if (tid < NT && m_of_tile < n_mine) {
-                const TileInfo tn = tile_info(a, item, f_lo, n_mine, m_of_tile);
-                if (c < tn.ntok) {
-                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->gpre[c])),
-                                 "l"(a.gate + tn.tok0 + (size_t)c * a.heads) : "memory");
-                    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->lpre[c])),
-                                 "l"(a.lam + tn.tok0 + (size_t)c * a.heads) : "memory");
-                    if (beta_p)
-                        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->bpre[c])),
-                                     "l"(beta_p + tn.tok0 + (size_t)c * a.heads) : "memory");
-                    if (alpha_p)
-                        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(&sc->apre[c])),
-                                     "l"(alpha_p + tn.tok0 + (size_t)c * a.heads) : "memory");
-                } else {
-                    sc->gpre[c] = 1.f;
-                    sc->lpre[c] = 1.f;
-                    sc->bpre[c] = 1.f;
-                    sc->apre[c] = 1.f;
-                }
-            }
-        };
-        prefetch_gates(0);
 
         int tile = 0;
+        bool stopped_early = false;
         for (int m = 0; m < n_mine; ++tile) {       // m: index of the tile's first chunk inside the block's range
             const int stage = tile & 1;
             const uint32_t off_k = stage ? OFF_K1 : OFF_K0;
@@ -597,35 +634,22 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     if (ti.m_next < n_mine)
                         issue_tma(&tmK, f_lo + ti.m_next, stage ? OFF_K0 : OFF_K1, stage ? BAR_K0 : BAR_K1);
                 }
-                // ---- gates: cumulative log2 decay by a scan over the tile (threads 0..127 own token c = tid)
-                if (tid < NT) {
-                    asm volatile("cp.async.wait_all;" ::: "memory");
-                    const float g = sc->gpre[c], lamv = sc->lpre[c];
-                    TSTAMP(21);
-                    const float lgc = fmaxf(log2f(g), -115.f);
-                    const float G2c = affine_scan(cx, 1.f, lgc, 0.f, 0);
-                    TSTAMP(22);
-                    const float mc = fmaxf(G2c, -60.f);
-                    sc->lg[c] = lgc;
-                    sc->G2[c] = G2c;
-                    sc->ac[c] = G2c - mc;
-                    sc->zt[c] = exp2f(mc);
-                    sc->iz[c] = exp2f(-mc);
-                    sc->lam[c] = lamv;
-                    if (beta_p) sc->sb[c] = sqrtf(fmaxf(sc->bpre[c], 0.f));
-                    if (alpha_p) sc->al[c] = sc->apre[c];
-                    TSTAMP(23);
-                }
+                // ---- the tile's gate scalars were prepared by the helper warp during the previous tile
+                GateScalars *const gs = &sc->g[stage];
+                if (tile >= 1 && ti.m_next < n_mine) asm volatile("bar.arrive 4, 544;" ::: "memory");   // the other buffer is free
+                wait_bar(cx, stage ? BAR_G1 : BAR_G0, (uint32_t)((tile >> 1) & 1));
+                if (tid < NT) sc->G2cur[c] = gs->G2[c];      // published by the barriers below, long before the solve loop
+                TSTAMP(23);
                 // ---- K tile has landed (it was fetched during the previous tile): Gram matrix under the set-up
                 wait_bar(cx, stage ? BAR_K1 : BAR_K0, (uint32_t)((tile >> 1) & 1));
                 if (beta_p) {      // beta k k^T is the plain write of sqrt(beta) k: rescale the key rows in place
                     cta_sync();
-                    scale_rows(smem + off_k, sc->sb, tid);
+                    scale_rows(smem + off_k, gs->sb, tid);
                     fence_async_smem();
                 }
                 sync_post(cx, OP_GRAM | (stage ? OPF_STAGE : 0));     // also publishes the gate scalars
                 TSTAMP(0);
-                const float Glast = sc->G2[ntok - 1];
+                const float Glast = gs->G2[ntok - 1];
                 clamped = Glast < -60.f;                      // the tile decays below 2^-60: per-element factors
                 pf = exp2f(-fmaxf(Glast, -60.f));             // Gamma[c][j] / zt_c = pf * w_j otherwise
                 const float decay = exp2f(Glast);             // zeta of the whole tile
@@ -636,7 +660,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     const int qi = tid + CT * i;               // 16-byte group index in the 32 KB tile
                     const int j = (qi & 1023) >> 3;            // key row of this group
                     uint4 v = *reinterpret_cast<const uint4 *>(smem + off_k + qi * 16);
-                    const float wj = (j < ntok) ? exp2f(Glast - sc->G2[j]) : 0.f;
+                    const float wj = (j < ntok) ? exp2f(Glast - gs->G2[j]) : 0.f;
                     uint32_t *pv = reinterpret_cast<uint32_t *>(&v);
 #pragma unroll
                     for (int u = 0; u < 4; ++u) pv[u] = pack_bf16(bf16_lo(pv[u]) * wj, bf16_hi(pv[u]) * wj);
@@ -666,7 +690,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 // ---- chunk-wise Frobenius norms: per key, k_j^T H_0 k_j and the decayed squared Gram entries of
                 // the earlier keys.  Thread = (key j = c, 32 columns).
                 {
-                    float kh = 0.f, gs = 0.f;
+                    float kh = 0.f, gsum = 0.f;
 #pragma unroll
                     for (int piece = 0; piece < 2; ++piece) {
                         uint32_t r[16];
@@ -685,7 +709,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                         }
                     }
                     if (cq <= cx.q) {
-                        const float G2j = sc->G2[c];
+                        const float G2j = gs->G2[c];
                         const int lim = (cq == cx.q) ? l : 32;   // keys i < lim come earlier, i == lim is the key itself
                         float gd = 0.f;                          // the key's own squared norm
                         uint64_t acc2 = 0ull;
@@ -702,7 +726,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                     if (ii == lim) gd = g0 * g0;
                                     if (ii + 1 == lim) gd = g1 * g1;
                                     const uint64_t gg = f2_pack(ii < lim ? g0 : 0.f, ii + 1 < lim ? g1 : 0.f);
-                                    const float2 z = *reinterpret_cast<const float2 *>(&sc->iz[32 * cq + ii]);
+                                    const float2 z = *reinterpret_cast<const float2 *>(&gs->iz[32 * cq + ii]);
                                     acc2 = f2_fma(f2_mul(gg, gg), f2_pack(z.x, z.y), acc2);
                                 }
                             } else {
@@ -711,17 +735,17 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                     const int ii = 16 * piece + i;
                                     const float g = __uint_as_float(r[i]);
                                     const float g2 = g * g;
-                                    if (ii < lim) gs = fmaf(2.f * ex2_fast(G2j - sc->G2[32 * cq + ii]), g2, gs);
+                                    if (ii < lim) gsum = fmaf(2.f * ex2_fast(G2j - gs->G2[32 * cq + ii]), g2, gsum);
                                     else if (ii == lim) gd = g2;
                                 }
                             }
                         }
                         float a0, a1;
                         f2_unpack(acc2, a0, a1);
-                        gs = fmaf(2.f * ex2_fast(G2j), a0 + a1, gs) + gd;
+                        gsum = fmaf(2.f * ex2_fast(G2j), a0 + a1, gsum) + gd;
                     }
                     sc->part[0][cq][c] = kh;
-                    sc->part[1][cq][c] = gs;
+                    sc->part[1][cq][c] = gsum;
                 }
                 fence_before();
                 cta_sync();
@@ -736,11 +760,11 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
                     for (int i = 0; i < 16; ++i) hh += sc->red[i];
                     const float kh = (sc->part[0][0][c] + sc->part[0][1][c]) + (sc->part[0][2][c] + sc->part[0][3][c]);
-                    const float gs = (sc->part[1][0][c] + sc->part[1][1][c]) + (sc->part[1][2][c] + sc->part[1][3][c]);
-                    const float dc = fmaf(2.f * exp2f(sc->G2[c]), kh, gs);
-                    const float s = affine_scan(cx, exp2f(2.f * sc->lg[c]), dc, hh, 1);
+                    const float gsum = (sc->part[1][0][c] + sc->part[1][1][c]) + (sc->part[1][2][c] + sc->part[1][3][c]);
+                    const float dc = fmaf(2.f * exp2f(gs->G2[c]), kh, gsum);
+                    const float s = affine_scan(cx, exp2f(2.f * gs->lg[c]), dc, hh, 1);
                     const float fc = sqrtf(fmaxf(s, 0.f));
-                    float lamc = sc->lam[c];
+                    float lamc = gs->lam[c];
                     if (adaptive) lamc *= fc;
                     const float Lpm = fc + 2.f * lamc;
                     const float rho = fc / Lpm;
@@ -758,7 +782,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             // ======================= phase 2: Algorithm 1 on the whole tile =======================
             {
                 // per-token scalars (this thread's token), x_0 = 2 q / (L + mu)
-                const float s0 = sc->s0[c], rho2 = sc->rho2[c], lamc = sc->lam[c], ztc = sc->zt[c], acc_c = sc->ac[c];
+                const float s0 = sc->s0[c], rho2 = sc->rho2[c], lamc = sc->lam[c], ztc = sc->g[stage].zt[c], acc_c = sc->g[stage].ac[c];
                 const unsigned char *qrow = smem + OFF_V;      // q tile: this thread reads row c, its 4 groups of 8 channels
                 uint64_t x2[16];   // the iterate (fp32 pairs), scaled by zt_c (the recurrence is linear), as the operand needs it
                 uint64_t xp2[16];  // the previous iterate
@@ -800,7 +824,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     ph_a ^= 1u;
                     fence_after();
                     TSTAMP(7);
-                    p_epilogue(cx, clamped ? PF_EXACT : PF_CONST, pf, acc_c);
+                    p_epilogue(cx, nullptr, clamped ? PF_EXACT : PF_CONST, pf, acc_c);
                     fence_before();
                     sync_post(cx, OP_ITER2 | rq);
                     TSTAMP(8);
@@ -848,7 +872,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 if (solve_only) {
                     // the solve is the result: x_c = x'_c / zt_c as bf16 into the X' buffer (no product reads it any
                     // more), stored by TMA after the tile's last barrier
-                    const float inv = sc->iz[c];
+                    const float inv = sc->g[tile & 1].iz[c];
                     auto stage_x = [&](const uint64_t(&x)[16]) {
 #pragma unroll
                         for (int ch = 0; ch < 4; ++ch) {
@@ -868,7 +892,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 }
                 if (mix) {
                     // alpha-connection (Section 4.4): X' <- zt (alpha x + (1 - alpha) q) = alpha x' + (1 - alpha) zt q
-                    const float alc = sc->al[c];
+                    const float alc = sc->g[tile & 1].al[c];
                     auto mix_x = [&](const uint64_t(&x)[16]) {
 #pragma unroll
                         for (int ch = 0; ch < 4; ++ch) {
@@ -899,7 +923,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                 int mm = m;
                 asm volatile("" : "+r"(mm));                   // recompute the tile's description
                 const TileInfo ti = tile_info(a, item, f_lo, n_mine, mm);
-                prefetch_gates(ti.m_next);
+                const GateScalars *const gs = &sc->g[tile & 1];
                 if (!solve_only) {
                     // q is no longer needed: its buffer takes the V tile
                     if (tid == 0) issue_tma(&tmV, ti.f, OFF_V, BAR_V);
@@ -908,19 +932,19 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     const StartSrc src = {(ti.chained && a.start_from_scan) ? a.ws.start + (size_t)item * st : ti.seq_state,
                                           a.ws.delta, a.ws.decay, (ti.chained && !a.start_from_scan) ? chain_j0 : 0,
                                           (ti.chained && !a.start_from_scan) ? item : 0, st, (size_t)D * D + (size_t)c * D};
-                    master_pass<false>(cx, tmem + TM_U, ti.run_start, src, exp2f(sc->G2[ti.ntok - 1]));
+                    master_pass<false>(cx, tmem + TM_U, ti.run_start, src, exp2f(gs->G2[ti.ntok - 1]));
                     fence_async_smem();
                     wait_bar(cx, BAR_A, ph_a);
                     ph_a ^= 1u;
                     fence_after();
                     TSTAMP(15);
-                    p_epilogue(cx, clamped ? PF_EXACT : PF_TABLE, pf, sc->ac[c]);   // this P multiplies the unweighted V
+                    p_epilogue(cx, gs, clamped ? PF_EXACT : PF_TABLE, pf, gs->ac[c]);   // this P multiplies the unweighted V
                     fence_before();
                     TSTAMP(16);
                     // O = X' U_0^T + P V (the H buffer holds U_0 since the last score pass), U advance
                     wait_bar(cx, BAR_V, 1u);                       // V tile has landed
                     if (beta_p) {  // beta v k^T with sqrt(beta) k already in place: the value rows take the other sqrt(beta)
-                        scale_rows(smem + OFF_V, sc->sb, tid);
+                        scale_rows(smem + OFF_V, gs->sb, tid);
                         fence_async_smem();
                     }
                     sync_post(cx, OP_OUT | (stage ? OPF_STAGE : 0));
@@ -966,10 +990,14 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                          : "memory");
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
-                if (sc->stop) break;          // the same decision in every thread
+                if (sc->stop) {               // the same decision in every thread
+                    stopped_early = true;
+                    break;
+                }
                 m = ti.m_next;
             }
         }
+        if (stopped_early) asm volatile("bar.arrive 4, 544;" ::: "memory");   // releases the helper warp, which then sees the stop flag
         if (n_mine > 0) sync_post(cx, OP_EXIT);
         if (tid == 32) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // output stores are complete
     }
