@@ -647,8 +647,6 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     scale_rows(smem + off_k, gs->sb, tid);
                     fence_async_smem();
                 }
-                sync_post(cx, OP_GRAM | (stage ? OPF_STAGE : 0));     // also publishes the gate scalars
-                TSTAMP(0);
                 const float Glast = gs->G2[ntok - 1];
                 clamped = Glast < -60.f;                      // the tile decays below 2^-60: per-element factors
                 pf = exp2f(-fmaxf(Glast, -60.f));             // Gamma[c][j] / zt_c = pf * w_j otherwise
@@ -667,6 +665,9 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                     *reinterpret_cast<uint4 *>(smem + OFF_KW + qi * 16) = v;
                 }
                 TSTAMP(2);
+                // the Gram matrix runs under the state pass (the weighting above would fight it for shared memory)
+                sync_post(cx, OP_GRAM | (stage ? OPF_STAGE : 0));
+                TSTAMP(0);
 
                 // ---- H master, one pass: ||H_0||^2, bf16 copy, scale by the tile's decay
                 {
