@@ -34,6 +34,7 @@ from paper_2511_21016_b200 import shard, synth  # noqa: E402
 
 METRIC = "gka_layer_fwd_tokens_per_s"
 UNIT = "tokens/s"
+PROFILE_EVERY = 8          # one timed step in this many also times the main kernel alone
 L2_FLUSH_BYTES = 256 << 20
 
 # DRAM traffic per launch of the dominant kernels (dram__bytes_read.sum + dram__bytes_write.sum from the
@@ -256,16 +257,19 @@ def run_ours(args):
     shard.barrier()
     torch.cuda.synchronize()
     wall0 = time.perf_counter()
+    # Every PROFILE_EVERY-th step also brackets the main kernel alone with the library's profile events (the roofline's
+    # duration).  Those events sit between the summary kernel and the main kernel and so keep the main kernel from
+    # starting its prologue under the summary kernel's tail; the other steps run exactly as a user's call does.
     for i in range(K):
         flush.zero_()
         ev[i][0].record(stream)
-        fwd(profile=(ev[i][2].cuda_event, ev[i][3].cuda_event))
+        fwd(profile=(ev[i][2].cuda_event, ev[i][3].cuda_event) if i % PROFILE_EVERY == 0 else None)
         ev[i][1].record(stream)
     torch.cuda.synchronize()
     shard.barrier()
     wall = time.perf_counter() - wall0
     step_ms = [a.elapsed_time(b) for a, b, _, _ in ev]
-    main_ms = [c.elapsed_time(d) for _, _, c, d in ev]
+    main_ms = [c.elapsed_time(d) for i, (_, _, c, d) in enumerate(ev) if i % PROFILE_EVERY == 0]
     total_ms = shard.max_over_ranks(sum(step_ms), device)
     ms_per_step = total_ms / K
     tokens_per_step = cfg.B * cfg.T * world
@@ -309,7 +313,7 @@ def run_ours(args):
                 "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved_tf / peaks["bf16_tflops"],
                 "peak_source": peaks["source"] + " (burst cuBLAS bf16)",
                 "traffic": NCU_TRAFFIC_BYTES["fwd_main"], "flops_per_launch": flops,
-                "kernel_ms": main_avg_ms, "whole_call_frac": flops / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                "kernel_ms": main_avg_ms, "kernel_launches_timed": len(main_ms), "whole_call_frac": flops / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
                 "frac_of_nominal_2250": achieved_tf / 2250.0}
 
     work_items = gka.gka_fwd_num_work_items(cfg.B, cfg.T, cfg.heads, cfg.d)

@@ -149,6 +149,7 @@ static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, c
     a.flags = desc->flags;
     a.solve_only = solve_only ? 1 : 0;
     a.start_from_scan = 0;
+    a.after_summary = 0;
     a.plan.set(desc->B * desc->heads, chunks_of(desc->T), G);
     a.ws = carve_workspace(desc->workspace, G, desc->d_k, desc->d_v);
     a.ev_start = reinterpret_cast<cudaEvent_t>(desc->profile_start);

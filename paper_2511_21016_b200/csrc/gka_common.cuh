@@ -176,6 +176,7 @@ struct FwdArgs {
     FastDiv divH;          // sequence index -> batch entry (divisor: heads)
     int n_iter;
     unsigned flags;
+    int after_summary;     // tensor path: the main kernel is launched as a programmatic dependent of the summary kernel
     int start_from_scan;   // tensor path: start states were materialised by the scan kernel (long chains of summaries)
     int solve_only;        // write the solve x_t = CH(H_t + lambda_t I, q_t, r) itself instead of U_t x_t (v unused)
     WorkPlan plan;

@@ -34,6 +34,9 @@ __global__ void __launch_bounds__(SUM_CT + 32, 1)
 fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, FwdArgs a) {
     const WorkPlan &P = a.plan;
     const int item = blockIdx.x;
+    // the main kernel may be launched as a programmatic dependent: its blocks may take the SMs that this grid leaves
+    // and run their prologue; they wait for this grid's completion before they read a summary
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (!P.cut_out(item)) return;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t s_bars[SB_COUNT];
@@ -262,6 +265,8 @@ cudaError_t launch_fwd_tc(const FwdArgs &a_in, cudaStream_t stream) {
         if (a.start_from_scan) {
             err = launch_fwd_scan(a, (int)state_floats(D, D), stream);
             if (err != cudaSuccess) return err;
+        } else {
+            a.after_summary = 1;
         }
     }
     return launch_fwd_tile(a, stream);

@@ -613,6 +613,9 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         };
 
         if (tid == 0 && n_mine > 0) issue_tma(&tmK, f_lo, OFF_K0, BAR_K0);
+        // launched as a programmatic dependent of the summary kernel: everything above overlapped its tail; the
+        // summaries are read by these threads only (no effect when there is no such dependency)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
 
         int tile = 0;
         bool stopped_early = false;
@@ -1026,7 +1029,18 @@ cudaError_t launch_fwd_tile(const FwdArgs &a, cudaStream_t stream) {
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TILE_SMEM);
     if (err != cudaSuccess) return err;
     if (a.ev_start) cudaEventRecord(a.ev_start, stream);
-    kernel<<<a.plan.G, kThreadsTile, TILE_SMEM, stream>>>(tmK, tmV, tmQ, tmO, a);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)a.plan.G);
+    cfg.blockDim = dim3(kThreadsTile);
+    cfg.dynamicSmemBytes = TILE_SMEM;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.after_summary ? 1 : 0;
+    err = cudaLaunchKernelEx(&cfg, kernel, tmK, tmV, tmQ, tmO, a);
+    if (err != cudaSuccess) return err;
     if (a.ev_stop) cudaEventRecord(a.ev_stop, stream);
     return cudaGetLastError();
 }
