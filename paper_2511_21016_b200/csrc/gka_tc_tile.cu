@@ -87,7 +87,7 @@ constexpr uint32_t TILE_SMEM = OFF_SC + SC_BYTES + 1024;   // + slack for the 10
 constexpr uint32_t TM_H = 0, TM_U = 128, TM_S = 256, TM_Y = 384;
 
 enum { BAR_K0 = 0, BAR_K1, BAR_V, BAR_A, BAR_B, BAR_G0, BAR_G1, BAR_COUNT };   // G: gate scalars of a buffer are ready
-enum { OP_FROB = 1, OP_ITER1, OP_ITER1_LAST, OP_ITER2, OP_OUT, OP_EXIT, OP_GRAM, OP_NONE };
+enum { OP_FROB = 1, OP_ITER1, OP_ITER1_LAST, OP_ITER2, OP_OUT, OP_EXIT, OP_GRAM, OP_NONE, OP_OUT_U0 };
 constexpr int OPF_STAGE = 1 << 8, OPF_PLAIN_K = 1 << 9;   // request flags: K stage; pair P with K instead of w o K
 
 // ---- operand descriptor constants relative to (shared base >> 4); k-steps of 16
@@ -162,9 +162,12 @@ __device__ __forceinline__ void issuer_run(int req, uint32_t base14, uint32_t tm
         mma8_mm<K_mn, Kw_mn>(tm_H, kb, base14, I_MM);        // H += K^T (w o K)
         mma8_kk<0, K_k, H_k>(tm_Y, kb, base14, I_KK);        // K H_0
         mma_commit(bars + 8 * BAR_A);
+    } else if (op == OP_OUT_U0) {
+        // X' U_0^T (the H buffer holds U_0 now): posted as soon as U_0 is staged, it runs behind the last score product,
+        // under the score epilogue; completion is covered by OP_OUT's first commit
+        mma8_kk<0, X_k, H_k>(tm_Y, base14, base14, I_KK);
     } else if (op == OP_OUT) {
-        mma8_kk<0, X_k, H_k>(tm_Y, base14, base14, I_KK);    // X' U_0^T (the H buffer holds U_0 now)
-        mma8_pm<V_mn>(tm_Y, tm_S, base14, I_PM);             // + P V
+        mma8_pm<V_mn>(tm_Y, tm_S, base14, I_PM);             // O = X' U_0^T + P V
         mma_commit(bars + 8 * BAR_A);
         mma8_mm<V_mn, Kw_mn>(tm_U, base14, base14, I_MM);    // U += V^T (w o K)
         mma_commit(bars + 8 * BAR_B);
@@ -938,6 +941,8 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                                           (ti.chained && !a.start_from_scan) ? item : 0, st, (size_t)D * D + (size_t)c * D};
                     master_pass<false>(cx, tmem + TM_U, ti.run_start, src, exp2f(gs->G2[ti.ntok - 1]));
                     fence_async_smem();
+                    fence_before();
+                    sync_post(cx, OP_OUT_U0);
                     wait_bar(cx, BAR_A, ph_a);
                     ph_a ^= 1u;
                     fence_after();
