@@ -279,12 +279,12 @@ __device__ __forceinline__ float master_pass(const Ctx &cx, uint32_t tm_master, 
                 r[4 * i + 2] = __float_as_uint(v4.z); r[4 * i + 3] = __float_as_uint(v4.w);
             }
             for (int j = src.j0; j < src.j1; ++j) {
-                // summaries come from the kernel this one may overlap with as its programmatic dependent: read them past
-                // L1 (they were written before the dependency wait returned; no read-only path)
-                const float dj = __ldcg(src.decay + j);
+                // summaries come from the kernel this one may overlap with as its programmatic dependent: ordinary loads
+                // (visible after the dependency wait), not the read-only path, whose data must not change under the kernel
+                const float dj = *reinterpret_cast<const volatile float *>(src.decay + j);
                 float4 dd[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) dd[i] = __ldcg(reinterpret_cast<const float4 *>(src.delta + (size_t)j * src.st + e) + i);
+                for (int i = 0; i < 4; ++i) dd[i] = *(reinterpret_cast<const float4 *>(src.delta + (size_t)j * src.st + e) + i);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const float4 d4 = dd[i];
