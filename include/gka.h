@@ -153,7 +153,9 @@ gka_status gka_decode_tokens(const gka_desc *desc, float *state, const void *q, 
  * bytes, 256-byte aligned; desc->workspace is required as for gka_fwd_chunked, desc->state_in (if
  * any, as well as beta / alpha) stays a device pointer.  The call enqueues host-to-device copies of the
  * five inputs, the forward kernels and device-to-host copies of out (and state_out), and does not
- * synchronise.  Sequences being independent, the batch is cut into up to 8 slices that pass through the
+ * synchronise.  Sequences being independent, the batch is cut into up to 8 slices (and the sequences of the last
+ * slice into two pieces of whole 128-token tiles, whose state is carried on the device, so that little work is
+ * left when the last input byte has arrived) that pass through the
  * three stages on three streams (copies in and out on two helper streams the library creates once per
  * device, kernels on desc->stream), so both copy directions and the kernels overlap; work already on
  * desc->stream is waited for, and desc->stream waits for the last copy, so stream order is as if

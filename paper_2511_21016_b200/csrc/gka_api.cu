@@ -223,8 +223,9 @@ size_t gka_fwd_host_staging_bytes(const gka_desc *desc) {
     const size_t es = desc->io_dtype == GKA_BF16 ? 2 : 4;
     const size_t tok = (size_t)desc->B * desc->T * desc->heads;
     const size_t st = (size_t)desc->B * desc->heads * state_floats(desc->d_k, desc->d_v) * sizeof(float);
+    const size_t carry = 2 * (size_t)desc->heads * state_floats(desc->d_k, desc->d_v) * sizeof(float);
     return 2 * align256(tok * desc->d_k * es) + 2 * align256(tok * desc->d_v * es) + 2 * align256(tok * 4) +
-           align256(st);
+           align256(st) + align256(carry);
 }
 
 namespace {
@@ -281,56 +282,90 @@ gka_status gka_fwd_chunked_host(const gka_desc *desc, void *staging, const void 
     unsigned char *dout = p; p += align256(nv);
     unsigned char *dgate = p; p += align256(ng);
     unsigned char *dlam = p; p += align256(ng);
-    float *dstate = reinterpret_cast<float *>(p);
+    float *dstate = reinterpret_cast<float *>(p); p += align256((size_t)desc->B * desc->heads * st_floats * sizeof(float));
+    float *dcarry = reinterpret_cast<float *>(p);            // two states of one batch entry, for the pieces of a sequence
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(desc->stream);
 
     // Sequences are independent, so the batch is cut into slices that move through three stages on three
     // streams: copies in (helper stream), kernels (the caller's stream), copies out (second helper stream).
     // The two copy directions and the kernels overlap; the caller's stream ends up waiting for everything.
-    const int per = (desc->B + 7) / 8;                       // at most 8 slices
-    const int slices = (desc->B + per - 1) / per;
+    // What the pipeline cannot hide is its tail, the kernels and the copy out of the last piece, so the last
+    // batch entries are also cut along the sequence (the state is carried from piece to piece on the device).
+    struct Job { int b0, nb, t0, tn; bool first, last; };
+    std::vector<Job> jobs;
+    const int per = (desc->B + 7) / 8;                       // at most 8 batch slices
+    const int nslices = (desc->B + per - 1) / per;
+    // pieces of the sequences of the last slice: two halves measured best (every further piece costs about as much
+    // as it takes off the tail)
+    const int tpieces = (desc->T >= 4 * 2 * kChunk) ? 2 : 1;
+    for (int i = 0; i < nslices; ++i) {
+        const int b0 = i * per, nb = (b0 + per <= desc->B) ? per : desc->B - b0;
+        if (i + 1 < nslices || tpieces == 1) {
+            jobs.push_back({b0, nb, 0, desc->T, true, true});
+        } else {
+            const int tstep = ((desc->T / tpieces + 2 * kChunk - 1) / (2 * kChunk)) * (2 * kChunk);   // whole 128-token tiles
+            for (int b = b0; b < b0 + nb; ++b) {
+                for (int t0 = 0; t0 < desc->T; t0 += tstep)
+                    jobs.push_back({b, 1, t0, (t0 + tstep < desc->T) ? tstep : desc->T - t0, t0 == 0, t0 + tstep >= desc->T});
+            }
+        }
+    }
+    const int njobs = (int)jobs.size();
     HostPipe *hp = nullptr;
-    cudaError_t err = get_pipe(slices, &hp);
+    cudaError_t err = get_pipe(njobs, &hp);
     if (err != cudaSuccess) return cuda_result(err, "gka_fwd_chunked_host (helper streams)");
     if ((err = cudaEventRecord(hp->start, stream)) != cudaSuccess ||
         (err = cudaStreamWaitEvent(hp->in, hp->start, 0)) != cudaSuccess ||
         (err = cudaStreamWaitEvent(hp->out, hp->start, 0)) != cudaSuccess)
         return cuda_result(err, "gka_fwd_chunked_host (stream ordering)");
-    const size_t tok1 = (size_t)desc->T * desc->heads;       // tokens x heads of one batch element
-    for (int i = 0; i < slices; ++i) {
-        const int b0 = i * per, nb = (b0 + per <= desc->B) ? per : desc->B - b0;
-        const size_t oqk = (size_t)b0 * tok1 * desc->d_k * es, ov = (size_t)b0 * tok1 * desc->d_v * es, og = (size_t)b0 * tok1 * 4;
-        const size_t bqk = (size_t)nb * tok1 * desc->d_k * es, bv = (size_t)nb * tok1 * desc->d_v * es, bg = (size_t)nb * tok1 * 4;
-        err = cudaMemcpyAsync(dq + oqk, static_cast<const unsigned char *>(q) + oqk, bqk, cudaMemcpyHostToDevice, hp->in);
-        if (err == cudaSuccess) err = cudaMemcpyAsync(dk + oqk, static_cast<const unsigned char *>(k) + oqk, bqk, cudaMemcpyHostToDevice, hp->in);
-        if (err == cudaSuccess) err = cudaMemcpyAsync(dv + ov, static_cast<const unsigned char *>(v) + ov, bv, cudaMemcpyHostToDevice, hp->in);
-        if (err == cudaSuccess) err = cudaMemcpyAsync(dgate + og, reinterpret_cast<const unsigned char *>(gate) + og, bg, cudaMemcpyHostToDevice, hp->in);
-        if (err == cudaSuccess) err = cudaMemcpyAsync(dlam + og, reinterpret_cast<const unsigned char *>(lam) + og, bg, cudaMemcpyHostToDevice, hp->in);
+    const size_t hh = (size_t)desc->heads;
+    auto copy = [&](unsigned char *dst, const void *src, size_t off, size_t bytes, cudaMemcpyKind kind, cudaStream_t on) {
+        return kind == cudaMemcpyHostToDevice
+                   ? cudaMemcpyAsync(dst + off, static_cast<const unsigned char *>(src) + off, bytes, kind, on)
+                   : cudaMemcpyAsync(static_cast<unsigned char *>(const_cast<void *>(src)) + off, dst + off, bytes, kind, on);
+    };
+    for (int i = 0; i < njobs; ++i) {
+        const Job &j = jobs[i];
+        // a job's tokens are one contiguous range: whole batch entries, or a token range of one entry
+        const size_t tok0 = ((size_t)j.b0 * desc->T + j.t0) * hh, ntok = (size_t)j.nb * j.tn * hh;
+        err = copy(dq, q, tok0 * desc->d_k * es, ntok * desc->d_k * es, cudaMemcpyHostToDevice, hp->in);
+        if (err == cudaSuccess) err = copy(dk, k, tok0 * desc->d_k * es, ntok * desc->d_k * es, cudaMemcpyHostToDevice, hp->in);
+        if (err == cudaSuccess) err = copy(dv, v, tok0 * desc->d_v * es, ntok * desc->d_v * es, cudaMemcpyHostToDevice, hp->in);
+        if (err == cudaSuccess) err = copy(dgate, gate, tok0 * 4, ntok * 4, cudaMemcpyHostToDevice, hp->in);
+        if (err == cudaSuccess) err = copy(dlam, lam, tok0 * 4, ntok * 4, cudaMemcpyHostToDevice, hp->in);
         if (err == cudaSuccess) err = cudaEventRecord(hp->copied[i], hp->in);
         if (err != cudaSuccess) return cuda_result(err, "gka_fwd_chunked_host (host-to-device copies)");
     }
-    for (int i = 0; i < slices; ++i) {
-        const int b0 = i * per, nb = (b0 + per <= desc->B) ? per : desc->B - b0;
-        const size_t oqk = (size_t)b0 * tok1 * desc->d_k * es, ov = (size_t)b0 * tok1 * desc->d_v * es, og = (size_t)b0 * tok1 * 4;
-        const size_t ost = (size_t)b0 * desc->heads * st_floats;
+    int carry = 0;
+    for (int i = 0; i < njobs; ++i) {
+        const Job &j = jobs[i];
+        const size_t tok0 = ((size_t)j.b0 * desc->T + j.t0) * hh, ntok = (size_t)j.nb * j.tn * hh;
+        const size_t ost = (size_t)j.b0 * hh * st_floats;
         if ((err = cudaStreamWaitEvent(stream, hp->copied[i], 0)) != cudaSuccess)
             return cuda_result(err, "gka_fwd_chunked_host (stream ordering)");
         gka_desc sub = *desc;
-        sub.B = nb;
-        if (desc->state_in) sub.state_in = desc->state_in + ost;
-        if (desc->fro_out) sub.fro_out = desc->fro_out + (size_t)b0 * tok1;
-        if (desc->beta) sub.beta = desc->beta + (size_t)b0 * tok1;
-        if (desc->alpha) sub.alpha = desc->alpha + (size_t)b0 * tok1;
+        sub.B = j.nb;
+        sub.T = j.tn;
+        // the first piece of a sequence starts from the caller's state (or zero), the others from the state the
+        // piece before left in the carry buffer; the last one writes the caller's state_out
+        if (j.first) sub.state_in = desc->state_in ? desc->state_in + ost : nullptr;
+        else sub.state_in = dcarry + (size_t)carry * hh * st_floats;
+        float *piece_state = j.last ? (state_out ? dstate + ost : nullptr) : dcarry + (size_t)(carry ^ 1) * hh * st_floats;
+        if (!j.last) carry ^= 1;
+        if (desc->fro_out) sub.fro_out = desc->fro_out + tok0;
+        if (desc->beta) sub.beta = desc->beta + tok0;
+        if (desc->alpha) sub.alpha = desc->alpha + tok0;
         if (i > 0) sub.profile_start = sub.profile_stop = nullptr;
-        s = gka_fwd_chunked(&sub, dq + oqk, dk + oqk, dv + ov, reinterpret_cast<const float *>(dgate + og),
-                            reinterpret_cast<const float *>(dlam + og), n_iter, chunk, dout + ov,
-                            state_out ? dstate + ost : nullptr);
+        s = gka_fwd_chunked(&sub, dq + tok0 * desc->d_k * es, dk + tok0 * desc->d_k * es, dv + tok0 * desc->d_v * es,
+                            reinterpret_cast<const float *>(dgate + tok0 * 4), reinterpret_cast<const float *>(dlam + tok0 * 4),
+                            n_iter, chunk, dout + tok0 * desc->d_v * es, piece_state);
         if (s != GKA_OK) return s;
-        const size_t bv = (size_t)nb * tok1 * desc->d_v * es, bst = (size_t)nb * desc->heads * st_floats * sizeof(float);
         err = cudaEventRecord(hp->computed[i], stream);
         if (err == cudaSuccess) err = cudaStreamWaitEvent(hp->out, hp->computed[i], 0);
-        if (err == cudaSuccess) err = cudaMemcpyAsync(static_cast<unsigned char *>(out) + ov, dout + ov, bv, cudaMemcpyDeviceToHost, hp->out);
-        if (err == cudaSuccess && state_out) err = cudaMemcpyAsync(state_out + ost, dstate + ost, bst, cudaMemcpyDeviceToHost, hp->out);
+        if (err == cudaSuccess) err = copy(dout, out, tok0 * desc->d_v * es, ntok * desc->d_v * es, cudaMemcpyDeviceToHost, hp->out);
+        if (err == cudaSuccess && state_out && j.last)
+            err = cudaMemcpyAsync(state_out + ost, dstate + ost, (size_t)j.nb * hh * st_floats * sizeof(float),
+                                  cudaMemcpyDeviceToHost, hp->out);
         if (err != cudaSuccess) return cuda_result(err, "gka_fwd_chunked_host (device-to-host copies)");
     }
     err = cudaEventRecord(hp->done, hp->out);

@@ -551,10 +551,11 @@ def test_fwd_bf16_native_tile_shapes(B, heads, T):
 
 # --------------------------------------------------------------------------- host-buffer entry point
 @pytest.mark.parametrize("bf16,B,T", [(False, 3, 64 * 6), (True, 5, 64 * 6), (True, 11, 64 * 6), (True, 5, 64 * 6 + 21),
-                                      (False, 2, 64 + 9)])
+                                      (False, 2, 64 + 9), (True, 3, 64 * 20 + 5), (False, 1, 64 * 9), (True, 10, 64 * 8)])
 def test_fwd_host_buffers_match_device_call_and_oracle(bf16, B, T):
     """gka_fwd_chunked_host (pinned host buffers in, pinned host buffers out; the batch moves through the copy
-    and kernel stages in slices) against the oracle and against the device-pointer call."""
+    and kernel stages in slices, the last batch entries also in pieces along the sequence whose state is carried on
+    the device) against the oracle and against the device-pointer call."""
     cfg = synth.shrink(synth.CONFIGS[1 if bf16 else 0], B=B, heads=2, T=T, d=128, n_iter=4)
     inp = synth.make_inputs(cfg)
     ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], cfg.n_iter)
