@@ -177,6 +177,25 @@ def test_fwd_is_deterministic():
     assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
 
 
+def test_fwd_back_to_back_calls_share_a_workspace():
+    """Two different problems enqueued back to back on one stream with the same workspace: the second result must not
+    see the first call's segment summaries (the main kernel starts under the summary kernel's tail and waits for the
+    summaries only where it reads them)."""
+    cfg = synth.shrink(synth.CONFIGS[1], B=2, heads=5, T=64 * 60, n_iter=3)
+    a = synth.make_inputs(cfg)
+    b = synth.make_inputs(synth.shrink(cfg, seed=77))
+    ws = gka.alloc_workspace(cfg.B, cfg.T, cfg.heads, cfg.d, DEV)
+    dev_a = [to_dev(a[n], n in ("q", "k", "v")) for n in ("q", "k", "v", "gate", "lam")]
+    dev_b = [to_dev(b[n], n in ("q", "k", "v")) for n in ("q", "k", "v", "gate", "lam")]
+    alone, st_alone = gka.gka_fwd_chunked(*dev_b, 3, 64, workspace=ws)
+    torch.cuda.synchronize()
+    for _ in range(5):
+        gka.gka_fwd_chunked(*dev_a, 3, 64, workspace=ws)
+        after, st_after = gka.gka_fwd_chunked(*dev_b, 3, 64, workspace=ws)
+    torch.cuda.synchronize()
+    assert torch.equal(alone, after) and torch.equal(st_alone, st_after)
+
+
 def test_fwd_gpu_argument_errors():
     q = torch.zeros(1, 100, 1, 64, device=DEV)
     v = torch.zeros(1, 100, 1, 128, device=DEV)
