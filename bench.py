@@ -41,7 +41,7 @@ L2_FLUSH_BYTES = 256 << 20
 # ncu captures summarised under profiles/).  Both captures ran a quarter/half-size case of the same kernel
 # (forward: 2048 of 4096 chunks, 133.71 MB; decode: 2048 of 8192 (sequence, head) pairs, 480.67 MB) and
 # are scaled by the units per launch; traffic is proportional to the units in both kernels.
-NCU_TRAFFIC_BYTES = {"fwd_main": 2 * 133_384_960, "decode": 4 * 480_674_816}
+NCU_TRAFFIC_BYTES = {"fwd_main": 2 * 133_384_960, "decode": 4 * 481_565_440}
 
 
 def fwd_flops(n_chunks: int, n_iter: int, C: int = 64, D: int = 128) -> float:

@@ -205,6 +205,8 @@ gka_status gka_decode_tokens(const gka_desc *desc, float *state, const void *q, 
     if (n_iter < 0 || desc->T < 1) return GKA_ERR_SHAPE;
     if (!aligned16(state) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
         return GKA_ERR_ALIGN;
+    if (desc->T == 1)      // one token: the single-step kernel (same layouts) overlaps the state write-back better
+        return gka_decode_step(desc, state, q, k, v, gate, lam, n_iter, out);
     cudaError_t err = launch_decode_multi(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->T, desc->heads,
                                           desc->d_k, desc->io_dtype, desc->flags, desc->beta, desc->alpha,
                                           desc->device_status,

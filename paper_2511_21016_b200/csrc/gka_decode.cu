@@ -117,14 +117,15 @@ decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *_
     const float Lpm = fro + 2.f * lamv;
     const float rho = fro / Lpm, rho2 = rho * rho, s0 = 2.f / Lpm;
     float omega = 2.f;
-    float xr[RPT], xpr[RPT], qr[RPT];     // this thread's rows (held redundantly by the 8 lanes)
-#pragma unroll
-    for (int m = 0; m < RPT; ++m) {
-        qr[m] = sQ[rgrp + 32 * m];
-        xr[m] = s0 * qr[m];
-        xpr[m] = 0.f;
-        if (lane8 == 0) sX[rgrp + 32 * m] = xr[m];
-    }
+    // Row sums of the matvec are reduced across the 8 lanes of a row group so that each lane pair ends up with one
+    // of the group's RPT rows (a transposing butterfly: fewer shuffles than RPT full reductions, and every row's
+    // update is computed by two lanes instead of eight).  Lane pair p = lane8 >> 1 owns row rgrp + 32 p.
+    static_assert(RPT == 4 || RPT == 2, "row ownership below assumes 2 or 4 rows per thread");
+    const int myrow = rgrp + 32 * (RPT == 4 ? (lane8 >> 1) : (lane8 >> 2));
+    const bool row_writer = (RPT == 4 ? (lane8 & 1) : (lane8 & 3)) == 0;
+    const float qr = sQ[myrow];
+    float xr = s0 * qr, xpr = 0.f;
+    if (row_writer) sX[myrow] = xr;
     __syncthreads();
     int cur = 0;
     for (int it = 0; it < n_iter; ++it) {
@@ -137,6 +138,7 @@ decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *_
         }
         omega = 4.f / (4.f - rho2 * omega);
         const float step = s0 * omega, mom = omega - 1.f;
+        float sm[RPT];
 #pragma unroll
         for (int m = 0; m < RPT; ++m) {
             float s = 0.f;
@@ -147,15 +149,27 @@ decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *_
                 s = fmaf(Hr[m][n].z, xc[n][2], s);
                 s = fmaf(Hr[m][n].w, xc[n][3], s);
             }
-            s += __shfl_xor_sync(0xffffffffu, s, 1);
-            s += __shfl_xor_sync(0xffffffffu, s, 2);
-            s += __shfl_xor_sync(0xffffffffu, s, 4);
-            const float y = fmaf(lamv, xr[m], s);
-            const float xn = xr[m] - step * (y - qr[m]) + mom * (xr[m] - xpr[m]);
-            xpr[m] = xr[m];
-            xr[m] = xn;
-            if (lane8 == 0) sX[(cur ^ 1) * D + rgrp + 32 * m] = xn;
+            sm[m] = s;
         }
+        float tot;
+        const bool hi4 = (lane8 & 4) != 0;
+        if (RPT == 4) {
+            const bool hi2 = (lane8 & 2) != 0;
+            float a0 = hi4 ? sm[RPT - 2] : sm[0], a1 = hi4 ? sm[RPT - 1] : sm[1];
+            a0 += __shfl_xor_sync(0xffffffffu, hi4 ? sm[0] : sm[RPT - 2], 4);
+            a1 += __shfl_xor_sync(0xffffffffu, hi4 ? sm[1] : sm[RPT - 1], 4);
+            tot = (hi2 ? a1 : a0) + __shfl_xor_sync(0xffffffffu, hi2 ? a0 : a1, 2);
+            tot += __shfl_xor_sync(0xffffffffu, tot, 1);
+        } else {
+            tot = (hi4 ? sm[1] : sm[0]) + __shfl_xor_sync(0xffffffffu, hi4 ? sm[0] : sm[1], 4);
+            tot += __shfl_xor_sync(0xffffffffu, tot, 2);
+            tot += __shfl_xor_sync(0xffffffffu, tot, 1);
+        }
+        const float y = fmaf(lamv, xr, tot);
+        const float xn = xr - step * (y - qr) + mom * (xr - xpr);
+        xpr = xr;
+        xr = xn;
+        if (row_writer) sX[(cur ^ 1) * D + myrow] = xn;
         cur ^= 1;
         __syncthreads();
     }

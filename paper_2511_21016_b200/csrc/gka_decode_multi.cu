@@ -92,6 +92,8 @@ decode_multi_kernel(float *__restrict__ state, const IoT *__restrict__ q, const 
                 h4.w = fmaf(gam, h4.w, kr[m] * kc[n][3]);
                 Hr[m][n] = h4;
                 ss += h4.x * h4.x + h4.y * h4.y + h4.z * h4.z + h4.w * h4.w;
+                // the last token's H is final: it goes back at once, under the iterations that follow
+                if (t == T - 1) __stcs(reinterpret_cast<float4 *>(gH + (size_t)(rgrp + 32 * m) * D + 4 * (lane8 + 8 * n)), h4);
             }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -203,7 +205,8 @@ decode_multi_kernel(float *__restrict__ state, const IoT *__restrict__ q, const 
                 u4.y = fmaf(gam, u4.y, vr * kc[n][1]);
                 u4.z = fmaf(gam, u4.z, vr * kc[n][2]);
                 u4.w = fmaf(gam, u4.w, vr * kc[n][3]);
-                *pu = u4;
+                if (t == T - 1) __stcs(reinterpret_cast<float4 *>(gU + (size_t)row * D + 4 * (lane8 + 8 * n)), u4);   // final U
+                else *pu = u4;
             }
             s += __shfl_xor_sync(0xffffffffu, s, 1);
             s += __shfl_xor_sync(0xffffffffu, s, 2);
@@ -213,15 +216,6 @@ decode_multi_kernel(float *__restrict__ state, const IoT *__restrict__ q, const 
         __syncthreads();      // the token's vectors and iterate buffers are free for the next token
     }
 
-    // ---- state back to HBM, once
-#pragma unroll
-    for (int m = 0; m < RPT; ++m)
-#pragma unroll
-        for (int n = 0; n < CG; ++n) {
-            const size_t e = (size_t)(rgrp + 32 * m) * D + 4 * (lane8 + 8 * n);
-            __stcs(reinterpret_cast<float4 *>(gH + e), Hr[m][n]);
-            __stcs(reinterpret_cast<float4 *>(gU + e), *reinterpret_cast<const float4 *>(sU + e));
-        }
 }
 
 template <int D, typename IoT>
