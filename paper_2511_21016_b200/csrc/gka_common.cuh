@@ -186,7 +186,8 @@ struct FwdArgs {
 
 // Launchers implemented in the kernel translation units.  Each returns a cudaError_t.
 cudaError_t launch_fwd_simt(const FwdArgs &a, int d, int io_dtype, cudaStream_t stream);
-cudaError_t launch_fwd_scan(const FwdArgs &a, int st, cudaStream_t stream);   // cross-item scan of the summaries
+// cross-item scan of the summaries; after_summary: launched as a programmatic dependent of the summary kernel
+cudaError_t launch_fwd_scan(const FwdArgs &a, int st, cudaStream_t stream, bool after_summary);
 cudaError_t launch_decode(float *state, const void *q, const void *k, const void *v,
                           const float *gate, const float *lam, int n_iter, void *out, int nseq,
                           int heads, int d, int io_dtype, unsigned flags, const float *beta, const float *alpha, int *device_status,

@@ -226,6 +226,10 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_summary(FwdArgs a) {
 // item folds its own short chain independently: blockIdx.y = item, four state elements per thread.
 // ------------------------------------------------------------------------------------------
 __global__ void fwd_scan(FwdArgs a, int st) {
+    // On the tensor-core path this kernel is a programmatic dependent of the summary kernel and the main kernel one of
+    // this kernel: both may be scheduled early, and each waits here for its producer (no effect on plain launches).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const WorkPlan &P = a.plan;
     const int i = blockIdx.y + 1;
     __shared__ int s_j0, s_seq;           // the chain is found once per block (64-bit divisions are slow)
@@ -551,9 +555,18 @@ cudaError_t launch_typed(const FwdArgs &a, cudaStream_t stream) {
 
 }  // namespace
 
-cudaError_t launch_fwd_scan(const FwdArgs &a, int st, cudaStream_t stream) {
-    if (a.plan.G > 1) fwd_scan<<<dim3((st / 4 + 255) / 256, a.plan.G - 1), 256, 0, stream>>>(a, st);
-    return cudaGetLastError();
+cudaError_t launch_fwd_scan(const FwdArgs &a, int st, cudaStream_t stream, bool after_summary) {
+    if (a.plan.G <= 1) return cudaSuccess;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((st / 4 + 255) / 256, a.plan.G - 1);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_summary ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, fwd_scan, a, st);
 }
 
 cudaError_t launch_fwd_simt(const FwdArgs &a, int d, int io_dtype, cudaStream_t stream) {

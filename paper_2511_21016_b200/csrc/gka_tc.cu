@@ -263,11 +263,10 @@ cudaError_t launch_fwd_tc(const FwdArgs &a_in, cudaStream_t stream) {
         if (err != cudaSuccess) return err;
         fwd_tc_summary_kernel<<<a.plan.G, SUM_CT + 32, SUM_SMEM, stream>>>(tmK, tmV, a);
         if (a.start_from_scan) {
-            err = launch_fwd_scan(a, (int)state_floats(D, D), stream);
+            err = launch_fwd_scan(a, (int)state_floats(D, D), stream, true);
             if (err != cudaSuccess) return err;
-        } else {
-            a.after_summary = 1;
         }
+        a.after_summary = 1;     // the main kernel follows its producer (summary or scan kernel) as a programmatic dependent
     }
     return launch_fwd_tile(a, stream);
 }

@@ -274,7 +274,8 @@ __device__ __forceinline__ float master_pass(const Ctx &cx, uint32_t tm_master, 
             const size_t e = src.off + 32 * cx.cq + 16 * piece;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                float4 v4 = src.state ? ldg_stream_f32x4(src.state + e + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                // ordinary loads: the start states may come from the scan kernel this kernel overlaps with
+                float4 v4 = src.state ? *reinterpret_cast<const float4 *>(src.state + e + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
                 r[4 * i + 0] = __float_as_uint(v4.x); r[4 * i + 1] = __float_as_uint(v4.y);
                 r[4 * i + 2] = __float_as_uint(v4.z); r[4 * i + 3] = __float_as_uint(v4.w);
             }
