@@ -259,43 +259,54 @@ struct StartSrc {
     int j0, j1;
     size_t st, off;
 };
+// Start of a run: the master's value (this thread's row, 32 columns at `taddr`) is written to TMEM from global
+// memory; the regular pass then reads it from there.  Compiled as a function of its own: it runs once per run and
+// must not weigh on the register allocation of the per-tile code.  All loads of a step go out together (the
+// thread's 128 bytes are one line), so the fold costs one round trip per chain item.
+__device__ __noinline__ void master_seed(uint32_t taddr, const float *state, const float *delta, const float *decay,
+                                         int j0, int j1, size_t st, size_t e) {
+    float g[32];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        // ordinary loads: the start states may come from the scan kernel this kernel overlaps with
+        const float4 v4 = state ? *reinterpret_cast<const float4 *>(state + e + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        g[4 * i + 0] = v4.x; g[4 * i + 1] = v4.y; g[4 * i + 2] = v4.z; g[4 * i + 3] = v4.w;
+    }
+    for (int j = j0; j < j1; ++j) {
+        // summaries come from the kernel this one may overlap with as its programmatic dependent: ordinary loads
+        // (visible after the dependency wait), not the read-only path, whose data must not change under the kernel
+        const float dj = *reinterpret_cast<const volatile float *>(decay + j);
+        float4 dd[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) dd[i] = *(reinterpret_cast<const float4 *>(delta + (size_t)j * st + e) + i);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            g[4 * i + 0] = fmaf(dj, g[4 * i + 0], dd[i].x);
+            g[4 * i + 1] = fmaf(dj, g[4 * i + 1], dd[i].y);
+            g[4 * i + 2] = fmaf(dj, g[4 * i + 2], dd[i].z);
+            g[4 * i + 3] = fmaf(dj, g[4 * i + 3], dd[i].w);
+        }
+    }
+    uint32_t r[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(g[i]);
+    TMEM_ST32(taddr, r);
+    tmem_wait_st();
+}
+
 template <bool SUMSQ>
 __device__ __forceinline__ float master_pass(const Ctx &cx, uint32_t tm_master, bool from_global, const StartSrc &src,
                                              float decay) {
+    if (from_global)
+        master_seed(tm_master + cx.lane_addr + 32 * cx.cq, src.state, src.delta, src.decay, src.j0, src.j1, src.st,
+                    src.off + 32 * cx.cq);
     float ss = 0.f;
 #pragma unroll
     for (int piece = 0; piece < 2; ++piece) {       // 16 columns at a time keeps the transient registers few
         uint32_t r[16];
         const uint32_t taddr = tm_master + cx.lane_addr + 32 * cx.cq + 16 * piece;
-        if (!from_global) {
-            TMEM_LD16(taddr, r);
-            tmem_wait_ld();
-        } else {
-            const size_t e = src.off + 32 * cx.cq + 16 * piece;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                // ordinary loads: the start states may come from the scan kernel this kernel overlaps with
-                float4 v4 = src.state ? *reinterpret_cast<const float4 *>(src.state + e + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
-                r[4 * i + 0] = __float_as_uint(v4.x); r[4 * i + 1] = __float_as_uint(v4.y);
-                r[4 * i + 2] = __float_as_uint(v4.z); r[4 * i + 3] = __float_as_uint(v4.w);
-            }
-            for (int j = src.j0; j < src.j1; ++j) {
-                // summaries come from the kernel this one may overlap with as its programmatic dependent: ordinary loads
-                // (visible after the dependency wait), not the read-only path, whose data must not change under the kernel
-                const float dj = *reinterpret_cast<const volatile float *>(src.decay + j);
-                float4 dd[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) dd[i] = *(reinterpret_cast<const float4 *>(src.delta + (size_t)j * src.st + e) + i);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float4 d4 = dd[i];
-                    r[4 * i + 0] = __float_as_uint(fmaf(dj, __uint_as_float(r[4 * i + 0]), d4.x));
-                    r[4 * i + 1] = __float_as_uint(fmaf(dj, __uint_as_float(r[4 * i + 1]), d4.y));
-                    r[4 * i + 2] = __float_as_uint(fmaf(dj, __uint_as_float(r[4 * i + 2]), d4.z));
-                    r[4 * i + 3] = __float_as_uint(fmaf(dj, __uint_as_float(r[4 * i + 3]), d4.w));
-                }
-            }
-        }
+        TMEM_LD16(taddr, r);
+        tmem_wait_ld();
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
             uint32_t pk[4];
