@@ -2,6 +2,7 @@
 
     python -m paper_2511_21016_b200.run_case fwd    B heads T n_iter reps
     python -m paper_2511_21016_b200.run_case decode N heads reps
+    python -m paper_2511_21016_b200.run_case tokens N heads T reps
 
 Used for profiling captures (a case of a few hundred MB that ends by itself) and as a usage example
 of the binding: inputs with the benchmark's distributions, one workspace allocation, repeated calls.
@@ -51,11 +52,28 @@ def run_decode(N: int, heads: int, reps: int, d: int = 128, dev: str = "cuda:0")
     return float(out.float().abs().mean())
 
 
+def run_tokens(N: int, heads: int, T: int, reps: int, d: int = 128, dev: str = "cuda:0") -> float:
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+    state = torch.randn(N, heads, 2 * d * d, device=dev, generator=gen) * 0.05
+    q, k = _unit((N, T, heads, d), gen, dev), _unit((N, T, heads, d), gen, dev)
+    v = torch.randn(N, T, heads, d, device=dev, generator=gen).bfloat16()
+    gate = torch.sigmoid(torch.randn(N, T, heads, device=dev, generator=gen) + 2)
+    lam = torch.nn.functional.softplus(torch.randn(N, T, heads, device=dev, generator=gen)) + 1e-2
+    out = torch.empty_like(v)
+    for _ in range(reps):
+        gka.gka_decode_tokens(state, q, k, v, gate, lam, 10, out=out)
+    torch.cuda.synchronize()
+    return float(out.float().abs().mean())
+
+
 def main(argv) -> int:
     if len(argv) >= 6 and argv[0] == "fwd":
         print("ok", run_fwd(*(int(x) for x in argv[1:6])))
     elif len(argv) >= 4 and argv[0] == "decode":
         print("ok", run_decode(*(int(x) for x in argv[1:4])))
+    elif len(argv) >= 5 and argv[0] == "tokens":
+        print("ok", run_tokens(*(int(x) for x in argv[1:5])))
     else:
         print(__doc__)
         return 2
