@@ -8,9 +8,9 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libgka.so")
-SOURCES = ["gka_api.cu", "gka_simt.cu", "gka_decode.cu", "gka_decode_multi.cu", "gka_tc.cu", "gka_tc_tile.cu", "gka_noalloc.cu"]
+SOURCES = ["gka_api.cu", "gka_simt.cu", "gka_decode.cu", "gka_decode_multi.cu", "gka_tc_state.cu", "gka_tc_solve.cu", "gka_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "--use_fast_math=false", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
+              "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
 
 def _nvcc() -> str:
@@ -33,7 +33,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         return LIB
     obj_dir = os.path.join(_HERE, "build")
     os.makedirs(obj_dir, exist_ok=True)
-    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+    flags = list(NVCC_FLAGS)
     objs = []
     procs = []
     for src in SOURCES:

@@ -57,9 +57,16 @@ gka_status check_fwd_shape(const gka_desc *d, int chunk) {
     return GKA_OK;
 }
 
+// bf16 I/O with bf16 tensor-core operands and head dimension 128: the tcgen05 kernels, which work on 128-token tiles
+bool wants_tensor_path(const gka_desc *d) {
+    return d->io_dtype == GKA_BF16 && d->precision == GKA_PREC_NATIVE && d->d_k == 128;
+}
+long long work_units(const gka_desc *d) {
+    return (long long)d->B * d->heads * (wants_tensor_path(d) ? tiles_of(d->T) : chunks_of(d->T));
+}
 // Upper bound on work items used for sizing (independent of the device).
 int work_items_cap(const gka_desc *d, int chunk) {
-    long long nc = (long long)d->B * d->heads * chunks_of(d->T);
+    const long long nc = work_units(d);
     return (int)(nc < kMaxWorkItems ? nc : kMaxWorkItems);
 }
 
@@ -88,6 +95,7 @@ const char *gka_status_string(int status) {
 
 size_t gka_fwd_workspace_bytes(const gka_desc *desc, int chunk) {
     if (check_fwd_shape(desc, chunk) != GKA_OK) return 0;
+    if (wants_tensor_path(desc)) return tc_workspace_bytes_for(work_items_cap(desc, chunk), work_units(desc));
     return workspace_bytes_for(work_items_cap(desc, chunk), desc->d_k, desc->d_v);
 }
 
@@ -107,10 +115,15 @@ gka_status gka_fwd_work_range(const gka_desc *desc, int chunk, int num_items, in
     if (s != GKA_OK) return s;
     if (!first_chunk || !end_chunk || !cut_in || !cut_out) return GKA_ERR_NULL;
     WorkPlan p;
-    p.set(desc->B * desc->heads, chunks_of(desc->T), num_items > 0 ? num_items : 1);
+    const bool tiles = wants_tensor_path(desc);       // that path plans in 128-token tiles = pairs of chunks
+    if (tiles) p.set(desc->B * desc->heads, tiles_of(desc->T), num_items > 0 ? num_items : 1, false);
+    else p.set(desc->B * desc->heads, chunks_of(desc->T), num_items > 0 ? num_items : 1);
     if (num_items <= 0 || num_items > p.NC || item < 0 || item >= num_items) return GKA_ERR_SHAPE;
-    *first_chunk = p.lo(item);
-    *end_chunk = p.lo(item + 1);
+    // a tile is two chunks (the last tile of a sequence with an odd number of chunks holds one)
+    const long long N = chunks_of(desc->T);
+    auto chunk_of = [&](long long f) { return tiles ? (f / p.N) * N + 2 * (f % p.N) : f; };
+    *first_chunk = chunk_of(p.lo(item));
+    *end_chunk = chunk_of(p.lo(item + 1));
     *cut_in = p.cut_in(item) ? 1 : 0;
     *cut_out = p.cut_out(item) ? 1 : 0;
     return GKA_OK;
@@ -150,15 +163,28 @@ static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, c
     a.solve_only = solve_only ? 1 : 0;
     a.start_from_scan = 0;
     a.after_summary = 0;
-    a.plan.set(desc->B * desc->heads, chunks_of(desc->T), G);
-    a.ws = carve_workspace(desc->workspace, G, desc->d_k, desc->d_v);
+    const bool tensor_path = wants_tensor_path(desc) && fwd_tc_available();
+    a.tile_hh = nullptr;
+    a.tile_hu = nullptr;
+    if (tensor_path) {
+        a.plan.set(desc->B * desc->heads, tiles_of(desc->T), G, false);
+        const TcWorkspace w = carve_tc_workspace(desc->workspace, G, a.plan.NC);
+        a.ws.start = w.start;
+        a.ws.delta = w.delta;
+        a.ws.cur = nullptr;
+        a.ws.decay = w.decay;
+        a.tile_hh = w.hh;
+        a.tile_hu = w.hu;
+    } else {
+        if (wants_tensor_path(desc)) return GKA_ERR_CUDA;   // no driver entry point for tensor maps
+        a.plan.set(desc->B * desc->heads, chunks_of(desc->T), G);
+        a.ws = carve_workspace(desc->workspace, G, desc->d_k, desc->d_v);
+    }
     a.ev_start = reinterpret_cast<cudaEvent_t>(desc->profile_start);
     a.ev_stop = reinterpret_cast<cudaEvent_t>(desc->profile_stop);
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(desc->stream);
 
     cudaError_t err;
-    const bool tensor_path = desc->io_dtype == GKA_BF16 && desc->precision == GKA_PREC_NATIVE &&
-                             desc->d_k == 128 && fwd_tc_available();
     if (tensor_path)
         err = launch_fwd_tc(a, stream);
     else

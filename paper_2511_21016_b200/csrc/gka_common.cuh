@@ -51,13 +51,13 @@ struct WorkPlan {
     int unit;      // granularity of the range boundaries in chunks (1 or 2)
     FastDiv divN;  // flat chunk index -> sequence
     __host__ __device__ long long lo(int i) const { return unit * (((long long)i * (NC / unit)) / G); }
-    __host__ __device__ void set(int bh, int n, int g) {
+    __host__ __device__ void set(int bh, int n, int g, bool pairs = true) {
         BH = bh;
         N = n;
         NC = (long long)bh * n;
         G = g;
         divN.set((unsigned)n);
-        unit = (n % 2 == 0 && 2LL * g <= NC) ? 2 : 1;
+        unit = (pairs && n % 2 == 0 && 2LL * g <= NC) ? 2 : 1;
     }
     // start of the last run of item i (flat chunk index)
     __host__ __device__ long long last_run_start(int i) const {
@@ -95,6 +95,41 @@ inline Workspace carve_workspace(void *base, int G, int dk, int dv) {
     w.delta = w.start + (size_t)G * st;
     w.cur = w.delta + (size_t)G * st;
     w.decay = w.cur + (size_t)G * st;
+    return w;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Tensor-core path (bf16 I/O, d = 128).  Its unit of work is a tile of 128 consecutive tokens of one sequence;
+// a sequence is ceil(T / 128) tiles and the WorkPlan above is then a plan over tiles (N = tiles per sequence,
+// unit 1).  A state kernel walks the plan's items, carries the fp32 (H, U) on chip and stores, for every tile,
+// the bf16 operand copies of the tile-initial H_0 and U_0 and ||H_0||_F^2; the solve kernel then treats the
+// tiles as independent problems.  Workspace: start states [G][st], summaries [G][st], decay products [G],
+// ||H_0||_F^2 [tiles], bf16 copies [tiles][2][128][128].
+// ---------------------------------------------------------------------------------------------
+constexpr int kTile = 128;
+__host__ __device__ constexpr int tiles_of(int T) { return (T + kTile - 1) / kTile; }
+constexpr size_t kTileStateBytes = 2 * 128 * 128 * 2;   // bf16 H_0 and U_0 of one tile
+
+struct TcWorkspace {
+    float *start, *delta, *decay, *hh;
+    unsigned char *hu;
+};
+inline size_t tc_workspace_bytes_for(int G, long long ntiles) {
+    const size_t st = state_floats(128, 128);
+    auto up = [](size_t n) { return (n + 255) / 256 * 256; };
+    return 2 * up((size_t)G * st * sizeof(float)) + up((size_t)G * sizeof(float)) + up((size_t)ntiles * sizeof(float)) +
+           (size_t)ntiles * kTileStateBytes;
+}
+inline TcWorkspace carve_tc_workspace(void *base, int G, long long ntiles) {
+    const size_t st = state_floats(128, 128);
+    auto up = [](size_t n) { return (n + 255) / 256 * 256; };
+    unsigned char *p = reinterpret_cast<unsigned char *>(base);
+    TcWorkspace w;
+    w.start = reinterpret_cast<float *>(p); p += up((size_t)G * st * sizeof(float));
+    w.delta = reinterpret_cast<float *>(p); p += up((size_t)G * st * sizeof(float));
+    w.decay = reinterpret_cast<float *>(p); p += up((size_t)G * sizeof(float));
+    w.hh = reinterpret_cast<float *>(p); p += up((size_t)ntiles * sizeof(float));
+    w.hu = p;
     return w;
 }
 
@@ -181,6 +216,8 @@ struct FwdArgs {
     int solve_only;        // write the solve x_t = CH(H_t + lambda_t I, q_t, r) itself instead of U_t x_t (v unused)
     WorkPlan plan;
     Workspace ws;
+    float *tile_hh;        // tensor path: ||H_0||_F^2 of every 128-token tile
+    unsigned char *tile_hu; // tensor path: bf16 H_0, U_0 of every 128-token tile
     cudaEvent_t ev_start, ev_stop;   // optional, recorded around the main kernel (host side only)
 };
 

@@ -148,9 +148,9 @@ def gka_fwd_num_work_items(B, T, heads, d, io_dtype=GKA_BF16, chunk=64) -> int:
     return int(load_library().gka_fwd_num_work_items(ctypes.byref(desc), chunk))
 
 
-def gka_fwd_work_range(B, T, heads, d, num_items, item, chunk=64):
+def gka_fwd_work_range(B, T, heads, d, num_items, item, chunk=64, io_dtype=GKA_BF16):
     """(first_chunk, end_chunk, cut_in, cut_out) of one work item; host arithmetic only."""
-    desc = make_desc(B, T, heads, d, d, GKA_BF16)
+    desc = make_desc(B, T, heads, d, d, io_dtype)
     lo, hi = ctypes.c_longlong(), ctypes.c_longlong()
     ci_, co_ = ctypes.c_int(), ctypes.c_int()
     rc = load_library().gka_fwd_work_range(ctypes.byref(desc), chunk, num_items, item,
@@ -161,8 +161,9 @@ def gka_fwd_work_range(B, T, heads, d, num_items, item, chunk=64):
     return lo.value, hi.value, bool(ci_.value), bool(co_.value)
 
 
-def alloc_workspace(B, T, heads, d, device, chunk=64) -> torch.Tensor:
-    n = gka_fwd_workspace_bytes(B, T, heads, d, chunk=chunk)
+def alloc_workspace(B, T, heads, d, device, chunk=64, io_dtype=GKA_BF16, precision=GKA_PREC_NATIVE) -> torch.Tensor:
+    desc = make_desc(B, T, heads, d, d, io_dtype, precision)
+    n = int(load_library().gka_fwd_workspace_bytes(ctypes.byref(desc), chunk))
     if n == 0:
         raise GkaError(2, "gka_fwd_workspace_bytes")
     return torch.empty(n, dtype=torch.uint8, device=device)
@@ -182,7 +183,7 @@ def gka_fwd_chunked(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=No
     if state_out is None:
         state_out = torch.empty(B, heads, 2 * d * d, dtype=torch.float32, device=q.device)
     if workspace is None:
-        workspace = alloc_workspace(B, T, heads, d, q.device, chunk)
+        workspace = alloc_workspace(B, T, heads, d, q.device, chunk, _io_code(q), precision)
     if stream is None:
         stream = torch.cuda.current_stream(q.device).cuda_stream
     desc = make_desc(B, T, heads, d, v.shape[-1], _io_code(q), precision, flags, stream, workspace,
@@ -206,7 +207,7 @@ def gka_solve_chunked(rhs, k, gate, lam, n_iter, chunk=64, out=None, *, state_in
     if out is None:
         out = torch.empty_like(rhs)
     if workspace is None:
-        workspace = alloc_workspace(B, T, heads, d, rhs.device, chunk)
+        workspace = alloc_workspace(B, T, heads, d, rhs.device, chunk, _io_code(rhs), precision)
     if stream is None:
         stream = torch.cuda.current_stream(rhs.device).cuda_stream
     desc = make_desc(B, T, heads, d, d, _io_code(rhs), precision, flags, stream, workspace, state_in, device_status,

@@ -41,11 +41,15 @@ def test_status_strings(lib):
 
 def test_workspace_bytes_arithmetic(lib):
     st = 2 * 128 * 128
-    # 64 sequences x 64 chunks = 4096 chunks -> capped at 296 work items
-    n = gka.gka_fwd_workspace_bytes(4, 4096, 16, 128)
+    up = lambda n: (n + 255) // 256 * 256
+    # fp32 path: 64 sequences x 64 chunks = 4096 chunks -> capped at 296 work items
+    n = gka.gka_fwd_workspace_bytes(4, 4096, 16, 128, io_dtype=gka.GKA_F32)
     assert n == ((3 * 296 * st + 296) * 4 + 255) // 256 * 256
+    # tensor-core path (bf16, d = 128): 2048 tiles of 128 tokens, each with bf16 copies of H_0 and U_0 and a norm
+    n = gka.gka_fwd_workspace_bytes(4, 4096, 16, 128)
+    assert n == 2 * up(296 * st * 4) + up(296 * 4) + up(2048 * 4) + 2048 * 65536
     # tiny problem: 2 sequences x 4 chunks = 8 items
-    n = gka.gka_fwd_workspace_bytes(1, 256, 2, 64)
+    n = gka.gka_fwd_workspace_bytes(1, 256, 2, 64, io_dtype=gka.GKA_F32)
     assert n == ((3 * 8 * 2 * 64 * 64 + 8) * 4 + 255) // 256 * 256
     # T need not be a multiple of the chunk: 100 tokens are two chunks, the second one short
     assert gka.gka_fwd_workspace_bytes(1, 100, 2, 64) == gka.gka_fwd_workspace_bytes(1, 128, 2, 64)
@@ -93,24 +97,34 @@ def test_argument_errors_are_reported_before_any_launch(lib):
     assert lib.gka_decode_tokens(ctypes.byref(dd), ok + 4, ok, ok, ok, ok, ok, 3, ok) == 9
 
 
-@pytest.mark.parametrize("B,T,heads,G", [(4, 4096, 16, 148), (1, 131072, 32, 148), (1, 256, 2, 8),
+@pytest.mark.parametrize("B,T,heads,G", [(4, 4096, 16, 148), (1, 131072, 32, 148), (1, 256, 2, 4),
                                          (1, 6400, 3, 148), (3, 192, 5, 7), (1, 64, 1, 1)])
-def test_work_ranges_partition_the_chunk_list(lib, B, T, heads, G):
+@pytest.mark.parametrize("io", ["bf16", "f32"])
+def test_work_ranges_partition_the_chunk_list(lib, B, T, heads, G, io):
+    """bf16 I/O with head dimension 128 is planned in 128-token tiles (pairs of chunks, the last tile of a
+    sequence with an odd number of chunks holding one), everything else in chunks."""
     N = T // 64
     NC = B * heads * N
+    tiles = io == "bf16"
     prev_hi = 0
     sizes = []
     for i in range(G):
-        lo, hi, cin, cout = gka.gka_fwd_work_range(B, T, heads, 128, G, i)
+        lo, hi, cin, cout = gka.gka_fwd_work_range(B, T, heads, 128, G, i,
+                                                   io_dtype=gka.GKA_BF16 if tiles else gka.GKA_F32)
         assert lo == prev_hi and hi > lo
         assert cin == (lo % N != 0) and cout == (hi % N != 0)
+        if tiles:
+            assert (lo % N) % 2 == 0          # boundaries between tiles
         sizes.append(hi - lo)
         prev_hi = hi
     assert prev_hi == NC
-    unit = 2 if (N % 2 == 0 and 2 * G <= NC) else 1    # even boundaries where pairs of chunks can be kept whole
-    assert max(sizes) - min(sizes) <= unit       # balanced to within one unit
-    if unit == 2:
-        assert all(sz % 2 == 0 for sz in sizes)
+    if tiles:
+        assert max(sizes) - min(sizes) <= 2 + (N % 2)   # one tile, and a short last tile counts one chunk
+    else:
+        unit = 2 if (N % 2 == 0 and 2 * G <= NC) else 1    # even boundaries where pairs of chunks can be kept whole
+        assert max(sizes) - min(sizes) <= unit       # balanced to within one unit
+        if unit == 2:
+            assert all(sz % 2 == 0 for sz in sizes)
     with pytest.raises(gka.GkaError):
         gka.gka_fwd_work_range(B, T, heads, 128, G, G)
 

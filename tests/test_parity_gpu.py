@@ -601,7 +601,7 @@ def test_fwd_host_buffers_match_device_call_and_oracle(bf16, B, T):
     st_pin = torch.empty(B, cfg.heads, 2 * cfg.d * cfg.d, dtype=torch.float32).pin_memory()
     staging = torch.empty(gka.gka_fwd_host_staging_bytes(B, cfg.T, cfg.heads, cfg.d, gka.GKA_BF16 if bf16 else gka.GKA_F32),
                           dtype=torch.uint8, device=DEV)
-    ws = gka.alloc_workspace(B, cfg.T, cfg.heads, cfg.d, DEV)
+    ws = gka.alloc_workspace(B, cfg.T, cfg.heads, cfg.d, DEV, io_dtype=gka.GKA_BF16 if bf16 else gka.GKA_F32)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     for _ in range(2):      # the second call reuses staging and helper streams while the first is still in flight
         gka.gka_fwd_chunked_host(pin["q"], pin["k"], pin["v"], pin["gate"], pin["lam"], cfg.n_iter, 64, out_pin, st_pin,
