@@ -221,7 +221,7 @@ __device__ __forceinline__ float affine_scan(const Ctx &cx, TileScalars *sc, flo
 }
 
 // Batches of products the issuing thread runs, one per arrival phase of B_RDY, in this order per tile:
-// FROB, then n_iter times (ITER1, ITER2), then (unless the solve itself is the result) OUT_HI, OUT_LO, OUT_PV.
+// FROB, then n_iter times (ITER1, ITER2), then (unless the solve itself is the result) OUT_S, OUT_O.
 __device__ __forceinline__ void issue_batch(int op, uint32_t base14, uint32_t tm, uint32_t bars) {
     const uint32_t kb = base14 + (BUF_K >> 4), hb = base14 + (BUF_H >> 4), db = base14 + (BUF_D >> 4);
     const uint32_t tm_S = tm + TM_S, tm_R = tm + TM_R;
@@ -240,17 +240,13 @@ __device__ __forceinline__ void issue_batch(int op, uint32_t base14, uint32_t tm
             mma8_pm(tm_R, tm_S, kb, kIdescPM);
             mma_commit(bars + 8 * B_MMA_R);
             break;
-        case 3:   // OUT_HI: S = X_hi Khat^T, O = X_hi U_0^T
+        case 3:   // OUT_S: scores of the final iterate, S = X_hi Khat^T + X_lo Khat^T (X_lo sits in the H_0 buffer)
             mma8_kk<0>(tm_S, db, kb, kIdescKK);
+            mma8_kk<1>(tm_S, hb, kb, kIdescKK);
+            mma_commit(bars + 8 * B_MMA_S);
+            break;
+        default:  // OUT_O: O = X_hi U_0^T + P Vhat
             mma8_kk<0>(tm_R, db, hb, kIdescKK);
-            mma_commit(bars + 8 * B_MMA_S);
-            break;
-        case 4:   // OUT_LO: S += X_lo Khat^T, O += X_lo U_0^T
-            mma8_kk<1>(tm_S, db, kb, kIdescKK);
-            mma8_kk<1>(tm_R, db, hb, kIdescKK);
-            mma_commit(bars + 8 * B_MMA_S);
-            break;
-        default:  // OUT_PV: O += P Vhat
             mma8_pm(tm_R, tm_S, kb, kIdescPM);
             mma_commit(bars + 8 * B_MMA_R);
             break;
@@ -383,8 +379,8 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 auto batch = [&](int op, int k) {
                     wait_bar(bars + 8 * B_RDY, n_rdy & 1u, abort_addr);
                     ++n_rdy;
-                    // the read's first batch also needs the U_0 tile (TMA, issued by a compute thread)
-                    if (op == 3) wait_bar(bars + 8 * B_LD_U, (uint32_t)(k & 1), abort_addr);
+                    // the read's last batch also needs the U_0 tile (TMA, issued by a compute thread)
+                    if (op == 4) wait_bar(bars + 8 * B_LD_U, (uint32_t)(k & 1), abort_addr);
                     fence_after();
                     issue_batch(op, base14, tmem, bars);
                 };
@@ -397,7 +393,6 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     if (!solve_only) {
                         batch(3, k);
                         batch(4, k);
-                        batch(5, k);
                     }
                 }
                 // every product is complete before the block gives its tensor memory back
@@ -433,7 +428,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         auto wait_r = [&]() { wait_bar(bars + 8 * B_MMA_R, n_r & 1u, abort_addr); ++n_r; fence_after(); };
         auto arrive_rdy = [&]() { warp_arrive(bars + 8 * B_RDY, l); };
         // stage -xs (times `scale`) as bf16: its leading part, or the remainder after the leading part
-        auto stage_x = [&](bool lo, float scale) {
+        auto stage_x = [&](unsigned char *dst, bool lo, float scale) {
 #pragma unroll
             for (int g8 = 0; g8 < 8; ++g8) {
                 uint32_t pk[4];
@@ -447,7 +442,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     if (lo) p = pack_bf16(xa - bf16_lo(p), xb - bf16_hi(p));
                     pk[u] = p;
                 }
-                *reinterpret_cast<uint4 *>(bufd + tile_off(c, 8 * hf + g8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4 *>(dst + tile_off(c, 8 * hf + g8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
         };
 
@@ -456,6 +451,8 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             const GateScalars *const gs = &sc->g[k & 1];
             const TileInfo ti = tile_info(a, tile);
             const bool valid = c < ti.ntok;
+            // ||H_0||_F^2 of the tile (state kernel): fetched now, used by the scan
+            const float hh = tid < NT ? ldg_stream_f32(a.tile_hh + tile) : 0.f;
             // ---- gate scalars (helper warp) and the K, H_0 tiles (TMA) of this tile
             wait_bar(bars + 8 * (B_GS0 + (k & 1)), (uint32_t)((k >> 1) & 1), abort_addr);
             wait_bar(bars + 8 * B_LD_KH, (uint32_t)(k & 1), abort_addr);
@@ -469,18 +466,20 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             {
                 float kh = 0.f, gsum = 0.f;
 #pragma unroll
-                for (int piece = 0; piece < 4; ++piece) {
-                    uint32_t r[16];
-                    TMEM_LD16(tm_r + cx.lane_addr + 64 * hf + 16 * piece, r);
+                for (int piece = 0; piece < 2; ++piece) {
+                    uint32_t r[32];
+                    TMEM_LD32(tm_r + cx.lane_addr + 64 * hf + 32 * piece, r);
+                    uint4 kv[4];
+#pragma unroll
+                    for (int h4 = 0; h4 < 4; ++h4) kv[h4] = *reinterpret_cast<const uint4 *>(bufk + tile_off(c, 8 * hf + 4 * piece + h4));
                     tmem_wait_ld();
 #pragma unroll
-                    for (int h2 = 0; h2 < 2; ++h2) {
-                        const uint4 kv = *reinterpret_cast<const uint4 *>(bufk + tile_off(c, 8 * hf + 2 * piece + h2));
-                        const uint32_t *pk = reinterpret_cast<const uint32_t *>(&kv);
+                    for (int h4 = 0; h4 < 4; ++h4) {
+                        const uint32_t *pk = reinterpret_cast<const uint32_t *>(&kv[h4]);
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
-                            kh = fmaf(__uint_as_float(r[8 * h2 + 2 * u]), bf16_lo(pk[u]), kh);
-                            kh = fmaf(__uint_as_float(r[8 * h2 + 2 * u + 1]), bf16_hi(pk[u]), kh);
+                            kh = fmaf(__uint_as_float(r[8 * h4 + 2 * u]), bf16_lo(pk[u]), kh);
+                            kh = fmaf(__uint_as_float(r[8 * h4 + 2 * u + 1]), bf16_hi(pk[u]), kh);
                         }
                     }
                 }
@@ -491,20 +490,16 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     if (kb > cx.q) continue;
                     const int lim = (kb == cx.q) ? l : 32;   // keys i < lim come earlier, i == lim is the key itself
                     float gs2 = 0.f, gd = 0.f;
+                    uint32_t r[32];
+                    TMEM_LD32(tm_s + cx.lane_addr + 32 * kb, r);
+                    tmem_wait_ld();
 #pragma unroll
-                    for (int piece = 0; piece < 2; ++piece) {
-                        uint32_t r[16];
-                        TMEM_LD16(tm_s + cx.lane_addr + 32 * kb + 16 * piece, r);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const int ii = 16 * piece + i;
-                            const float g = __uint_as_float(r[i]);
-                            const float g2 = g * g;
-                            if (ii == lim) gd = g2;
-                            if (!exact) gs2 += (ii < lim) ? g2 : 0.f;
-                            else if (ii < lim) gs2 = fmaf(ex2_fast(G2j - gs->G2[32 * kb + ii]), g2, gs2);
-                        }
+                    for (int ii = 0; ii < 32; ++ii) {
+                        const float g = __uint_as_float(r[ii]);
+                        const float g2 = g * g;
+                        if (ii == lim) gd = g2;
+                        if (!exact) gs2 += (ii < lim) ? g2 : 0.f;
+                        else if (ii < lim) gs2 = fmaf(ex2_fast(G2j - gs->G2[32 * kb + ii]), g2, gs2);
                     }
                     gsum += 2.f * gs2 + gd;
                 }
@@ -516,7 +511,6 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             asm volatile("bar.sync 1, 256;" ::: "memory");
             // ---- f_c by an affine scan (s_c = gamma_c^2 s_{c-1} + d_c, s_{-1} = ||H_0||^2), Chebyshev set-up
             if (tid < NT) {
-                const float hh = a.tile_hh[tile];
                 const float kh = sc->part[0][0][c] + sc->part[0][1][c];
                 const float gsum = sc->part[1][0][c] + sc->part[1][1][c];
                 const float G2c = gs->G2[c];
@@ -540,20 +534,25 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             const float rho2 = sc->rho2[c], czb = sc->czb[c], lz = sc->lz[c];
             // ---- x_0: R = q, E_0 = czb q (in place of q), xs = E_0
 #pragma unroll
-            for (int g8 = 0; g8 < 8; ++g8) {
-                const uint4 qv = *reinterpret_cast<const uint4 *>(bufd + tile_off(c, 8 * hf + g8));
-                const uint32_t *qq = reinterpret_cast<const uint32_t *>(&qv);
-                uint32_t rr[8], pk[4];
+            for (int g16 = 0; g16 < 4; ++g16) {
+                uint32_t rr[16];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const float qa = bf16_lo(qq[u]), qb = bf16_hi(qq[u]);
-                    rr[2 * u] = __float_as_uint(qa);
-                    rr[2 * u + 1] = __float_as_uint(qb);
-                    pk[u] = pack_bf16(czb * qa, czb * qb);
-                    xs[4 * g8 + u] = f2_pack(bf16_lo(pk[u]), bf16_hi(pk[u]));
+                for (int h2 = 0; h2 < 2; ++h2) {
+                    const int g8 = 2 * g16 + h2;
+                    const uint4 qv = *reinterpret_cast<const uint4 *>(bufd + tile_off(c, 8 * hf + g8));
+                    const uint32_t *qq = reinterpret_cast<const uint32_t *>(&qv);
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const float qa = bf16_lo(qq[u]), qb = bf16_hi(qq[u]);
+                        rr[8 * h2 + 2 * u] = __float_as_uint(qa);
+                        rr[8 * h2 + 2 * u + 1] = __float_as_uint(qb);
+                        pk[u] = pack_bf16(czb * qa, czb * qb);
+                        xs[4 * g8 + u] = f2_pack(bf16_lo(pk[u]), bf16_hi(pk[u]));
+                    }
+                    *reinterpret_cast<uint4 *>(bufd + tile_off(c, 8 * hf + g8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
-                TMEM_ST8(tm_r + cx.lane_addr + 64 * hf + 8 * g8, rr);
-                *reinterpret_cast<uint4 *>(bufd + tile_off(c, 8 * hf + g8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                TMEM_ST16(tm_r + cx.lane_addr + 64 * hf + 16 * g16, rr);
             }
             tmem_wait_st();
             // ---- Algorithm 1
@@ -618,7 +617,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             // ---- final iterate
             if (solve_only) {
                 // the solve is the result: x_c = -xs / zt_c as bf16, stored by TMA
-                stage_x(false, gs->iz[c]);
+                stage_x(bufd, false, gs->iz[c]);
                 fence_async_smem();
                 warp_arrive(bars + 8 * (B_GF0 + (k & 1)), l);
                 warp_arrive(bars + 8 * B_RDY_ST, l);
@@ -648,22 +647,20 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 }
                 asm volatile("bar.sync 1, 256;" ::: "memory");   // every thread has read q: U_0 may overwrite it
             }
-            if (tid == 0) {               // U_0 into the H_0 buffer (every product on H_0 is complete)
-                mbar_expect_tx(bars + 8 * B_LD_U, 32768u);
-                tma_load_tile2(&tmS, sbase + BUF_H, bars + 8 * B_LD_U, (int)(tile * 256 + 128));
-            }
-            stage_x(false, 1.f);
+            // The read uses the final iterate as two bf16 terms in the score product (the recent keys resolve directions
+            // of x that one bf16 rounding would lose); the second term takes the H_0 buffer, which no product reads
+            // any more.
+            stage_x(bufd, false, 1.f);
+            stage_x(bufh, true, 1.f);
             fence_async_smem();
             fence_before();
-            arrive_rdy();                                        // -> OUT_HI
-            wait_s();                                            // the products on X_hi are complete
-            stage_x(true, 1.f);
-            fence_async_smem();
-            arrive_rdy();                                        // -> OUT_LO
+            arrive_rdy();                                        // -> OUT_S
             wait_s();
-            if (tid == 0) {               // the keys are no longer needed: their buffer takes the V tile
+            if (tid == 0) {               // the keys and the second term are no longer needed: V and U_0 take their buffers
                 mbar_expect_tx(bars + 8 * B_LD_V, 32768u);
                 tma_load_tile3(&tmV, sbase + BUF_K, bars + 8 * B_LD_V, ti.h * D, ti.n * NT, ti.b);
+                mbar_expect_tx(bars + 8 * B_LD_U, 32768u);
+                tma_load_tile2(&tmS, sbase + BUF_H, bars + 8 * B_LD_U, (int)(tile * 256 + 128));
             }
             p_epilogue(cx, tm_s, gs->G2, exact, gs->ac[c]);
             wait_bar(bars + 8 * B_LD_V, n_v & 1u, abort_addr);
@@ -672,7 +669,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             scale_rows(bufk, gs, exact, tid);
             fence_async_smem();
             fence_before();
-            arrive_rdy();                                        // -> OUT_PV
+            arrive_rdy();                                        // -> OUT_O
             wait_r();
             // O as bf16 into the operand buffer (no product reads it any more), stored by TMA
 #pragma unroll
