@@ -78,7 +78,8 @@ static_assert(kBlocksPerSM * (SOLVE_SMEM + 1024 + 256) <= 233472, "shared memory
 constexpr uint32_t TM_S = 0, TM_R = 128;
 
 enum {
-    B_LD_KH = 0,   // K and H_0 tiles have landed (TMA)
+    B_LD_K = 0,    // K tile has landed (TMA)
+    B_LD_H,        // H_0 tile
     B_LD_Q,        // q tile
     B_LD_U,        // U_0 tile
     B_LD_V,        // V tile
@@ -340,11 +341,14 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         } else if (hw == 1) {
             // ================= TMA: loads of every tile's K, H_0, q; stores of the output tiles =================
             if (lane == 0) {
-                auto load_kh = [&](int k) {      // K goes with H_0 on one barrier
+                auto load_k = [&](int k) {
                     const TileInfo ti = tile_info(a, t_lo + k);
-                    mbar_expect_tx(bars + 8 * B_LD_KH, 65536u);
-                    tma_load_tile3(&tmK, sbase + BUF_K, bars + 8 * B_LD_KH, ti.h * D, ti.n * NT, ti.b);
-                    tma_load_tile2(&tmS, sbase + BUF_H, bars + 8 * B_LD_KH, (int)((t_lo + k) * 256));
+                    mbar_expect_tx(bars + 8 * B_LD_K, 32768u);
+                    tma_load_tile3(&tmK, sbase + BUF_K, bars + 8 * B_LD_K, ti.h * D, ti.n * NT, ti.b);
+                };
+                auto load_h = [&](int k) {
+                    mbar_expect_tx(bars + 8 * B_LD_H, 32768u);
+                    tma_load_tile2(&tmS, sbase + BUF_H, bars + 8 * B_LD_H, (int)((t_lo + k) * 256));
                 };
                 auto load_q = [&](int k) {
                     const TileInfo ti = tile_info(a, t_lo + k);
@@ -352,22 +356,35 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     tma_load_tile3(&tmQ, sbase + BUF_D, bars + 8 * B_LD_Q, ti.h * D, ti.n * NT, ti.b);
                 };
                 // the inputs do not depend on the state kernel; its per-tile states do
-                if (n_mine > 0) load_q(0);
+                if (n_mine > 0) {
+                    load_q(0);
+                    load_k(0);
+                }
                 asm volatile("griddepcontrol.wait;" ::: "memory");
-                if (n_mine > 0) load_kh(0);
+                if (n_mine > 0) load_h(0);
+                // The result tile is staged in the H_0 / U_0 buffer (the solve alone: in the operand buffer).  The other
+                // two buffers of the next tile are loaded by a compute thread as soon as the last product is complete;
+                // the staging buffer's next content follows once the store has read it.
+                const uint32_t stage_buf = solve_only ? BUF_D : BUF_H;
                 for (int k = 0; k < n_mine; ++k) {
                     wait_bar(bars + 8 * B_RDY_ST, (uint32_t)(k & 1), abort_addr);
                     const TileInfo ti = tile_info(a, t_lo + k);
                     for (int hf = 0; hf < 2; ++hf)     // rows past the sequence are clipped
                         asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::
                                          "l"(reinterpret_cast<uint64_t>(&tmO)), "r"(ti.h * D + 64 * hf), "r"(ti.n * NT),
-                                     "r"(ti.b), "r"(sbase + BUF_D + 16384 * hf)
+                                     "r"(ti.b), "r"(sbase + stage_buf + 16384 * hf)
                                      : "memory");
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     const bool more = k + 1 < n_mine && !aborted(abort_addr);
-                    if (more) load_kh(k + 1);
+                    if (more && solve_only) {
+                        load_k(k + 1);
+                        load_h(k + 1);
+                    }
                     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the staged tile has been read
-                    if (more) load_q(k + 1);
+                    if (more) {
+                        if (solve_only) load_q(k + 1);
+                        else load_h(k + 1);
+                    }
                 }
                 asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // output stores are complete
             }
@@ -379,7 +396,8 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 auto batch = [&](int op, int k) {
                     wait_bar(bars + 8 * B_RDY, n_rdy & 1u, abort_addr);
                     ++n_rdy;
-                    // the read's last batch also needs the U_0 tile (TMA, issued by a compute thread)
+                    // the first batch also needs the H_0 tile, the last one the U_0 tile (TMA)
+                    if (op == 0) wait_bar(bars + 8 * B_LD_H, (uint32_t)(k & 1), abort_addr);
                     if (op == 4) wait_bar(bars + 8 * B_LD_U, (uint32_t)(k & 1), abort_addr);
                     fence_after();
                     issue_batch(op, base14, tmem, bars);
@@ -455,7 +473,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             const float hh = tid < NT ? ldg_stream_f32(a.tile_hh + tile) : 0.f;
             // ---- gate scalars (helper warp) and the K, H_0 tiles (TMA) of this tile
             wait_bar(bars + 8 * (B_GS0 + (k & 1)), (uint32_t)((k >> 1) & 1), abort_addr);
-            wait_bar(bars + 8 * B_LD_KH, (uint32_t)(k & 1), abort_addr);
+            wait_bar(bars + 8 * B_LD_K, (uint32_t)(k & 1), abort_addr);
             const bool exact = gs->G2[ti.ntok - 1] < -60.f;     // the tile decays below 2^-60: per-element factors
             scale_rows(bufk, gs, exact, tid);
             fence_async_smem();
@@ -515,15 +533,16 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 const float gsum = sc->part[1][0][c] + sc->part[1][1][c];
                 const float G2c = gs->G2[c];
                 // pre-scaled keys: both sums carry 2^(-2 G_c); plain keys: k H_0 k carries zeta_c
-                const float dc = exact ? fmaf(2.f * exp2f(G2c), kh, gsum) : exp2f(2.f * G2c) * fmaf(2.f, kh, gsum);
-                const float s = affine_scan(cx, sc, exp2f(2.f * gs->lg[c]), dc, hh);
+                const float dc = exact ? fmaf(2.f * ex2_fast(G2c), kh, gsum) : ex2_fast(2.f * G2c) * fmaf(2.f, kh, gsum);
+                const float s = affine_scan(cx, sc, ex2_fast(2.f * gs->lg[c]), dc, hh);
                 const float fc = sqrtf(fmaxf(s, 0.f));
                 float lamc = gs->lam[c];
                 if (adaptive) lamc *= fc;
                 const float Lpm = fc + 2.f * lamc;
-                const float rho = fc / Lpm;
+                const float iL = 1.f / Lpm;
+                const float rho = fc * iL;
                 sc->rho2[c] = rho * rho;
-                sc->czb[c] = valid ? -gs->zt[c] * (2.f / Lpm) : 0.f;
+                sc->czb[c] = valid ? -gs->zt[c] * (2.f * iL) : 0.f;
                 sc->lz[c] = lamc * gs->iz[c];
                 if (a.fro_out && valid) a.fro_out[ti.tok0 + (size_t)c * a.heads] = fc;
             }
@@ -671,7 +690,15 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             fence_before();
             arrive_rdy();                                        // -> OUT_O
             wait_r();
-            // O as bf16 into the operand buffer (no product reads it any more), stored by TMA
+            // every product of the tile is complete: the next tile's K and q can come in (H_0 follows the store)
+            if (tid == 0 && k + 1 < n_mine) {
+                const TileInfo tn = tile_info(a, tile + 1);
+                mbar_expect_tx(bars + 8 * B_LD_K, 32768u);
+                tma_load_tile3(&tmK, sbase + BUF_K, bars + 8 * B_LD_K, tn.h * D, tn.n * NT, tn.b);
+                mbar_expect_tx(bars + 8 * B_LD_Q, 32768u);
+                tma_load_tile3(&tmQ, sbase + BUF_D, bars + 8 * B_LD_Q, tn.h * D, tn.n * NT, tn.b);
+            }
+            // O as bf16 into the U_0 buffer (no product reads it any more), stored by TMA
 #pragma unroll
             for (int piece = 0; piece < 4; ++piece) {
                 uint32_t r[16];
@@ -680,8 +707,8 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 uint32_t pk[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) pk[u] = pack_bf16(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1]));
-                *reinterpret_cast<uint4 *>(bufd + tile_off(c, 8 * hf + 2 * piece)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                *reinterpret_cast<uint4 *>(bufd + tile_off(c, 8 * hf + 2 * piece + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                *reinterpret_cast<uint4 *>(bufh + tile_off(c, 8 * hf + 2 * piece)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4 *>(bufh + tile_off(c, 8 * hf + 2 * piece + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
             }
             fence_async_smem();
             fence_before();
