@@ -48,7 +48,7 @@ static_assert(kThreadsSolve * kRegsLaunch * kBlocksPerSM <= 65536, "launch regis
 static_assert(CT * kRegsCompute + 128 * kRegsHelper <= kThreadsSolve * kRegsLaunch, "register split exceeds the launch allocation");
 
 // ---- shared memory map (bytes; operand buffers 1024-byte aligned): three operand tiles and the scalars
-constexpr uint32_t BUF_K = 0;                  // Khat, later Vhat
+constexpr uint32_t BUF_K = 0;                  // Khat, later V
 constexpr uint32_t BUF_H = kTileBytes;         // bf16 H_0, later U_0
 constexpr uint32_t BUF_D = 2 * kTileBytes;     // q, then the operand E, then the output tile
 constexpr uint32_t OFF_SC = 3 * kTileBytes;    // scalars
@@ -62,6 +62,7 @@ struct GateScalars {       // per token of a tile, from the gates and the other 
     float lam[NT];         // lambda_c as given
     float al[NT];          // alpha_c (alpha-connection)
     float sb[NT];          // sqrt(beta_j) (beta-augmented write)
+    float ks[NT];          // row factor of the staged keys: sb_j 2^(-G_j / 2), or sb_j alone when the tile decays below 2^-60
 };
 struct TileScalars {
     GateScalars g[2];
@@ -139,8 +140,8 @@ __device__ __forceinline__ TileInfo tile_info(const FwdArgs &a, long long tile) 
 // block of the scores).  A thread owns token c = 32 q + l and the key blocks kb = 2 hf, 2 hf + 1 (keys 32 kb + i):
 // blocks above the diagonal are zero, blocks below it need no mask.  EXACT: per-element factor 2^(ac_c - G_j)
 // (strongly decaying tiles, whose keys are not pre-scaled).
-template <bool EXACT, bool DIAG>
-__device__ __forceinline__ void p_block(const Ctx &cx, const float *G2kb, uint32_t taddr, float ac_c) {
+template <bool EXACT, bool DIAG, bool KEYF>
+__device__ __forceinline__ void p_block(const Ctx &cx, const float *G2kb, const float *kskb, uint32_t taddr, float ac_c) {
 #pragma unroll
     for (int piece = 0; piece < 2; ++piece) {
         uint32_t r[16], pk[8];
@@ -154,6 +155,11 @@ __device__ __forceinline__ void p_block(const Ctx &cx, const float *G2kb, uint32
                 p0 *= ex2_fast(fminf(ac_c - G2kb[i0], 126.f));
                 p1 *= ex2_fast(fminf(ac_c - G2kb[i0 + 1], 126.f));
             }
+            if (KEYF) {                     // the values are not pre-scaled: their row factor rides on the scores
+                const float2 f = *reinterpret_cast<const float2 *>(kskb + i0);
+                p0 *= f.x;
+                p1 *= f.y;
+            }
             if (DIAG) {                     // keys i <= l are visible
                 p0 = (i0 <= cx.l) ? p0 : 0.f;
                 p1 = (i0 + 1 <= cx.l) ? p1 : 0.f;
@@ -163,11 +169,14 @@ __device__ __forceinline__ void p_block(const Ctx &cx, const float *G2kb, uint32
         TMEM_ST8(taddr + 8 * piece, pk);
     }
 }
-__device__ __forceinline__ void p_epilogue(const Ctx &cx, uint32_t tm_s, const float *G2, bool exact, float ac_c) {
+// keyf: multiply key j's column by ks[j] as well (the pass whose P meets the unscaled V)
+template <bool KEYF>
+__device__ __forceinline__ void p_epilogue(const Ctx &cx, uint32_t tm_s, const GateScalars *gs, bool exact, float ac_c) {
 #pragma unroll
     for (int b2 = 0; b2 < 2; ++b2) {
         const int kb = 2 * cx.hf + b2;
         const uint32_t taddr = tm_s + cx.lane_addr + 32 * kb;
+        const float *G2kb = gs->G2 + 32 * kb, *kskb = gs->ks + 32 * kb;
         if (kb > cx.q) {
             uint32_t z[8];
 #pragma unroll
@@ -175,27 +184,31 @@ __device__ __forceinline__ void p_epilogue(const Ctx &cx, uint32_t tm_s, const f
             TMEM_ST8(taddr, z);
             TMEM_ST8(taddr + 8, z);
         } else if (kb == cx.q) {
-            if (exact) p_block<true, true>(cx, G2 + 32 * kb, taddr, ac_c);
-            else p_block<false, true>(cx, G2 + 32 * kb, taddr, ac_c);
+            if (exact) p_block<true, true, KEYF>(cx, G2kb, kskb, taddr, ac_c);
+            else p_block<false, true, KEYF>(cx, G2kb, kskb, taddr, ac_c);
         } else {
-            if (exact) p_block<true, false>(cx, G2 + 32 * kb, taddr, ac_c);
-            else p_block<false, false>(cx, G2 + 32 * kb, taddr, ac_c);
+            if (exact) p_block<true, false, KEYF>(cx, G2kb, kskb, taddr, ac_c);
+            else p_block<false, false, KEYF>(cx, G2kb, kskb, taddr, ac_c);
         }
     }
     tmem_wait_st();
 }
 
-// Scale the 128 rows of a bf16 operand tile in place: row j by sb_j 2^(-G_j / 2), or by sb_j alone (exact mode).
-__device__ __forceinline__ void scale_rows(unsigned char *tile, const GateScalars *gs, bool exact, int tid) {
+// Scale the 128 rows of a bf16 operand tile in place by the per-row factors f[j].
+__device__ __forceinline__ void scale_rows(unsigned char *tile, const float *f, int tid) {
 #pragma unroll
     for (int i = 0; i < 2048 / CT; ++i) {
         const int qi = tid + CT * i;               // 16-byte group index in the 32 KB tile
-        const int j = (qi & 1023) >> 3;            // row of this group
-        const float f = exact ? gs->sb[j] : gs->sb[j] * ex2_fast(-0.5f * gs->G2[j]);
+        const float fj = f[(qi & 1023) >> 3];      // row of this group
+        const uint64_t f2 = f2_pack(fj, fj);
         uint4 v = *reinterpret_cast<const uint4 *>(tile + qi * 16);
         uint32_t *pv = reinterpret_cast<uint32_t *>(&v);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) pv[u] = pack_bf16(bf16_lo(pv[u]) * f, bf16_hi(pv[u]) * f);
+        for (int u = 0; u < 4; ++u) {
+            float lo, hi;
+            f2_unpack(f2_mul(f2_pack(bf16_lo(pv[u]), bf16_hi(pv[u])), f2), lo, hi);
+            pv[u] = pack_bf16(lo, hi);
+        }
         *reinterpret_cast<uint4 *>(tile + qi * 16) = v;
     }
 }
@@ -246,7 +259,7 @@ __device__ __forceinline__ void issue_batch(int op, uint32_t base14, uint32_t tm
             mma8_kk<1>(tm_S, hb, kb, kIdescKK);
             mma_commit(bars + 8 * B_MMA_S);
             break;
-        default:  // OUT_O: O = X_hi U_0^T + P Vhat
+        default:  // OUT_O: O = X_hi U_0^T + P V
             mma8_kk<0>(tm_R, db, hb, kIdescKK);
             mma8_pm(tm_R, tm_S, kb, kIdescPM);
             mma_commit(bars + 8 * B_MMA_R);
@@ -307,7 +320,8 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 const TileInfo ti = tile_info(a, t_lo + k);
                 GateScalars *g = &sc->g[k & 1];
                 float run = 0.f;
-#pragma unroll 1
+                float ks_g[4], ks_s[4];
+#pragma unroll
                 for (int grp = 0; grp < 4; ++grp) {
                     const int cc = 32 * grp + lane;
                     const bool in = cc < ti.ntok;       // tokens past the sequence: no decay, unit lambda / strengths
@@ -334,6 +348,16 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     g->lam[cc] = lamv;
                     g->sb[cc] = sqrtf(fmaxf(bv, 0.f));
                     g->al[cc] = av;
+                    ks_g[grp] = G2c;
+                    ks_s[grp] = sqrtf(fmaxf(bv, 0.f));
+                }
+                {
+                    // the decay of the whole tile decides how the keys are staged (ti.ntok - 1 is the last token)
+                    const float Glast = __shfl_sync(0xffffffffu, ks_g[(ti.ntok - 1) >> 5], (ti.ntok - 1) & 31);
+                    const bool exact = Glast < -60.f;
+#pragma unroll
+                    for (int grp = 0; grp < 4; ++grp)
+                        g->ks[32 * grp + lane] = exact ? ks_s[grp] : ks_s[grp] * exp2f(-0.5f * ks_g[grp]);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bars + 8 * (B_GS0 + (k & 1)));
@@ -398,7 +422,10 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     ++n_rdy;
                     // the first batch also needs the H_0 tile, the last one the U_0 tile (TMA)
                     if (op == 0) wait_bar(bars + 8 * B_LD_H, (uint32_t)(k & 1), abort_addr);
-                    if (op == 4) wait_bar(bars + 8 * B_LD_U, (uint32_t)(k & 1), abort_addr);
+                    if (op == 4) {
+                        wait_bar(bars + 8 * B_LD_U, (uint32_t)(k & 1), abort_addr);
+                        wait_bar(bars + 8 * B_LD_V, (uint32_t)(k & 1), abort_addr);
+                    }
                     fence_after();
                     issue_batch(op, base14, tmem, bars);
                 };
@@ -441,7 +468,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         asm volatile("griddepcontrol.wait;" ::: "memory");
 
         uint64_t xs[32];                    // -zt_c x_c, this thread's 64 channels as fp32 pairs
-        uint32_t n_s = 0, n_r = 0, n_q = 0, n_v = 0;   // completed phases of MMA_S, MMA_R, LD_Q, LD_V
+        uint32_t n_s = 0, n_r = 0, n_q = 0;   // completed phases of MMA_S, MMA_R, LD_Q
         auto wait_s = [&]() { wait_bar(bars + 8 * B_MMA_S, n_s & 1u, abort_addr); ++n_s; fence_after(); };
         auto wait_r = [&]() { wait_bar(bars + 8 * B_MMA_R, n_r & 1u, abort_addr); ++n_r; fence_after(); };
         auto arrive_rdy = [&]() { warp_arrive(bars + 8 * B_RDY, l); };
@@ -475,7 +502,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             wait_bar(bars + 8 * (B_GS0 + (k & 1)), (uint32_t)((k >> 1) & 1), abort_addr);
             wait_bar(bars + 8 * B_LD_K, (uint32_t)(k & 1), abort_addr);
             const bool exact = gs->G2[ti.ntok - 1] < -60.f;     // the tile decays below 2^-60: per-element factors
-            scale_rows(bufk, gs, exact, tid);
+            scale_rows(bufk, gs->ks, tid);
             fence_async_smem();
             arrive_rdy();                                        // -> FROB
             wait_s();
@@ -586,7 +613,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 omega = 4.f / (4.f - rho2 * omega);              // weight schedule
                 const float beta = omega - 1.f, cz = czb * omega;
                 wait_s();
-                p_epilogue(cx, tm_s, gs->G2, exact, gs->ac[c]);
+                p_epilogue<false>(cx, tm_s, gs, exact, gs->ac[c]);
                 fence_before();
                 arrive_rdy();                                    // -> ITER2
                 const uint64_t beta2 = f2_pack(beta, beta), cz2 = f2_pack(cz, cz), lz2 = f2_pack(lz, lz);
@@ -681,12 +708,8 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 mbar_expect_tx(bars + 8 * B_LD_U, 32768u);
                 tma_load_tile2(&tmS, sbase + BUF_H, bars + 8 * B_LD_U, (int)(tile * 256 + 128));
             }
-            p_epilogue(cx, tm_s, gs->G2, exact, gs->ac[c]);
-            wait_bar(bars + 8 * B_LD_V, n_v & 1u, abort_addr);
-            ++n_v;
-            // Vhat_j = sqrt(beta_j) 2^(-G_j / 2) v_j pairs with the scores on Khat
-            scale_rows(bufk, gs, exact, tid);
-            fence_async_smem();
+            // the values stay as loaded: their row factor sqrt(beta_j) 2^(-G_j / 2) rides on the masked scores
+            p_epilogue<true>(cx, tm_s, gs, exact, gs->ac[c]);
             fence_before();
             arrive_rdy();                                        // -> OUT_O
             wait_r();

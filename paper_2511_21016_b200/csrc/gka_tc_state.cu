@@ -357,16 +357,18 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             chain_j0 = item - 1;
             while (P.lo(chain_j0) > seq_start) --chain_j0;
         }
-        auto load_scalars = [&](int m, float &g, float &bt) {
-            g = 1.f;
-            bt = 0.f;
+        // gate and write strength of this thread's token of tile m (threads 0..127; 1 and 0 past the sequence); returned
+        // by value so that the loads stay in registers until they are used a tile later
+        auto load_scalars = [&](int m) -> float2 {
+            float g = 1.f, bt = 0.f;
             if (t < NT && m < n_mine) {
                 const Pos p = pos_of(m);
-                if (t < p.ntok) {      // issued here and now (the values are used a tile later)
+                if (t < p.ntok) {
                     g = ldg_stream_f32(a.gate + p.tok0 + (size_t)t * a.heads);
                     bt = a.beta ? fmaxf(ldg_stream_f32(a.beta + p.tok0 + (size_t)t * a.heads), 0.f) : 1.f;
                 }
             }
+            return make_float2(g, bt);
         };
         // Tile m: row factors sqrt(beta_j 2^(G_last - G_j)) (0 past the sequence), rows scaled in place, products posted.
         // (g, bt): this thread's gate and write strength of the tile (threads 0..127).
@@ -400,19 +402,18 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         };
 
         float mH[32], mU[32];
-        float g_nx, b_nx;
-        load_scalars(0, g_nx, b_nx);
-        prepare(0, g_nx, b_nx);
-        load_scalars(1, g_nx, b_nx);
+        float2 nx = load_scalars(0);
+        prepare(0, nx.x, nx.y);
+        nx = load_scalars(1);
         // summaries and start states are read after this point only
         asm volatile("griddepcontrol.wait;" ::: "memory");
 
         for (int m = 0; m < n_mine; ++m) {
             const Pos p = pos_of(m);
             if (m + 1 < n_mine) {
-                const float g1 = g_nx, b1 = b_nx;
-                load_scalars(m + 2, g_nx, b_nx);
-                prepare(m + 1, g1, b1);                          // its products run under this tile's passes
+                const float2 cur = nx;
+                nx = load_scalars(m + 2);
+                prepare(m + 1, cur.x, cur.y);                    // its products run under this tile's passes
             }
             const long long tile = f_lo + m;
             if (p.run_start) {
