@@ -205,7 +205,8 @@ gka_status gka_fwd_work_range(const gka_desc *desc, int chunk, int num_items, in
  *   - Calls no cudaMalloc / cudaFree and no allocating library routine.
  *   - Problems whose scan needs more than the array (gka_fwd_workspace_bytes(desc, chunk) >
  *     gka_noalloc_scratch_bytes()) are rejected with GKA_ERR_WORKSPACE before anything is launched:
- *     d_k = 64 fits up to 170 chunks in total (B * heads * T / chunk), d_k = 128 up to 42 chunks.
+ *     fp32 arithmetic: d_k = 64 fits up to 170 chunks in total (B * heads * ceil(T / chunk)), d_k = 128 up to 42;
+ *     bf16 tensor-core path (d_k = 128): up to 52 tiles of 128 tokens in total (B * heads * ceil(T / 128)).
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) with
  *     that device current; make that first call before any stream capture.
  *   - All calls on one device share the array.  Calls that overlap on the GPU race, whatever their

@@ -371,7 +371,11 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
         }
         __syncthreads();
 
-        // ---- Algorithm 1 on the whole chunk
+        // ---- Algorithm 1 on the whole chunk, in residual form: with d_i = x_i - x_{i-1} (x_{-1} = 0, d_0 = x_0) the update
+        // x_{i+1} = x_i + (omega - 1) d_i + (2 omega / (L + mu)) (q - A x_i) reads r_i = r_{i-1} - A d_i (r_{-1} = q),
+        // d_{i+1} = (omega - 1) d_i + (2 omega / (L + mu)) r_i, x_{i+1} = x_i + d_{i+1}: the same iterates in exact
+        // arithmetic, but the matrix meets the shrinking increment, so its rounding errors shrink with it.
+        // xm: iterate x; xp: increment d (the published operand); qm: q - (A - lambda) x (the lambda term uses x itself)
         float xm[4][NCH], xp[4][NCH], qm[4][NCH];
         float omega[4], rho2[4], s0[4], lamr[4], zet[4];
 #pragma unroll
@@ -394,18 +398,19 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
             }
 #pragma unroll
             for (int u = 0; u < NCH; ++u) {
-                xm[t][u] = s0[t] * qm[t][u];            // xi_0 = 2 q / (L + mu)
-                xp[t][u] = 0.f;                         // xi_{-1} = 0
+                xp[t][u] = s0[t] * qm[t][u];            // d_0 = xi_0 = 2 q / (L + mu)
+                xm[t][u] = 0.f;                         // xi_{-1} = 0
             }
         }
-        auto publish_x = [&]() {
+        auto publish = [&](const float(&x)[4][NCH]) {
 #pragma unroll
             for (int g = 0; g < DG; ++g)
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
                     st4(sXt + (64 * g + 4 * td + u) * XS + 4 * tc,
-                        make_float4(xm[0][4 * g + u], xm[1][4 * g + u], xm[2][4 * g + u], xm[3][4 * g + u]));
+                        make_float4(x[0][4 * g + u], x[1][4 * g + u], x[2][4 * g + u], x[3][4 * g + u]));
         };
+        auto publish_x = [&]() { publish(xm); };
         auto masked_scores = [&]() {   // sPt[j][c] = Gamma[c][j] * (x_c . k_j), j <= c
             float s[4][4];
             gemm_tok_tok<D>(s, sXt, sKt, tc, td);
@@ -421,17 +426,17 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
                 st4(sPt + j * XS + 4 * tc, make_float4(p[0], p[1], p[2], p[3]));
             }
         };
-        publish_x();
+        publish(xp);
         __syncthreads();
         for (int it = 0; it < a.n_iter; ++it) {
-            masked_scores();
+            masked_scores();                                   // of the increment
             __syncthreads();
             float acc[4][NCH];
 #pragma unroll
             for (int t = 0; t < 4; ++t)
 #pragma unroll
                 for (int u = 0; u < NCH; ++u) acc[t][u] = 0.f;
-            gemm_tok_mat<D>(acc, sXt, sH, D, tc, td);          // X H_0
+            gemm_tok_mat<D>(acc, sXt, sH, D, tc, td);          // D H_0
 #pragma unroll
             for (int t = 0; t < 4; ++t)
 #pragma unroll
@@ -444,13 +449,21 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
                 const float mom = omega[t] - 1.f;
 #pragma unroll
                 for (int u = 0; u < NCH; ++u) {
-                    const float y = fmaf(lamr[t], xm[t][u], acc[t][u]);       // (H_c + lambda_c I) x_c
-                    const float xn = xm[t][u] - step * (y - qm[t][u]) + mom * (xm[t][u] - xp[t][u]);
-                    xp[t][u] = xm[t][u];
-                    xm[t][u] = xn;
+                    xm[t][u] += xp[t][u];                                      // x_i
+                    qm[t][u] -= acc[t][u];                                     // q - H_c x_i
+                    const float res = fmaf(-lamr[t], xm[t][u], qm[t][u]);      // r_i = q - (H_c + lambda_c I) x_i
+                    xp[t][u] = fmaf(step, res, mom * xp[t][u]);                // d_{i+1}
                 }
             }
             __syncthreads();      // every read of sXt / sPt of this iteration is done
+            publish(xp);
+            __syncthreads();
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t)
+#pragma unroll
+            for (int u = 0; u < NCH; ++u) xm[t][u] += xp[t][u];               // the final iterate
+        if (!a.solve_only && !a.alpha) {
             publish_x();
             __syncthreads();
         }
@@ -468,11 +481,18 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
         if (a.alpha && !a.solve_only) {    // alpha-connection (Section 4.4): the read uses alpha x + (1 - alpha) q
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
-                const float al = (4 * tc + t < nvalid) ? a.alpha[tok0 + (size_t)(4 * tc + t) * a.heads] : 1.f;
+                const int c = 4 * tc + t;
+                const float al = (c < nvalid) ? a.alpha[tok0 + (size_t)c * a.heads] : 1.f;
 #pragma unroll
-                for (int u = 0; u < NCH; ++u) xm[t][u] = fmaf(al, xm[t][u] - qm[t][u], qm[t][u]);
+                for (int g = 0; g < DG; ++g) {      // the query again (its registers hold the residual)
+                    float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (c < nvalid) qv = Io<IoT>::load4(gq + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td);
+                    xm[t][4 * g + 0] = fmaf(al, xm[t][4 * g + 0] - qv.x, qv.x);
+                    xm[t][4 * g + 1] = fmaf(al, xm[t][4 * g + 1] - qv.y, qv.y);
+                    xm[t][4 * g + 2] = fmaf(al, xm[t][4 * g + 2] - qv.z, qv.z);
+                    xm[t][4 * g + 3] = fmaf(al, xm[t][4 * g + 3] - qv.w, qv.w);
+                }
             }
-            __syncthreads();      // every read of the published iterate is done
             publish_x();
             __syncthreads();
         }

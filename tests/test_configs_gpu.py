@@ -3,7 +3,8 @@
 The oracle cannot recompute a whole full-size tensor in a test, so whole (batch, head) pairs are
 sampled: every pair is an independent problem whose outputs the oracle computes one by one from the
 same seeded inputs (per-(b,h) substreams make a pair's inputs identical whether drawn alone or with
-the rest).  Tolerances: relative L2 of 1e-4 (fp32 I/O) and 2e-2 (bf16 I/O).
+the rest).  Tolerances: relative L2 of 1e-4 (fp32 I/O) and 2e-2 (bf16 I/O) over each compared pair, and the same
+bound over every 128-token tile of a compared pair, so that one wrong tile cannot hide in a long sequence.
 """
 import numpy as np
 import pytest
@@ -25,6 +26,16 @@ def rel(a, b):
 def dev(x, bf16=False):
     t = torch.from_numpy(np.ascontiguousarray(x)).to(DEV)
     return t.to(torch.bfloat16) if bf16 else t
+
+
+def tile_max(out, ref, tile=128):
+    """Largest relative L2 error over the 128-token tiles of a [T, d] sequence."""
+    out = np.asarray(out, np.float64)
+    ref = np.asarray(ref, np.float64)
+    T = ref.shape[0] // tile * tile
+    num = np.sqrt(((out[:T] - ref[:T]) ** 2).reshape(-1, tile * ref.shape[1]).sum(1))
+    den = np.sqrt((ref[:T] ** 2).reshape(-1, tile * ref.shape[1]).sum(1))
+    return float((num / np.maximum(den, 1e-300)).max())
 
 
 def head_inputs(inp, pairs):
@@ -61,34 +72,45 @@ def test_config1_full_size_sampled_pairs():
     # per-pair too: no pair hides behind the others
     for i in range(len(pairs)):
         assert rel(got[0, :, i], ref["out"][0, :, i]) <= 2e-2
+        et = tile_max(got[0, :, i], ref["out"][0, :, i])
+        assert et <= 2e-2, f"pair {pairs[i]}: worst 128-token tile rel L2 {et:.3e}"
 
 
-def test_config3_long_context_one_head_of_32():
-    """T=131072, d=128, bf16, slow-fading gates: the full sequence length with the full head count
-    in the launch (B=1, heads=32); the oracle recomputes one whole head."""
+def test_config3_long_context_three_heads_of_32():
+    """T=131072, d=128, bf16, slow-fading gates, B=1, heads=32: the benchmark's launch with real inputs for every
+    head (drawn on the device with the configuration's distributions; the host recipe would take minutes).  Every
+    head is spread over several work items; the oracle recomputes three whole heads (first, middle, last) from the
+    same inputs, and every 128-token tile of each is bounded."""
     cfg = synth.CONFIGS[3]
-    pairs = [(0, 5)]
-    # only the sampled head needs real data for the comparison; the others get cheap valid inputs
-    inp = synth.make_inputs(cfg, pairs=pairs)
-    rng = np.random.default_rng(123)
-    fill = rng.standard_normal((cfg.T, cfg.d)).astype(np.float32)
-    fill /= np.linalg.norm(fill, axis=1, keepdims=True)
-    fill = synth.round_bf16(fill)
-    for h in range(cfg.heads):
-        if (0, h) not in pairs:
-            inp["q"][0, :, h] = fill
-            inp["k"][0, :, h] = fill
-            inp["v"][0, :, h] = fill
-            inp["gate"][0, :, h] = 0.98
-            inp["lam"][0, :, h] = 0.3
-    out, st = run_full(cfg, inp)
-    assert np.all(np.isfinite(out))
-    hi = head_inputs(inp, pairs)
-    ref = oracle.fwd(hi["q"], hi["k"], hi["v"], hi["gate"], hi["lam"], cfg.n_iter)
-    e = rel(out[0, :, 5], ref["out"][0, :, 0])
-    es = rel(st[0, 5], ref["state"][0, 0])
-    print("config3 head rel L2 out %.3e state %.3e" % (e, es))
-    assert e <= 2e-2 and es <= 5e-3
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(cfg.seed)
+    B, T, Hh, d = cfg.B, cfg.T, cfg.heads, cfg.d
+
+    def unit(shape):
+        x = torch.randn(shape, generator=gen, device=DEV)
+        return (x / x.norm(dim=-1, keepdim=True)).to(torch.bfloat16)
+
+    q, k = unit((B, T, Hh, d)), unit((B, T, Hh, d))
+    v = torch.randn((B, T, Hh, d), generator=gen, device=DEV).to(torch.bfloat16)
+    gate = torch.sigmoid(torch.randn((B, T, Hh), generator=gen, device=DEV) + 4.0)
+    lam = torch.nn.functional.softplus(torch.randn((B, T, Hh), generator=gen, device=DEV) - 1.0) + 1e-3
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out, st = gka.gka_fwd_chunked(q, k, v, gate, lam, cfg.n_iter, cfg.chunk, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert bool(torch.isfinite(out.float()).all())
+    heads = [0, 13, 31]
+    f64 = lambda t: np.ascontiguousarray(t.float().cpu().numpy().astype(np.float64))
+    ref = oracle.fwd(f64(q[:, :, heads]), f64(k[:, :, heads]), f64(v[:, :, heads]), f64(gate[:, :, heads]),
+                     f64(lam[:, :, heads]), cfg.n_iter)
+    for i, h in enumerate(heads):
+        got = out[0, :, h].float().cpu().numpy()
+        e = rel(got, ref["out"][0, :, i])
+        et = tile_max(got, ref["out"][0, :, i])
+        es = rel(st[0, h].cpu().numpy(), ref["state"][0, i])
+        print("config3 head %d rel L2 out %.3e (worst tile %.3e) state %.3e" % (h, e, et, es))
+        assert e <= 2e-2 and es <= 5e-3
+        assert et <= 2e-2
 
 
 def test_config2_decode_full_size_sampled_heads():
@@ -157,10 +179,7 @@ def test_config4_conditioning_stress_table():
         x_f32 = rel(pick(o_f32), exact)
         rows.append((r, e_f32, e_hi, e_nat, x_ch, x_f32))
         assert np.all(np.isfinite(o_nat))
-        # fp32 arithmetic (unit roundoff 6e-8) on a matrix with ||H||_F ~ 100 and kappa ~ 1e6: every matvec
-        # injects ~1e-6 |x| and the momentum recurrence amplifies it with the iteration count; 32 iterations
-        # sit at ~1.3e-4, so the 1e-4 bar is applied up to 16 iterations and 3e-4 at 32
-        assert e_f32 <= (1e-4 if r <= 16 else 3e-4), f"fp32 I/O n_iter={r}: {e_f32:.3e}"
+        assert e_f32 <= 1e-4, f"fp32 I/O n_iter={r}: {e_f32:.3e}"
         assert e_hi <= 2e-2, f"bf16 I/O fp32 math n_iter={r}: {e_hi:.3e}"
     print("\nconfig4: n_iter | vs CH oracle: f32 io, bf16 io (fp32 math), bf16 operands | vs Cholesky: oracle CH, f32 kernel")
     for row in rows:

@@ -1,6 +1,8 @@
 """Parity of the CUDA path (through the C ABI) against the fp64 CPU oracle, element by element
 on the same seeded inputs.  Tolerances: relative L2 over the whole tensor of 1e-4 for fp32 I/O
-and 2e-2 for bf16 I/O (the figures the benchmark spec states)."""
+and 2e-2 for bf16 I/O, and, so that no single stretch of tokens hides behind the rest, a bound on the
+relative L2 of every 128-token tile of every (batch, head) pair: the same two figures (measured: the
+worst tile sits within a factor of two of the whole-tensor error)."""
 import numpy as np
 import pytest
 import torch
@@ -12,7 +14,21 @@ pytestmark = pytest.mark.gpu
 
 TOL_F32 = 1e-4
 TOL_BF16 = 2e-2
+TILE_TOL_F32 = 1e-4
+TILE_TOL_BF16 = 2e-2
 DEV = "cuda:0"
+
+
+def tile_max(out, ref, tile=128):
+    """Largest relative L2 error over the 128-token tiles of every (batch, head) pair; [B, T, heads, d] arrays."""
+    out = np.asarray(out, np.float64)
+    ref = np.asarray(ref, np.float64)
+    worst = 0.0
+    for t0 in range(0, ref.shape[1], tile):
+        num = np.sqrt(((out[:, t0:t0 + tile] - ref[:, t0:t0 + tile]) ** 2).sum(axis=(1, 3)))
+        den = np.sqrt((ref[:, t0:t0 + tile] ** 2).sum(axis=(1, 3)))
+        worst = max(worst, float((num / np.maximum(den, 1e-300)).max()))
+    return worst
 
 
 def rel(a, b):
@@ -55,9 +71,11 @@ def check_fwd(cfg, n_iter=None, precision=gka.GKA_PREC_NATIVE, flags=0, tol=None
     assert np.all(np.isfinite(out))
     e_out, e_st, e_fro = rel(out, ref["out"]), rel(st, ref["state"]), rel(fro, ref["fro"])
     assert e_out <= tol, f"out rel L2 {e_out:.3e} > {tol}"
+    e_tile = tile_max(out, ref["out"])
+    assert e_tile <= (TILE_TOL_BF16 if bf16 else TILE_TOL_F32), f"worst 128-token tile rel L2 {e_tile:.3e}"
     assert e_st <= state_tol, f"state rel L2 {e_st:.3e} > {state_tol}"
     assert e_fro <= (1e-5 if fp32_math else 5e-3), f"fro rel L2 {e_fro:.3e}"
-    return e_out, e_st, e_fro
+    return e_out, e_st, e_fro, e_tile
 
 
 SMALL = synth.GkaConfig("small", B=2, heads=3, T=128, d=64, chunk=64, n_iter=4, io_dtype="f32", seed=7)
@@ -151,20 +169,29 @@ def test_fwd_adaptive_lambda_mode():
     assert rel(out, ref["out"]) < TOL_F32
 
 
-@pytest.mark.parametrize("T", [256, 457])
-def test_fwd_adaptive_lambda_mode_bf16(T):
+@pytest.mark.parametrize("T,n_iter", [(256, 8), (457, 8), (64 * 30, 30)])
+def test_fwd_adaptive_lambda_mode_bf16(T, n_iter):
     """The adaptive rule with the paper's a = 0.02 makes every solve as ill-conditioned as the rule allows
-    (kappa = 51): bf16 operands perturb H_t by eps_bf16 ||H_t||, which the solve amplifies by up to
-    ||H_t|| / lambda_t = 1 / a, so the tensor-core path is held to 6e-2 here (3 - 4 % measured) and the
-    fp32-arithmetic mode of the same call to 5e-3."""
-    cfg = synth.shrink(synth.CONFIGS[1], B=3, heads=5, T=T, n_iter=8, seed=49)
+    (kappa = 51), and the paper runs 30 iterations: the tensor-core path (bf16 operands on the increments,
+    fp32 iterate, two-term read) meets the bf16 bar there, and so does the fp32-arithmetic mode of the same call."""
+    cfg = synth.shrink(synth.CONFIGS[1], B=3, heads=5, T=T, n_iter=n_iter, seed=49)
     inp = synth.make_inputs(cfg)
     inp["lam"] = np.full_like(inp["lam"], 0.02)
-    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], 8, lam_mode=1)
-    out, _, _ = run_fwd(inp, 8, True, flags=gka.GKA_FLAG_ADAPTIVE_LAMBDA)
-    assert rel(out, ref["out"]) <= 6e-2
-    out, _, _ = run_fwd(inp, 8, True, precision=gka.GKA_PREC_HIGH, flags=gka.GKA_FLAG_ADAPTIVE_LAMBDA)
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], n_iter, lam_mode=1)
+    out, _, _ = run_fwd(inp, n_iter, True, flags=gka.GKA_FLAG_ADAPTIVE_LAMBDA)
+    e, et = rel(out, ref["out"]), tile_max(out, ref["out"])
+    print("adaptive a=0.02 T=%d r=%d tensor path: rel L2 %.3e, worst tile %.3e" % (T, n_iter, e, et))
+    assert e <= TOL_BF16 and et <= TILE_TOL_BF16
+    out, _, _ = run_fwd(inp, n_iter, True, precision=gka.GKA_PREC_HIGH, flags=gka.GKA_FLAG_ADAPTIVE_LAMBDA)
     assert rel(out, ref["out"]) <= 5e-3
+
+
+def test_fwd_bf16_native_paper_iteration_count():
+    """30 iterations (the paper's setting in every experiment) on configuration-1-like inputs, sequences cut by
+    work items: tensor-core path against the oracle."""
+    cfg = synth.shrink(synth.CONFIGS[1], B=2, heads=3, T=64 * 70, n_iter=30)
+    e = check_fwd(cfg)
+    print("bf16 native r=30 rel L2 (out, state, fro, worst tile):", e)
 
 
 def test_fwd_degenerate_inputs():
@@ -477,14 +504,7 @@ def test_fwd_ragged_sequence_length(bf16, d, B, heads, T):
     assert bool((big[B * T * heads * d:] == 7.0).all()) and bool((fbig[B * T * heads:] == -3.0).all())
     tensor_path = bf16 and d == 128
     o = out.float().cpu().numpy()
-    if tensor_path and T == 1:
-        # a single token per sequence: o = v (k . x) reads only the component of x along k, which bf16 operands
-        # resolve to eps * |x|, so the bound is the forward error of o = U x under a relative perturbation of x
-        U = ref["state"][..., d * d:].reshape(B, heads, d, d)
-        bound = TOL_BF16 * np.linalg.norm(U, axis=(-2, -1)) * np.linalg.norm(ref["x"][:, 0], axis=-1)
-        assert np.all(np.linalg.norm(o[:, 0] - ref["out"][:, 0], axis=-1) <= bound)
-    else:
-        assert rel(o, ref["out"]) <= (TOL_BF16 if bf16 else TOL_F32)
+    assert rel(o, ref["out"]) <= (TOL_BF16 if bf16 else TOL_F32)
     assert rel(fro.cpu().numpy(), ref["fro"]) <= (5e-3 if tensor_path else 1e-5)
     assert rel(st.cpu().numpy(), ref["state"]) <= (5e-3 if tensor_path else 1e-5)
 

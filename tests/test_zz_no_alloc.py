@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2511_21016_b200 import gka, synth
 
 pytestmark = pytest.mark.gpu
@@ -34,7 +35,7 @@ def _rel(a, b):
     # fp32 path, d = 64: several work items, sequences cut between items (scan scratch is used)
     ("f32_d64", synth.GkaConfig("na0", B=1, heads=3, T=64 * 50, d=64, chunk=64, n_iter=3,
                                 io_dtype="f32", seed=11), 1e-4),
-    # tensor-core path, d = 128, 40 chunks: below the built-in scratch limit of 42 chunks
+    # tensor-core path, d = 128, 20 tiles of 128 tokens: below the built-in scratch limit of 52 tiles
     ("bf16_d128", synth.GkaConfig("na1", B=1, heads=2, T=64 * 20, d=128, chunk=64, n_iter=4,
                                   io_dtype="bf16", seed=12), 2e-2),
 ])
@@ -45,6 +46,7 @@ def test_noalloc_matches_regular_entry_point_twice(name, cfg, tol):
     gate, lam = _dev(inp["gate"]), _dev(inp["lam"])
     ref_out, ref_state = gka.gka_fwd_chunked(q, k, v, gate, lam, cfg.n_iter, cfg.chunk)
     torch.cuda.synchronize()
+    want = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], cfg.n_iter)     # and both against the oracle
     for call in range(2):
         out = torch.full_like(ref_out, float("nan"))
         state = torch.full_like(ref_state, float("nan"))
@@ -53,6 +55,8 @@ def test_noalloc_matches_regular_entry_point_twice(name, cfg, tol):
         assert torch.isfinite(out.float()).all() and torch.isfinite(state).all()
         assert _rel(out, ref_out) <= tol, f"{name}: call {call}: out differs"
         assert _rel(state, ref_state) <= tol, f"{name}: call {call}: state differs"
+        e = float(np.linalg.norm(out.double().cpu().numpy() - want["out"]) / np.linalg.norm(want["out"]))
+        assert e <= tol, f"{name}: call {call}: rel L2 {e:.3e} against the oracle"
 
 
 def test_noalloc_rejects_problems_beyond_the_builtin_scratch():
