@@ -119,6 +119,28 @@ def _check_cuda(*ts):
                 raise ValueError("tensors must be contiguous")
 
 
+def _expect(name, t, dtype, shape):
+    """Raise ValueError unless tensor ``t`` (None is allowed: an optional argument) has this dtype and shape.
+    The kernels trust the descriptor: a tensor of another size or type would be read or written out of bounds."""
+    if t is None:
+        return
+    if t.dtype != dtype:
+        raise ValueError(f"{name}: dtype {t.dtype}, expected {dtype}")
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: shape {tuple(t.shape)}, expected {tuple(shape)}")
+
+
+def _expect_tokens(q, k, v, gate, lam, out, names=("q", "k", "v", "out"), **scalars):
+    """q, k, v, out: one I/O dtype and shape [.., heads, d]; gate, lam and the other per-token scalars: float32 [.., heads]."""
+    if q.dim() < 3:
+        raise ValueError(f"{names[0]}: expected [..., heads, d], got shape {tuple(q.shape)}")
+    _io_code(q)
+    for n, t in zip(names[1:], (k, v, out)):
+        _expect(n, t, q.dtype, q.shape)
+    for n, t in dict(gate=gate, lam=lam, **scalars).items():
+        _expect(n, t, torch.float32, q.shape[:-1])
+
+
 def make_desc(B, T, heads, d_k, d_v, io_dtype, precision=GKA_PREC_NATIVE, flags=0, stream=None,
               workspace=None, state_in=None, device_status=None, fro_out=None,
               profile_events=None, beta=None, alpha=None) -> GkaDesc:
@@ -176,14 +198,22 @@ def gka_fwd_chunked(q, k, v, gate, lam, n_iter, chunk=64, out=None, state_out=No
 
     Returns (out, state_out).  Work is enqueued on ``stream`` (default: torch's current stream).
     """
-    _check_cuda(q, k, v, gate, lam, out, state_out, state_in, workspace, fro_out, device_status, beta, alpha)
+    if q.dim() != 4:
+        raise ValueError(f"q: expected [B, T, heads, d], got shape {tuple(q.shape)}")
     B, T, heads, d = q.shape
+    _expect_tokens(q, k, v, gate, lam, out, fro_out=fro_out, beta=beta, alpha=alpha)
+    _expect("state_out", state_out, torch.float32, (B, heads, 2 * d * d))
+    _expect("state_in", state_in, torch.float32, (B, heads, 2 * d * d))
+    _expect("device_status", device_status, torch.int32, (1,))
+    _check_cuda(q, k, v, gate, lam, out, state_out, state_in, workspace, fro_out, device_status, beta, alpha)
     if out is None:
         out = torch.empty_like(v)
     if state_out is None:
         state_out = torch.empty(B, heads, 2 * d * d, dtype=torch.float32, device=q.device)
     if workspace is None:
         workspace = alloc_workspace(B, T, heads, d, q.device, chunk, _io_code(q), precision)
+    elif workspace.dtype != torch.uint8:
+        raise ValueError("workspace: expected a uint8 tensor")
     if stream is None:
         stream = torch.cuda.current_stream(q.device).cuda_stream
     desc = make_desc(B, T, heads, d, v.shape[-1], _io_code(q), precision, flags, stream, workspace,
@@ -202,8 +232,13 @@ def gka_solve_chunked(rhs, k, gate, lam, n_iter, chunk=64, out=None, *, state_in
 
     With rhs = q this is the iterate the forward multiplies by U_t; with rhs = dL/dx it is dL/dq.
     """
-    _check_cuda(rhs, k, gate, lam, out, state_in, workspace, device_status)
+    if rhs.dim() != 4:
+        raise ValueError(f"rhs: expected [B, T, heads, d], got shape {tuple(rhs.shape)}")
     B, T, heads, d = rhs.shape
+    _expect_tokens(rhs, k, None, gate, lam, out, names=("rhs", "k", "v", "x_out"), beta=beta)
+    _expect("state_in", state_in, torch.float32, (B, heads, 2 * d * d))
+    _expect("device_status", device_status, torch.int32, (1,))
+    _check_cuda(rhs, k, gate, lam, out, state_in, workspace, device_status)
     if out is None:
         out = torch.empty_like(rhs)
     if workspace is None:
@@ -228,11 +263,21 @@ def gka_fwd_chunked_host(q, k, v, gate, lam, n_iter, chunk, out, state_out, *, s
                          precision=GKA_PREC_NATIVE, flags=0, stream=None, device_status=None):
     """Host-buffer forward: q, k, v, gate, lam, out, state_out are (pinned) CPU tensors; staging and
     workspace are CUDA byte tensors.  Copies and kernels are enqueued on the stream; no synchronisation."""
+    if q.dim() != 4:
+        raise ValueError(f"q: expected [B, T, heads, d], got shape {tuple(q.shape)}")
+    B, T, heads, d = q.shape
+    if out is None:
+        raise ValueError("out: the host-buffer call writes into a caller-provided CPU tensor")
+    _expect_tokens(q, k, v, gate, lam, out)
+    _expect("state_out", state_out, torch.float32, (B, heads, 2 * d * d))
+    _expect("device_status", device_status, torch.int32, (1,))
     for t in (q, k, v, gate, lam, out, state_out):
         if t is not None and (t.is_cuda or not t.is_contiguous()):
             raise ValueError("host-buffer call takes contiguous CPU tensors")
     _check_cuda(staging, workspace, device_status)
-    B, T, heads, d = q.shape
+    need = gka_fwd_host_staging_bytes(B, T, heads, d, _io_code(q))
+    if staging.dtype != torch.uint8 or staging.numel() < need:
+        raise ValueError(f"staging: expected a uint8 tensor of at least {need} bytes")
     if stream is None:
         stream = torch.cuda.current_stream(staging.device).cuda_stream
     desc = make_desc(B, T, heads, d, v.shape[-1], _io_code(q), precision, flags, stream, workspace,
@@ -250,8 +295,13 @@ def gka_fwd_chunked_noalloc(q, k, v, gate, lam, n_iter, chunk=64, out=None, stat
     """Chunk-wise forward for callers that cannot provide scratch memory: the library's built-in
     scratch array is used instead of a workspace.  ``out`` and ``state_out`` must be given by such
     callers; they are only created here (with torch) when omitted, for convenience in tests."""
-    _check_cuda(q, k, v, gate, lam, out, state_out, state_in)
+    if q.dim() != 4:
+        raise ValueError(f"q: expected [B, T, heads, d], got shape {tuple(q.shape)}")
     B, T, heads, d = q.shape
+    _expect_tokens(q, k, v, gate, lam, out)
+    _expect("state_out", state_out, torch.float32, (B, heads, 2 * d * d))
+    _expect("state_in", state_in, torch.float32, (B, heads, 2 * d * d))
+    _check_cuda(q, k, v, gate, lam, out, state_out, state_in)
     if out is None:
         out = torch.empty_like(v)
     if state_out is None:
@@ -271,8 +321,13 @@ def gka_fwd_chunked_noalloc(q, k, v, gate, lam, n_iter, chunk=64, out=None, stat
 def gka_decode_step(state, q, k, v, gate, lam, n_iter, out=None, *, flags=0, device_status=None,
                     stream=None, profile_events=None, beta=None, alpha=None):
     """One recurrent step.  state: [N,heads,2*d*d] f32, updated in place; q,k,v: [N,heads,d]."""
-    _check_cuda(state, q, k, v, gate, lam, out, device_status)
+    if q.dim() != 3:
+        raise ValueError(f"q: expected [N, heads, d], got shape {tuple(q.shape)}")
     N, heads, d = q.shape
+    _expect_tokens(q, k, v, gate, lam, out, beta=beta, alpha=alpha)
+    _expect("state", state, torch.float32, (N, heads, 2 * d * d))
+    _expect("device_status", device_status, torch.int32, (1,))
+    _check_cuda(state, q, k, v, gate, lam, out, device_status, beta, alpha)
     if out is None:
         out = torch.empty_like(v)
     if stream is None:
@@ -291,8 +346,13 @@ def gka_decode_tokens(state, q, k, v, gate, lam, n_iter, out=None, *, flags=0, d
                       stream=None, profile_events=None, beta=None, alpha=None):
     """The recurrent step over T consecutive tokens.  state: [N,heads,2*d*d] f32, updated in place;
     q,k,v: [N,T,heads,d]; gate, lam (beta, alpha): [N,T,heads]."""
-    _check_cuda(state, q, k, v, gate, lam, out, device_status)
+    if q.dim() != 4:
+        raise ValueError(f"q: expected [N, T, heads, d], got shape {tuple(q.shape)}")
     N, T, heads, d = q.shape
+    _expect_tokens(q, k, v, gate, lam, out, beta=beta, alpha=alpha)
+    _expect("state", state, torch.float32, (N, heads, 2 * d * d))
+    _expect("device_status", device_status, torch.int32, (1,))
+    _check_cuda(state, q, k, v, gate, lam, out, device_status, beta, alpha)
     if out is None:
         out = torch.empty_like(v)
     if stream is None:

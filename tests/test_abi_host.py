@@ -144,6 +144,44 @@ def test_cpu_tensors_are_rejected():
         gka.gka_fwd_chunked(t, t, t, g, g, 1)
 
 
+def test_binding_rejects_mismatched_tensors():
+    """The kernels trust the descriptor, so the binding compares every tensor's dtype and shape with q before it
+    calls the library: a mismatch is a ValueError, never a launch (CPU tensors suffice to show it)."""
+    import torch
+    B, T, H, d = 2, 64, 3, 64
+    q = torch.zeros(B, T, H, d)
+    g = torch.ones(B, T, H)
+    st = torch.zeros(B, H, 2 * d * d)
+    cases = [
+        dict(k=q.double()), dict(k=q[:, :32]), dict(v=q.bfloat16()), dict(gate=g.double()), dict(lam=g[:, :, :2]),
+        dict(gate=g.bfloat16()), dict(out=q.bfloat16()), dict(state_out=st[:, :, :-4]), dict(state_out=st.double()),
+        dict(state_in=st[:1]), dict(fro_out=g.double()), dict(beta=g[:, :10]), dict(alpha=g.half()),
+        dict(device_status=torch.zeros(1, dtype=torch.int64)),
+    ]
+    for bad in cases:
+        kw = dict(k=q, v=q, gate=g, lam=g)
+        kw.update(bad)
+        k, v, gate, lam = (kw.pop(n) for n in ("k", "v", "gate", "lam"))
+        with pytest.raises(ValueError, match="dtype|shape"):
+            gka.gka_fwd_chunked(q, k, v, gate, lam, 1, **kw)
+    with pytest.raises(ValueError, match="dtype|shape"):
+        gka.gka_solve_chunked(q, q.double(), g, g, 1)
+    with pytest.raises(TypeError):
+        gka.gka_fwd_chunked(q.double(), q.double(), q.double(), g, g, 1)          # unsupported I/O dtype
+    # decode: state of the wrong size, per-head scalars of the wrong shape
+    qd, gd = torch.zeros(4, H, d), torch.ones(4, H)
+    with pytest.raises(ValueError, match="shape"):
+        gka.gka_decode_step(torch.zeros(4, H, d * d), qd, qd, qd, gd, gd, 1)
+    with pytest.raises(ValueError, match="shape"):
+        gka.gka_decode_step(torch.zeros(4, H, 2 * d * d), qd, qd, qd, gd[:, :2], gd, 1)
+    with pytest.raises(ValueError, match="dtype"):
+        gka.gka_decode_tokens(torch.zeros(4, H, 2 * d * d).double(), q[:, :4].transpose(0, 1).contiguous(),
+                              q[:, :4].transpose(0, 1).contiguous(), q[:, :4].transpose(0, 1).contiguous(),
+                              torch.ones(4, 2, H), torch.ones(4, 2, H), 1)
+    with pytest.raises(ValueError, match="dtype|shape"):
+        gka.gka_fwd_chunked_noalloc(q, q, q, g, g.double(), 1)
+
+
 def test_synth_substreams_and_distributions():
     cfg = synth.shrink(synth.CONFIGS[1], B=2, heads=3, T=128)
     full = synth.make_inputs(cfg)
