@@ -1,11 +1,11 @@
 // tcgen05 / TMEM solve kernel of the chunk-wise GKA forward (bf16 operands, fp32 accumulation) for sm_100a.
 //
 // Input: for every tile of 128 consecutive tokens of a sequence, the bf16 copies of the tile-initial states
-// H_0, U_0 and ||H_0||_F^2 (written by the state kernel, gka_tc_state.cu).  Tiles are independent problems.  Two
-// persistent thread blocks share an SM, each with one tile in flight (half of the SM's shared memory and tensor
-// memory each), so that the tensor-core products of one block run under the CUDA-core epilogues of the other
-// without any coupling in the code.  A tile puts one token on each TMEM lane; every product of the chunk-wise
-// form (Section 4.2.1; Algorithm 1 on the whole tile) is an M = 128 tile.
+// H_0, U_0 and ||H_0||_F^2 (written by the state kernel, gka_tc_state.cu).  Tiles are independent problems.  One
+// persistent thread block per SM keeps two tiles ("slots") in flight and runs them in opposite phases: while the
+// tensor pipe works on the products of one slot, the CUDA cores run the fp32 update of the other.  A tile puts one
+// token on each TMEM lane; every product of the chunk-wise form (Section 4.2.1; Algorithm 1 on the whole tile) is
+// an M = 128 tile.
 //
 // Algorithm 1 in residual form.  With d_i = x_i - x_{i-1} (x_{-1} = 0, d_0 = x_0 = 2 q / (L + mu)) the update
 // x_{i+1} = x_i + (omega_{i+1} - 1) d_i + (2 omega_{i+1} / (L + mu)) (q - A x_i) reads
@@ -23,10 +23,17 @@
 // bf16 terms (x is dominated by directions that U barely reads; a single bf16 rounding of x would swamp the rest).
 // Chunk-wise Frobenius norms of Section 4.2.1 come from Khat H_0, the Gram matrix Khat Khat^T and an affine scan.
 //
-// Warp roles: 8 compute warps (warp quadrant q = TMEM lanes 32 q .. 32 q + 31, column half hf = 64 of the 128
-// columns: a thread holds one token's 64 channels of the iterate in registers); one warp prepares the gate scalars
-// one tile ahead; one thread issues the TMA loads and stores of the tiles; one thread issues every tcgen05.mma.
-// The compute warps hand work over through mbarriers (one arrival per warp) and wait for tcgen05.commit.
+// On-chip layout.  Tensor memory (512 columns): one score tile S shared by the two slots (only one slot at a time
+// is between its score product and the product that consumes the masked scores: the issuing thread hands S from
+// slot to slot, which is also what keeps the slots in opposite phases), and per slot the fp32 accumulator R (128
+// columns) and the operand E as packed bf16 (64 columns).  E and P feed the products from tensor memory, so a
+// product reads only its B operand (keys, H_0, U_0, values) from shared memory and leaves half of the shared-memory
+// bandwidth to everything else.  Shared memory per slot: keys, H_0 (later U_0), q (later V, then the result).
+//
+// Warp roles: 4 compute warps per slot, a thread owns one token (one TMEM lane) and all 128 channels of its
+// iterate in registers; one warp prepares the gate scalars one tile ahead; one thread per slot issues that slot's
+// TMA stores and the loads that follow them; one thread issues every tcgen05.mma for both slots.  Hand-overs go
+// through mbarriers (one arrival per warp) and tcgen05.commit.
 #include <cuda.h>
 
 #include "gka_common.cuh"
@@ -39,19 +46,20 @@ using namespace tcu;
 
 constexpr int D = 128;
 constexpr int NT = kTile;                  // tokens per tile: one per TMEM lane
-constexpr int CT = 256;                    // compute threads
-constexpr int NW = CT / 32;                // compute warps
-constexpr int kThreadsSolve = CT + 128;    // + helper warpgroup: gate scalars, TMA, MMA issue
-constexpr int kBlocksPerSM = 2;
-constexpr int kRegsLaunch = 80, kRegsCompute = 104, kRegsHelper = 32;   // register split after setmaxnreg
-static_assert(kThreadsSolve * kRegsLaunch * kBlocksPerSM <= 65536, "launch registers");
+constexpr int kSlots = 2;
+constexpr int ST = 128;                    // compute threads per slot
+constexpr int CT = kSlots * ST;            // compute threads
+constexpr int kThreadsSolve = CT + 128;    // + helper warpgroup: gate scalars, TMA (one warp per slot), MMA issue
+constexpr int kRegsLaunch = 168, kRegsCompute = 232, kRegsHelper = 40;   // register split after setmaxnreg
+static_assert(kThreadsSolve * kRegsLaunch <= 65536, "launch registers");
 static_assert(CT * kRegsCompute + 128 * kRegsHelper <= kThreadsSolve * kRegsLaunch, "register split exceeds the launch allocation");
 
-// ---- shared memory map (bytes; operand buffers 1024-byte aligned): three operand tiles and the scalars
-constexpr uint32_t BUF_K = 0;                  // Khat, later V
-constexpr uint32_t BUF_H = kTileBytes;         // bf16 H_0, later U_0
-constexpr uint32_t BUF_D = 2 * kTileBytes;     // q, then the operand E, then the output tile
-constexpr uint32_t OFF_SC = 3 * kTileBytes;    // scalars
+// ---- shared memory map (bytes; operand buffers 1024-byte aligned): three operand tiles per slot, then the scalars
+constexpr uint32_t BUF_A = 0;                  // keys (Khat)
+constexpr uint32_t BUF_B = kTileBytes;         // bf16 H_0, later U_0
+constexpr uint32_t BUF_C = 2 * kTileBytes;     // q, later V, then the result tile
+constexpr uint32_t SLOT_BYTES = 3 * kTileBytes;
+constexpr uint32_t OFF_SC = kSlots * SLOT_BYTES;
 
 struct GateScalars {       // per token of a tile, from the gates and the other per-token inputs alone
     float lg[NT];          // log2 gamma_c
@@ -61,44 +69,44 @@ struct GateScalars {       // per token of a tile, from the gates and the other 
     float iz[NT];          // 1 / zt_c
     float lam[NT];         // lambda_c as given
     float al[NT];          // alpha_c (alpha-connection)
-    float sb[NT];          // sqrt(beta_j) (beta-augmented write)
-    float ks[NT];          // row factor of the staged keys: sb_j 2^(-G_j / 2), or sb_j alone when the tile decays below 2^-60
+    float ks[NT];          // row factor of the staged keys: sqrt(beta_j) 2^(-G_j / 2), or sqrt(beta_j) alone when the tile decays below 2^-60
 };
-struct TileScalars {
+struct SlotScalars {
     GateScalars g[2];
-    float rho2[NT], czb[NT], lz[NT];   // rho^2;  -zt 2 / (L + mu) (0 past the sequence);  lambda / zt
-    float part[2][2][NT];              // Frobenius partial sums: [k H_0 k | Gram part][column half][key]
-    float carry[2][4];                 // per-warp totals (a, b) of the affine scan
-    int stop;
+    float carry[2][4];     // per-warp totals (a, b) of the affine scan
 };
-constexpr uint32_t SC_BYTES = (sizeof(TileScalars) + 127) / 128 * 128;
-constexpr uint32_t SOLVE_SMEM = OFF_SC + SC_BYTES + 1024;   // + slack for the 1024-byte alignment of the base
-static_assert(kBlocksPerSM * (SOLVE_SMEM + 1024 + 256) <= 233472, "shared memory budget of two blocks per SM");
+constexpr uint32_t SC_BYTES = (sizeof(SlotScalars) + 127) / 128 * 128;
+constexpr uint32_t SOLVE_SMEM = OFF_SC + kSlots * SC_BYTES + 1024;   // + slack for the 1024-byte alignment of the base
+static_assert(SOLVE_SMEM + 2048 <= 232448, "shared memory budget");
 
-// ---- TMEM columns: score accumulator S (P overwrites it in place), residual / output accumulator R
-constexpr uint32_t TM_S = 0, TM_R = 128;
+// ---- TMEM columns: shared score accumulator S (P overwrites it in place); per slot the residual / output
+// accumulator R and the bf16 operand E
+constexpr uint32_t TM_S = 0;
+__host__ __device__ constexpr uint32_t tm_r_of(int s) { return 128u + 128u * (uint32_t)s; }
+__host__ __device__ constexpr uint32_t tm_e_of(int s) { return 384u + 64u * (uint32_t)s; }
 
-enum {
-    B_LD_K = 0,    // K tile has landed (TMA)
-    B_LD_H,        // H_0 tile
-    B_LD_Q,        // q tile
-    B_LD_U,        // U_0 tile
-    B_LD_V,        // V tile
-    B_RDY,         // compute warps -> MMA issuer: operands of the next batch are in place (one arrival per warp)
-    B_RDY_ST,      // compute warps -> TMA thread: the output tile is staged
-    B_MMA_S,       // tcgen05.commit: score-side batch complete
-    B_MMA_R,       // tcgen05.commit: accumulator-side batch complete
-    B_GS0, B_GS1,  // gate scalars of buffer 0 / 1 are ready
-    B_GF0, B_GF1,  // compute warps -> gate helper: buffer 0 / 1 is free
-    B_DRAIN,       // every product is complete (before the tensor memory is given back)
-    B_COUNT
+enum {                 // per slot
+    B_LD_K = 0,        // K tile has landed (TMA)
+    B_LD_H,            // H_0 tile
+    B_LD_Q,            // q tile
+    B_LD_U,            // U_0 tile
+    B_LD_V,            // V tile
+    B_RDY_ST,          // compute warps -> TMA thread: the result tile is staged
+    B_QF,              // compute warps -> TMA thread: q has been read, V may take its buffer
+    B_MMA_S,           // tcgen05.commit: score-side batch complete
+    B_MMA_R,           // tcgen05.commit: accumulator-side batch complete
+    B_GS0, B_GS1,      // gate scalars of buffer 0 / 1 are ready
+    B_GF0, B_GF1,      // compute warps -> gate helper: buffer 0 / 1 is free
+    B_PER_SLOT
 };
+constexpr int B_DRAIN = kSlots * B_PER_SLOT;   // every product is complete (before the tensor memory is given back)
+constexpr int B_COUNT = B_DRAIN + 1;
 
-struct Ctx {
-    int tid, l, q, hf, c;         // thread, lane, TMEM lane quadrant, column half, token / TMEM lane
-    uint32_t lane_addr, sbase, bars, tmem, abort_addr;
-    unsigned char *smem;
-};
+// Requests a slot makes to the issuing thread: every warp of the slot adds one to the slot's request counter in
+// shared memory (a poll of both counters is one 40-cycle load, where a test of an mbarrier phase takes 100 cycles);
+// request n of a slot is ready when its counter has reached 4 (n + 1).  In this order per tile:
+// FROB, then n_iter times (ITER1, ITER2), then (unless the solve itself is the result) OUT_S, OUT_O
+enum { OP_FROB = 0, OP_ITER1, OP_ITER2, OP_OUT_S, OP_OUT_O };
 
 __device__ __forceinline__ bool aborted(uint32_t abort_addr) {
     int v;
@@ -108,11 +116,37 @@ __device__ __forceinline__ bool aborted(uint32_t abort_addr) {
 __device__ __forceinline__ void set_abort(uint32_t abort_addr) {
     asm volatile("st.volatile.shared.b32 [%0], %1;" ::"r"(abort_addr), "r"(1) : "memory");
 }
-// Bounded wait; once any wait of the block has given up every later wait returns at once, so the block runs to its
-// end without further delays and reports GKA_ERR_TIMEOUT.
+// Bounded wait (about a second; the wait suspends in hardware between polls); once any wait of the block has given up
+// every later wait returns at once, so the block runs to its end without further delays and reports
+// GKA_ERR_TIMEOUT.  One compact loop in a single asm block: the wait is inlined at some thirty places.
 __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, uint32_t abort_addr) {
-    if (aborted(abort_addr)) return;
-    if (!mbar_spin_bounded(bar, parity)) set_abort(abort_addr);
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .u32 n, ab;\n\t"
+        "mov.u32 n, 0;\n\t"
+        "ld.volatile.shared.b32 ab, [%4];\n\t"
+        "setp.ne.u32 p, ab, 0;\n\t"
+        "@p bra WAIT_DONE;\n"
+        "WAIT_LOOP:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "@p bra WAIT_DONE;\n\t"
+        "add.u32 n, n, 1;\n\t"
+        "setp.lt.u32 q, n, 200000;\n\t"
+        "@q bra WAIT_LOOP;\n"
+        "WAIT_DONE:\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(5000u), "r"(abort_addr)
+        : "memory");
+    if (!ok) set_abort(abort_addr);
+}
+// one count per warp on a shared-memory counter, after every lane's writes and fences (release); acquire load of a pair
+__device__ __forceinline__ void warp_post(uint32_t addr, int lane) {
+    __syncwarp();
+    if (lane == 0) asm volatile("red.release.cta.shared::cta.add.u32 [%0], 1;" ::"r"(addr) : "memory");
+}
+__device__ __forceinline__ void ld_acquire_pair(uint32_t addr, uint32_t &a, uint32_t &b) {
+    asm volatile("ld.acquire.cta.shared::cta.v2.u32 {%0, %1}, [%2];" : "=r"(a), "=r"(b) : "r"(addr) : "memory");
 }
 // one arrival per warp, after every lane's writes and fences
 __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
@@ -136,86 +170,188 @@ __device__ __forceinline__ TileInfo tile_info(const FwdArgs &a, long long tile) 
     return t;
 }
 
-// Masked score epilogue: S (TMEM, fp32) -> P (packed bf16 pairs, written over the first 16 columns of each 32-column
-// block of the scores).  A thread owns token c = 32 q + l and the key blocks kb = 2 hf, 2 hf + 1 (keys 32 kb + i):
-// blocks above the diagonal are zero, blocks below it need no mask.  EXACT: per-element factor 2^(ac_c - G_j)
-// (strongly decaying tiles, whose keys are not pre-scaled).
-template <bool EXACT, bool DIAG, bool KEYF>
-__device__ __forceinline__ void p_block(const Ctx &cx, const float *G2kb, const float *kskb, uint32_t taddr, float ac_c) {
-#pragma unroll
-    for (int piece = 0; piece < 2; ++piece) {
-        uint32_t r[16], pk[8];
-        TMEM_LD16(taddr + 16 * piece, r);
-        tmem_wait_ld();
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int i0 = 16 * piece + 2 * u;
-            float p0 = __uint_as_float(r[2 * u]), p1 = __uint_as_float(r[2 * u + 1]);
-            if (EXACT) {
-                p0 *= ex2_fast(fminf(ac_c - G2kb[i0], 126.f));
-                p1 *= ex2_fast(fminf(ac_c - G2kb[i0 + 1], 126.f));
-            }
-            if (KEYF) {                     // the values are not pre-scaled: their row factor rides on the scores
-                const float2 f = *reinterpret_cast<const float2 *>(kskb + i0);
-                p0 *= f.x;
-                p1 *= f.y;
-            }
-            if (DIAG) {                     // keys i <= l are visible
-                p0 = (i0 <= cx.l) ? p0 : 0.f;
-                p1 = (i0 + 1 <= cx.l) ? p1 : 0.f;
-            }
-            pk[u] = pack_bf16(p0, p1);
-        }
-        TMEM_ST8(taddr + 8 * piece, pk);
+// Products of the issuing thread: 8 k-steps of 16 each.  The three products of an iteration are unrolled with
+// immediate descriptor offsets (the issue then keeps up with the tensor pipe: one tcgen05.mma per 64 cycles); the
+// products that run once per tile are issued from rolled loops with run-time descriptors, at about 100 cycles per
+// instruction, which keeps the code of the issuing warp small in the instruction cache.
+// D (+)= A x B with A (packed bf16 pairs, 8 columns per k-step of 16) in TMEM and B in shared memory
+template <int ACC, uint32_t B_CONST>
+__device__ __forceinline__ void mma_ts_c(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_base, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .b64 db;\n\t.reg .b32 lb;\n\t"
+        "add.u32 lb, %2, %5;\n\tmov.b64 db, {lb, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, %6;\n\t}" ::"r"(d_tmem), "r"(a_tmem), "r"(b_base), "r"(idesc),
+        "r"(kDescHi), "n"(B_CONST), "n"(ACC)
+        : "memory");
+}
+// A = operand tile in TMEM (64 columns: channels 2 u, 2 u + 1 of a token in column u), B K-major
+template <int ACC0, int KS = 0>
+__device__ __forceinline__ void mma8_ek(uint32_t d, uint32_t e_tmem, uint32_t b_base, uint32_t idesc) {
+    if constexpr (KS < 8) {
+        mma_ts_c<(KS == 0 ? ACC0 : 1), t_kmaj(0) + t_kstep(KS)>(d, e_tmem + 8 * KS, b_base, idesc);
+        mma8_ek<ACC0, KS + 1>(d, e_tmem, b_base, idesc);
     }
 }
-// keyf: multiply key j's column by ks[j] as well (the pass whose P meets the unscaled V)
-template <bool KEYF>
-__device__ __forceinline__ void p_epilogue(const Ctx &cx, uint32_t tm_s, const GateScalars *gs, bool exact, float ac_c) {
+// low descriptor word of k-step ks of a K-major operand tile / an MN-major operand tile (relative to its base)
+__device__ __forceinline__ uint32_t kmaj_lo(uint32_t base14, int ks) {
+    return base14 + t_kmaj(0) + (uint32_t)((ks >> 2) * 1024 + (ks & 3) * 2);
+}
+__device__ __forceinline__ uint32_t mn_lo(uint32_t base14, int ks) { return base14 + t_mn(0) + (uint32_t)(ks * 128); }
+__device__ __forceinline__ void mma_ss_rt(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
+        "mov.b64 da, {%1, %4};\n\tmov.b64 db, {%2, %4};\n\tsetp.ne.u32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc),
+        "r"(kDescHi), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ts_rt(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .b64 db;\n\t.reg .pred p;\n\t"
+        "mov.b64 db, {%2, %4};\n\tsetp.ne.u32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}" ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc),
+        "r"(kDescHi), "r"(acc)
+        : "memory");
+}
+// both operands in shared memory, K-major
+__device__ __forceinline__ void prod_kk(uint32_t d, uint32_t a14, uint32_t b14, uint32_t acc0) {
+#pragma unroll 1
+    for (int ks = 0; ks < 8; ++ks) mma_ss_rt(d, kmaj_lo(a14, ks), kmaj_lo(b14, ks), kIdescKK, ks ? 1u : acc0);
+}
+// A = operand tile in TMEM (64 columns: channels 2 u, 2 u + 1 of a token in column u), B K-major
+__device__ __forceinline__ void prod_ek(uint32_t d, uint32_t e_tmem, uint32_t b14, uint32_t acc0) {
+#pragma unroll 1
+    for (int ks = 0; ks < 8; ++ks) mma_ts_rt(d, e_tmem + 8 * ks, kmaj_lo(b14, ks), kIdescKK, ks ? 1u : acc0);
+}
+// A = masked scores P in TMEM (key block kb in the first 16 columns of the 32-column block kb of the score tile),
+// B MN-major; accumulates
+__device__ __forceinline__ void prod_pm(uint32_t d, uint32_t p_tmem, uint32_t b14) {
+#pragma unroll 1
+    for (int ks = 0; ks < 8; ++ks) mma_ts_rt(d, p_tmem + 32 * (ks >> 1) + 8 * (ks & 1), mn_lo(b14, ks), kIdescPM, 1u);
+}
+
+// The products of one request.  kb, hb, cb: descriptor bases (shared address >> 4) of the slot's buffers.
+__device__ __forceinline__ void issue_batch(int op, uint32_t kb, uint32_t hb, uint32_t cb, uint32_t tm_S, uint32_t tm_R,
+                                            uint32_t tm_E, uint32_t bar_s, uint32_t bar_r) {
+    switch (op) {
+        case OP_FROB:    // Gram matrix Khat Khat^T and Khat H_0
+            prod_kk(tm_S, kb, kb, 0u);
+            prod_kk(tm_R, kb, hb, 0u);
+            mma_commit(bar_s);
+            break;
+        case OP_ITER1:   // S = E Khat^T, R += E H_0^T (the second runs under the masked-score epilogue)
+            mma8_ek<0>(tm_S, tm_E, kb, kIdescKK);
+            mma_commit(bar_s);
+            mma8_ek<1>(tm_R, tm_E, hb, kIdescKK);
+            break;
+        case OP_ITER2:   // R += P Khat
+            mma8_pm(tm_R, tm_S, kb, kIdescPM);
+            mma_commit(bar_r);
+            break;
+        case OP_OUT_S:   // scores of the final iterate: S = X_hi Khat^T + X_lo Khat^T (X_lo sits in the first columns of R)
+            prod_ek(tm_S, tm_E, kb, 0u);
+            prod_ek(tm_S, tm_R, kb, 1u);
+            mma_commit(bar_s);
+            break;
+        case OP_OUT_O:   // O = X_hi U_0^T + P V
+            prod_ek(tm_R, tm_E, hb, 0u);
+            prod_pm(tm_R, tm_S, cb);
+            mma_commit(bar_r);
+            break;
+        default:
+            break;
+    }
+}
+
+struct Ctx {
+    int l, q, c;                  // lane, TMEM lane quadrant, token / TMEM lane of the slot's tile
+    uint32_t tm_s, tm_r, tm_e;    // TMEM addresses of this thread's lane: scores, accumulator, operand
+};
+
+// Masked scores of 16 keys: S (fp32, 16 columns) -> P (packed bf16 pairs in 8 registers).  EXACT: per-element factor
+// 2^(ac_c - G_j) (strongly decaying tiles, whose keys are not pre-scaled); KEYF: key j's column times ks[j] (the pass
+// whose P meets the unscaled V); DIAG: keys i <= l of the 32-key block are visible (i0: first key of this half).
+template <bool EXACT, bool KEYF, bool DIAG>
+__device__ __forceinline__ void p_half(const uint32_t (&r)[16], uint32_t (&pk)[8], const float *G2h, const float *ksh,
+                                       float ac_c, int l, int i0) {
 #pragma unroll
-    for (int b2 = 0; b2 < 2; ++b2) {
-        const int kb = 2 * cx.hf + b2;
-        const uint32_t taddr = tm_s + cx.lane_addr + 32 * kb;
-        const float *G2kb = gs->G2 + 32 * kb, *kskb = gs->ks + 32 * kb;
-        if (kb > cx.q) {
-            uint32_t z[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) z[i] = 0u;
-            TMEM_ST8(taddr, z);
-            TMEM_ST8(taddr + 8, z);
-        } else if (kb == cx.q) {
-            if (exact) p_block<true, true, KEYF>(cx, G2kb, kskb, taddr, ac_c);
-            else p_block<false, true, KEYF>(cx, G2kb, kskb, taddr, ac_c);
-        } else {
-            if (exact) p_block<true, false, KEYF>(cx, G2kb, kskb, taddr, ac_c);
-            else p_block<false, false, KEYF>(cx, G2kb, kskb, taddr, ac_c);
+    for (int u = 0; u < 8; ++u) {
+        float p0 = __uint_as_float(r[2 * u]), p1 = __uint_as_float(r[2 * u + 1]);
+        if (EXACT) {
+            p0 *= ex2_fast(fminf(ac_c - G2h[2 * u], 126.f));
+            p1 *= ex2_fast(fminf(ac_c - G2h[2 * u + 1], 126.f));
         }
+        if (KEYF) {
+            const float2 f = *reinterpret_cast<const float2 *>(ksh + 2 * u);
+            p0 *= f.x;
+            p1 *= f.y;
+        }
+        if (DIAG) {
+            p0 = (i0 + 2 * u <= l) ? p0 : 0.f;
+            p1 = (i0 + 2 * u + 1 <= l) ? p1 : 0.f;
+        }
+        pk[u] = pack_bf16(p0, p1);
+    }
+}
+// Masked-score epilogue of token c = 32 q + l: key blocks below q need no mask, block q is the diagonal block, the
+// blocks above it are zero.  P for keys 32 kb + 2 u, 2 u + 1 goes to column 32 kb + u of the score tile.  One 32-key
+// block per pass of a rolled loop (the code stays small; the two loads of a pass are in flight together).
+template <bool EXACT, bool KEYF>
+__device__ __forceinline__ void p_epilogue_t(const Ctx &cx, const GateScalars *gs, float ac_c) {
+#pragma unroll 1
+    for (int kb = 0; kb < 4; ++kb) {
+        const uint32_t taddr = cx.tm_s + 32 * kb;
+        uint32_t pa[8], pb[8];
+        if (kb > cx.q) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pa[i] = 0u;
+            TMEM_ST8(taddr, pa);
+            TMEM_ST8(taddr + 8, pa);
+            continue;
+        }
+        uint32_t ra[16], rb[16];
+        TMEM_LD16(taddr, ra);
+        TMEM_LD16(taddr + 16, rb);
+        const float *G2kb = gs->G2 + 32 * kb, *kskb = gs->ks + 32 * kb;
+        tmem_wait_ld();
+        if (kb == cx.q) {
+            p_half<EXACT, KEYF, true>(ra, pa, G2kb, kskb, ac_c, cx.l, 0);
+            p_half<EXACT, KEYF, true>(rb, pb, G2kb + 16, kskb + 16, ac_c, cx.l, 16);
+        } else {
+            p_half<EXACT, KEYF, false>(ra, pa, G2kb, kskb, ac_c, cx.l, 0);
+            p_half<EXACT, KEYF, false>(rb, pb, G2kb + 16, kskb + 16, ac_c, cx.l, 16);
+        }
+        TMEM_ST8(taddr, pa);
+        TMEM_ST8(taddr + 8, pb);
     }
     tmem_wait_st();
 }
-
-// Scale the 128 rows of a bf16 operand tile in place by the per-row factors f[j].
-__device__ __forceinline__ void scale_rows(unsigned char *tile, const float *f, int tid) {
-#pragma unroll
-    for (int i = 0; i < 2048 / CT; ++i) {
-        const int qi = tid + CT * i;               // 16-byte group index in the 32 KB tile
-        const float fj = f[(qi & 1023) >> 3];      // row of this group
-        const uint64_t f2 = f2_pack(fj, fj);
-        uint4 v = *reinterpret_cast<const uint4 *>(tile + qi * 16);
-        uint32_t *pv = reinterpret_cast<uint32_t *>(&v);
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            float lo, hi;
-            f2_unpack(f2_mul(f2_pack(bf16_lo(pv[u]), bf16_hi(pv[u])), f2), lo, hi);
-            pv[u] = pack_bf16(lo, hi);
-        }
-        *reinterpret_cast<uint4 *>(tile + qi * 16) = v;
-    }
+template <bool KEYF>
+__device__ __forceinline__ void p_epilogue(const Ctx &cx, const GateScalars *gs, bool exact, float ac_c) {
+    if (exact) p_epilogue_t<true, KEYF>(cx, gs, ac_c);
+    else p_epilogue_t<false, KEYF>(cx, gs, ac_c);
 }
 
-// Inclusive scan over the tile's 128 tokens (threads 0..127 = warps 0..3, one token each) of the affine maps
+// Sum over one 32-key block of the squared Gram entries of the earlier keys (decayed when the keys are not
+// pre-scaled) and the key's own squared norm.
+template <bool DIAG>
+__device__ __forceinline__ void gram_block(const uint32_t (&r)[32], const float *G2kb, float G2j, bool exact, int l, float &gsum) {
+    float gs2 = 0.f, gd = 0.f;
+#pragma unroll
+    for (int ii = 0; ii < 32; ++ii) {
+        const float g = __uint_as_float(r[ii]);
+        const float g2 = g * g;
+        if (DIAG && ii == l) gd = g2;
+        const bool in = !DIAG || ii < l;
+        if (!exact) gs2 += in ? g2 : 0.f;
+        else if (in) gs2 = fmaf(ex2_fast(G2j - G2kb[ii]), g2, gs2);
+    }
+    gsum += 2.f * gs2 + gd;
+}
+
+// Inclusive scan over the tile's 128 tokens (the slot's four warps, one token per thread) of the affine maps
 // s -> a s + b, composed in token order; returns the map's value at `seed`.
-__device__ __forceinline__ float affine_scan(const Ctx &cx, TileScalars *sc, float a, float b, float seed) {
+__device__ __forceinline__ float affine_scan(const Ctx &cx, SlotScalars *sc, int slot, float a, float b, float seed) {
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const float pa = __shfl_up_sync(0xffffffffu, a, o), pb = __shfl_up_sync(0xffffffffu, b, o);
@@ -224,51 +360,19 @@ __device__ __forceinline__ float affine_scan(const Ctx &cx, TileScalars *sc, flo
             a *= pa;
         }
     }
+    // (the previous tile's carries have long been read: every warp of the slot has passed several hand-overs since)
     if (cx.l == 31) {
         sc->carry[0][cx.q] = a;
         sc->carry[1][cx.q] = b;
     }
-    asm volatile("bar.sync 2, 128;" ::: "memory");
+    asm volatile("bar.sync %0, 128;" ::"r"(slot + 1) : "memory");
     float s = seed;
     for (int w = 0; w < cx.q; ++w) s = fmaf(sc->carry[0][w], s, sc->carry[1][w]);
     return fmaf(a, s, b);
 }
 
-// Batches of products the issuing thread runs, one per arrival phase of B_RDY, in this order per tile:
-// FROB, then n_iter times (ITER1, ITER2), then (unless the solve itself is the result) OUT_S, OUT_O.
-__device__ __forceinline__ void issue_batch(int op, uint32_t base14, uint32_t tm, uint32_t bars) {
-    const uint32_t kb = base14 + (BUF_K >> 4), hb = base14 + (BUF_H >> 4), db = base14 + (BUF_D >> 4);
-    const uint32_t tm_S = tm + TM_S, tm_R = tm + TM_R;
-    switch (op) {
-        case 0:   // FROB: Gram matrix Khat Khat^T and Khat H_0
-            mma8_kk<0>(tm_S, kb, kb, kIdescKK);
-            mma8_kk<0>(tm_R, kb, hb, kIdescKK);
-            mma_commit(bars + 8 * B_MMA_S);
-            break;
-        case 1:   // ITER1: S = E Khat^T, R += E H_0^T (the second runs under the masked-score epilogue)
-            mma8_kk<0>(tm_S, db, kb, kIdescKK);
-            mma_commit(bars + 8 * B_MMA_S);
-            mma8_kk<1>(tm_R, db, hb, kIdescKK);
-            break;
-        case 2:   // ITER2: R += P Khat
-            mma8_pm(tm_R, tm_S, kb, kIdescPM);
-            mma_commit(bars + 8 * B_MMA_R);
-            break;
-        case 3:   // OUT_S: scores of the final iterate, S = X_hi Khat^T + X_lo Khat^T (X_lo sits in the H_0 buffer)
-            mma8_kk<0>(tm_S, db, kb, kIdescKK);
-            mma8_kk<1>(tm_S, hb, kb, kIdescKK);
-            mma_commit(bars + 8 * B_MMA_S);
-            break;
-        default:  // OUT_O: O = X_hi U_0^T + P V
-            mma8_kk<0>(tm_R, db, hb, kIdescKK);
-            mma8_pm(tm_R, tm_S, kb, kIdescPM);
-            mma_commit(bars + 8 * B_MMA_R);
-            break;
-    }
-}
-
 template <bool EXTRA>
-__global__ void __launch_bounds__(kThreadsSolve, kBlocksPerSM)
+__global__ void __launch_bounds__(kThreadsSolve, 1)
 fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
                     const __grid_constant__ CUtensorMap tmS, FwdArgs a, long long ntiles) {
@@ -276,6 +380,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     __shared__ __align__(8) uint64_t s_bars[B_COUNT];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
+    __shared__ __align__(16) uint32_t s_req[4];     // per slot: requests posted (warps), Gram matrices read (warps)
 
     unsigned char *smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     const int tid = threadIdx.x;
@@ -284,14 +389,16 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
     if (tid == 0) {
         s_abort = 0;
+        s_req[0] = s_req[1] = s_req[2] = s_req[3] = 0u;
         for (int i = 0; i < B_COUNT; ++i) {
-            const int count = (i == B_RDY || i == B_RDY_ST || i == B_GF0 || i == B_GF1) ? NW : 1;
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bars + 8 * i), "r"(count));
+            const int b = i % B_PER_SLOT;
+            const bool per_warp = i < B_DRAIN && (b == B_RDY_ST || b == B_QF || b == B_GF0 || b == B_GF1);
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bars + 8 * i), "r"(per_warp ? ST / 32 : 1));
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid < 32) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(&s_tmem_base))
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&s_tmem_base))
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -300,9 +407,8 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     fence_after();
     const uint32_t tmem = s_tmem_base;
     const uint32_t sbase = smem_u32(smem);
-    TileScalars *const sc = reinterpret_cast<TileScalars *>(smem + OFF_SC);
 
-    // this block's tiles: a contiguous range
+    // this block's tiles: a contiguous range, dealt to the two slots in turn
     const long long t_lo = (ntiles * blockIdx.x) / gridDim.x, t_hi = (ntiles * (blockIdx.x + 1)) / gridDim.x;
     const int n_mine = (int)(t_hi - t_lo);
     const bool solve_only = EXTRA && a.solve_only != 0;   // the result is the solve itself: no V, no U, no output product
@@ -310,15 +416,19 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const float *const alpha_p = EXTRA ? a.alpha : nullptr;
     const bool mix = alpha_p != nullptr && !solve_only;   // alpha-connection: the read uses alpha x + (1 - alpha) q
 
-    if (tid >= CT) {
+    // The helper warps come first: when a scheduler changes warps it prefers the oldest eligible one, and the thread
+    // that issues the products must not wait behind the compute warps of its scheduler.
+    if (tid < 128) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsHelper));
-        const int hw = (tid - CT) >> 5, lane = tid & 31;
+        const int hw = tid >> 5, lane = tid & 31;
         if (hw == 0) {
             // ================= gate scalars of every tile, one tile ahead of the compute warps =================
             for (int k = 0; k < n_mine; ++k) {
-                if (k >= 2) wait_bar(bars + 8 * (B_GF0 + (k & 1)), (uint32_t)(((k - 2) >> 1) & 1), abort_addr);
+                const int slot = k & 1, j = k >> 1;
+                const uint32_t sb = bars + 8 * (slot * B_PER_SLOT);
+                if (j >= 2) wait_bar(sb + 8 * (B_GF0 + (j & 1)), (uint32_t)(((j - 2) >> 1) & 1), abort_addr);
                 const TileInfo ti = tile_info(a, t_lo + k);
-                GateScalars *g = &sc->g[k & 1];
+                GateScalars *g = &reinterpret_cast<SlotScalars *>(smem + OFF_SC + slot * SC_BYTES)->g[j & 1];
                 float run = 0.f;
                 float ks_g[4], ks_s[4];
 #pragma unroll
@@ -346,7 +456,6 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     g->zt[cc] = exp2f(mc);
                     g->iz[cc] = exp2f(-mc);
                     g->lam[cc] = lamv;
-                    g->sb[cc] = sqrtf(fmaxf(bv, 0.f));
                     g->al[cc] = av;
                     ks_g[grp] = G2c;
                     ks_s[grp] = sqrtf(fmaxf(bv, 0.f));
@@ -360,86 +469,153 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         g->ks[32 * grp + lane] = exact ? ks_s[grp] : ks_s[grp] * exp2f(-0.5f * ks_g[grp]);
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bars + 8 * (B_GS0 + (k & 1)));
+                if (lane == 0) mbar_arrive(sb + 8 * (B_GS0 + (j & 1)));
             }
-        } else if (hw == 1) {
-            // ================= TMA: loads of every tile's K, H_0, q; stores of the output tiles =================
-            if (lane == 0) {
-                auto load_k = [&](int k) {
-                    const TileInfo ti = tile_info(a, t_lo + k);
-                    mbar_expect_tx(bars + 8 * B_LD_K, 32768u);
-                    tma_load_tile3(&tmK, sbase + BUF_K, bars + 8 * B_LD_K, ti.h * D, ti.n * NT, ti.b);
-                };
-                auto load_h = [&](int k) {
-                    mbar_expect_tx(bars + 8 * B_LD_H, 32768u);
-                    tma_load_tile2(&tmS, sbase + BUF_H, bars + 8 * B_LD_H, (int)((t_lo + k) * 256));
-                };
+        } else if (hw == 1 || hw == 3) {
+            // ========== TMA thread of a slot: first loads, V once q has been read, result stores, the next q ==========
+            const int slot = hw >> 1;
+            const int n_slot = (n_mine - slot + 1) >> 1;       // tiles of this slot: k = slot, slot + 2, ...
+            if (lane == 0 && n_slot > 0) {
+                const uint32_t sb = bars + 8 * (slot * B_PER_SLOT);
+                const uint32_t sl = sbase + slot * SLOT_BYTES;
                 auto load_q = [&](int k) {
                     const TileInfo ti = tile_info(a, t_lo + k);
-                    mbar_expect_tx(bars + 8 * B_LD_Q, 32768u);
-                    tma_load_tile3(&tmQ, sbase + BUF_D, bars + 8 * B_LD_Q, ti.h * D, ti.n * NT, ti.b);
+                    mbar_expect_tx(sb + 8 * B_LD_Q, 32768u);
+                    tma_load_tile3(&tmQ, sl + BUF_C, sb + 8 * B_LD_Q, ti.h * D, ti.n * NT, ti.b);
                 };
                 // the inputs do not depend on the state kernel; its per-tile states do
-                if (n_mine > 0) {
-                    load_q(0);
-                    load_k(0);
+                {
+                    const TileInfo ti = tile_info(a, t_lo + slot);
+                    load_q(slot);
+                    mbar_expect_tx(sb + 8 * B_LD_K, 32768u);
+                    tma_load_tile3(&tmK, sl + BUF_A, sb + 8 * B_LD_K, ti.h * D, ti.n * NT, ti.b);
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    mbar_expect_tx(sb + 8 * B_LD_H, 32768u);
+                    tma_load_tile2(&tmS, sl + BUF_B, sb + 8 * B_LD_H, (int)((t_lo + slot) * 256));
                 }
-                asm volatile("griddepcontrol.wait;" ::: "memory");
-                if (n_mine > 0) load_h(0);
-                // The result tile is staged in the H_0 / U_0 buffer (the solve alone: in the operand buffer).  The other
-                // two buffers of the next tile are loaded by a compute thread as soon as the last product is complete;
-                // the staging buffer's next content follows once the store has read it.
-                const uint32_t stage_buf = solve_only ? BUF_D : BUF_H;
-                for (int k = 0; k < n_mine; ++k) {
-                    wait_bar(bars + 8 * B_RDY_ST, (uint32_t)(k & 1), abort_addr);
+                for (int j = 0; j < n_slot; ++j) {
+                    const int k = slot + 2 * j;
                     const TileInfo ti = tile_info(a, t_lo + k);
+                    if (!solve_only) {
+                        wait_bar(sb + 8 * B_QF, (uint32_t)(j & 1), abort_addr);
+                        mbar_expect_tx(sb + 8 * B_LD_V, 32768u);
+                        tma_load_tile3(&tmV, sl + BUF_C, sb + 8 * B_LD_V, ti.h * D, ti.n * NT, ti.b);
+                    }
+                    wait_bar(sb + 8 * B_RDY_ST, (uint32_t)(j & 1), abort_addr);
                     for (int hf = 0; hf < 2; ++hf)     // rows past the sequence are clipped
                         asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::
                                          "l"(reinterpret_cast<uint64_t>(&tmO)), "r"(ti.h * D + 64 * hf), "r"(ti.n * NT),
-                                     "r"(ti.b), "r"(sbase + stage_buf + 16384 * hf)
+                                     "r"(ti.b), "r"(sl + BUF_C + 16384 * hf)
                                      : "memory");
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    const bool more = k + 1 < n_mine && !aborted(abort_addr);
-                    if (more && solve_only) {
-                        load_k(k + 1);
-                        load_h(k + 1);
-                    }
                     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the staged tile has been read
-                    if (more) {
-                        if (solve_only) load_q(k + 1);
-                        else load_h(k + 1);
-                    }
+                    if (j + 1 < n_slot && !aborted(abort_addr)) load_q(k + 2);
                 }
                 asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // output stores are complete
             }
-        } else if (hw == 2) {
+        } else {
             // ================================ MMA issuing thread ================================
+            // Serves the requests of both slots in the order they become ready.  The score tile S is held by a slot
+            // from its FROB request until its warps have read the Gram matrix (counted in shared memory), from ITER1 to the issue of
+            // ITER2 and from OUT_S to the issue of OUT_O (products run in issue order, so the next owner's score
+            // product follows the last read of P).
             if (lane == 0) {
                 const uint32_t base14 = (sbase >> 4) & 0x3FFF;
-                uint32_t n_rdy = 0;
-                auto batch = [&](int op, int k) {
-                    wait_bar(bars + 8 * B_RDY, n_rdy & 1u, abort_addr);
-                    ++n_rdy;
-                    // the first batch also needs the H_0 tile, the last one the U_0 tile (TMA)
-                    if (op == 0) wait_bar(bars + 8 * B_LD_H, (uint32_t)(k & 1), abort_addr);
-                    if (op == 4) {
-                        wait_bar(bars + 8 * B_LD_U, (uint32_t)(k & 1), abort_addr);
-                        wait_bar(bars + 8 * B_LD_V, (uint32_t)(k & 1), abort_addr);
-                    }
+                // Per-slot state in scalars (arrays indexed by the slot would live in local memory).  Every instruction
+                // of this thread competes with the compute warps of its scheduler, so the paths between a request and
+                // its products are kept as short as possible.
+                int op0 = OP_FROB, op1 = OP_FROB, it0 = 0, it1 = 0, left0 = (n_mine + 1) >> 1, left1 = n_mine >> 1;
+                uint32_t thr0 = 4u, thr1 = 4u;          // request counter values at which the next request of a slot is complete
+                uint32_t gthr0 = 4u, gthr1 = 4u;        // the same for the Gram-read counters
+                uint32_t til0 = 0, til1 = 0;            // tiles done (phase of the per-tile TMA barriers)
+                const uint32_t req_addr = smem_u32(&s_req[0]);
+                int owner = -1;                         // slot that holds S while its warps read the Gram matrix
+                int prefer = 0;                         // slot to serve first when both are ready
+                bool gave_up = false;
+                auto issue = [&](int sl, int o) {
+                    const uint32_t sbb = bars + 8 * (sl * B_PER_SLOT);
+                    const uint32_t sl14 = base14 + ((sl * SLOT_BYTES) >> 4);
                     fence_after();
-                    issue_batch(op, base14, tmem, bars);
+                    issue_batch(o, sl14 + (BUF_A >> 4), sl14 + (BUF_B >> 4), sl14 + (BUF_C >> 4), tmem + TM_S, tmem + tm_r_of(sl),
+                                tmem + tm_e_of(sl), sbb + 8 * B_MMA_S, sbb + 8 * B_MMA_R);
                 };
-                for (int k = 0; k < n_mine; ++k) {
-                    batch(0, k);
-                    for (int it = 0; it < a.n_iter; ++it) {
-                        batch(1, k);
-                        batch(2, k);
+                while ((left0 > 0 || left1 > 0) && !gave_up) {
+                    // ---- a slot whose next request (FROB, ITER1 or OUT_S: all need the score tile) is posted and may have S
+                    int s = -1;
+                    for (int polls = 0;;) {
+                        uint32_t c0, c1, g0, g1;
+                        asm volatile("ld.volatile.shared::cta.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(c0), "=r"(c1), "=r"(g0), "=r"(g1)
+                                     : "r"(req_addr)
+                                     : "memory");
+                        if (owner == 0 && (int)(g0 - gthr0) >= 0) { gthr0 += 4u; owner = -1; }
+                        if (owner == 1 && (int)(g1 - gthr1) >= 0) { gthr1 += 4u; owner = -1; }
+                        const bool r0 = left0 > 0 && owner != 1 && (int)(c0 - thr0) >= 0;
+                        const bool r1 = left1 > 0 && owner != 0 && (int)(c1 - thr1) >= 0;
+                        if (r0 | r1) {
+                            s = (r0 && !(r1 && prefer == 1)) ? 0 : 1;
+                            break;
+                        }
+                        if ((++polls & 1023) == 0 && (aborted(abort_addr) || polls > (1 << 24))) {
+                            gave_up = true;
+                            break;
+                        }
                     }
-                    if (!solve_only) {
-                        batch(3, k);
-                        batch(4, k);
+                    if (gave_up) break;
+                    prefer = 1 - s;
+                    const int o = s ? op1 : op0;
+                    const uint32_t sb = bars + 8 * (s * B_PER_SLOT);
+                    // a request of the slot that still holds S for its Gram reads implies that those are done
+                    if (owner == s) {
+                        if (s) gthr1 += 4u; else gthr0 += 4u;
+                        owner = -1;
                     }
+                    if (o == OP_FROB) wait_bar(sb + 8 * B_LD_H, (s ? til1 : til0) & 1u, abort_addr);   // the H_0 tile (TMA)
+                    issue(s, o);
+                    if (s) thr1 += 4u; else thr0 += 4u;
+                    bool tile_done = false;
+                    int it = s ? it1 : it0, nop;
+                    if (o == OP_FROB) {
+                        owner = s;                           // until the Gram matrix has been read
+                        nop = it < a.n_iter ? OP_ITER1 : OP_OUT_S;
+                        if (a.n_iter == 0 && solve_only) tile_done = true;
+                    } else {
+                        // ---- ITER1 or OUT_S: the slot's next request (ITER2, OUT_O) is the only one that can be served now
+                        const uint32_t thr = s ? thr1 : thr0;
+                        const uint32_t my_addr = req_addr + 4u * (uint32_t)s;
+                        for (int polls = 0;;) {
+                            uint32_t c;
+                            asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(c) : "r"(my_addr) : "memory");
+                            if ((int)(c - thr) >= 0) break;
+                            if ((++polls & 1023) == 0 && (aborted(abort_addr) || polls > (1 << 24))) {
+                                gave_up = true;
+                                break;
+                            }
+                        }
+                        if (gave_up) break;
+                        if (o == OP_OUT_S) {                 // the U_0 and V tiles (TMA)
+                            wait_bar(sb + 8 * B_LD_U, (s ? til1 : til0) & 1u, abort_addr);
+                            wait_bar(sb + 8 * B_LD_V, (s ? til1 : til0) & 1u, abort_addr);
+                        }
+                        issue(s, o == OP_ITER1 ? OP_ITER2 : OP_OUT_O);
+                        if (s) thr1 += 4u; else thr0 += 4u;
+                        if (o == OP_ITER1) {
+                            ++it;
+                            nop = it < a.n_iter ? OP_ITER1 : OP_OUT_S;
+                            if (it >= a.n_iter && solve_only) tile_done = true;
+                        } else {
+                            nop = OP_FROB;
+                            tile_done = true;
+                        }
+                    }
+                    if (tile_done) {
+                        nop = OP_FROB;
+                        it = 0;
+                    }
+                    if (s) { op1 = nop; it1 = it; if (tile_done) { --left1; ++til1; } }
+                    else { op0 = nop; it0 = it; if (tile_done) { --left0; ++til0; } }
                 }
+                if (gave_up) set_abort(abort_addr);
                 // every product is complete before the block gives its tensor memory back
                 mma_commit(bars + 8 * B_DRAIN);
                 if (!mbar_spin_bounded(bars + 8 * B_DRAIN, 0u)) set_abort(abort_addr);
@@ -448,163 +624,191 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     } else {
         // ================================= compute threads =================================
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsCompute));
+        const int slot = (tid >> 7) - 1;
         Ctx cx;
-        cx.tid = tid;
         cx.l = tid & 31;
         cx.q = (tid >> 5) & 3;
-        cx.hf = tid >> 7;
         cx.c = 32 * cx.q + cx.l;
-        cx.lane_addr = (uint32_t)(32 * cx.q) << 16;
-        cx.smem = smem;
-        cx.sbase = sbase;
-        cx.bars = bars;
-        cx.tmem = tmem;
-        cx.abort_addr = abort_addr;
-        const int c = cx.c, hf = cx.hf, l = cx.l;
+        const uint32_t lane_addr = (uint32_t)(32 * cx.q) << 16;
+        cx.tm_s = tmem + TM_S + lane_addr;
+        cx.tm_r = tmem + tm_r_of(slot) + lane_addr;
+        cx.tm_e = tmem + tm_e_of(slot) + lane_addr;
+        const int c = cx.c, l = cx.l;
+        const bool leader = c == 0;                              // issues the slot's loads that follow a product
         const bool adaptive = (a.flags & GKA_FLAG_ADAPTIVE_LAMBDA) != 0;
-        const uint32_t tm_s = tmem + TM_S, tm_r = tmem + TM_R;
-        unsigned char *const bufk = smem + BUF_K, *const bufh = smem + BUF_H, *const bufd = smem + BUF_D;
+        const uint32_t sb = bars + 8 * (slot * B_PER_SLOT);
+        const uint32_t sl = sbase + slot * SLOT_BYTES;
+        unsigned char *const bufa = smem + slot * SLOT_BYTES + BUF_A, *const bufc = smem + slot * SLOT_BYTES + BUF_C;
+        SlotScalars *const sc = reinterpret_cast<SlotScalars *>(smem + OFF_SC + slot * SC_BYTES);
         // the per-tile states and norms come from the state kernel
         asm volatile("griddepcontrol.wait;" ::: "memory");
 
-        uint64_t xs[32];                    // -zt_c x_c, this thread's 64 channels as fp32 pairs
-        uint32_t n_s = 0, n_r = 0, n_q = 0;   // completed phases of MMA_S, MMA_R, LD_Q
-        auto wait_s = [&]() { wait_bar(bars + 8 * B_MMA_S, n_s & 1u, abort_addr); ++n_s; fence_after(); };
-        auto wait_r = [&]() { wait_bar(bars + 8 * B_MMA_R, n_r & 1u, abort_addr); ++n_r; fence_after(); };
-        auto arrive_rdy = [&]() { warp_arrive(bars + 8 * B_RDY, l); };
-        // stage -xs (times `scale`) as bf16: its leading part, or the remainder after the leading part
-        auto stage_x = [&](unsigned char *dst, bool lo, float scale) {
+        uint64_t xs[64];                      // -zt_c x_c: the token's 128 channels as fp32 pairs
+        uint32_t n_s = 0, n_r = 0;            // completed phases of MMA_S, MMA_R
+        auto wait_s = [&]() { wait_bar(sb + 8 * B_MMA_S, n_s & 1u, abort_addr); ++n_s; fence_after(); };
+        // the same waits without suspending, for the iterations (a suspended wait wakes up late, and a poll of an
+        // mbarrier takes about 100 cycles, so a polling warp leaves nearly all issue slots to the working warps)
+        auto wait_s_spin = [&]() {      // one lane polls (32 lanes on one mbarrier would crowd the shared-memory pipe)
+            if (l == 0 && !aborted(abort_addr) && !mbar_spin_bounded(sb + 8 * B_MMA_S, n_s & 1u)) set_abort(abort_addr);
+            __syncwarp();
+            ++n_s;
+            fence_after();
+        };
+        auto wait_r_spin = [&]() {
+            if (!aborted(abort_addr) && !mbar_spin_bounded(sb + 8 * B_MMA_R, n_r & 1u)) set_abort(abort_addr);
+            ++n_r;
+            fence_after();
+        };
+        auto wait_r = [&]() { wait_bar(sb + 8 * B_MMA_R, n_r & 1u, abort_addr); ++n_r; fence_after(); };
+        const uint32_t req_addr = smem_u32(&s_req[slot]), grd_addr = smem_u32(&s_req[2 + slot]);
+        auto arrive_rdy = [&]() { warp_post(req_addr, l); };
+        // -xs (times `scale`) as packed bf16 pairs of channel group g8 (8 channels): its leading part, or the remainder
+        auto pack_x = [&](int g8, bool lo, float scale, uint32_t(&pk)[4]) {
 #pragma unroll
-            for (int g8 = 0; g8 < 8; ++g8) {
-                uint32_t pk[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    float xa, xb;
-                    f2_unpack(xs[4 * g8 + u], xa, xb);
-                    xa *= -scale;
-                    xb *= -scale;
-                    uint32_t p = pack_bf16(xa, xb);
-                    if (lo) p = pack_bf16(xa - bf16_lo(p), xb - bf16_hi(p));
-                    pk[u] = p;
-                }
-                *reinterpret_cast<uint4 *>(dst + tile_off(c, 8 * hf + g8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            for (int u = 0; u < 4; ++u) {
+                float xa, xb;
+                f2_unpack(xs[4 * g8 + u], xa, xb);
+                xa *= -scale;
+                xb *= -scale;
+                uint32_t p = pack_bf16(xa, xb);
+                if (lo) p = pack_bf16(xa - bf16_lo(p), xb - bf16_hi(p));
+                pk[u] = p;
             }
         };
 
-        for (int k = 0; k < n_mine; ++k) {
+        for (int k = slot, j = 0; k < n_mine; k += kSlots, ++j) {
             const long long tile = t_lo + k;
-            const GateScalars *const gs = &sc->g[k & 1];
+            const bool more = k + kSlots < n_mine;
+            const GateScalars *const gs = &sc->g[j & 1];
             const TileInfo ti = tile_info(a, tile);
             const bool valid = c < ti.ntok;
+            // loads of the slot's next tile, issued by the leader as soon as the buffer's last reader is done
+            auto load_next_k = [&]() {
+                if (leader && more) {
+                    const TileInfo tn = tile_info(a, tile + kSlots);
+                    mbar_expect_tx(sb + 8 * B_LD_K, 32768u);
+                    tma_load_tile3(&tmK, sl + BUF_A, sb + 8 * B_LD_K, tn.h * D, tn.n * NT, tn.b);
+                }
+            };
+            auto load_next_h = [&]() {
+                if (leader && more) {
+                    mbar_expect_tx(sb + 8 * B_LD_H, 32768u);
+                    tma_load_tile2(&tmS, sl + BUF_B, sb + 8 * B_LD_H, (int)((tile + kSlots) * 256));
+                }
+            };
+            auto after_last_h0_product = [&]() {      // H_0 has been read for the last time
+                if (solve_only) {
+                    load_next_k();
+                    load_next_h();
+                } else if (leader) {
+                    mbar_expect_tx(sb + 8 * B_LD_U, 32768u);
+                    tma_load_tile2(&tmS, sl + BUF_B, sb + 8 * B_LD_U, (int)(tile * 256 + 128));
+                }
+            };
             // ||H_0||_F^2 of the tile (state kernel): fetched now, used by the scan
-            const float hh = tid < NT ? ldg_stream_f32(a.tile_hh + tile) : 0.f;
-            // ---- gate scalars (helper warp) and the K, H_0 tiles (TMA) of this tile
-            wait_bar(bars + 8 * (B_GS0 + (k & 1)), (uint32_t)((k >> 1) & 1), abort_addr);
-            wait_bar(bars + 8 * B_LD_K, (uint32_t)(k & 1), abort_addr);
+            const float hh = ldg_stream_f32(a.tile_hh + tile);
+            // ---- gate scalars (helper warp) and the K tile (TMA) of this tile
+            wait_bar(sb + 8 * (B_GS0 + (j & 1)), (uint32_t)((j >> 1) & 1), abort_addr);
+            wait_bar(sb + 8 * B_LD_K, (uint32_t)(j & 1), abort_addr);
             const bool exact = gs->G2[ti.ntok - 1] < -60.f;     // the tile decays below 2^-60: per-element factors
-            scale_rows(bufk, gs->ks, tid);
+            const float G2c = gs->G2[c], ac_c = gs->ac[c];
+            {
+                // Khat: the token's key row scaled in place
+                const float fj = gs->ks[c];
+                const uint64_t f2 = f2_pack(fj, fj);
+#pragma unroll 1
+                for (int g = 0; g < 16; ++g) {                   // (rolled: code that runs once per tile is kept small)
+                    uint4 v = *reinterpret_cast<const uint4 *>(bufa + tile_off(c, g));
+                    uint32_t *pv = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        float lo, hi;
+                        f2_unpack(f2_mul(f2_pack(bf16_lo(pv[u]), bf16_hi(pv[u])), f2), lo, hi);
+                        pv[u] = pack_bf16(lo, hi);
+                    }
+                    *reinterpret_cast<uint4 *>(bufa + tile_off(c, g)) = v;
+                }
+            }
             fence_async_smem();
             arrive_rdy();                                        // -> FROB
             wait_s();
-            // ---- chunk-wise Frobenius norms: per key, k_j^T H_0 k_j and the decayed squared Gram entries of the
-            // earlier keys.  Thread = (key j = c, 64 columns).
+            if (a.n_iter == 0) after_last_h0_product();
+            // ---- chunk-wise Frobenius norms: for the token's key, k^T H_0 k and the decayed squared Gram entries of
+            // the earlier keys
+            float kh = 0.f, gsum = 0.f;
             {
-                float kh = 0.f, gsum = 0.f;
-#pragma unroll
-                for (int piece = 0; piece < 2; ++piece) {
-                    uint32_t r[32];
-                    TMEM_LD32(tm_r + cx.lane_addr + 64 * hf + 32 * piece, r);
+                uint32_t ra[32];
+#pragma unroll 1
+                for (int p = 0; p < 4; ++p) {
+                    TMEM_LD32(cx.tm_r + 32 * p, ra);
                     uint4 kv[4];
 #pragma unroll
-                    for (int h4 = 0; h4 < 4; ++h4) kv[h4] = *reinterpret_cast<const uint4 *>(bufk + tile_off(c, 8 * hf + 4 * piece + h4));
+                    for (int h4 = 0; h4 < 4; ++h4) kv[h4] = *reinterpret_cast<const uint4 *>(bufa + tile_off(c, 4 * p + h4));
                     tmem_wait_ld();
 #pragma unroll
                     for (int h4 = 0; h4 < 4; ++h4) {
                         const uint32_t *pk = reinterpret_cast<const uint32_t *>(&kv[h4]);
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
-                            kh = fmaf(__uint_as_float(r[8 * h4 + 2 * u]), bf16_lo(pk[u]), kh);
-                            kh = fmaf(__uint_as_float(r[8 * h4 + 2 * u + 1]), bf16_hi(pk[u]), kh);
+                            kh = fmaf(__uint_as_float(ra[8 * h4 + 2 * u]), bf16_lo(pk[u]), kh);
+                            kh = fmaf(__uint_as_float(ra[8 * h4 + 2 * u + 1]), bf16_hi(pk[u]), kh);
                         }
                     }
                 }
-                const float G2j = gs->G2[c];
-#pragma unroll
-                for (int b2 = 0; b2 < 2; ++b2) {
-                    const int kb = 2 * hf + b2;
-                    if (kb > cx.q) continue;
-                    const int lim = (kb == cx.q) ? l : 32;   // keys i < lim come earlier, i == lim is the key itself
-                    float gs2 = 0.f, gd = 0.f;
-                    uint32_t r[32];
-                    TMEM_LD32(tm_s + cx.lane_addr + 32 * kb, r);
+#pragma unroll 1
+                for (int kb = 0; kb <= cx.q; ++kb) {
+                    TMEM_LD32(cx.tm_s + 32 * kb, ra);
                     tmem_wait_ld();
-#pragma unroll
-                    for (int ii = 0; ii < 32; ++ii) {
-                        const float g = __uint_as_float(r[ii]);
-                        const float g2 = g * g;
-                        if (ii == lim) gd = g2;
-                        if (!exact) gs2 += (ii < lim) ? g2 : 0.f;
-                        else if (ii < lim) gs2 = fmaf(ex2_fast(G2j - gs->G2[32 * kb + ii]), g2, gs2);
-                    }
-                    gsum += 2.f * gs2 + gd;
+                    if (kb == cx.q) gram_block<true>(ra, gs->G2 + 32 * kb, G2c, exact, l, gsum);
+                    else gram_block<false>(ra, gs->G2 + 32 * kb, G2c, exact, l, gsum);
                 }
-                sc->part[0][hf][c] = kh;
-                sc->part[1][hf][c] = gsum;
             }
             fence_before();
-            if (tid == 0) sc->stop = aborted(abort_addr) ? 1 : 0;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
+            warp_post(grd_addr, l);                              // the Gram matrix has been read: S is free again
             // ---- f_c by an affine scan (s_c = gamma_c^2 s_{c-1} + d_c, s_{-1} = ||H_0||^2), Chebyshev set-up
-            if (tid < NT) {
-                const float kh = sc->part[0][0][c] + sc->part[0][1][c];
-                const float gsum = sc->part[1][0][c] + sc->part[1][1][c];
-                const float G2c = gs->G2[c];
+            float rho2, czb, lz;
+            {
                 // pre-scaled keys: both sums carry 2^(-2 G_c); plain keys: k H_0 k carries zeta_c
                 const float dc = exact ? fmaf(2.f * ex2_fast(G2c), kh, gsum) : ex2_fast(2.f * G2c) * fmaf(2.f, kh, gsum);
-                const float s = affine_scan(cx, sc, ex2_fast(2.f * gs->lg[c]), dc, hh);
+                const float s = affine_scan(cx, sc, slot, ex2_fast(2.f * gs->lg[c]), dc, hh);
                 const float fc = sqrtf(fmaxf(s, 0.f));
                 float lamc = gs->lam[c];
                 if (adaptive) lamc *= fc;
                 const float Lpm = fc + 2.f * lamc;
                 const float iL = 1.f / Lpm;
                 const float rho = fc * iL;
-                sc->rho2[c] = rho * rho;
-                sc->czb[c] = valid ? -gs->zt[c] * (2.f * iL) : 0.f;
-                sc->lz[c] = lamc * gs->iz[c];
+                rho2 = rho * rho;
+                czb = valid ? -gs->zt[c] * (2.f * iL) : 0.f;
+                lz = lamc * gs->iz[c];
                 if (a.fro_out && valid) a.fro_out[ti.tok0 + (size_t)c * a.heads] = fc;
             }
-            wait_bar(bars + 8 * B_LD_Q, n_q & 1u, abort_addr);   // q tile has landed
-            ++n_q;
-            asm volatile("bar.sync 1, 256;" ::: "memory");       // the set-up values are published
-            if (sc->stop) break;                                 // the same decision in every thread
-            const float rho2 = sc->rho2[c], czb = sc->czb[c], lz = sc->lz[c];
-            // ---- x_0: R = q, E_0 = czb q (in place of q), xs = E_0
+            wait_bar(sb + 8 * B_LD_Q, (uint32_t)(j & 1), abort_addr);   // q tile has landed
+            // ---- x_0: R = q, E_0 = czb q, xs = E_0
 #pragma unroll
-            for (int g16 = 0; g16 < 4; ++g16) {
-                uint32_t rr[16];
+            for (int g16 = 0; g16 < 8; ++g16) {
+                uint32_t rr[16], pk[8];
 #pragma unroll
                 for (int h2 = 0; h2 < 2; ++h2) {
-                    const int g8 = 2 * g16 + h2;
-                    const uint4 qv = *reinterpret_cast<const uint4 *>(bufd + tile_off(c, 8 * hf + g8));
+                    const uint4 qv = *reinterpret_cast<const uint4 *>(bufc + tile_off(c, 2 * g16 + h2));
                     const uint32_t *qq = reinterpret_cast<const uint32_t *>(&qv);
-                    uint32_t pk[4];
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const float qa = bf16_lo(qq[u]), qb = bf16_hi(qq[u]);
                         rr[8 * h2 + 2 * u] = __float_as_uint(qa);
                         rr[8 * h2 + 2 * u + 1] = __float_as_uint(qb);
-                        pk[u] = pack_bf16(czb * qa, czb * qb);
-                        xs[4 * g8 + u] = f2_pack(bf16_lo(pk[u]), bf16_hi(pk[u]));
+                        const uint32_t p = pack_bf16(czb * qa, czb * qb);
+                        pk[4 * h2 + u] = p;
+                        xs[8 * g16 + 4 * h2 + u] = f2_pack(bf16_lo(p), bf16_hi(p));
                     }
-                    *reinterpret_cast<uint4 *>(bufd + tile_off(c, 8 * hf + g8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
-                TMEM_ST16(tm_r + cx.lane_addr + 64 * hf + 16 * g16, rr);
+                TMEM_ST16(cx.tm_r + 16 * g16, rr);
+                TMEM_ST8(cx.tm_e + 8 * g16, pk);
             }
+            if (!solve_only && !mix) warp_arrive(sb + 8 * B_QF, l);      // q has been read: V may take its buffer
             tmem_wait_st();
             // ---- Algorithm 1
             float omega = 2.f;
             if (a.n_iter > 0) {
-                fence_async_smem();
                 fence_before();
                 arrive_rdy();                                    // -> ITER1
             }
@@ -612,76 +816,72 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 const bool last = it + 1 == a.n_iter;
                 omega = 4.f / (4.f - rho2 * omega);              // weight schedule
                 const float beta = omega - 1.f, cz = czb * omega;
-                wait_s();
-                p_epilogue<false>(cx, tm_s, gs, exact, gs->ac[c]);
+                wait_s_spin();
+                p_epilogue<false>(cx, gs, exact, ac_c);
                 fence_before();
                 arrive_rdy();                                    // -> ITER2
                 const uint64_t beta2 = f2_pack(beta, beta), cz2 = f2_pack(cz, cz), lz2 = f2_pack(lz, lz);
                 wait_r();
-                // e_new = beta e_old + cz (R + lz xs); xs += e_new (as rounded for the operand, unless last).  Eight
+                if (last) after_last_h0_product();
+                // e_new = beta e_old + cz (R + lz xs) as bf16, xs += e_new (the value the operand holds).  Sixteen
                 // channels at a time; the next group's loads are in flight while a group is computed.
                 {
-                    uint32_t ra[8], rb[8];
-                    uint4 eva, evb;
-                    TMEM_LD8(tm_r + cx.lane_addr + 64 * hf, ra);
-                    eva = *reinterpret_cast<const uint4 *>(bufd + tile_off(c, 8 * hf));
+                    uint32_t ra[16], rb[16], ea[8], eb[8];
+                    TMEM_LD16(cx.tm_r, ra);
+                    TMEM_LD8(cx.tm_e, ea);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int g8 = 0; g8 < 8; ++g8) {
-                        uint32_t(&r)[8] = (g8 & 1) ? rb : ra;
-                        uint32_t(&rn)[8] = (g8 & 1) ? ra : rb;
-                        uint4 &ev = (g8 & 1) ? evb : eva;
-                        uint4 &evn = (g8 & 1) ? eva : evb;
-                        if (g8 < 7) {
-                            TMEM_LD8(tm_r + cx.lane_addr + 64 * hf + 8 * (g8 + 1), rn);
-                            evn = *reinterpret_cast<const uint4 *>(bufd + tile_off(c, 8 * hf + g8 + 1));
+                    for (int g = 0; g < 8; ++g) {
+                        uint32_t(&r)[16] = (g & 1) ? rb : ra;
+                        uint32_t(&rn)[16] = (g & 1) ? ra : rb;
+                        uint32_t(&e)[8] = (g & 1) ? eb : ea;
+                        uint32_t(&en_)[8] = (g & 1) ? ea : eb;
+                        if (g < 7) {
+                            TMEM_LD16(cx.tm_r + 16 * (g + 1), rn);
+                            TMEM_LD8(cx.tm_e + 8 * (g + 1), en_);
                         }
-                        const uint32_t *ee = reinterpret_cast<const uint32_t *>(&ev);
-                        uint32_t pk[4];
+                        uint32_t pk[8];
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int i = 4 * g8 + u;
+                        for (int u = 0; u < 8; ++u) {
+                            const int i = 8 * g + u;
                             const uint64_t res = f2_fma(lz2, xs[i], f2_pack(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1])));
-                            const uint64_t en = f2_fma(cz2, res, f2_mul(beta2, f2_pack(bf16_lo(ee[u]), bf16_hi(ee[u]))));
-                            float ea, eb;
-                            f2_unpack(en, ea, eb);
-                            pk[u] = pack_bf16(ea, eb);
-                            xs[i] = f2_add(xs[i], last ? en : f2_pack(bf16_lo(pk[u]), bf16_hi(pk[u])));
+                            const uint64_t en = f2_fma(cz2, res, f2_mul(beta2, f2_pack(bf16_lo(e[u]), bf16_hi(e[u]))));
+                            float ea_, eb_;
+                            f2_unpack(en, ea_, eb_);
+                            pk[u] = pack_bf16(ea_, eb_);
+                            xs[i] = f2_add(xs[i], f2_pack(bf16_lo(pk[u]), bf16_hi(pk[u])));
                         }
-                        if (!last) {
-                            *reinterpret_cast<uint4 *>(bufd + tile_off(c, 8 * hf + g8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                            if (g8 == 7) {
-                                fence_async_smem();
-                                fence_before();     // the accumulator R has been read completely
-                                arrive_rdy();       // -> ITER1
-                            }
-                        }
-                        if (g8 < 7) tmem_wait_ld();
+                        TMEM_ST8(cx.tm_e + 8 * g, pk);
+                                        if (g < 7) tmem_wait_ld();
+                    }
+                    if (!last) {
+                        tmem_wait_st();
+                        fence_before();
+                        arrive_rdy();                            // -> ITER1
                     }
                 }
             }
             // ---- final iterate
             if (solve_only) {
-                // the solve is the result: x_c = -xs / zt_c as bf16, stored by TMA
-                stage_x(bufd, false, gs->iz[c]);
+                // the solve is the result: x_c = -xs / zt_c as bf16, staged in the q buffer and stored by TMA
+                const float izc = gs->iz[c];
+#pragma unroll
+                for (int g8 = 0; g8 < 16; ++g8) {
+                    uint32_t pk[4];
+                    pack_x(g8, false, izc, pk);
+                    *reinterpret_cast<uint4 *>(bufc + tile_off(c, g8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
                 fence_async_smem();
-                warp_arrive(bars + 8 * (B_GF0 + (k & 1)), l);
-                warp_arrive(bars + 8 * B_RDY_ST, l);
+                warp_arrive(sb + 8 * (B_GF0 + (j & 1)), l);
+                warp_arrive(sb + 8 * B_RDY_ST, l);
                 continue;
             }
             if (mix) {
-                // alpha-connection (Section 4.3): the read uses alpha x + (1 - alpha) q; q comes back into the H_0
-                // buffer, which no product reads any more
-                if (tid == 0) {
-                    mbar_expect_tx(bars + 8 * B_LD_Q, 32768u);
-                    tma_load_tile3(&tmQ, sbase + BUF_H, bars + 8 * B_LD_Q, ti.h * D, ti.n * NT, ti.b);
-                }
-                wait_bar(bars + 8 * B_LD_Q, n_q & 1u, abort_addr);
-                ++n_q;
+                // alpha-connection (Section 4.3): the read uses alpha x + (1 - alpha) q; q is still in its buffer
                 const float alc = gs->al[c], nzt = valid ? -gs->zt[c] : 0.f;
 #pragma unroll
-                for (int g8 = 0; g8 < 8; ++g8) {
-                    const uint4 qv = *reinterpret_cast<const uint4 *>(bufh + tile_off(c, 8 * hf + g8));
+                for (int g8 = 0; g8 < 16; ++g8) {
+                    const uint4 qv = *reinterpret_cast<const uint4 *>(bufc + tile_off(c, g8));
                     const uint32_t *qq = reinterpret_cast<const uint32_t *>(&qv);
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
@@ -691,54 +891,53 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         xs[4 * g8 + u] = f2_pack(fmaf(alc, xa - qa, qa), fmaf(alc, xb - qb, qb));
                     }
                 }
-                asm volatile("bar.sync 1, 256;" ::: "memory");   // every thread has read q: U_0 may overwrite it
+                warp_arrive(sb + 8 * B_QF, l);                   // q has been read: V may take its buffer
             }
             // The read uses the final iterate as two bf16 terms in the score product (the recent keys resolve directions
-            // of x that one bf16 rounding would lose); the second term takes the H_0 buffer, which no product reads
-            // any more.
-            stage_x(bufd, false, 1.f);
-            stage_x(bufh, true, 1.f);
-            fence_async_smem();
+            // of x that one bf16 rounding would lose): the leading term takes the operand columns, the remainder the
+            // first columns of the accumulator, whose content is no longer needed.
+#pragma unroll
+            for (int g8 = 0; g8 < 16; g8 += 2) {
+                uint32_t hi[8], lo[8];
+                pack_x(g8, false, 1.f, *reinterpret_cast<uint32_t(*)[4]>(&hi[0]));
+                pack_x(g8 + 1, false, 1.f, *reinterpret_cast<uint32_t(*)[4]>(&hi[4]));
+                pack_x(g8, true, 1.f, *reinterpret_cast<uint32_t(*)[4]>(&lo[0]));
+                pack_x(g8 + 1, true, 1.f, *reinterpret_cast<uint32_t(*)[4]>(&lo[4]));
+                TMEM_ST8(cx.tm_e + 4 * g8, hi);
+                TMEM_ST8(cx.tm_r + 4 * g8, lo);
+            }
+            tmem_wait_st();
             fence_before();
             arrive_rdy();                                        // -> OUT_S
             wait_s();
-            if (tid == 0) {               // the keys and the second term are no longer needed: V and U_0 take their buffers
-                mbar_expect_tx(bars + 8 * B_LD_V, 32768u);
-                tma_load_tile3(&tmV, sbase + BUF_K, bars + 8 * B_LD_V, ti.h * D, ti.n * NT, ti.b);
-                mbar_expect_tx(bars + 8 * B_LD_U, 32768u);
-                tma_load_tile2(&tmS, sbase + BUF_H, bars + 8 * B_LD_U, (int)(tile * 256 + 128));
-            }
+            load_next_k();                                       // the keys have been read for the last time
             // the values stay as loaded: their row factor sqrt(beta_j) 2^(-G_j / 2) rides on the masked scores
-            p_epilogue<true>(cx, tm_s, gs, exact, gs->ac[c]);
+            p_epilogue<true>(cx, gs, exact, ac_c);
             fence_before();
             arrive_rdy();                                        // -> OUT_O
             wait_r();
-            // every product of the tile is complete: the next tile's K and q can come in (H_0 follows the store)
-            if (tid == 0 && k + 1 < n_mine) {
-                const TileInfo tn = tile_info(a, tile + 1);
-                mbar_expect_tx(bars + 8 * B_LD_K, 32768u);
-                tma_load_tile3(&tmK, sbase + BUF_K, bars + 8 * B_LD_K, tn.h * D, tn.n * NT, tn.b);
-                mbar_expect_tx(bars + 8 * B_LD_Q, 32768u);
-                tma_load_tile3(&tmQ, sbase + BUF_D, bars + 8 * B_LD_Q, tn.h * D, tn.n * NT, tn.b);
-            }
-            // O as bf16 into the U_0 buffer (no product reads it any more), stored by TMA
+            load_next_h();                                       // every product of the tile is complete
+            // O as bf16 into the V buffer (no product reads it any more), stored by TMA
+            {
+                uint32_t r[32];
+#pragma unroll 1
+                for (int p = 0; p < 4; ++p) {
+                    TMEM_LD32(cx.tm_r + 32 * p, r);
+                    tmem_wait_ld();
 #pragma unroll
-            for (int piece = 0; piece < 4; ++piece) {
-                uint32_t r[16];
-                TMEM_LD16(tm_r + cx.lane_addr + 64 * hf + 16 * piece, r);
-                tmem_wait_ld();
-                uint32_t pk[8];
+                    for (int h4 = 0; h4 < 4; ++h4) {
+                        uint32_t pk[4];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) pk[u] = pack_bf16(__uint_as_float(r[2 * u]), __uint_as_float(r[2 * u + 1]));
-                *reinterpret_cast<uint4 *>(bufh + tile_off(c, 8 * hf + 2 * piece)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                *reinterpret_cast<uint4 *>(bufh + tile_off(c, 8 * hf + 2 * piece + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                        for (int u = 0; u < 4; ++u) pk[u] = pack_bf16(__uint_as_float(r[8 * h4 + 2 * u]), __uint_as_float(r[8 * h4 + 2 * u + 1]));
+                        *reinterpret_cast<uint4 *>(bufc + tile_off(c, 4 * p + h4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                }
             }
             fence_async_smem();
             fence_before();
-            warp_arrive(bars + 8 * (B_GF0 + (k & 1)), l);
-            warp_arrive(bars + 8 * B_RDY_ST, l);
+            warp_arrive(sb + 8 * (B_GF0 + (j & 1)), l);
+            warp_arrive(sb + 8 * B_RDY_ST, l);
         }
-        if (aborted(abort_addr)) set_abort(abort_addr);
     }
 
     fence_before();
@@ -748,7 +947,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
         if (tid == 0 && a.device_status) atomicExch(a.device_status, (int)GKA_ERR_TIMEOUT);
     }
-    if (tid < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem) : "memory");
+    if (tid < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
 }
 
 }  // namespace
@@ -768,10 +967,10 @@ cudaError_t launch_fwd_solve(const FwdArgs &a, cudaStream_t stream) {
     int dev = 0, sms = 0;
     if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
     if ((err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return err;
-    const long long want = (long long)kBlocksPerSM * sms;
+    const long long want = ntiles < sms ? ntiles : (long long)sms;   // one persistent block per SM, two tiles in flight each
     if (a.ev_start) cudaEventRecord(a.ev_start, stream);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(ntiles < want ? ntiles : want));
+    cfg.gridDim = dim3((unsigned)(want < 1 ? 1 : want));
     cfg.blockDim = dim3(kThreadsSolve);
     cfg.dynamicSmemBytes = SOLVE_SMEM;
     cfg.stream = stream;
