@@ -539,10 +539,12 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     issue_batch(o, sl14 + (BUF_A >> 4), sl14 + (BUF_B >> 4), sl14 + (BUF_C >> 4), tmem + TM_S, tmem + tm_r_of(sl),
                                 tmem + tm_e_of(sl), sbb + 8 * B_MMA_S, sbb + 8 * B_MMA_R);
                 };
+                int next_s = -1;                        // slot known to have its request posted (no poll needed)
                 while ((left0 > 0 || left1 > 0) && !gave_up) {
                     // ---- a slot whose next request (FROB, ITER1 or OUT_S: all need the score tile) is posted and may have S
-                    int s = -1;
-                    for (int polls = 0;;) {
+                    int s = next_s;
+                    next_s = -1;
+                    for (int polls = 0; s < 0;) {
                         uint32_t c0, c1, g0, g1;
                         asm volatile("ld.volatile.shared::cta.v4.u32 {%0, %1, %2, %3}, [%4];"
                                      : "=r"(c0), "=r"(c1), "=r"(g0), "=r"(g1)
@@ -572,48 +574,52 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     }
                     if (o == OP_FROB) wait_bar(sb + 8 * B_LD_H, (s ? til1 : til0) & 1u, abort_addr);   // the H_0 tile (TMA)
                     issue(s, o);
-                    if (s) thr1 += 4u; else thr0 += 4u;
+                    // ---- the slot's state after this request and its follow-up (worked out while the products run)
                     bool tile_done = false;
                     int it = s ? it1 : it0, nop;
+                    uint32_t thr = (s ? thr1 : thr0) + 4u;
                     if (o == OP_FROB) {
                         owner = s;                           // until the Gram matrix has been read
                         nop = it < a.n_iter ? OP_ITER1 : OP_OUT_S;
                         if (a.n_iter == 0 && solve_only) tile_done = true;
+                    } else if (o == OP_ITER1) {
+                        ++it;
+                        nop = it < a.n_iter ? OP_ITER1 : OP_OUT_S;
+                        if (it >= a.n_iter && solve_only) tile_done = true;
                     } else {
-                        // ---- ITER1 or OUT_S: the slot's next request (ITER2, OUT_O) is the only one that can be served now
-                        const uint32_t thr = s ? thr1 : thr0;
-                        const uint32_t my_addr = req_addr + 4u * (uint32_t)s;
-                        for (int polls = 0;;) {
-                            uint32_t c;
-                            asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(c) : "r"(my_addr) : "memory");
-                            if ((int)(c - thr) >= 0) break;
-                            if ((++polls & 1023) == 0 && (aborted(abort_addr) || polls > (1 << 24))) {
-                                gave_up = true;
-                                break;
-                            }
-                        }
-                        if (gave_up) break;
-                        if (o == OP_OUT_S) {                 // the U_0 and V tiles (TMA)
-                            wait_bar(sb + 8 * B_LD_U, (s ? til1 : til0) & 1u, abort_addr);
-                            wait_bar(sb + 8 * B_LD_V, (s ? til1 : til0) & 1u, abort_addr);
-                        }
-                        issue(s, o == OP_ITER1 ? OP_ITER2 : OP_OUT_O);
-                        if (s) thr1 += 4u; else thr0 += 4u;
-                        if (o == OP_ITER1) {
-                            ++it;
-                            nop = it < a.n_iter ? OP_ITER1 : OP_OUT_S;
-                            if (it >= a.n_iter && solve_only) tile_done = true;
-                        } else {
-                            nop = OP_FROB;
-                            tile_done = true;
-                        }
+                        nop = OP_FROB;
+                        tile_done = true;
                     }
                     if (tile_done) {
                         nop = OP_FROB;
                         it = 0;
                     }
-                    if (s) { op1 = nop; it1 = it; if (tile_done) { --left1; ++til1; } }
-                    else { op0 = nop; it0 = it; if (tile_done) { --left0; ++til0; } }
+                    const uint32_t til = s ? til1 : til0;
+                    const uint32_t thr_other = s ? thr0 : thr1;
+                    const bool other_left = (s ? left0 : left1) > 0;
+                    if (s) { op1 = nop; it1 = it; thr1 = thr + (o == OP_FROB ? 0u : 4u); if (tile_done) { --left1; ++til1; } }
+                    else { op0 = nop; it0 = it; thr0 = thr + (o == OP_FROB ? 0u : 4u); if (tile_done) { --left0; ++til0; } }
+                    if (o == OP_FROB) continue;
+                    // ---- ITER1 or OUT_S: the slot's next request (ITER2, OUT_O) is the only one that can be served now
+                    uint32_t c_other = 0u;
+                    for (int polls = 0;;) {
+                        uint32_t c0, c1;
+                        asm volatile("ld.volatile.shared::cta.v2.u32 {%0, %1}, [%2];" : "=r"(c0), "=r"(c1) : "r"(req_addr) : "memory");
+                        c_other = s ? c0 : c1;
+                        if ((int)((s ? c1 : c0) - thr) >= 0) break;
+                        if ((++polls & 1023) == 0 && (aborted(abort_addr) || polls > (1 << 24))) {
+                            gave_up = true;
+                            break;
+                        }
+                    }
+                    if (gave_up) break;
+                    if (o == OP_OUT_S) {                     // the U_0 and V tiles (TMA)
+                        wait_bar(sb + 8 * B_LD_U, til & 1u, abort_addr);
+                        wait_bar(sb + 8 * B_LD_V, til & 1u, abort_addr);
+                    }
+                    issue(s, o == OP_ITER1 ? OP_ITER2 : OP_OUT_O);
+                    // the other slot's request, if it was already posted, is served next without a poll
+                    if (other_left && (int)(c_other - thr_other) >= 0) next_s = 1 - s;
                 }
                 if (gave_up) set_abort(abort_addr);
                 // every product is complete before the block gives its tensor memory back
