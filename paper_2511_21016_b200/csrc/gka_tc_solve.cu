@@ -49,10 +49,12 @@ constexpr int NT = kTile;                  // tokens per tile: one per TMEM lane
 constexpr int kSlots = 2;
 constexpr int ST = 128;                    // compute threads per slot
 constexpr int CT = kSlots * ST;            // compute threads
-constexpr int kThreadsSolve = CT + 128;    // + helper warpgroup: gate scalars, TMA (one warp per slot), MMA issue
-constexpr int kRegsLaunch = 168, kRegsCompute = 232, kRegsHelper = 40;   // register split after setmaxnreg
+// Warpgroups: 0 = helpers (gate scalars, TMA: one warp per slot, MMA issue), 1 = score warps (the masked-score
+// epilogue of both slots, one warp per TMEM lane quadrant), 2 and 3 = the compute warps of slot 0 and slot 1.
+constexpr int kThreadsSolve = 256 + CT;
+constexpr int kRegsLaunch = 128, kRegsCompute = 200, kRegsScore = 72, kRegsHelper = 40;   // register split after setmaxnreg
 static_assert(kThreadsSolve * kRegsLaunch <= 65536, "launch registers");
-static_assert(CT * kRegsCompute + 128 * kRegsHelper <= kThreadsSolve * kRegsLaunch, "register split exceeds the launch allocation");
+static_assert(CT * kRegsCompute + 128 * kRegsScore + 128 * kRegsHelper <= kThreadsSolve * kRegsLaunch, "register split exceeds the launch allocation");
 
 // ---- shared memory map (bytes; operand buffers 1024-byte aligned): three operand tiles per slot, then the scalars
 constexpr uint32_t BUF_A = 0;                  // keys (Khat)
@@ -74,6 +76,7 @@ struct GateScalars {       // per token of a tile, from the gates and the other 
 struct SlotScalars {
     GateScalars g[2];
     float carry[2][4];     // per-warp totals (a, b) of the affine scan
+    int exact[2];          // the tile of gate buffer 0 / 1 decays below 2^-60 (per-element factors in the score epilogue)
 };
 constexpr uint32_t SC_BYTES = (sizeof(SlotScalars) + 127) / 128 * 128;
 constexpr uint32_t SOLVE_SMEM = OFF_SC + kSlots * SC_BYTES + 1024;   // + slack for the 1024-byte alignment of the base
@@ -93,14 +96,15 @@ enum {                 // per slot
     B_LD_V,            // V tile
     B_RDY_ST,          // compute warps -> TMA thread: the result tile is staged
     B_QF,              // compute warps -> TMA thread: q has been read, V may take its buffer
-    B_MMA_S,           // tcgen05.commit: score-side batch complete
+    B_MMA_S,           // tcgen05.commit: the Frobenius batch (Gram matrix, K H_0) is complete
     B_MMA_R,           // tcgen05.commit: accumulator-side batch complete
     B_GS0, B_GS1,      // gate scalars of buffer 0 / 1 are ready
     B_GF0, B_GF1,      // compute warps -> gate helper: buffer 0 / 1 is free
     B_PER_SLOT
 };
 constexpr int B_DRAIN = kSlots * B_PER_SLOT;   // every product is complete (before the tensor memory is given back)
-constexpr int B_COUNT = B_DRAIN + 1;
+constexpr int B_SC = B_DRAIN + 1;              // tcgen05.commit: a score product of either slot is complete (-> score warps)
+constexpr int B_COUNT = B_SC + 1;
 
 // Requests a slot makes to the issuing thread: every warp of the slot adds one to the slot's request counter in
 // shared memory (a poll of both counters is one 40-cycle load, where a test of an mbarrier phase takes 100 cycles);
@@ -232,7 +236,7 @@ __device__ __forceinline__ void prod_pm(uint32_t d, uint32_t p_tmem, uint32_t b1
 
 // The products of one request.  kb, hb, cb: descriptor bases (shared address >> 4) of the slot's buffers.
 __device__ __forceinline__ void issue_batch(int op, uint32_t kb, uint32_t hb, uint32_t cb, uint32_t tm_S, uint32_t tm_R,
-                                            uint32_t tm_E, uint32_t bar_s, uint32_t bar_r) {
+                                            uint32_t tm_E, uint32_t bar_s, uint32_t bar_r, uint32_t bar_sc) {
     switch (op) {
         case OP_FROB:    // Gram matrix Khat Khat^T and Khat H_0
             prod_kk(tm_S, kb, kb, 0u);
@@ -241,7 +245,7 @@ __device__ __forceinline__ void issue_batch(int op, uint32_t kb, uint32_t hb, ui
             break;
         case OP_ITER1:   // S = E Khat^T, R += E H_0^T (the second runs under the masked-score epilogue)
             mma8_ek<0>(tm_S, tm_E, kb, kIdescKK);
-            mma_commit(bar_s);
+            mma_commit(bar_sc);
             mma8_ek<1>(tm_R, tm_E, hb, kIdescKK);
             break;
         case OP_ITER2:   // R += P Khat
@@ -251,7 +255,7 @@ __device__ __forceinline__ void issue_batch(int op, uint32_t kb, uint32_t hb, ui
         case OP_OUT_S:   // scores of the final iterate: S = X_hi Khat^T + X_lo Khat^T (X_lo sits in the first columns of R)
             prod_ek(tm_S, tm_E, kb, 0u);
             prod_ek(tm_S, tm_R, kb, 1u);
-            mma_commit(bar_s);
+            mma_commit(bar_sc);
             break;
         case OP_OUT_O:   // O = X_hi U_0^T + P V
             prod_ek(tm_R, tm_E, hb, 0u);
@@ -294,35 +298,43 @@ __device__ __forceinline__ void p_half(const uint32_t (&r)[16], uint32_t (&pk)[8
     }
 }
 // Masked-score epilogue of token c = 32 q + l: key blocks below q need no mask, block q is the diagonal block, the
-// blocks above it are zero.  P for keys 32 kb + 2 u, 2 u + 1 goes to column 32 kb + u of the score tile.  One 32-key
-// block per pass of a rolled loop (the code stays small; the two loads of a pass are in flight together).
+// blocks above it are zero.  P for keys 32 kb + 2 u, 2 u + 1 goes to column 32 kb + u of the score tile.  The epilogue
+// is a chain of tensor-memory round trips, so the zero blocks are stored first, and while a block is converted the
+// next block's scores are already in flight (two passes of two 32-key blocks).
+template <bool EXACT, bool KEYF>
+__device__ __forceinline__ void p_convert(const Ctx &cx, const GateScalars *gs, float ac_c, int kb, const uint32_t (&ra)[16],
+                                          const uint32_t (&rb)[16]) {
+    uint32_t pa[8], pb[8];
+    const float *G2kb = gs->G2 + 32 * kb, *kskb = gs->ks + 32 * kb;
+    if (kb == cx.q) {
+        p_half<EXACT, KEYF, true>(ra, pa, G2kb, kskb, ac_c, cx.l, 0);
+        p_half<EXACT, KEYF, true>(rb, pb, G2kb + 16, kskb + 16, ac_c, cx.l, 16);
+    } else {
+        p_half<EXACT, KEYF, false>(ra, pa, G2kb, kskb, ac_c, cx.l, 0);
+        p_half<EXACT, KEYF, false>(rb, pb, G2kb + 16, kskb + 16, ac_c, cx.l, 16);
+    }
+    TMEM_ST8(cx.tm_s + 32 * kb, pa);
+    TMEM_ST8(cx.tm_s + 32 * kb + 8, pb);
+}
 template <bool EXACT, bool KEYF>
 __device__ __forceinline__ void p_epilogue_t(const Ctx &cx, const GateScalars *gs, float ac_c) {
-#pragma unroll 1
-    for (int kb = 0; kb < 4; ++kb) {
-        const uint32_t taddr = cx.tm_s + 32 * kb;
-        uint32_t pa[8], pb[8];
-        if (kb > cx.q) {
+    {
+        uint32_t z[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) pa[i] = 0u;
-            TMEM_ST8(taddr, pa);
-            TMEM_ST8(taddr + 8, pa);
-            continue;
+        for (int i = 0; i < 8; ++i) z[i] = 0u;
+#pragma unroll 1
+        for (int kb = cx.q + 1; kb < 4; ++kb) {
+            TMEM_ST8(cx.tm_s + 32 * kb, z);
+            TMEM_ST8(cx.tm_s + 32 * kb + 8, z);
         }
+    }
+#pragma unroll 1
+    for (int kb = 0; kb <= cx.q; ++kb) {
         uint32_t ra[16], rb[16];
-        TMEM_LD16(taddr, ra);
-        TMEM_LD16(taddr + 16, rb);
-        const float *G2kb = gs->G2 + 32 * kb, *kskb = gs->ks + 32 * kb;
+        TMEM_LD16(cx.tm_s + 32 * kb, ra);
+        TMEM_LD16(cx.tm_s + 32 * kb + 16, rb);
         tmem_wait_ld();
-        if (kb == cx.q) {
-            p_half<EXACT, KEYF, true>(ra, pa, G2kb, kskb, ac_c, cx.l, 0);
-            p_half<EXACT, KEYF, true>(rb, pb, G2kb + 16, kskb + 16, ac_c, cx.l, 16);
-        } else {
-            p_half<EXACT, KEYF, false>(ra, pa, G2kb, kskb, ac_c, cx.l, 0);
-            p_half<EXACT, KEYF, false>(rb, pb, G2kb + 16, kskb + 16, ac_c, cx.l, 16);
-        }
-        TMEM_ST8(taddr, pa);
-        TMEM_ST8(taddr + 8, pb);
+        p_convert<EXACT, KEYF>(cx, gs, ac_c, kb, ra, rb);
     }
     tmem_wait_st();
 }
@@ -381,6 +393,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ __align__(16) uint32_t s_req[4];     // per slot: requests posted (warps), Gram matrices read (warps)
+    __shared__ uint32_t s_sinfo[2];                 // score event n (parity): slot | read pass << 1 | gate buffer << 2
 
     unsigned char *smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     const int tid = threadIdx.x;
@@ -532,12 +545,19 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 int owner = -1;                         // slot that holds S while its warps read the Gram matrix
                 int prefer = 0;                         // slot to serve first when both are ready
                 bool gave_up = false;
+                uint32_t sev = 0;                       // score events so far
+                const uint32_t sinfo_addr = smem_u32(&s_sinfo[0]);
                 auto issue = [&](int sl, int o) {
                     const uint32_t sbb = bars + 8 * (sl * B_PER_SLOT);
                     const uint32_t sl14 = base14 + ((sl * SLOT_BYTES) >> 4);
+                    if (o == OP_ITER1 || o == OP_OUT_S) {   // tell the score warps whose scores come next
+                        const uint32_t info = (uint32_t)sl | (o == OP_OUT_S ? 2u : 0u) | (((sl ? til1 : til0) & 1u) << 2);
+                        asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(sinfo_addr + 4u * (sev & 1u)), "r"(info) : "memory");
+                        ++sev;
+                    }
                     fence_after();
                     issue_batch(o, sl14 + (BUF_A >> 4), sl14 + (BUF_B >> 4), sl14 + (BUF_C >> 4), tmem + TM_S, tmem + tm_r_of(sl),
-                                tmem + tm_e_of(sl), sbb + 8 * B_MMA_S, sbb + 8 * B_MMA_R);
+                                tmem + tm_e_of(sl), sbb + 8 * B_MMA_S, sbb + 8 * B_MMA_R, bars + 8 * B_SC);
                 };
                 int next_s = -1;                        // slot known to have its request posted (no poll needed)
                 while ((left0 > 0 || left1 > 0) && !gave_up) {
@@ -627,10 +647,40 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 if (!mbar_spin_bounded(bars + 8 * B_DRAIN, 0u)) set_abort(abort_addr);
             }
         }
+    } else if (tid < 256) {
+        // ================================== score warps ==================================
+        // The masked-score epilogue of both slots: S (fp32) -> P (packed bf16) in place, for the scores of an iteration
+        // and for those of the read.  These warps hold no iterate, so they are not short of registers, and the compute
+        // warps go from their update straight to the wait for the accumulator.
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsScore));
+        Ctx cx;
+        cx.l = tid & 31;
+        cx.q = (tid >> 5) & 3;
+        cx.c = 32 * cx.q + cx.l;
+        cx.tm_s = tmem + TM_S + ((uint32_t)(32 * cx.q) << 16);
+        cx.tm_r = cx.tm_e = 0u;
+        const int per_tile = a.n_iter + (solve_only ? 0 : 1);
+        const long long n_events = (long long)n_mine * per_tile;
+        for (long long ev = 0; ev < n_events; ++ev) {
+            if (cx.l == 0 && !aborted(abort_addr) && !mbar_spin_bounded(bars + 8 * B_SC, (uint32_t)(ev & 1))) set_abort(abort_addr);
+            __syncwarp();
+            fence_after();
+            uint32_t info;
+            asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(info) : "r"(smem_u32(&s_sinfo[ev & 1])) : "memory");
+            const int sl_ = (int)(info & 1u);
+            const SlotScalars *const scs = reinterpret_cast<const SlotScalars *>(smem + OFF_SC + sl_ * SC_BYTES);
+            const GateScalars *const gs = &scs->g[(info >> 2) & 1u];
+            const bool exact = scs->exact[(info >> 2) & 1u] != 0;
+            const float ac_c = gs->ac[cx.c];
+            if (info & 2u) p_epilogue<true>(cx, gs, exact, ac_c);
+            else p_epilogue<false>(cx, gs, exact, ac_c);
+            fence_before();
+            warp_post(smem_u32(&s_req[sl_]), cx.l);          // -> ITER2 / OUT_O of that slot
+        }
     } else {
         // ================================= compute threads =================================
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsCompute));
-        const int slot = (tid >> 7) - 1;
+        const int slot = (tid >> 7) - 2;
         Ctx cx;
         cx.l = tid & 31;
         cx.q = (tid >> 5) & 3;
@@ -717,6 +767,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             wait_bar(sb + 8 * (B_GS0 + (j & 1)), (uint32_t)((j >> 1) & 1), abort_addr);
             wait_bar(sb + 8 * B_LD_K, (uint32_t)(j & 1), abort_addr);
             const bool exact = gs->G2[ti.ntok - 1] < -60.f;     // the tile decays below 2^-60: per-element factors
+            if (leader) sc->exact[j & 1] = exact ? 1 : 0;       // (for the score warps; published by the FROB request)
             const float G2c = gs->G2[c], ac_c = gs->ac[c];
             {
                 // Khat: the token's key row scaled in place
@@ -822,10 +873,6 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 const bool last = it + 1 == a.n_iter;
                 omega = 4.f / (4.f - rho2 * omega);              // weight schedule
                 const float beta = omega - 1.f, cz = czb * omega;
-                wait_s_spin();
-                p_epilogue<false>(cx, gs, exact, ac_c);
-                fence_before();
-                arrive_rdy();                                    // -> ITER2
                 const uint64_t beta2 = f2_pack(beta, beta), cz2 = f2_pack(cz, cz), lz2 = f2_pack(lz, lz);
                 wait_r();
                 if (last) after_last_h0_product();
@@ -915,14 +962,11 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             tmem_wait_st();
             fence_before();
             arrive_rdy();                                        // -> OUT_S
-            wait_s();
-            load_next_k();                                       // the keys have been read for the last time
-            // the values stay as loaded: their row factor sqrt(beta_j) 2^(-G_j / 2) rides on the masked scores
-            p_epilogue<true>(cx, gs, exact, ac_c);
-            fence_before();
-            arrive_rdy();                                        // -> OUT_O
+            // (the score warps mask the scores and post OUT_O; the values stay as loaded: their row factor
+            // sqrt(beta_j) 2^(-G_j / 2) rides on the masked scores)
             wait_r();
-            load_next_h();                                       // every product of the tile is complete
+            load_next_k();                                       // every product of the tile is complete
+            load_next_h();
             // O as bf16 into the V buffer (no product reads it any more), stored by TMA
             {
                 uint32_t r[32];
