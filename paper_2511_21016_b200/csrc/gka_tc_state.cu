@@ -242,7 +242,10 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 // stores the bf16 copies of its part of the tile-initial H_0, U_0 (and adds up ||H_0||_F^2), then advances its
 // masters: H <- zeta H + dH, U <- zeta U + dU.
 // ------------------------------------------------------------------------------------------------------------
-enum { TB_KV0 = 0, TB_D0 = NS, TB_D1, TB_STG_RDY, TB_COUNT };
+// TB_STG0 + stage: one barrier per stage, like the loads.  (With a single barrier the compute warps could complete two
+// phases, tiles m + 1 and m + 2, while the TMA thread was still held up behind tile m's store; the phase parity it
+// then polled looked incomplete, and the compute warps in turn waited for the load that only this thread issues.)
+enum { TB_KV0 = 0, TB_D0 = NS, TB_D1, TB_STG0, TB_COUNT = TB_STG0 + NS };
 
 __global__ void __launch_bounds__(kThreadsStateK, 1)
 fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
@@ -261,7 +264,7 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (t == 0) {
         s_abort = 0;
         for (int i = 0; i < TB_COUNT; ++i)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bars + 8 * i), "r"(i == TB_STG_RDY ? CT / 32 : 1));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bars + 8 * i), "r"(i >= TB_STG0 ? CT / 32 : 1));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (t < 32) {
@@ -313,7 +316,7 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             for (int m = 0; m < n_mine; ++m) {
                 // the compute warps have written the bf16 copies of H_0, U_0 over the tile's K and V (the tile's
                 // products are complete): store them, then the stage takes the tile three further on
-                wait(TB_STG_RDY, (uint32_t)(m & 1));
+                wait(TB_STG0 + m % NS, (uint32_t)((m / NS) & 1));
                 const uint32_t src = sb + (uint32_t)(m % NS) * STAGE;
                 for (int which = 0; which < 2; ++which)
                     for (int hf = 0; hf < 2; ++hf)
@@ -476,7 +479,7 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 if (which == 1) {
                     fence_async_smem();
                     __syncwarp();
-                    if (l == 0) mbar_arrive(bars + 8 * TB_STG_RDY);  // -> the TMA thread stores both copies
+                    if (l == 0) mbar_arrive(bars + 8 * (TB_STG0 + m % NS));  // -> the TMA thread stores both copies
                 }
                 // advance the master: zeta m + increment
 #pragma unroll

@@ -16,6 +16,24 @@ def env_rank_world() -> Tuple[int, int, int]:
             int(os.environ.get("WORLD_SIZE", "1")))
 
 
+def free_port() -> int:
+    """A TCP port that is free on the loopback interface right now."""
+    import socket
+    sk = socket.socket()
+    sk.bind(("127.0.0.1", 0))
+    port = sk.getsockname()[1]
+    sk.close()
+    return port
+
+
+def rank_env(rank: int, world: int, port: int) -> dict:
+    """Environment of local rank `rank` of `world` (what torchrun would set), for launching ranks without it."""
+    env = dict(os.environ)
+    env.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+               MASTER_PORT=str(port))
+    return env
+
+
 def shard_seed(base_seed: int, rank: int) -> int:
     """Seed of a rank's shard: every rank draws its own batch of the same shape (weak scaling)."""
     return base_seed + 1000 * rank

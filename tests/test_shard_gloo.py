@@ -64,3 +64,28 @@ def test_batch_slices_cover_without_overlap():
                 lo, hi = shard.batch_slice(total, r, world)
                 seen.extend(range(lo, hi))
             assert seen == list(range(total))
+
+
+def test_local_launcher_starts_ranks_with_the_torchrun_environment(tmp_path):
+    """`bench.py --gpus N` without torchrun starts N ranks itself; here the same environment is given to two CPU
+    processes that meet in a gloo barrier and take the max of their ranks."""
+    import subprocess
+    import sys
+    code = (
+        "import os, sys; sys.path.insert(0, os.environ['GKA_ROOT'])\n"
+        "from paper_2511_21016_b200 import shard\n"
+        "r, lr, w = shard.env_rank_world(); assert lr == r and w == 2\n"
+        "shard.init_process_group('gloo'); shard.barrier()\n"
+        "m = shard.max_over_ranks(float(r))\n"
+        "open(os.path.join(os.environ['GKA_OUT'], f'rank{r}.txt'), 'w').write(str(m))\n"
+        "import torch.distributed as dist; dist.destroy_process_group()\n")
+    port = shard.free_port()
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    procs = []
+    for r in range(2):
+        env = shard.rank_env(r, 2, port)
+        env.update(GKA_ROOT=root, GKA_OUT=str(tmp_path))
+        assert env["MASTER_ADDR"] == "127.0.0.1" and env["WORLD_SIZE"] == "2" and env["LOCAL_RANK"] == str(r)
+        procs.append(subprocess.Popen([sys.executable, "-c", code], env=env))
+    assert [p.wait(timeout=120) for p in procs] == [0, 0]
+    assert [open(tmp_path / f"rank{r}.txt").read() for r in range(2)] == ["1.0", "1.0"]
