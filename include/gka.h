@@ -11,7 +11,7 @@
  * Algorithm 1 run for exactly n_iter matrix-vector products with eigenvalue bounds
  * L = ||H_t||_F + lambda_t, mu = lambda_t (Section 4.1, "Adaptive Regularization").
  * ||H_t||_F is evaluated per token inside each chunk from the chunk-initial state
- * (Section 4.2.1).  The spec name M_t is the paper's U_t; this header uses U.
+ * (Section 4.2.1).  (Descriptions of the layer that speak of a memory M_t mean the paper's U_t.)
  * Optional per-token inputs in the descriptor: write strengths beta_t (beta_t k k^T, beta_t v k^T)
  * and alpha-connection weights alpha_t (o_t = U_t (alpha_t x_t + (1 - alpha_t) q_t)).
  *
@@ -30,7 +30,8 @@
  *     desc->stream and the call returns.
  *   - Argument errors are reported by the return value before anything is launched.  Nothing
  *     throws or aborts.  Device-side waits are bounded; if one runs out the kernel stores
- *     GKA_ERR_TIMEOUT into *desc->device_status (when given) and returns cleanly.
+ *     GKA_ERR_TIMEOUT into *desc->device_status (when given), stops waiting and returns; the outputs
+ *     and the states written by that call are then undefined (partly updated), the device stays usable.
  *   - Supported: d_k == d_v in {64, 128}; chunk == 64; any T >= 1 (a sequence is ceil(T / chunk) chunks, the
  *     last one holds the remaining T mod chunk tokens); n_iter >= 0.
  */
@@ -50,7 +51,8 @@ typedef enum {
     GKA_ERR_DTYPE = 3,       /* unknown io_dtype / precision value                           */
     GKA_ERR_UNSUPPORTED = 4, /* a shape or mode outside the supported set                    */
     GKA_ERR_WORKSPACE = 5,   /* workspace missing, misaligned or smaller than required       */
-    GKA_ERR_DOMAIN = 6,      /* reserved: input outside its domain                           */
+    GKA_ERR_DOMAIN = 6,      /* written to *device_status by the validation pass (GKA_FLAG_VALIDATE): a gate outside
+                                (0, 1], a lambda (or a) that is not positive, a negative beta, a non-finite value */
     GKA_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed (launch, attribute, map) */
     GKA_ERR_TIMEOUT = 8,     /* written to *device_status by a kernel whose bounded wait ran out */
     GKA_ERR_ALIGN = 9        /* a data pointer is not aligned as required                    */
@@ -65,7 +67,12 @@ typedef enum {
 } gka_precision;
 
 enum {
-    GKA_FLAG_ADAPTIVE_LAMBDA = 1u /* lam[] holds a; lambda_t = a * ||H_t||_F (Section 4.1, eq. (4)) */
+    GKA_FLAG_ADAPTIVE_LAMBDA = 1u, /* lam[] holds a; lambda_t = a * ||H_t||_F (Section 4.1, eq. (4)) */
+    GKA_FLAG_VALIDATE = 2u         /* one extra pass over gate, lam (beta, alpha) before the kernels: gamma_t in (0, 1]
+                                      (Section 4.1, "Adaptive Weighting"), lambda_t > 0 so that L >= mu > 0 (input
+                                      condition of Algorithm 1), beta_t >= 0, all finite; a violation stores
+                                      GKA_ERR_DOMAIN into *device_status (which must be given and hold GKA_OK); the
+                                      kernels run all the same */
 };
 
 typedef struct {
@@ -82,14 +89,16 @@ typedef struct {
     const float *state_in; /* optional initial state of the chunked forward; NULL = zero state */
     int *device_status;  /* optional device int, set by kernels on a bounded-wait timeout     */
     float *fro_out;      /* optional [B, T, heads] float32: ||H_t||_F per token (debug output) */
-    void *profile_start; /* optional cudaEvent_t recorded on the stream right before the dominant  */
-    void *profile_stop;  /* kernel (main forward kernel / decode kernel) and right after it        */
+    void *profile_start; /* optional cudaEvent_t pair recorded on the stream right before and right after the    */
+    void *profile_stop;  /* dominant kernel of the call (solve kernel / decode kernel): a forward call is several
+                            kernels, so events of the caller cannot bracket one of them                          */
     const float *beta;   /* optional write strengths beta_t (device pointer): [B, T, heads] for the chunked
                             calls, [B, heads] for the decode step; H_t = gamma_t H_{t-1} + beta_t k_t k_t^T,
                             U_t = gamma_t U_{t-1} + beta_t v_t k_t^T (Remark "canonical beta_t-augmented
                             variant", Section 4.1).  NULL = 1, the recurrence of eq. (CH).  Must be >= 0. */
     const float *alpha;  /* optional alpha-connection weights alpha_t (device pointer, same shapes as beta): the
-                            read becomes out_t = U_t (alpha_t x_t + (1 - alpha_t) q_t) (Section 4.4).  NULL = 1.
+                            read becomes out_t = U_t (alpha_t x_t + (1 - alpha_t) q_t) (Section 4.3, "Architectural
+                            Consideration").  NULL = 1.
                             Ignored by gka_solve_chunked.                                                     */
 } gka_desc;
 
@@ -116,8 +125,8 @@ gka_status gka_fwd_chunked(const gka_desc *desc, const void *q, const void *k, c
  * bounds L, mu as in gka_fwd_chunked (Algorithm 1; H_t from k and gate only).  With rhs = q it returns the
  * iterate x_t that gka_fwd_chunked multiplies by U_t; with rhs = dL/dx_t it returns dL/dq_t, the first
  * step of the backward pass: the fixed-iteration Chebyshev map is linear in its right-hand side and
- * self-adjoint, so the gradient is the same solve with a different right-hand side (Section 4.3,
- * implicit differentiation, Lemma 2).  rhs, k, x_out : [B, T, heads, d_k] (d_v is ignored and must
+ * self-adjoint, so the gradient is the same solve with a different right-hand side (Section 4.2.2,
+ * "Backward Pass", implicit differentiation, Lemma 2).  rhs, k, x_out : [B, T, heads, d_k] (d_v is ignored and must
  * equal d_k in the descriptor); gate, lam : [B, T, heads].  Same dtype rules, workspace, state_in (H part
  * used), flags and error behaviour as gka_fwd_chunked; no state is written.
  */
@@ -166,6 +175,14 @@ size_t gka_fwd_host_staging_bytes(const gka_desc *desc);
 gka_status gka_fwd_chunked_host(const gka_desc *desc, void *staging, const void *q, const void *k,
                                 const void *v, const float *gate, const float *lam, int n_iter,
                                 int chunk, void *out, float *state_out);
+
+/*
+ * Self-test of the bounded device-side waits (no counterpart in the paper; failure detection): one thread block polls,
+ * at most `polls` times (1 .. 2^20), an mbarrier that nothing arrives at, with no copy or product outstanding, then
+ * stores GKA_ERR_TIMEOUT into *desc->device_status (required) and returns.  Uses desc->stream and desc->device_status
+ * only.  The device and the library stay fully usable afterwards.
+ */
+gka_status gka_selftest_bounded_wait(const gka_desc *desc, int polls);
 
 /* Static, human-readable name of a status code. */
 const char *gka_status_string(int status);

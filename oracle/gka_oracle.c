@@ -13,7 +13,7 @@
  *   - beta_t-augmented write, Remark "canonical beta_t-augmented variant" (Section 4.1) and the
  *     appendix's modified eq. (CH): H_t = gamma_t H_{t-1} + beta_t k_t k_t^T,
  *     U_t = gamma_t U_{t-1} + beta_t v_t k_t^T (beta == NULL means beta_t = 1, the paper's experiments)
- *   - alpha-connection, Section 4.4 "Architectural Consideration": the read uses the convex combination
+ *   - alpha-connection, Section 4.3 "Architectural Consideration": the read uses the convex combination
  *     alpha_t x_t + (1 - alpha_t) q_t in place of x_t (alpha == NULL means alpha_t = 1: y_t = U_t x_t)
  *   - Chebyshev Iteration, Algorithm 1 (weight schedule, grad descent, momentum)
  *   - eigenvalue bounds, Section 4.1 "Adaptive Regularization":
@@ -21,7 +21,7 @@
  *   - exact target, Section 4.1 "Motivation" (closed form of eq. (3)):
  *         y_t = U_t (H_t + lambda_t I)^{-1} q_t          (solved by Cholesky)
  *
- * Readings where the paper is silent (see the design notes of the repository):
+ * Readings where the paper is silent:
  *   - lambda_t is a per-token input (absolute value); the optional adaptive mode
  *     lambda_t = a ||H_t||_F of Section 4.1 is selected with lam_mode = 1, in
  *     which case lam[] holds the per-token constant a.

@@ -14,7 +14,8 @@ bool fwd_tc_available();
 
 namespace {
 
-int g_sm_count = 0;
+constexpr int kMaxDevices = 64;
+int g_sm_count[kMaxDevices] = {};      // per device ordinal; filled on first use (a benign race: every writer stores the same value)
 thread_local char g_detail[256] = "";
 
 gka_status cuda_result(cudaError_t err, const char *where) {
@@ -25,13 +26,56 @@ gka_status cuda_result(cudaError_t err, const char *where) {
 }
 
 int sm_count() {
-    if (g_sm_count == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return -1;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
-        g_sm_count = n;
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+    if (dev >= 0 && dev < kMaxDevices && g_sm_count[dev] > 0) return g_sm_count[dev];
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+    if (dev >= 0 && dev < kMaxDevices) g_sm_count[dev] = n;
+    return n;
+}
+
+// Domain check of the per-token scalars (GKA_FLAG_VALIDATE): gamma_t in (0, 1] (Section 4.1, "Adaptive Weighting"),
+// lambda_t > 0, or a > 0 with the adaptive rule, so that L >= mu > 0 (the input condition of Algorithm 1), beta_t >= 0,
+// all finite.  One pass; the first violation stores GKA_ERR_DOMAIN.
+__global__ void validate_kernel(const float *gate, const float *lam, const float *beta, const float *alpha, size_t n,
+                                int *device_status) {
+    bool bad = false;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const float g = gate[i], l = lam[i];
+        bad |= !(g > 0.f && g <= 1.f) || !(l > 0.f && l < INFINITY);
+        if (beta) bad |= !(beta[i] >= 0.f && beta[i] < INFINITY);
+        if (alpha) bad |= !(fabsf(alpha[i]) < INFINITY);
     }
-    return g_sm_count;
+    if (__syncthreads_or(bad) && threadIdx.x == 0) atomicCAS(device_status, (int)GKA_OK, (int)GKA_ERR_DOMAIN);
+}
+cudaError_t launch_validate(const gka_desc *d, const float *gate, const float *lam, size_t n, cudaStream_t stream) {
+    if (!(d->flags & GKA_FLAG_VALIDATE) || !d->device_status) return cudaSuccess;
+    const int blocks = (int)((n + 255) / 256 < 592 ? (n + 255) / 256 : 592);
+    validate_kernel<<<blocks, 256, 0, stream>>>(gate, lam, d->beta, d->alpha, n, d->device_status);
+    return cudaGetLastError();
+}
+
+// Self-test of the bounded waits: one block waits, with a limit of a few thousand polls, on an mbarrier that nothing
+// arrives at (no copy and no product is outstanding), stores GKA_ERR_TIMEOUT and returns.
+__global__ void bounded_wait_selftest_kernel(int polls, int *device_status) {
+    __shared__ __align__(8) uint64_t bar;
+    const uint32_t addr = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(addr));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool done = false;
+    for (int i = 0; i < polls && !done; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(addr), "r"(0u)
+            : "memory");
+        done = ok != 0;
+    }
+    if (__syncthreads_or(!done) && threadIdx.x == 0 && device_status) atomicExch(device_status, (int)GKA_ERR_TIMEOUT);
 }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -44,7 +88,7 @@ gka_status check_desc_common(const gka_desc *d) {
     if (d->io_dtype != GKA_F32 && d->io_dtype != GKA_BF16) return GKA_ERR_DTYPE;
     if (d->precision != GKA_PREC_NATIVE && d->precision != GKA_PREC_HIGH) return GKA_ERR_DTYPE;
     if (d->d_k != 64 && d->d_k != 128) return GKA_ERR_UNSUPPORTED;
-    if (d->flags & ~(unsigned)GKA_FLAG_ADAPTIVE_LAMBDA) return GKA_ERR_UNSUPPORTED;
+    if (d->flags & ~(unsigned)(GKA_FLAG_ADAPTIVE_LAMBDA | GKA_FLAG_VALIDATE)) return GKA_ERR_UNSUPPORTED;
     return GKA_OK;
 }
 
@@ -184,7 +228,8 @@ static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, c
     a.ev_stop = reinterpret_cast<cudaEvent_t>(desc->profile_stop);
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(desc->stream);
 
-    cudaError_t err;
+    cudaError_t err = launch_validate(desc, gate, lam, (size_t)desc->B * desc->T * desc->heads, stream);
+    if (err != cudaSuccess) return cuda_result(err, "gka_fwd_chunked (validation pass)");
     if (tensor_path)
         err = launch_fwd_tc(a, stream);
     else
@@ -214,7 +259,9 @@ gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, co
     if (n_iter < 0) return GKA_ERR_SHAPE;
     if (!aligned16(state) || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
         return GKA_ERR_ALIGN;
-    cudaError_t err = launch_decode(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->heads,
+    cudaError_t err = launch_validate(desc, gate, lam, (size_t)desc->B * desc->heads, reinterpret_cast<cudaStream_t>(desc->stream));
+    if (err != cudaSuccess) return cuda_result(err, "gka_decode_step (validation pass)");
+    err = launch_decode(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->heads,
                                     desc->d_k, desc->io_dtype, desc->flags, desc->beta, desc->alpha, desc->device_status,
                                     reinterpret_cast<cudaEvent_t>(desc->profile_start),
                                     reinterpret_cast<cudaEvent_t>(desc->profile_stop),
@@ -233,7 +280,9 @@ gka_status gka_decode_tokens(const gka_desc *desc, float *state, const void *q, 
         return GKA_ERR_ALIGN;
     if (desc->T == 1)      // one token: the single-step kernel (same layouts) overlaps the state write-back better
         return gka_decode_step(desc, state, q, k, v, gate, lam, n_iter, out);
-    cudaError_t err = launch_decode_multi(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->T, desc->heads,
+    cudaError_t err = launch_validate(desc, gate, lam, (size_t)desc->B * desc->T * desc->heads, reinterpret_cast<cudaStream_t>(desc->stream));
+    if (err != cudaSuccess) return cuda_result(err, "gka_decode_tokens (validation pass)");
+    err = launch_decode_multi(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->T, desc->heads,
                                           desc->d_k, desc->io_dtype, desc->flags, desc->beta, desc->alpha,
                                           desc->device_status,
                                           reinterpret_cast<cudaEvent_t>(desc->profile_start),
@@ -243,6 +292,13 @@ gka_status gka_decode_tokens(const gka_desc *desc, float *state, const void *q, 
 }
 
 const char *gka_last_error_detail(void) { return g_detail; }
+
+gka_status gka_selftest_bounded_wait(const gka_desc *desc, int polls) {
+    if (!desc || !desc->device_status) return GKA_ERR_NULL;
+    if (polls < 1 || polls > (1 << 20)) return GKA_ERR_SHAPE;
+    bounded_wait_selftest_kernel<<<1, 128, 0, reinterpret_cast<cudaStream_t>(desc->stream)>>>(polls, desc->device_status);
+    return cuda_result(cudaGetLastError(), "gka_selftest_bounded_wait");
+}
 
 static size_t align256(size_t n) { return (n + 255) / 256 * 256; }
 

@@ -182,7 +182,7 @@ decode_kernel(float *__restrict__ state, const IoT *__restrict__ q, const IoT *_
         }
     }
     const float *xs = sX + cur * D;
-    const float al = (EXTRA && alpha) ? alpha[head] : 1.f;   // alpha-connection (Section 4.4): the read uses alpha x + (1 - alpha) q
+    const float al = (EXTRA && alpha) ? alpha[head] : 1.f;   // alpha-connection (Section 4.3): the read uses alpha x + (1 - alpha) q
     float xc[CG][4];
     float kx = 0.f;
 #pragma unroll

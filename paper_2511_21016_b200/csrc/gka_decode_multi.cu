@@ -68,7 +68,7 @@ decode_multi_kernel(float *__restrict__ state, const IoT *__restrict__ q, const 
         }
         const float gam = gate[tok];
         float lamv = lam[tok];
-        const float al = alpha ? alpha[tok] : 1.f;   // alpha-connection (Section 4.4): the read uses alpha x + (1 - alpha) q
+        const float al = alpha ? alpha[tok] : 1.f;   // alpha-connection (Section 4.3): the read uses alpha x + (1 - alpha) q
         __syncthreads();
 
         // ---- H <- gamma H + k k^T (kept in registers), Frobenius norm

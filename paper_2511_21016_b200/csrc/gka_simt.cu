@@ -468,7 +468,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
             __syncthreads();
         }
 
-        if (a.solve_only) {      // the solve itself is the result (Section 4.3: the same solve gives dq from dx)
+        if (a.solve_only) {      // the solve itself is the result (Section 4.2.2, Lemma 2: the same solve gives dq from dx)
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
                 const int c = 4 * tc + t;
@@ -478,7 +478,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
                                     make_float4(xm[t][4 * g + 0], xm[t][4 * g + 1], xm[t][4 * g + 2], xm[t][4 * g + 3]));
             }
         }
-        if (a.alpha && !a.solve_only) {    // alpha-connection (Section 4.4): the read uses alpha x + (1 - alpha) q
+        if (a.alpha && !a.solve_only) {    // alpha-connection (Section 4.3): the read uses alpha x + (1 - alpha) q
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
                 const int c = 4 * tc + t;

@@ -19,11 +19,12 @@ GKA_OK = 0
 GKA_F32, GKA_BF16 = 0, 1
 GKA_PREC_NATIVE, GKA_PREC_HIGH = 0, 1
 GKA_FLAG_ADAPTIVE_LAMBDA = 1
+GKA_FLAG_VALIDATE = 2
 GKA_ERR_TIMEOUT = 8
 
 EXPORTS = ("gka_fwd_workspace_bytes", "gka_fwd_chunked", "gka_decode_step", "gka_status_string",
            "gka_fwd_num_work_items", "gka_fwd_work_range", "gka_last_error_detail",
-           "gka_fwd_chunked_noalloc", "gka_noalloc_scratch_bytes",
+           "gka_fwd_chunked_noalloc", "gka_noalloc_scratch_bytes", "gka_selftest_bounded_wait",
            "gka_fwd_chunked_host", "gka_fwd_host_staging_bytes", "gka_solve_chunked", "gka_decode_tokens")
 
 
@@ -88,6 +89,8 @@ def load_library():
         lib.gka_fwd_work_range.restype = ci
         lib.gka_last_error_detail.argtypes = []
         lib.gka_last_error_detail.restype = ctypes.c_char_p
+        lib.gka_selftest_bounded_wait.argtypes = [dp, ci]
+        lib.gka_selftest_bounded_wait.restype = ci
         lib.gka_status_string.argtypes = [ci]
         lib.gka_status_string.restype = ctypes.c_char_p
         _lib = lib
@@ -365,3 +368,17 @@ def gka_decode_tokens(state, q, k, v, gate, lam, n_iter, out=None, *, flags=0, d
     if rc != GKA_OK:
         raise GkaError(rc, "gka_decode_tokens")
     return out
+
+
+def gka_selftest_bounded_wait(device_status, polls=4096, stream=None):
+    """Self-test of the bounded device-side waits: a one-block kernel polls an mbarrier that nothing arrives at,
+    gives up after ``polls`` polls and stores GKA_ERR_TIMEOUT into ``device_status`` (an int32 CUDA tensor)."""
+    _expect("device_status", device_status, torch.int32, (1,))
+    _check_cuda(device_status)
+    if stream is None:
+        stream = torch.cuda.current_stream(device_status.device).cuda_stream
+    desc = make_desc(1, 1, 1, 128, 128, GKA_BF16, stream=stream, device_status=device_status)
+    rc = load_library().gka_selftest_bounded_wait(ctypes.byref(desc), int(polls))
+    if rc != 0:
+        raise GkaError(rc, "gka_selftest_bounded_wait")
+

@@ -419,7 +419,7 @@ def test_adaptive_regularisation_gives_kappa_bound():
 
 # --------------------------------------------------------------------------- backward solve for dq
 def test_fixed_iteration_solve_is_linear_and_self_adjoint():
-    """Section 4.3 (implicit differentiation), Lemma 2: with r fixed the Chebyshev map q -> x is x = p_r(A) q,
+    """Section 4.2.2 ("Backward Pass", implicit differentiation), Lemma 2: with r fixed the Chebyshev map q -> x is x = p_r(A) q,
     a polynomial in the symmetric matrix A = H_t + lambda_t I whose coefficients depend on (L, mu, r) only.
     Hence it is linear in the right-hand side and self-adjoint, so dL/dq = CH(A, dL/dx, r): the same solve
     with another right-hand side.  Checked on the oracle's per-token solves: <CH(u), w> = <u, CH(w)> and
@@ -490,7 +490,7 @@ def test_beta_zero_tokens_write_nothing():
 
 # --------------------------------------------------------------------------- alpha-connection
 def test_alpha_connection_is_a_convex_combination_of_two_reads():
-    """Section 4.4: the read uses alpha_t x_t + (1 - alpha_t) q_t.  By linearity of the read,
+    """Section 4.3 ("Architectural Consideration"): the read uses alpha_t x_t + (1 - alpha_t) q_t.  By linearity of the read,
     y_t(alpha) = alpha_t U_t x_t + (1 - alpha_t) U_t q_t, where U_t x_t is the alpha == 1 output (pinned above) and
     U_t q_t is gated linear attention, written out here by brute force from the definition of U_t."""
     T, D, r = 30, 10, 5

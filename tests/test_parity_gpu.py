@@ -435,7 +435,7 @@ def test_decode_beta_write():
 # --------------------------------------------------------------------------- alpha-connection
 @pytest.mark.parametrize("bf16,n_iter", [(False, 8), (True, 10), (True, 0), (True, 3)])
 def test_fwd_alpha_connection(bf16, n_iter):
-    """out_t = U_t (alpha_t x_t + (1 - alpha_t) q_t) (Section 4.4), both forward paths, with write strengths too."""
+    """out_t = U_t (alpha_t x_t + (1 - alpha_t) q_t) (Section 4.3, "Architectural Consideration"), both forward paths, with write strengths too."""
     cfg = synth.shrink(synth.CONFIGS[1 if bf16 else 0], B=2, heads=3, T=64 * 9, d=128)
     inp = synth.make_inputs(cfg)
     alpha, beta = _beta_for(inp, 11), _beta_for(inp, 12)
@@ -633,3 +633,46 @@ def test_fwd_host_buffers_match_device_call_and_oracle(bf16, B, T):
     dev_out, dev_st, _ = run_fwd(inp, cfg.n_iter, bf16, want_fro=False)
     assert rel(out, dev_out) <= (1e-2 if bf16 else 1e-5)
     assert rel(st, dev_st) <= (5e-3 if bf16 else 1e-5)
+
+
+# ------------------------------------------------------------------------------- failure detection on the device
+def test_bounded_wait_runs_out_and_the_library_stays_usable():
+    """A bounded device-side wait that nothing satisfies gives up after its poll limit, reports GKA_ERR_TIMEOUT
+    through device_status and returns; the next ordinary call works (nothing was in flight, nothing hangs)."""
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    gka.gka_selftest_bounded_wait(status, polls=2000)
+    torch.cuda.synchronize()
+    assert int(status.item()) == gka.GKA_ERR_TIMEOUT
+    check_fwd(synth.shrink(synth.CONFIGS[1], B=1, heads=2, T=256))
+
+
+def test_validate_flag_reports_inputs_outside_their_domain():
+    """GKA_FLAG_VALIDATE: gamma in (0, 1] and lambda > 0 (L >= mu > 0, the input condition of Algorithm 1) are checked in
+    one pass on the device; a violation stores GKA_ERR_DOMAIN, valid inputs leave the status at 0."""
+    cfg = synth.shrink(synth.CONFIGS[1], B=1, heads=2, T=128)
+    inp = synth.make_inputs(cfg)
+    q, k, v = (to_dev(inp[n], True) for n in ("q", "k", "v"))
+    gate, lam = to_dev(inp["gate"]), to_dev(inp["lam"])
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    gka.gka_fwd_chunked(q, k, v, gate, lam, 2, flags=gka.GKA_FLAG_VALIDATE, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for bad_gate, bad_lam in ((1.5, None), (0.0, None), (None, 0.0), (None, float("nan"))):
+        g2, l2 = gate.clone(), lam.clone()
+        if bad_gate is not None:
+            g2[0, 77, 1] = bad_gate
+        if bad_lam is not None:
+            l2[0, 5, 0] = bad_lam
+        status.zero_()
+        gka.gka_fwd_chunked(q, k, v, g2, l2, 2, flags=gka.GKA_FLAG_VALIDATE, device_status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 6, (bad_gate, bad_lam)
+    # the decode step checks its scalars the same way
+    st = torch.zeros(1, 2, 2 * 128 * 128, device=DEV)
+    gd = torch.full((1, 2), 2.0, device=DEV)
+    status.zero_()
+    gka.gka_decode_step(st, q[:, 0], k[:, 0], v[:, 0], gd, lam[:, 0].contiguous(), 1, flags=gka.GKA_FLAG_VALIDATE,
+                        device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 6
+
