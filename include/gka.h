@@ -103,9 +103,11 @@ typedef struct {
 } gka_desc;
 
 /*
- * Scratch the chunked forward needs for this descriptor (segment summaries and segment start
- * states of the cross-chunk state scan; Section 4.2.1 stores the initial state of every chunk,
- * this library stores one state per work segment instead and carries the rest on chip).
+ * Scratch the chunked forward needs for this descriptor: segment summaries and segment start
+ * states of the cross-chunk state scan (one fp32 state per work segment) and, on the bf16
+ * tensor-core path, the bf16 copies of the initial H and U of every 128-token tile plus its
+ * ||H||_F^2 (64 KB + 4 B per tile; Section 4.2.1 stores the initial state of every chunk as well).
+ * The fp32 path carries the states on chip and stores none per chunk.
  * Returns 0 if the descriptor is invalid.  Pure host arithmetic; no CUDA call.
  */
 size_t gka_fwd_workspace_bytes(const gka_desc *desc, int chunk);
@@ -223,7 +225,7 @@ gka_status gka_fwd_work_range(const gka_desc *desc, int chunk, int num_items, in
  *   - Problems whose scan needs more than the array (gka_fwd_workspace_bytes(desc, chunk) >
  *     gka_noalloc_scratch_bytes()) are rejected with GKA_ERR_WORKSPACE before anything is launched:
  *     fp32 arithmetic: d_k = 64 fits up to 170 chunks in total (B * heads * ceil(T / chunk)), d_k = 128 up to 42;
- *     bf16 tensor-core path (d_k = 128): up to 52 tiles of 128 tokens in total (B * heads * ceil(T / 128)).
+ *     bf16 tensor-core path (d_k = 128): up to 51 tiles of 128 tokens in total (B * heads * ceil(T / 128)).
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) with
  *     that device current; make that first call before any stream capture.
  *   - All calls on one device share the array.  Calls that overlap on the GPU race, whatever their

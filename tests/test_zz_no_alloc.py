@@ -35,7 +35,7 @@ def _rel(a, b):
     # fp32 path, d = 64: several work items, sequences cut between items (scan scratch is used)
     ("f32_d64", synth.GkaConfig("na0", B=1, heads=3, T=64 * 50, d=64, chunk=64, n_iter=3,
                                 io_dtype="f32", seed=11), 1e-4),
-    # tensor-core path, d = 128, 20 tiles of 128 tokens: below the built-in scratch limit of 52 tiles
+    # tensor-core path, d = 128, 20 tiles of 128 tokens: below the built-in scratch limit of 51 tiles
     ("bf16_d128", synth.GkaConfig("na1", B=1, heads=2, T=64 * 20, d=128, chunk=64, n_iter=4,
                                   io_dtype="bf16", seed=12), 2e-2),
 ])
