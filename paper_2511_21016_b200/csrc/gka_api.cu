@@ -101,9 +101,10 @@ gka_status check_fwd_shape(const gka_desc *d, int chunk) {
     return GKA_OK;
 }
 
-// bf16 I/O with bf16 tensor-core operands and head dimension 128: the tcgen05 kernels, which work on 128-token tiles
+// bf16 I/O with bf16 tensor-core operands: the tcgen05 kernels, which work on 128-token tiles of 128 channels (head
+// dimension 64 is zero-extended on chip: the loads of the upper 64 channels read past the tensor, i.e. zeros)
 bool wants_tensor_path(const gka_desc *d) {
-    return d->io_dtype == GKA_BF16 && d->precision == GKA_PREC_NATIVE && d->d_k == 128;
+    return d->io_dtype == GKA_BF16 && d->precision == GKA_PREC_NATIVE && (d->d_k == 128 || d->d_k == 64);
 }
 long long work_units(const gka_desc *d) {
     return (long long)d->B * d->heads * (wants_tensor_path(d) ? tiles_of(d->T) : chunks_of(d->T));
@@ -201,6 +202,7 @@ static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, c
     a.alpha = solve_only ? nullptr : desc->alpha;
     a.device_status = desc->device_status;
     a.B = desc->B; a.T = desc->T; a.heads = desc->heads;
+    a.d = desc->d_k;
     a.divH.set((unsigned)desc->heads);
     a.n_iter = n_iter;
     a.flags = desc->flags;

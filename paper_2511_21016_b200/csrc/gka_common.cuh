@@ -208,6 +208,7 @@ struct FwdArgs {
     const float *alpha;    // optional alpha-connection weights [B, T, heads]; nullptr = 1
     int *device_status;
     int B, T, heads;
+    int d;                 // head dimension of the caller's tensors (the tensor path works on 128 channels on chip: 64 is zero-extended)
     FastDiv divH;          // sequence index -> batch entry (divisor: heads)
     int n_iter;
     unsigned flags;

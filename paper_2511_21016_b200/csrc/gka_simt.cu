@@ -250,7 +250,17 @@ __global__ void fwd_scan(FwdArgs a, int st) {
     if (j0 < 0) return;
     const int e = 4 * (blockIdx.x * blockDim.x + threadIdx.x);
     if (e >= st) return;
-    float4 carry = a.state_in ? ld4(a.state_in + (size_t)seq * st + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 carry = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (a.state_in) {
+        const int dd = 2 * a.d * a.d;
+        if (dd == st) {
+            carry = ld4(a.state_in + (size_t)seq * st + e);
+        } else {
+            // tensor path with head dimension 64: the workspace holds states zero-extended to 128 x 128
+            const int which = e >> 14, row = (e >> 7) & 127, col = e & 127;
+            if (row < a.d && col < a.d) carry = ld4(a.state_in + (size_t)seq * dd + (size_t)which * a.d * a.d + (size_t)row * a.d + col);
+        }
+    }
     for (int j = j0; j < i; ++j) {
         const float dcy = a.ws.decay[j];
         const float4 d = ld4(a.ws.delta + (size_t)j * st + e);

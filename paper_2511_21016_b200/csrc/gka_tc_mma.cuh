@@ -76,15 +76,19 @@ constexpr uint32_t kIdescMM = make_idesc(128, 128, 1, 1);   // both MN-major
                  "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])                     \
                  : "memory")
 
-// TMA: one [128 rows][128 columns] operand tile = two boxes; `bar` gets 32768 bytes of transactions
-__device__ __forceinline__ void tma_load_tile3(const CUtensorMap *map, uint32_t dst, uint32_t bar, int x, int y, int z) {
+// TMA: one [128 rows][128 columns] operand tile = two boxes of 64 columns, the second one at column x_hi; `bar` gets
+// 32768 bytes of transactions.  With head dimension 64 the second box lies past the last column of the tensor and
+// reads as zeros (the tile is the head's rows zero-extended to 128 channels).
+__device__ __forceinline__ void tma_load_tile3(const CUtensorMap *map, uint32_t dst, uint32_t bar, int x, int x_hi, int y, int z) {
 #pragma unroll
     for (int hf = 0; hf < 2; ++hf)
         asm volatile(
             "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::
-                "r"(dst + 16384 * hf), "l"(reinterpret_cast<uint64_t>(map)), "r"(x + 64 * hf), "r"(y), "r"(z), "r"(bar)
+                "r"(dst + 16384 * hf), "l"(reinterpret_cast<uint64_t>(map)), "r"(hf ? x_hi : x), "r"(y), "r"(z), "r"(bar)
             : "memory");
 }
+// column of the second box of head h's tile: the head's upper 64 channels, or past the tensor for head dimension 64
+__host__ __device__ __forceinline__ int tile_x_hi(int h, int d, int heads) { return d == 128 ? h * 128 + 64 : heads * d; }
 __device__ __forceinline__ void tma_load_tile2(const CUtensorMap *map, uint32_t dst, uint32_t bar, int y) {
 #pragma unroll
     for (int hf = 0; hf < 2; ++hf)

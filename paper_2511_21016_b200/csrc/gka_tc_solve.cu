@@ -494,14 +494,14 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 auto load_q = [&](int k) {
                     const TileInfo ti = tile_info(a, t_lo + k);
                     mbar_expect_tx(sb + 8 * B_LD_Q, 32768u);
-                    tma_load_tile3(&tmQ, sl + BUF_C, sb + 8 * B_LD_Q, ti.h * D, ti.n * NT, ti.b);
+                    tma_load_tile3(&tmQ, sl + BUF_C, sb + 8 * B_LD_Q, ti.h * a.d, tile_x_hi(ti.h, a.d, a.heads), ti.n * NT, ti.b);
                 };
                 // the inputs do not depend on the state kernel; its per-tile states do
                 {
                     const TileInfo ti = tile_info(a, t_lo + slot);
                     load_q(slot);
                     mbar_expect_tx(sb + 8 * B_LD_K, 32768u);
-                    tma_load_tile3(&tmK, sl + BUF_A, sb + 8 * B_LD_K, ti.h * D, ti.n * NT, ti.b);
+                    tma_load_tile3(&tmK, sl + BUF_A, sb + 8 * B_LD_K, ti.h * a.d, tile_x_hi(ti.h, a.d, a.heads), ti.n * NT, ti.b);
                     asm volatile("griddepcontrol.wait;" ::: "memory");
                     mbar_expect_tx(sb + 8 * B_LD_H, 32768u);
                     tma_load_tile2(&tmS, sl + BUF_B, sb + 8 * B_LD_H, (int)((t_lo + slot) * 256));
@@ -512,12 +512,12 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     if (!solve_only) {
                         wait_bar(sb + 8 * B_QF, (uint32_t)(j & 1), abort_addr);
                         mbar_expect_tx(sb + 8 * B_LD_V, 32768u);
-                        tma_load_tile3(&tmV, sl + BUF_C, sb + 8 * B_LD_V, ti.h * D, ti.n * NT, ti.b);
+                        tma_load_tile3(&tmV, sl + BUF_C, sb + 8 * B_LD_V, ti.h * a.d, tile_x_hi(ti.h, a.d, a.heads), ti.n * NT, ti.b);
                     }
                     wait_bar(sb + 8 * B_RDY_ST, (uint32_t)(j & 1), abort_addr);
-                    for (int hf = 0; hf < 2; ++hf)     // rows past the sequence are clipped
+                    for (int hf = 0; hf < a.d / 64; ++hf)   // rows past the sequence are clipped; channels from a.d on are not stored
                         asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::
-                                         "l"(reinterpret_cast<uint64_t>(&tmO)), "r"(ti.h * D + 64 * hf), "r"(ti.n * NT),
+                                         "l"(reinterpret_cast<uint64_t>(&tmO)), "r"(ti.h * a.d + 64 * hf), "r"(ti.n * NT),
                                      "r"(ti.b), "r"(sl + BUF_C + 16384 * hf)
                                      : "memory");
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -743,7 +743,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 if (leader && more) {
                     const TileInfo tn = tile_info(a, tile + kSlots);
                     mbar_expect_tx(sb + 8 * B_LD_K, 32768u);
-                    tma_load_tile3(&tmK, sl + BUF_A, sb + 8 * B_LD_K, tn.h * D, tn.n * NT, tn.b);
+                    tma_load_tile3(&tmK, sl + BUF_A, sb + 8 * B_LD_K, tn.h * a.d, tile_x_hi(tn.h, a.d, a.heads), tn.n * NT, tn.b);
                 }
             };
             auto load_next_h = [&]() {
@@ -1004,7 +1004,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
 cudaError_t launch_fwd_solve(const FwdArgs &a, cudaStream_t stream) {
     alignas(64) CUtensorMap tmK, tmV, tmQ, tmO, tmS;
-    const int cols = a.heads * D;
+    const int cols = a.heads * a.d;
     const long long ntiles = a.plan.NC;
     if (!make_tile_map(&tmK, a.k, a.B, a.T, cols, NT) || !make_tile_map(&tmV, a.v, a.B, a.T, cols, NT) ||
         !make_tile_map(&tmQ, a.q, a.B, a.T, cols, NT) || !make_tile_map(&tmO, a.out, a.B, a.T, cols, NT) ||

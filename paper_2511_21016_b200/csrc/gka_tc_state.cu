@@ -131,8 +131,8 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
             const uint32_t dst = sb + (uint32_t)(n % NS) * STAGE;
             const uint32_t bar = bars + 8 * (SB_KV0 + n % NS);
             mbar_expect_tx(bar, 65536u);
-            tma_load_tile3(&tmK, dst, bar, h * D, (n0 + n) * NT, b);
-            tma_load_tile3(&tmV, dst + 32768, bar, h * D, (n0 + n) * NT, b);
+            tma_load_tile3(&tmK, dst, bar, h * a.d, tile_x_hi(h, a.d, a.heads), (n0 + n) * NT, b);
+            tma_load_tile3(&tmV, dst + 32768, bar, h * a.d, tile_x_hi(h, a.d, a.heads), (n0 + n) * NT, b);
         };
         if (t == 0)
             for (int n = 0; n < ntiles && n < NS; ++n) issue_tma(n);
@@ -309,8 +309,8 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 const Pos p = pos_of(m);
                 const uint32_t dst = sb + (uint32_t)(m % NS) * STAGE, bar = bars + 8 * (TB_KV0 + m % NS);
                 mbar_expect_tx(bar, 65536u);
-                tma_load_tile3(&tmK, dst, bar, p.h * D, p.n * NT, p.b);
-                tma_load_tile3(&tmV, dst + 32768, bar, p.h * D, p.n * NT, p.b);
+                tma_load_tile3(&tmK, dst, bar, p.h * a.d, tile_x_hi(p.h, a.d, a.heads), p.n * NT, p.b);
+                tma_load_tile3(&tmV, dst + 32768, bar, p.h * a.d, tile_x_hi(p.h, a.d, a.heads), p.n * NT, p.b);
             };
             for (int m = 0; m < n_mine && m < NS; ++m) issue_tma(m);
             for (int m = 0; m < n_mine; ++m) {
@@ -427,13 +427,20 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                                   : (a.state_in ? a.state_in + (size_t)p.seq * st : nullptr);
                 const int j0 = (chained && !a.start_from_scan) ? chain_j0 : 0, j1 = (chained && !a.start_from_scan) ? item : 0;
                 const size_t e = (size_t)c * D + 32 * cq;
+                // the caller's state has head dimension a.d (rows and columns from a.d on are zero on chip); the scan
+                // kernel's start states are in the on-chip layout
+                const bool ext = s0 != nullptr && !(chained && a.start_from_scan);
+                const float *const s0e = ext ? a.state_in + (size_t)p.seq * 2 * a.d * a.d + (size_t)c * a.d + 32 * cq : nullptr;
+                const bool in_ext = c < a.d && 32 * cq < a.d;
 #pragma unroll
                 for (int which = 0; which < 2; ++which) {
                     float(&mm)[32] = which ? mU : mH;
                     const size_t eo = e + which * (size_t)D * D;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
-                        const float4 v4 = s0 ? *reinterpret_cast<const float4 *>(s0 + eo + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        const float4 v4 = ext ? (in_ext ? *reinterpret_cast<const float4 *>(s0e + which * (size_t)a.d * a.d + 4 * i)
+                                                        : make_float4(0.f, 0.f, 0.f, 0.f))
+                                          : (s0 ? *reinterpret_cast<const float4 *>(s0 + eo + 4 * i) : make_float4(0.f, 0.f, 0.f, 0.f));
                         mm[4 * i + 0] = v4.x; mm[4 * i + 1] = v4.y; mm[4 * i + 2] = v4.z; mm[4 * i + 3] = v4.w;
                     }
                     for (int j = j0; j < j1; ++j) {
@@ -493,14 +500,14 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             }
             fence_before();
             // ---- final state of the sequence
-            if (p.seq_end && a.state_out) {
-                float *so = a.state_out + (size_t)p.seq * st + (size_t)c * D + 32 * cq;
+            if (p.seq_end && a.state_out && c < a.d && 32 * cq < a.d) {      // in the caller's layout (head dimension a.d)
+                float *so = a.state_out + (size_t)p.seq * 2 * a.d * a.d + (size_t)c * a.d + 32 * cq;
 #pragma unroll
                 for (int which = 0; which < 2; ++which) {
                     const float(&mm)[32] = which ? mU : mH;
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
-                        *reinterpret_cast<float4 *>(so + which * (size_t)D * D + 4 * i) = make_float4(mm[4 * i], mm[4 * i + 1], mm[4 * i + 2], mm[4 * i + 3]);
+                        *reinterpret_cast<float4 *>(so + which * (size_t)a.d * a.d + 4 * i) = make_float4(mm[4 * i], mm[4 * i + 1], mm[4 * i + 2], mm[4 * i + 3]);
                 }
             }
             // ||H_0||_F^2 of the previous tile: its per-warp sums were written before this tile's hand-over barrier
@@ -551,7 +558,7 @@ cudaError_t launch_fwd_tc(const FwdArgs &a_in, cudaStream_t stream) {
     // states once instead.
     a.start_from_scan = longest > 4 ? 1 : 0;
     alignas(64) CUtensorMap tmK, tmV, tmS;      // boxes of 128 tokens x 64 channels; per-tile bf16 state copies
-    const int cols = a.heads * D;
+    const int cols = a.heads * a.d;
     if (!make_tile_map(&tmK, a.k, a.B, a.T, cols, NT) || !make_tile_map(&tmV, a.v, a.B, a.T, cols, NT) ||
         !make_state_map(&tmS, a.tile_hu, (unsigned long long)a.plan.NC * 256ull))
         return cudaErrorInvalidValue;

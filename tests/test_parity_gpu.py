@@ -66,7 +66,7 @@ def check_fwd(cfg, n_iter=None, precision=gka.GKA_PREC_NATIVE, flags=0, tol=None
                      lam_mode=1 if flags & gka.GKA_FLAG_ADAPTIVE_LAMBDA else 0)
     out, st, fro = run_fwd(inp, n_iter, bf16, precision, flags=flags)
     tol = tol if tol is not None else (TOL_BF16 if bf16 else TOL_F32)
-    fp32_math = (not bf16) or precision == gka.GKA_PREC_HIGH or cfg.d != 128
+    fp32_math = (not bf16) or precision == gka.GKA_PREC_HIGH     # bf16 I/O in native precision: tensor cores, d = 64 or 128
     state_tol = state_tol if state_tol is not None else (1e-5 if fp32_math else 5e-3)
     assert np.all(np.isfinite(out))
     e_out, e_st, e_fro = rel(out, ref["out"]), rel(st, ref["state"]), rel(fro, ref["fro"])
@@ -139,9 +139,40 @@ def test_fwd_bf16_native_iteration_counts(n_iter):
     check_fwd(cfg, n_iter=n_iter)
 
 
-def test_fwd_bf16_native_items_cut_sequences():
-    cfg = synth.shrink(synth.CONFIGS[1], B=1, heads=3, T=64 * 101, n_iter=4)
+@pytest.mark.parametrize("d", [128, 64])
+def test_fwd_bf16_native_items_cut_sequences(d):
+    cfg = synth.shrink(synth.CONFIGS[1], B=1, heads=3, T=64 * 101, n_iter=4, d=d)
     check_fwd(cfg)
+
+
+def test_fwd_bf16_native_head_dimension_64_every_option():
+    """Head dimension 64 on the tensor-core path (bf16 I/O, native precision): several heads side by side (a head's
+    upper half on chip must read as zeros, not as the next head's channels), write strengths, alpha-connection,
+    adaptive lambda at the paper's iteration count, the solve alone, and a 1e-4 comparison of the final state's
+    layout against the fp32 path."""
+    cfg = synth.shrink(synth.CONFIGS[1], B=2, heads=5, T=64 * 9 + 30, n_iter=10, d=64)
+    inp = synth.make_inputs(cfg)
+    rng = np.random.default_rng(5)
+    beta = rng.uniform(0.2, 1.0, inp["gate"].shape).astype(np.float32)
+    alpha = rng.uniform(0.0, 1.0, inp["gate"].shape).astype(np.float32)
+    q, k, v = (to_dev(inp[n], True) for n in ("q", "k", "v"))
+    gate, lam = to_dev(inp["gate"]), to_dev(inp["lam"])
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], 10, beta=beta, alpha=alpha, want_x=True)
+    out, st = gka.gka_fwd_chunked(q, k, v, gate, lam, 10, 64, beta=to_dev(beta), alpha=to_dev(alpha), device_status=status)
+    x = gka.gka_solve_chunked(q, k, gate, lam, 10, 64, beta=to_dev(beta), device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert rel(out.float().cpu().numpy(), ref["out"]) <= TOL_BF16
+    assert tile_max(out.float().cpu().numpy(), ref["out"]) <= TILE_TOL_BF16
+    assert rel(st.cpu().numpy(), ref["state"]) <= 5e-3
+    assert rel(x.float().cpu().numpy(), ref["x"]) <= TOL_BF16
+    lam_a = np.full_like(inp["lam"], 0.02)
+    ref_a = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], lam_a, 30, lam_mode=1)
+    out_a, _ = gka.gka_fwd_chunked(q, k, v, gate, to_dev(lam_a), 30, 64, flags=gka.GKA_FLAG_ADAPTIVE_LAMBDA, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert rel(out_a.float().cpu().numpy(), ref_a["out"]) <= TOL_BF16
 
 
 def test_fwd_state_in_split_prefill_equals_whole():
@@ -501,7 +532,7 @@ def test_fwd_ragged_sequence_length(bf16, d, B, heads, T):
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert bool((big[B * T * heads * d:] == 7.0).all()) and bool((fbig[B * T * heads:] == -3.0).all())
-    tensor_path = bf16 and d == 128
+    tensor_path = bf16
     o = out.float().cpu().numpy()
     assert rel(o, ref["out"]) <= (TOL_BF16 if bf16 else TOL_F32)
     assert rel(fro.cpu().numpy(), ref["fro"]) <= (5e-3 if tensor_path else 1e-5)
@@ -581,12 +612,13 @@ def test_decode_tokens_matches_the_token_recurrence(d, bf16, T, extras):
 
 
 # --------------------------------------------------------------------------- tile shapes of the tensor-core path
+@pytest.mark.parametrize("d", [128, 64])
 @pytest.mark.parametrize("B,heads,T", [(1, 1, 64), (1, 1, 64 * 5), (1, 2, 64 * 7), (3, 1, 64 * 3), (1, 1, 64 * 300)])
-def test_fwd_bf16_native_tile_shapes(B, heads, T):
+def test_fwd_bf16_native_tile_shapes(B, heads, T, d):
     """One-chunk sequences, odd chunk counts (half-filled 128-token tiles at run ends), one chunk per work item
     (every start state comes through a chain of summaries), one long sequence over all work items; with a
-    caller-supplied initial state."""
-    cfg = synth.shrink(synth.CONFIGS[1], B=B, heads=heads, T=T, n_iter=3)
+    caller-supplied initial state.  Head dimension 64 runs on the same kernels, zero-extended on chip."""
+    cfg = synth.shrink(synth.CONFIGS[1], B=B, heads=heads, T=T, n_iter=3, d=d)
     inp = synth.make_inputs(cfg)
     rng = np.random.default_rng(21)
     d = cfg.d
