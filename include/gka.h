@@ -32,11 +32,12 @@
  *     throws or aborts.  Device-side waits are bounded; if one runs out the kernel stores
  *     GKA_ERR_TIMEOUT into *desc->device_status (when given), stops waiting and returns; the outputs
  *     and the states written by that call are then undefined (partly updated), the device stays usable.
- *   - Supported: d_k == d_v in {64, 128}; chunk == 64; any T >= 1 (a sequence is ceil(T / chunk) chunks, the
+ *   - Supported: d_k == d_v in {16, 32, 64, 128}; chunk == 64; any T >= 1 (a sequence is ceil(T / chunk) chunks, the
  *     last one holds the remaining T mod chunk tokens); n_iter >= 0.
  *   - bf16 I/O with GKA_PREC_NATIVE runs on the tensor cores (tiles of 128 tokens x 128 channels; head dimension
- *     64 is zero-extended on chip, so it costs the time of 128); f32 I/O and GKA_PREC_HIGH run in fp32 arithmetic
- *     on the CUDA cores.
+ *     64 is zero-extended on chip, so it costs the time of 128); f32 I/O, GKA_PREC_HIGH and head dimensions 16 and
+ *     32 run in fp32 arithmetic on the CUDA cores (16 and 32 zero-extended to 64 on chip in the chunked calls; the
+ *     decode calls handle them with one warp per (sequence, head) pair).
  */
 #ifndef GKA_H_
 #define GKA_H_
@@ -227,7 +228,7 @@ gka_status gka_fwd_work_range(const gka_desc *desc, int chunk, int num_items, in
  *   - Calls no cudaMalloc / cudaFree and no allocating library routine.
  *   - Problems whose scan needs more than the array (gka_fwd_workspace_bytes(desc, chunk) >
  *     gka_noalloc_scratch_bytes()) are rejected with GKA_ERR_WORKSPACE before anything is launched:
- *     fp32 arithmetic: d_k = 64 fits up to 170 chunks in total (B * heads * ceil(T / chunk)), d_k = 128 up to 42;
+ *     fp32 arithmetic: d_k <= 64 fits up to 170 chunks in total (B * heads * ceil(T / chunk)), d_k = 128 up to 42;
  *     bf16 tensor-core path (d_k = 64 or 128): up to 51 tiles of 128 tokens in total (B * heads * ceil(T / 128)).
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) with
  *     that device current; make that first call before any stream capture.

@@ -8,7 +8,7 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libgka.so")
-SOURCES = ["gka_api.cu", "gka_simt.cu", "gka_decode.cu", "gka_decode_multi.cu", "gka_tc_state.cu", "gka_tc_solve.cu", "gka_noalloc.cu"]
+SOURCES = ["gka_api.cu", "gka_simt.cu", "gka_decode.cu", "gka_decode_multi.cu", "gka_decode_small.cu", "gka_tc_state.cu", "gka_tc_solve.cu", "gka_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -87,7 +87,7 @@ gka_status check_desc_common(const gka_desc *d) {
     if (d->d_k != d->d_v) return GKA_ERR_SHAPE;
     if (d->io_dtype != GKA_F32 && d->io_dtype != GKA_BF16) return GKA_ERR_DTYPE;
     if (d->precision != GKA_PREC_NATIVE && d->precision != GKA_PREC_HIGH) return GKA_ERR_DTYPE;
-    if (d->d_k != 64 && d->d_k != 128) return GKA_ERR_UNSUPPORTED;
+    if (d->d_k != 16 && d->d_k != 32 && d->d_k != 64 && d->d_k != 128) return GKA_ERR_UNSUPPORTED;
     if (d->flags & ~(unsigned)(GKA_FLAG_ADAPTIVE_LAMBDA | GKA_FLAG_VALIDATE)) return GKA_ERR_UNSUPPORTED;
     return GKA_OK;
 }
@@ -106,6 +106,8 @@ gka_status check_fwd_shape(const gka_desc *d, int chunk) {
 bool wants_tensor_path(const gka_desc *d) {
     return d->io_dtype == GKA_BF16 && d->precision == GKA_PREC_NATIVE && (d->d_k == 128 || d->d_k == 64);
 }
+// head dimension the fp32 kernels work with on chip: 16 and 32 are zero-extended to 64
+int simt_dim(const gka_desc *d) { return d->d_k <= 64 ? 64 : 128; }
 long long work_units(const gka_desc *d) {
     return (long long)d->B * d->heads * (wants_tensor_path(d) ? tiles_of(d->T) : chunks_of(d->T));
 }
@@ -141,7 +143,7 @@ const char *gka_status_string(int status) {
 size_t gka_fwd_workspace_bytes(const gka_desc *desc, int chunk) {
     if (check_fwd_shape(desc, chunk) != GKA_OK) return 0;
     if (wants_tensor_path(desc)) return tc_workspace_bytes_for(work_items_cap(desc, chunk), work_units(desc));
-    return workspace_bytes_for(work_items_cap(desc, chunk), desc->d_k, desc->d_v);
+    return workspace_bytes_for(work_items_cap(desc, chunk), simt_dim(desc), simt_dim(desc));
 }
 
 int gka_fwd_num_work_items(const gka_desc *desc, int chunk) {
@@ -224,7 +226,7 @@ static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, c
     } else {
         if (wants_tensor_path(desc)) return GKA_ERR_CUDA;   // no driver entry point for tensor maps
         a.plan.set(desc->B * desc->heads, chunks_of(desc->T), G);
-        a.ws = carve_workspace(desc->workspace, G, desc->d_k, desc->d_v);
+        a.ws = carve_workspace(desc->workspace, G, simt_dim(desc), simt_dim(desc));
     }
     a.ev_start = reinterpret_cast<cudaEvent_t>(desc->profile_start);
     a.ev_stop = reinterpret_cast<cudaEvent_t>(desc->profile_stop);
@@ -263,7 +265,12 @@ gka_status gka_decode_step(const gka_desc *desc, float *state, const void *q, co
         return GKA_ERR_ALIGN;
     cudaError_t err = launch_validate(desc, gate, lam, (size_t)desc->B * desc->heads, reinterpret_cast<cudaStream_t>(desc->stream));
     if (err != cudaSuccess) return cuda_result(err, "gka_decode_step (validation pass)");
-    err = launch_decode(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->heads,
+    if (desc->d_k < 64)      // small head dimensions: one warp per (sequence, head) pair
+        err = launch_decode_small(state, q, k, v, gate, lam, n_iter, out, desc->B, 1, desc->heads, desc->d_k, desc->io_dtype,
+                                  desc->flags, desc->beta, desc->alpha, reinterpret_cast<cudaEvent_t>(desc->profile_start),
+                                  reinterpret_cast<cudaEvent_t>(desc->profile_stop), reinterpret_cast<cudaStream_t>(desc->stream));
+    else
+        err = launch_decode(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->heads,
                                     desc->d_k, desc->io_dtype, desc->flags, desc->beta, desc->alpha, desc->device_status,
                                     reinterpret_cast<cudaEvent_t>(desc->profile_start),
                                     reinterpret_cast<cudaEvent_t>(desc->profile_stop),
@@ -284,7 +291,12 @@ gka_status gka_decode_tokens(const gka_desc *desc, float *state, const void *q, 
         return gka_decode_step(desc, state, q, k, v, gate, lam, n_iter, out);
     cudaError_t err = launch_validate(desc, gate, lam, (size_t)desc->B * desc->T * desc->heads, reinterpret_cast<cudaStream_t>(desc->stream));
     if (err != cudaSuccess) return cuda_result(err, "gka_decode_tokens (validation pass)");
-    err = launch_decode_multi(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->T, desc->heads,
+    if (desc->d_k < 64)
+        err = launch_decode_small(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->T, desc->heads, desc->d_k, desc->io_dtype,
+                                  desc->flags, desc->beta, desc->alpha, reinterpret_cast<cudaEvent_t>(desc->profile_start),
+                                  reinterpret_cast<cudaEvent_t>(desc->profile_stop), reinterpret_cast<cudaStream_t>(desc->stream));
+    else
+        err = launch_decode_multi(state, q, k, v, gate, lam, n_iter, out, desc->B, desc->T, desc->heads,
                                           desc->d_k, desc->io_dtype, desc->flags, desc->beta, desc->alpha,
                                           desc->device_status,
                                           reinterpret_cast<cudaEvent_t>(desc->profile_start),

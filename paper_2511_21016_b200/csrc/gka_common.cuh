@@ -230,6 +230,11 @@ cudaError_t launch_decode(float *state, const void *q, const void *k, const void
                           const float *gate, const float *lam, int n_iter, void *out, int nseq,
                           int heads, int d, int io_dtype, unsigned flags, const float *beta, const float *alpha, int *device_status,
                           cudaEvent_t ev_start, cudaEvent_t ev_stop, cudaStream_t stream);
+// head dimensions 16 and 32, T >= 1 tokens per sequence: one warp per (sequence, head) pair
+cudaError_t launch_decode_small(float *state, const void *q, const void *k, const void *v, const float *gate,
+                                const float *lam, int n_iter, void *out, int nseq, int T, int heads, int d, int io_dtype,
+                                unsigned flags, const float *beta, const float *alpha, cudaEvent_t ev_start,
+                                cudaEvent_t ev_stop, cudaStream_t stream);
 // the same step over T consecutive tokens per sequence, the state read and written once
 cudaError_t launch_decode_multi(float *state, const void *q, const void *k, const void *v, const float *gate,
                                 const float *lam, int n_iter, void *out, int nseq, int T, int heads, int d, int io_dtype,

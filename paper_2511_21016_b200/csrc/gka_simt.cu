@@ -123,16 +123,17 @@ __device__ __forceinline__ void state_update(float *M, const float *A, const flo
 // Section 4.1) key and value rows are scaled by sqrt(beta_t): beta k k^T and beta v k^T are the plain writes of
 // the scaled rows, and every later use of a key in the chunk-wise form carries exactly this factor.
 // Rows from nvalid on (the last chunk of a sequence whose length is not a multiple of C) are zero: a zero key
-// and value write nothing, a zero query solves to zero.
+// and value write nothing, a zero query solves to zero.  The caller's rows hold dx <= D channels (head dimensions 16
+// and 32 run on the 64-channel kernels, zero-extended: zero channels write nothing and solve to zero).
 template <int D, typename IoT>
 __device__ __forceinline__ void load_rows(const IoT *src, size_t row0_elem, size_t row_stride_elem,
-                                          float *dst, float *dstT, int nvalid, const float *beta = nullptr,
+                                          float *dst, float *dstT, int nvalid, int dx, const float *beta = nullptr,
                                           size_t tok0 = 0, int heads = 0) {
     constexpr int F4 = D / 4;
     for (int idx = threadIdx.x; idx < kChunk * F4; idx += kThreads) {
         const int row = idx / F4, c4 = idx % F4;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (row < nvalid) v = Io<IoT>::load4(src + row0_elem + (size_t)row * row_stride_elem + 4 * c4);
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);      // channels from dx on (a smaller head dimension, zero-extended) are zero
+        if (row < nvalid && 4 * c4 < dx) v = Io<IoT>::load4(src + row0_elem + (size_t)row * row_stride_elem + 4 * c4);
         if (beta && row < nvalid) {
             const float sb = sqrtf(fmaxf(beta[tok0 + (size_t)row * heads], 0.f));
             v.x *= sb; v.y *= sb; v.z *= sb; v.w *= sb;
@@ -201,14 +202,14 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_summary(FwdArgs a) {
     float *dU = dH + (size_t)D * D;
     const long long f0 = P.last_run_start(item), f1 = P.lo(item + 1);
     const int seq = (int)(f0 / P.N), b = seq / a.heads, h = seq % a.heads;
-    const size_t rs = (size_t)a.heads * D;
+    const size_t rs = (size_t)a.heads * a.d;
     float decay_log = 0.f;
     for (long long f = f0; f < f1; ++f) {
         const int n = (int)(f % P.N);
         const size_t tok0 = ((size_t)b * a.T + (size_t)n * kChunk) * a.heads + h;
         const int nvalid = min(kChunk, a.T - n * kChunk);
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, nullptr, nvalid, a.beta, tok0, a.heads);
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr, nvalid, a.beta, tok0, a.heads);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * a.d, rs, sK, nullptr, nvalid, a.d, a.beta, tok0, a.heads);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * a.d, rs, sV, nullptr, nvalid, a.d, a.beta, tok0, a.heads);
         load_gates(a.gate, a.lam, tok0, a.heads, nvalid, sG, sZeta, sLam, sW);
         const float zc = sZeta[kChunk - 1];
         decay_log += sG[kChunk - 1];
@@ -256,8 +257,9 @@ __global__ void fwd_scan(FwdArgs a, int st) {
         if (dd == st) {
             carry = ld4(a.state_in + (size_t)seq * st + e);
         } else {
-            // tensor path with head dimension 64: the workspace holds states zero-extended to 128 x 128
-            const int which = e >> 14, row = (e >> 7) & 127, col = e & 127;
+            // the workspace holds states zero-extended to the on-chip head dimension (128 or 64)
+            const int Dw = st == 2 * 128 * 128 ? 128 : 64;
+            const int which = e / (Dw * Dw), row = (e / Dw) % Dw, col = e % Dw;
             if (row < a.d && col < a.d) carry = ld4(a.state_in + (size_t)seq * dd + (size_t)which * a.d * a.d + (size_t)row * a.d + col);
         }
     }
@@ -298,7 +300,9 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
     float *mU = mH + (size_t)D * D;
     const IoT *gq = reinterpret_cast<const IoT *>(a.q);
     IoT *gout = reinterpret_cast<IoT *>(a.out);
-    const size_t rs = (size_t)a.heads * D;
+    const size_t rs = (size_t)a.heads * a.d;
+    const int dx = a.d;                         // channels of the caller's rows and states (dx <= D)
+    const size_t ste = 2 * (size_t)dx * dx;
     const bool adaptive = (a.flags & GKA_FLAG_ADAPTIVE_LAMBDA) != 0;
 
     const long long f_lo = P.lo(item), f_hi = P.lo(item + 1);
@@ -310,16 +314,26 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
 
         // ---- run start: fetch the start state into the running masters
         if (f == f_lo || n == 0) {
-            const float *src = (n == 0) ? (a.state_in ? a.state_in + (size_t)seq * st : nullptr)
-                                        : a.ws.start + (size_t)item * st;
-            for (size_t e = 4 * (size_t)tid; e < st; e += 4 * kThreads)
-                st4(mH + e, src ? ld4(src + e) : make_float4(0.f, 0.f, 0.f, 0.f));
+            if (n != 0 || dx == D) {
+                const float *src = (n == 0) ? (a.state_in ? a.state_in + (size_t)seq * st : nullptr)
+                                            : a.ws.start + (size_t)item * st;
+                for (size_t e = 4 * (size_t)tid; e < st; e += 4 * kThreads)
+                    st4(mH + e, src ? ld4(src + e) : make_float4(0.f, 0.f, 0.f, 0.f));
+            } else {
+                // the caller's state has dx x dx matrices: zero-extended to D x D
+                const float *src = a.state_in ? a.state_in + (size_t)seq * ste : nullptr;
+                for (size_t e = 4 * (size_t)tid; e < st; e += 4 * kThreads) {
+                    const int which = (int)(e / (D * D)), row = (int)(e / D) % D, col = (int)(e % D);
+                    const bool in = src && row < dx && col < dx;
+                    st4(mH + e, in ? ld4(src + (size_t)which * dx * dx + (size_t)row * dx + col) : make_float4(0.f, 0.f, 0.f, 0.f));
+                }
+            }
         }
         __syncthreads();
 
         // ---- stage the chunk
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * D, rs, sK, sKt, nvalid, a.beta, tok0, a.heads);
-        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * D, rs, sV, nullptr, nvalid, a.beta, tok0, a.heads);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.k), tok0 * dx, rs, sK, sKt, nvalid, dx, a.beta, tok0, a.heads);
+        load_rows<D, IoT>(reinterpret_cast<const IoT *>(a.v), tok0 * dx, rs, sV, nullptr, nvalid, dx, a.beta, tok0, a.heads);
         for (int e = 4 * tid; e < D * D; e += 4 * kThreads) st4(sH + e, ld4(mH + e));
         load_gates(a.gate, a.lam, tok0, a.heads, nvalid, sG, sZeta, sLam, sW);  // ends with a barrier
 
@@ -402,7 +416,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
 #pragma unroll
             for (int g = 0; g < DG; ++g) {
                 float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (c < nvalid) qv = Io<IoT>::load4(gq + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td);
+                if (c < nvalid && 64 * g + 4 * td < dx) qv = Io<IoT>::load4(gq + (tok0 + (size_t)c * a.heads) * dx + 64 * g + 4 * td);
                 qm[t][4 * g + 0] = qv.x; qm[t][4 * g + 1] = qv.y;
                 qm[t][4 * g + 2] = qv.z; qm[t][4 * g + 3] = qv.w;
             }
@@ -484,7 +498,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
                 const int c = 4 * tc + t;
 #pragma unroll
                 for (int g = 0; g < DG && c < nvalid; ++g)
-                    Io<IoT>::store4(gout + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td,
+                    if (64 * g + 4 * td < dx)
+                    Io<IoT>::store4(gout + (tok0 + (size_t)c * a.heads) * dx + 64 * g + 4 * td,
                                     make_float4(xm[t][4 * g + 0], xm[t][4 * g + 1], xm[t][4 * g + 2], xm[t][4 * g + 3]));
             }
         }
@@ -496,7 +511,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
 #pragma unroll
                 for (int g = 0; g < DG; ++g) {      // the query again (its registers hold the residual)
                     float4 qv = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (c < nvalid) qv = Io<IoT>::load4(gq + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td);
+                    if (c < nvalid && 64 * g + 4 * td < dx) qv = Io<IoT>::load4(gq + (tok0 + (size_t)c * a.heads) * dx + 64 * g + 4 * td);
                     xm[t][4 * g + 0] = fmaf(al, xm[t][4 * g + 0] - qv.x, qv.x);
                     xm[t][4 * g + 1] = fmaf(al, xm[t][4 * g + 1] - qv.y, qv.y);
                     xm[t][4 * g + 2] = fmaf(al, xm[t][4 * g + 2] - qv.z, qv.z);
@@ -534,7 +549,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
                 const int c = 4 * tc + t;
 #pragma unroll
                 for (int g = 0; g < DG && c < nvalid; ++g)
-                    Io<IoT>::store4(gout + (tok0 + (size_t)c * a.heads) * D + 64 * g + 4 * td,
+                    if (64 * g + 4 * td < dx)
+                    Io<IoT>::store4(gout + (tok0 + (size_t)c * a.heads) * dx + 64 * g + 4 * td,
                                     make_float4(acc[t][4 * g + 0], acc[t][4 * g + 1],
                                                 acc[t][4 * g + 2], acc[t][4 * g + 3]));
             }
@@ -546,8 +562,16 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_simt_main(FwdArgs a) {
         state_update<D>(mU, sV, sK, sW, zc, false);
         __syncthreads();
         if (n == P.N - 1 && a.state_out) {
-            float *dst = a.state_out + (size_t)seq * st;
-            for (size_t e = 4 * (size_t)tid; e < st; e += 4 * kThreads) st4(dst + e, ld4(mH + e));
+            if (dx == D) {
+                float *dst = a.state_out + (size_t)seq * st;
+                for (size_t e = 4 * (size_t)tid; e < st; e += 4 * kThreads) st4(dst + e, ld4(mH + e));
+            } else {                                   // the caller's dx x dx matrices out of the D x D masters
+                float *dst = a.state_out + (size_t)seq * ste;
+                for (size_t e = 4 * (size_t)tid; e < st; e += 4 * kThreads) {
+                    const int which = (int)(e / (D * D)), row = (int)(e / D) % D, col = (int)(e % D);
+                    if (row < dx && col < dx) st4(dst + (size_t)which * dx * dx + (size_t)row * dx + col, ld4(mH + e));
+                }
+            }
         }
         __syncthreads();
     }
@@ -600,6 +624,7 @@ cudaError_t launch_fwd_scan(const FwdArgs &a, int st, cudaStream_t stream, bool 
 }
 
 cudaError_t launch_fwd_simt(const FwdArgs &a, int d, int io_dtype, cudaStream_t stream) {
+    // head dimensions 16, 32 and 64 run on the 64-channel kernels (a.d is the caller's head dimension)
     if (d == 128) {
         return io_dtype == GKA_BF16 ? launch_typed<128, __nv_bfloat16>(a, stream)
                                     : launch_typed<128, float>(a, stream);

@@ -302,7 +302,7 @@ def decode_case(N, heads, d, n_iter, bf16, seed, prefix_T=96):
     return out.float().cpu().numpy(), st_dev.cpu().numpy(), ref
 
 
-@pytest.mark.parametrize("d,bf16", [(128, True), (128, False), (64, False), (64, True)])
+@pytest.mark.parametrize("d,bf16", [(128, True), (128, False), (64, False), (64, True), (32, False), (32, True), (16, False), (16, True)])
 @pytest.mark.parametrize("n_iter", [0, 1, 10])
 def test_decode_step(d, bf16, n_iter):
     out, st, ref = decode_case(5, 3, d, n_iter, bf16, seed=31)
@@ -568,9 +568,47 @@ def test_ragged_length_with_every_option(bf16):
     assert rel(st.cpu().numpy(), ref["state"]) <= (5e-3 if bf16 else 1e-5)
 
 
+# --------------------------------------------------------------------------- head dimensions 16 and 32
+@pytest.mark.parametrize("d,bf16,precision", [(16, False, 0), (32, False, 0), (16, True, 0), (32, True, 0), (32, True, 1)])
+def test_fwd_small_head_dimensions(d, bf16, precision):
+    """Head dimensions 16 and 32 run on the 64-channel fp32 kernels, zero-extended on chip (whatever the I/O dtype and
+    precision): several heads side by side, a ragged last chunk, work items that cut sequences, a caller-supplied
+    initial state in the caller's d x d layout, write strengths and the alpha-connection; outputs, norms, final state
+    and the solve alone against the oracle."""
+    B, heads, T = 2, 5, 64 * 40 + 23
+    cfg = synth.shrink(synth.CONFIGS[1 if bf16 else 0], B=B, heads=heads, T=T, d=d, n_iter=6)
+    inp = synth.make_inputs(cfg)
+    alpha, beta = _beta_for(inp, 8), _beta_for(inp, 9)
+    rng = np.random.default_rng(23)
+    s_in = np.zeros((B, heads, 2 * d * d), np.float32)
+    for b in range(B):
+        for h in range(heads):
+            A = rng.standard_normal((d, 4)) * 0.3
+            s_in[b, h, :d * d] = (A @ A.T).astype(np.float32).ravel()
+            s_in[b, h, d * d:] = (0.1 * rng.standard_normal(d * d)).astype(np.float32)
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], 6, state_in=s_in, alpha=alpha, beta=beta,
+                     want_x=True)
+    q, k, v = (to_dev(inp[n], bf16) for n in ("q", "k", "v"))
+    gate, lam = to_dev(inp["gate"]), to_dev(inp["lam"])
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    fro = torch.zeros(B, T, heads, dtype=torch.float32, device=DEV)
+    out, st = gka.gka_fwd_chunked(q, k, v, gate, lam, 6, 64, state_in=to_dev(s_in), alpha=to_dev(alpha), beta=to_dev(beta),
+                                  precision=precision, fro_out=fro, device_status=status)
+    x = gka.gka_solve_chunked(q, k, gate, lam, 6, 64, state_in=to_dev(s_in), beta=to_dev(beta), precision=precision,
+                              device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    tol = TOL_BF16 if bf16 else TOL_F32          # bf16 I/O: the output is rounded to bf16, the arithmetic is fp32
+    assert rel(out.float().cpu().numpy(), ref["out"]) <= tol
+    assert rel(x.float().cpu().numpy(), ref["x"]) <= tol
+    assert rel(fro.cpu().numpy(), ref["fro"]) <= 1e-5
+    assert rel(st.cpu().numpy(), ref["state"]) <= 1e-5
+
+
 # --------------------------------------------------------------------------- multi-token decode
 @pytest.mark.parametrize("d,bf16,T,extras", [(128, False, 1, False), (128, False, 7, True), (128, True, 16, False),
-                                              (64, False, 5, True), (64, True, 3, False), (128, True, 4, True)])
+                                              (64, False, 5, True), (64, True, 3, False), (128, True, 4, True),
+                                              (32, False, 1, False), (32, True, 6, True), (16, False, 9, True), (16, True, 1, False)])
 def test_decode_tokens_matches_the_token_recurrence(d, bf16, T, extras):
     """T tokens in one call continue a prefix state exactly like the token-by-token recurrence (eq. (CH)):
     outputs and final state against the oracle run on prefix + T tokens, and against T single-token calls."""
