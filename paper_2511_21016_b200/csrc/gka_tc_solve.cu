@@ -144,13 +144,10 @@ __device__ __forceinline__ void wait_bar(uint32_t bar, uint32_t parity, uint32_t
         : "memory");
     if (!ok) set_abort(abort_addr);
 }
-// one count per warp on a shared-memory counter, after every lane's writes and fences (release); acquire load of a pair
+// one count per warp on a shared-memory counter, after every lane's writes and fences (release)
 __device__ __forceinline__ void warp_post(uint32_t addr, int lane) {
     __syncwarp();
     if (lane == 0) asm volatile("red.release.cta.shared::cta.add.u32 [%0], 1;" ::"r"(addr) : "memory");
-}
-__device__ __forceinline__ void ld_acquire_pair(uint32_t addr, uint32_t &a, uint32_t &b) {
-    asm volatile("ld.acquire.cta.shared::cta.v2.u32 {%0, %1}, [%2];" : "=r"(a), "=r"(b) : "r"(addr) : "memory");
 }
 // one arrival per warp, after every lane's writes and fences
 __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane) {
@@ -299,8 +296,8 @@ __device__ __forceinline__ void p_half(const uint32_t (&r)[16], uint32_t (&pk)[8
 }
 // Masked-score epilogue of token c = 32 q + l: key blocks below q need no mask, block q is the diagonal block, the
 // blocks above it are zero.  P for keys 32 kb + 2 u, 2 u + 1 goes to column 32 kb + u of the score tile.  The epilogue
-// is a chain of tensor-memory round trips, so the zero blocks are stored first, and while a block is converted the
-// next block's scores are already in flight (two passes of two 32-key blocks).
+// is a chain of tensor-memory round trips (loads of a 32-key block, conversion, stores), so the zero blocks are stored
+// first.
 template <bool EXACT, bool KEYF>
 __device__ __forceinline__ void p_convert(const Ctx &cx, const GateScalars *gs, float ac_c, int kb, const uint32_t (&ra)[16],
                                           const uint32_t (&rb)[16]) {
@@ -702,19 +699,6 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         uint64_t xs[64];                      // -zt_c x_c: the token's 128 channels as fp32 pairs
         uint32_t n_s = 0, n_r = 0;            // completed phases of MMA_S, MMA_R
         auto wait_s = [&]() { wait_bar(sb + 8 * B_MMA_S, n_s & 1u, abort_addr); ++n_s; fence_after(); };
-        // the same waits without suspending, for the iterations (a suspended wait wakes up late, and a poll of an
-        // mbarrier takes about 100 cycles, so a polling warp leaves nearly all issue slots to the working warps)
-        auto wait_s_spin = [&]() {      // one lane polls (32 lanes on one mbarrier would crowd the shared-memory pipe)
-            if (l == 0 && !aborted(abort_addr) && !mbar_spin_bounded(sb + 8 * B_MMA_S, n_s & 1u)) set_abort(abort_addr);
-            __syncwarp();
-            ++n_s;
-            fence_after();
-        };
-        auto wait_r_spin = [&]() {
-            if (!aborted(abort_addr) && !mbar_spin_bounded(sb + 8 * B_MMA_R, n_r & 1u)) set_abort(abort_addr);
-            ++n_r;
-            fence_after();
-        };
         auto wait_r = [&]() { wait_bar(sb + 8 * B_MMA_R, n_r & 1u, abort_addr); ++n_r; fence_after(); };
         const uint32_t req_addr = smem_u32(&s_req[slot]), grd_addr = smem_u32(&s_req[2 + slot]);
         auto arrive_rdy = [&]() { warp_post(req_addr, l); };

@@ -15,35 +15,6 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn, int b_
 // Every operand of this kernel uses the 128-byte swizzle with 1024 bytes between 8-row groups, so all
 // shared-memory descriptors share one high word; the low word holds the start address and the leading offset.
 constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
-    return ((saddr >> 4) & 0x3FFF) | (((lbo_bytes >> 4) & 0x3FFF) << 16);
-}
-// Every operand of a slot lives at a compile-time offset from the slot's base, and a shared-memory address
-// fits the 14-bit address field without carry, so a descriptor's low word is (slot base >> 4) plus a constant
-// (tile offset, k-step, leading-byte-offset field).  The constants are immediates of the asm block: the
-// issuing thread keeps one register per slot instead of one per operand, and runs on a small register budget.
-template <int ACC, uint32_t A_CONST, uint32_t B_CONST>
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t base14, uint32_t idesc) {
-    asm volatile(
-        "{\n\t.reg .b64 da, db;\n\t.reg .b32 la, lb;\n\t"
-        "add.u32 la, %1, %4;\n\tadd.u32 lb, %1, %5;\n\t"
-        "mov.b64 da, {la, %3};\n\tmov.b64 db, {lb, %3};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %2, %6;\n\t}" ::"r"(d_tmem), "r"(base14), "r"(idesc),
-        "r"(kDescHi), "n"(A_CONST), "n"(B_CONST), "n"(ACC)
-        : "memory");
-}
-// the same with run-time low words and k-steps (summary kernel: operand stages rotate)
-template <int ACC>
-__device__ __forceinline__ void mma_ss_r(uint32_t d_tmem, uint32_t a_lo, uint32_t a_step, uint32_t b_lo, uint32_t b_step,
-                                         uint32_t idesc) {
-    asm volatile(
-        "{\n\t.reg .b64 da, db;\n\t.reg .b32 la, lb;\n\t"
-        "add.u32 la, %1, %5;\n\tadd.u32 lb, %2, %6;\n\t"
-        "mov.b64 da, {la, %4};\n\tmov.b64 db, {lb, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, %7;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc),
-        "r"(kDescHi), "r"(a_step), "r"(b_step), "n"(ACC)
-        : "memory");
-}
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -64,30 +35,10 @@ __device__ __forceinline__ bool mbar_spin_bounded(uint32_t bar, uint32_t parity)
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void slot_sync(int slot) { asm volatile("bar.sync %0, 256;" ::"r"(slot + 1) : "memory"); }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// non-blocking test of a phase (try_wait may suspend the thread; a thread that serves several barriers must not)
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return done != 0;
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return done != 0;
 }
 
 #define TMEM_LD16(taddr, r)                                                                                   \
@@ -170,28 +121,11 @@ __device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
-__device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
 // Streaming global loads that leave the small L1 (what 228 KB of shared memory leave of it) to the
 // thread-local spill slots.
-__device__ __forceinline__ uint32_t ldg_stream_u16(const unsigned short *p) {
-    unsigned short v;
-    asm volatile("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(v) : "l"(p));
-    return v;
-}
 __device__ __forceinline__ float ldg_stream_f32(const float *p) {
     float v;
     asm volatile("ld.global.nc.L1::no_allocate.f32 %0, [%1];" : "=f"(v) : "l"(p));
-    return v;
-}
-__device__ __forceinline__ float4 ldg_stream_f32x4(const float *p) {
-    float4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0, %1, %2, %3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                 : "l"(p));
     return v;
 }
 __device__ __forceinline__ float ex2_fast(float x) {
