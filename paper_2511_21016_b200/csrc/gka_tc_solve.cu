@@ -556,6 +556,33 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     issue_batch(o, sl14 + (BUF_A >> 4), sl14 + (BUF_B >> 4), sl14 + (BUF_C >> 4), tmem + TM_S, tmem + tm_r_of(sl),
                                 tmem + tm_e_of(sl), sbb + 8 * B_MMA_S, sbb + 8 * B_MMA_R, bars + 8 * B_SC);
                 };
+                // Bookkeeping of a request of slot sl that has just been issued, together with its follow-up (ITER2 after
+                // ITER1, OUT_O after OUT_S): the slot's next request, counters and tile count.  Returns the counter value
+                // at which the follow-up is posted.
+                auto book = [&](int sl, int o) -> uint32_t {
+                    bool tile_done = false;
+                    int it = sl ? it1 : it0, nop;
+                    const uint32_t thr = (sl ? thr1 : thr0) + 4u;
+                    if (o == OP_FROB) {
+                        owner = sl;                          // until the Gram matrix has been read
+                        nop = it < a.n_iter ? OP_ITER1 : OP_OUT_S;
+                        if (a.n_iter == 0 && solve_only) tile_done = true;
+                    } else if (o == OP_ITER1) {
+                        ++it;
+                        nop = it < a.n_iter ? OP_ITER1 : OP_OUT_S;
+                        if (it >= a.n_iter && solve_only) tile_done = true;
+                    } else {
+                        nop = OP_FROB;
+                        tile_done = true;
+                    }
+                    if (tile_done) {
+                        nop = OP_FROB;
+                        it = 0;
+                    }
+                    if (sl) { op1 = nop; it1 = it; thr1 = thr + (o == OP_FROB ? 0u : 4u); if (tile_done) { --left1; ++til1; } }
+                    else { op0 = nop; it0 = it; thr0 = thr + (o == OP_FROB ? 0u : 4u); if (tile_done) { --left0; ++til0; } }
+                    return thr;
+                };
                 int next_s = -1;                        // slot known to have its request posted (no poll needed)
                 while ((left0 > 0 || left1 > 0) && !gave_up) {
                     // ---- a slot whose next request (FROB, ITER1 or OUT_S: all need the score tile) is posted and may have S
@@ -582,61 +609,76 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     }
                     if (gave_up) break;
                     prefer = 1 - s;
-                    const int o = s ? op1 : op0;
-                    const uint32_t sb = bars + 8 * (s * B_PER_SLOT);
+                    int o = s ? op1 : op0;
                     // a request of the slot that still holds S for its Gram reads implies that those are done
                     if (owner == s) {
                         if (s) gthr1 += 4u; else gthr0 += 4u;
                         owner = -1;
                     }
-                    if (o == OP_FROB) wait_bar(sb + 8 * B_LD_H, (s ? til1 : til0) & 1u, abort_addr);   // the H_0 tile (TMA)
+                    uint32_t til = s ? til1 : til0;
+                    if (o == OP_FROB) wait_bar(bars + 8 * (s * B_PER_SLOT + B_LD_H), til & 1u, abort_addr);   // the H_0 tile (TMA)
                     issue(s, o);
-                    // ---- the slot's state after this request and its follow-up (worked out while the products run)
-                    bool tile_done = false;
-                    int it = s ? it1 : it0, nop;
-                    uint32_t thr = (s ? thr1 : thr0) + 4u;
-                    if (o == OP_FROB) {
-                        owner = s;                           // until the Gram matrix has been read
-                        nop = it < a.n_iter ? OP_ITER1 : OP_OUT_S;
-                        if (a.n_iter == 0 && solve_only) tile_done = true;
-                    } else if (o == OP_ITER1) {
-                        ++it;
-                        nop = it < a.n_iter ? OP_ITER1 : OP_OUT_S;
-                        if (it >= a.n_iter && solve_only) tile_done = true;
-                    } else {
-                        nop = OP_FROB;
-                        tile_done = true;
-                    }
-                    if (tile_done) {
-                        nop = OP_FROB;
-                        it = 0;
-                    }
-                    const uint32_t til = s ? til1 : til0;
-                    const uint32_t thr_other = s ? thr0 : thr1;
-                    const bool other_left = (s ? left0 : left1) > 0;
-                    if (s) { op1 = nop; it1 = it; thr1 = thr + (o == OP_FROB ? 0u : 4u); if (tile_done) { --left1; ++til1; } }
-                    else { op0 = nop; it0 = it; thr0 = thr + (o == OP_FROB ? 0u : 4u); if (tile_done) { --left0; ++til0; } }
+                    uint32_t thr = book(s, o);
                     if (o == OP_FROB) continue;
-                    // ---- ITER1 or OUT_S: the slot's next request (ITER2, OUT_O) is the only one that can be served now
-                    uint32_t c_other = 0u;
-                    for (int polls = 0;;) {
-                        uint32_t c0, c1;
-                        asm volatile("ld.volatile.shared::cta.v2.u32 {%0, %1}, [%2];" : "=r"(c0), "=r"(c1) : "r"(req_addr) : "memory");
-                        c_other = s ? c0 : c1;
-                        if ((int)((s ? c1 : c0) - thr) >= 0) break;
-                        if ((++polls & 1023) == 0 && (aborted(abort_addr) || polls > (1 << 24))) {
-                            gave_up = true;
+                    // ---- ITER1 or OUT_S of slot s is running: its follow-up (ITER2, OUT_O) comes next.  In the steady state
+                    // of the iterations the other slot's ITER1 follows at once; everything both need is worked out here,
+                    // while the products run and the score warps work, so that a handful of instructions lie between the
+                    // posts and the products.
+                    for (;;) {
+                        const int t = 1 - s;
+                        const uint32_t s14 = base14 + ((s * SLOT_BYTES) >> 4), t14 = base14 + ((t * SLOT_BYTES) >> 4);
+                        const uint32_t p_kb = s14 + (BUF_A >> 4), p_tmR = tmem + tm_r_of(s);
+                        const uint32_t p_barR = bars + 8 * (s * B_PER_SLOT + B_MMA_R);
+                        const bool t_iter = (t ? left1 : left0) > 0 && (t ? op1 : op0) == OP_ITER1;
+                        const uint32_t thr_t = t ? thr1 : thr0;
+                        const uint32_t n_kb = t14 + (BUF_A >> 4), n_hb = t14 + (BUF_B >> 4);
+                        const uint32_t n_tmR = tmem + tm_r_of(t), n_tmE = tmem + tm_e_of(t);
+                        const uint32_t n_info = (uint32_t)t | (((t ? til1 : til0) & 1u) << 2);
+                        const uint32_t n_sinfo = sinfo_addr + 4u * (sev & 1u);
+                        uint32_t c_t = 0u;
+                        for (int polls = 0;;) {
+                            uint32_t c0, c1;
+                            asm volatile("ld.volatile.shared::cta.v2.u32 {%0, %1}, [%2];" : "=r"(c0), "=r"(c1) : "r"(req_addr) : "memory");
+                            c_t = s ? c0 : c1;
+                            if ((int)((s ? c1 : c0) - thr) >= 0) break;
+                            if ((++polls & 1023) == 0 && (aborted(abort_addr) || polls > (1 << 24))) {
+                                gave_up = true;
+                                break;
+                            }
+                        }
+                        if (gave_up) break;
+                        if (o == OP_ITER1) {
+                            fence_after();
+                            mma8_pm(p_tmR, tmem + TM_S, p_kb, kIdescPM);       // ITER2: R += P Khat
+                            mma_commit(p_barR);
+                        } else {                                 // OUT_O: the U_0 and V tiles (TMA)
+                            wait_bar(bars + 8 * (s * B_PER_SLOT + B_LD_U), til & 1u, abort_addr);
+                            wait_bar(bars + 8 * (s * B_PER_SLOT + B_LD_V), til & 1u, abort_addr);
+                            issue(s, OP_OUT_O);
+                        }
+                        const bool t_posted = (int)(c_t - thr_t) >= 0;
+                        if (!(t_iter && t_posted)) {
+                            // the other slot's request, if it was already posted, is served next without a poll
+                            if ((t ? left1 : left0) > 0 && t_posted) next_s = t;
                             break;
                         }
+                        // ---- ITER1 of the other slot, at once
+                        asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(n_sinfo), "r"(n_info) : "memory");
+                        ++sev;
+                        fence_after();
+                        mma8_ek<0>(tmem + TM_S, n_tmE, n_kb, kIdescKK);        // S = E Khat^T
+                        mma_commit(bars + 8 * B_SC);
+                        mma8_ek<1>(n_tmR, n_tmE, n_hb, kIdescKK);               // R += E H_0^T
+                        if (owner == t) {                        // (its Gram reads are done: it has asked again)
+                            if (t) gthr1 += 4u; else gthr0 += 4u;
+                            owner = -1;
+                        }
+                        prefer = s;
+                        til = t ? til1 : til0;
+                        thr = book(t, OP_ITER1);
+                        o = OP_ITER1;
+                        s = t;
                     }
-                    if (gave_up) break;
-                    if (o == OP_OUT_S) {                     // the U_0 and V tiles (TMA)
-                        wait_bar(sb + 8 * B_LD_U, til & 1u, abort_addr);
-                        wait_bar(sb + 8 * B_LD_V, til & 1u, abort_addr);
-                    }
-                    issue(s, o == OP_ITER1 ? OP_ITER2 : OP_OUT_O);
-                    // the other slot's request, if it was already posted, is served next without a poll
-                    if (other_left && (int)(c_other - thr_other) >= 0) next_s = 1 - s;
                 }
                 if (gave_up) set_abort(abort_addr);
                 // every product is complete before the block gives its tensor memory back
