@@ -390,7 +390,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ __align__(16) uint32_t s_req[4];     // per slot: requests posted (warps), Gram matrices read (warps)
-    __shared__ uint32_t s_sinfo[2];                 // score event n (parity): slot | read pass << 1 | gate buffer << 2
+    __shared__ uint32_t s_sinfo[2];                 // score event n (parity): slot | read pass << 1 | gate buffer << 2 | (n + 1) << 8
 
     unsigned char *smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     const int tid = threadIdx.x;
@@ -400,6 +400,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (tid == 0) {
         s_abort = 0;
         s_req[0] = s_req[1] = s_req[2] = s_req[3] = 0u;
+        s_sinfo[0] = s_sinfo[1] = 0u;
         for (int i = 0; i < B_COUNT; ++i) {
             const int b = i % B_PER_SLOT;
             const bool per_warp = i < B_DRAIN && (b == B_RDY_ST || b == B_QF || b == B_GF0 || b == B_GF1);
@@ -548,9 +549,9 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     const uint32_t sbb = bars + 8 * (sl * B_PER_SLOT);
                     const uint32_t sl14 = base14 + ((sl * SLOT_BYTES) >> 4);
                     if (o == OP_ITER1 || o == OP_OUT_S) {   // tell the score warps whose scores come next
-                        const uint32_t info = (uint32_t)sl | (o == OP_OUT_S ? 2u : 0u) | (((sl ? til1 : til0) & 1u) << 2);
-                        asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(sinfo_addr + 4u * (sev & 1u)), "r"(info) : "memory");
                         ++sev;
+                        const uint32_t info = (uint32_t)sl | (o == OP_OUT_S ? 2u : 0u) | (((sl ? til1 : til0) & 1u) << 2) | (sev << 8);
+                        asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(sinfo_addr + 4u * ((sev - 1u) & 1u)), "r"(info) : "memory");
                     }
                     fence_after();
                     issue_batch(o, sl14 + (BUF_A >> 4), sl14 + (BUF_B >> 4), sl14 + (BUF_C >> 4), tmem + TM_S, tmem + tm_r_of(sl),
@@ -631,9 +632,8 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         const uint32_t p_barR = bars + 8 * (s * B_PER_SLOT + B_MMA_R);
                         const bool t_iter = (t ? left1 : left0) > 0 && (t ? op1 : op0) == OP_ITER1;
                         const uint32_t thr_t = t ? thr1 : thr0;
-                        const uint32_t n_kb = t14 + (BUF_A >> 4), n_hb = t14 + (BUF_B >> 4);
-                        const uint32_t n_tmR = tmem + tm_r_of(t), n_tmE = tmem + tm_e_of(t);
-                        const uint32_t n_info = (uint32_t)t | (((t ? til1 : til0) & 1u) << 2);
+                        const uint32_t n_kb = t14 + (BUF_A >> 4), n_tmE = tmem + tm_e_of(t);
+                        const uint32_t n_info = (uint32_t)t | (((t ? til1 : til0) & 1u) << 2) | ((sev + 1u) << 8);
                         const uint32_t n_sinfo = sinfo_addr + 4u * (sev & 1u);
                         uint32_t c_t = 0u;
                         for (int polls = 0;;) {
@@ -668,7 +668,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         fence_after();
                         mma8_ek<0>(tmem + TM_S, n_tmE, n_kb, kIdescKK);        // S = E Khat^T
                         mma_commit(bars + 8 * B_SC);
-                        mma8_ek<1>(n_tmR, n_tmE, n_hb, kIdescKK);               // R += E H_0^T
+                        mma8_ek<1>(tmem + tm_r_of(t), n_tmE, n_kb + ((BUF_B - BUF_A) >> 4), kIdescKK);   // R += E H_0^T
                         if (owner == t) {                        // (its Gram reads are done: it has asked again)
                             if (t) gthr1 += 4u; else gthr0 += 4u;
                             owner = -1;
@@ -701,16 +701,28 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const int per_tile = a.n_iter + (solve_only ? 0 : 1);
         const long long n_events = (long long)n_mine * per_tile;
         for (long long ev = 0; ev < n_events; ++ev) {
-            if (cx.l == 0 && !aborted(abort_addr) && !mbar_spin_bounded(bars + 8 * B_SC, (uint32_t)(ev & 1))) set_abort(abort_addr);
-            __syncwarp();
-            fence_after();
-            uint32_t info;
-            asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(info) : "r"(smem_u32(&s_sinfo[ev & 1])) : "memory");
+            // The issuing thread announces an event before it issues the score product: whose scores, which pass; the
+            // scalars the epilogue needs are fetched while the product runs.
+            uint32_t info = 0u;
+            if (cx.l == 0) {
+                for (int polls = 0;; ++polls) {
+                    asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(info) : "r"(smem_u32(&s_sinfo[ev & 1])) : "memory");
+                    if ((info >> 8) == (uint32_t)(ev + 1)) break;
+                    if ((polls & 1023) == 1023 && (aborted(abort_addr) || polls > (1 << 24))) {
+                        set_abort(abort_addr);
+                        break;
+                    }
+                }
+            }
+            info = __shfl_sync(0xffffffffu, info, 0);
             const int sl_ = (int)(info & 1u);
             const SlotScalars *const scs = reinterpret_cast<const SlotScalars *>(smem + OFF_SC + sl_ * SC_BYTES);
             const GateScalars *const gs = &scs->g[(info >> 2) & 1u];
             const bool exact = scs->exact[(info >> 2) & 1u] != 0;
             const float ac_c = gs->ac[cx.c];
+            if (cx.l == 0 && !aborted(abort_addr) && !mbar_spin_bounded(bars + 8 * B_SC, (uint32_t)(ev & 1))) set_abort(abort_addr);
+            __syncwarp();
+            fence_after();
             if (info & 2u) p_epilogue<true>(cx, gs, exact, ac_c);
             else p_epilogue<false>(cx, gs, exact, ac_c);
             fence_before();
