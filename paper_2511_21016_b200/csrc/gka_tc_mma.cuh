@@ -43,6 +43,13 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_
         "r"(kDescHi), "n"(B_CONST)
         : "memory");
 }
+template <int ACC0, int KS = 0>   // both K-major, 8 k-steps over the 128 columns
+__device__ __forceinline__ void mma8_kk(uint32_t d, uint32_t a_base, uint32_t b_base, uint32_t idesc) {
+    if constexpr (KS < 8) {
+        mma_ss2<(KS == 0 ? ACC0 : 1), t_kmaj(0) + t_kstep(KS), t_kmaj(0) + t_kstep(KS)>(d, a_base, b_base, idesc);
+        mma8_kk<ACC0, KS + 1>(d, a_base, b_base, idesc);
+    }
+}
 template <int ACC0, int KS = 0>   // both MN-major, 8 k-steps over the 128 rows
 __device__ __forceinline__ void mma8_mm(uint32_t d, uint32_t a_base, uint32_t b_base, uint32_t idesc) {
     if constexpr (KS < 8) {

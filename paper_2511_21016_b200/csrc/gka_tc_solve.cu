@@ -44,7 +44,6 @@ namespace {
 
 using namespace tcu;
 
-constexpr int D = 128;
 constexpr int NT = kTile;                  // tokens per tile: one per TMEM lane
 constexpr int kSlots = 2;
 constexpr int ST = 128;                    // compute threads per slot
@@ -171,10 +170,9 @@ __device__ __forceinline__ TileInfo tile_info(const FwdArgs &a, long long tile) 
     return t;
 }
 
-// Products of the issuing thread: 8 k-steps of 16 each.  The three products of an iteration are unrolled with
-// immediate descriptor offsets (the issue then keeps up with the tensor pipe: one tcgen05.mma per 64 cycles); the
-// products that run once per tile are issued from rolled loops with run-time descriptors, at about 100 cycles per
-// instruction, which keeps the code of the issuing warp small in the instruction cache.
+// Products of the issuing thread: 8 k-steps of 16 each, unrolled with immediate descriptor offsets: every instruction
+// of the issuing thread takes of the order of ten cycles beside the working warps of its scheduler, and the issue then
+// keeps up with the tensor pipe (one tcgen05.mma per 64 to 78 cycles).
 // D (+)= A x B with A (packed bf16 pairs, 8 columns per k-step of 16) in TMEM and B in shared memory
 template <int ACC, uint32_t B_CONST>
 __device__ __forceinline__ void mma_ts_c(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_base, uint32_t idesc) {
@@ -193,51 +191,13 @@ __device__ __forceinline__ void mma8_ek(uint32_t d, uint32_t e_tmem, uint32_t b_
         mma8_ek<ACC0, KS + 1>(d, e_tmem, b_base, idesc);
     }
 }
-// low descriptor word of k-step ks of a K-major operand tile / an MN-major operand tile (relative to its base)
-__device__ __forceinline__ uint32_t kmaj_lo(uint32_t base14, int ks) {
-    return base14 + t_kmaj(0) + (uint32_t)((ks >> 2) * 1024 + (ks & 3) * 2);
-}
-__device__ __forceinline__ uint32_t mn_lo(uint32_t base14, int ks) { return base14 + t_mn(0) + (uint32_t)(ks * 128); }
-__device__ __forceinline__ void mma_ss_rt(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc) {
-    asm volatile(
-        "{\n\t.reg .b64 da, db;\n\t.reg .pred p;\n\t"
-        "mov.b64 da, {%1, %4};\n\tmov.b64 db, {%2, %4};\n\tsetp.ne.u32 p, %5, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc),
-        "r"(kDescHi), "r"(acc)
-        : "memory");
-}
-__device__ __forceinline__ void mma_ts_rt(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc) {
-    asm volatile(
-        "{\n\t.reg .b64 db;\n\t.reg .pred p;\n\t"
-        "mov.b64 db, {%2, %4};\n\tsetp.ne.u32 p, %5, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}" ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc),
-        "r"(kDescHi), "r"(acc)
-        : "memory");
-}
-// both operands in shared memory, K-major
-__device__ __forceinline__ void prod_kk(uint32_t d, uint32_t a14, uint32_t b14, uint32_t acc0) {
-#pragma unroll 1
-    for (int ks = 0; ks < 8; ++ks) mma_ss_rt(d, kmaj_lo(a14, ks), kmaj_lo(b14, ks), kIdescKK, ks ? 1u : acc0);
-}
-// A = operand tile in TMEM (64 columns: channels 2 u, 2 u + 1 of a token in column u), B K-major
-__device__ __forceinline__ void prod_ek(uint32_t d, uint32_t e_tmem, uint32_t b14, uint32_t acc0) {
-#pragma unroll 1
-    for (int ks = 0; ks < 8; ++ks) mma_ts_rt(d, e_tmem + 8 * ks, kmaj_lo(b14, ks), kIdescKK, ks ? 1u : acc0);
-}
-// A = masked scores P in TMEM (key block kb in the first 16 columns of the 32-column block kb of the score tile),
-// B MN-major; accumulates
-__device__ __forceinline__ void prod_pm(uint32_t d, uint32_t p_tmem, uint32_t b14) {
-#pragma unroll 1
-    for (int ks = 0; ks < 8; ++ks) mma_ts_rt(d, p_tmem + 32 * (ks >> 1) + 8 * (ks & 1), mn_lo(b14, ks), kIdescPM, 1u);
-}
-
 // The products of one request.  kb, hb, cb: descriptor bases (shared address >> 4) of the slot's buffers.
 __device__ __forceinline__ void issue_batch(int op, uint32_t kb, uint32_t hb, uint32_t cb, uint32_t tm_S, uint32_t tm_R,
                                             uint32_t tm_E, uint32_t bar_s, uint32_t bar_r, uint32_t bar_sc) {
     switch (op) {
         case OP_FROB:    // Gram matrix Khat Khat^T and Khat H_0
-            prod_kk(tm_S, kb, kb, 0u);
-            prod_kk(tm_R, kb, hb, 0u);
+            mma8_kk<0>(tm_S, kb, kb, kIdescKK);
+            mma8_kk<0>(tm_R, kb, hb, kIdescKK);
             mma_commit(bar_s);
             break;
         case OP_ITER1:   // S = E Khat^T, R += E H_0^T (the second runs under the masked-score epilogue)
@@ -250,13 +210,13 @@ __device__ __forceinline__ void issue_batch(int op, uint32_t kb, uint32_t hb, ui
             mma_commit(bar_r);
             break;
         case OP_OUT_S:   // scores of the final iterate: S = X_hi Khat^T + X_lo Khat^T (X_lo sits in the first columns of R)
-            prod_ek(tm_S, tm_E, kb, 0u);
-            prod_ek(tm_S, tm_R, kb, 1u);
+            mma8_ek<0>(tm_S, tm_E, kb, kIdescKK);
+            mma8_ek<1>(tm_S, tm_R, kb, kIdescKK);
             mma_commit(bar_sc);
             break;
         case OP_OUT_O:   // O = X_hi U_0^T + P V
-            prod_ek(tm_R, tm_E, hb, 0u);
-            prod_pm(tm_R, tm_S, cb);
+            mma8_ek<0>(tm_R, tm_E, hb, kIdescKK);
+            mma8_pm(tm_R, tm_S, cb, kIdescPM);
             mma_commit(bar_r);
             break;
         default:
@@ -806,7 +766,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             wait_bar(sb + 8 * B_LD_K, (uint32_t)(j & 1), abort_addr);
             const bool exact = gs->G2[ti.ntok - 1] < -60.f;     // the tile decays below 2^-60: per-element factors
             if (leader) sc->exact[j & 1] = exact ? 1 : 0;       // (for the score warps; published by the FROB request)
-            const float G2c = gs->G2[c], ac_c = gs->ac[c];
+            const float G2c = gs->G2[c];
             {
                 // Khat: the token's key row scaled in place
                 const float fj = gs->ks[c];
