@@ -616,7 +616,16 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                             wait_bar(bars + 8 * (s * B_PER_SLOT + B_LD_V), til & 1u, abort_addr);
                             issue(s, OP_OUT_O);
                         }
-                        const bool t_posted = (int)(c_t - thr_t) >= 0;
+                        bool t_posted = (int)(c_t - thr_t) >= 0;
+                        if (t_iter && !t_posted) {
+                            // the other slot is in its iterations and its update is about to end (this slot's own next
+                            // request is a whole update away): wait for it here, where its products are prepared
+                            for (int polls = 0; polls < 4096 && !t_posted; ++polls) {
+                                uint32_t c0, c1;
+                                asm volatile("ld.volatile.shared::cta.v2.u32 {%0, %1}, [%2];" : "=r"(c0), "=r"(c1) : "r"(req_addr) : "memory");
+                                t_posted = (int)((t ? c1 : c0) - thr_t) >= 0;
+                            }
+                        }
                         if (!(t_iter && t_posted)) {
                             // the other slot's request, if it was already posted, is served next without a poll
                             if ((t ? left1 : left0) > 0 && t_posted) next_s = t;
