@@ -66,6 +66,25 @@ __device__ __forceinline__ void mma8_pm(uint32_t d, uint32_t p_tmem, uint32_t b_
         mma8_pm<KS + 1>(d, p_tmem, b_base, idesc);
     }
 }
+// D += A x B with A in TMEM, the lane quadrants below QLO of D left untouched (their rows of A need not be valid)
+template <uint32_t B_CONST, int QLO>
+__device__ __forceinline__ void mma_ts_rows(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_base, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .b64 db;\n\t.reg .b32 lb;\n\t.reg .pred p;\n\t"
+        "add.u32 lb, %2, %5;\n\tmov.b64 db, {lb, %4};\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, {%6, %7, %8, %9}, p;\n\t}" ::"r"(d_tmem), "r"(a_tmem), "r"(b_base),
+        "r"(idesc), "r"(kDescHi), "n"(B_CONST), "r"(QLO > 0 ? 0xFFFFFFFFu : 0u), "r"(QLO > 1 ? 0xFFFFFFFFu : 0u),
+        "r"(QLO > 2 ? 0xFFFFFFFFu : 0u), "r"(0u)
+        : "memory");
+}
+// P Khat with the masked scores of key block kb valid only for the lane quadrants kb .. 3 (tokens below see none of its keys)
+template <int KS = 0>
+__device__ __forceinline__ void mma8_pm_rows(uint32_t d, uint32_t p_tmem, uint32_t b_base, uint32_t idesc) {
+    if constexpr (KS < 8) {
+        mma_ts_rows<t_mn(0) + t_mnstep(KS), (KS >> 1)>(d, p_tmem + 32 * (KS >> 1) + 8 * (KS & 1), b_base, idesc);
+        mma8_pm_rows<KS + 1>(d, p_tmem, b_base, idesc);
+    }
+}
 
 constexpr uint32_t kIdescKK = make_idesc(128, 128, 0, 0);   // both operands K-major
 constexpr uint32_t kIdescPM = make_idesc(128, 128, 0, 1);   // A from TMEM, B MN-major

@@ -206,7 +206,7 @@ __device__ __forceinline__ void issue_batch(int op, uint32_t kb, uint32_t hb, ui
             mma8_ek<1>(tm_R, tm_E, hb, kIdescKK);
             break;
         case OP_ITER2:   // R += P Khat
-            mma8_pm(tm_R, tm_S, kb, kIdescPM);
+            mma8_pm_rows(tm_R, tm_S, kb, kIdescPM);
             mma_commit(bar_r);
             break;
         case OP_OUT_S:   // scores of the final iterate: S = X_hi Khat^T + X_lo Khat^T (X_lo sits in the first columns of R)
@@ -275,7 +275,7 @@ __device__ __forceinline__ void p_convert(const Ctx &cx, const GateScalars *gs, 
 }
 template <bool EXACT, bool KEYF>
 __device__ __forceinline__ void p_epilogue_t(const Ctx &cx, const GateScalars *gs, float ac_c) {
-    {
+    if (KEYF) {      // (the product of an iteration leaves out the rows whose key block is above the diagonal instead)
         uint32_t z[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) z[i] = 0u;
@@ -609,7 +609,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         if (gave_up) break;
                         if (o == OP_ITER1) {
                             fence_after();
-                            mma8_pm(p_tmR, tmem + TM_S, p_kb, kIdescPM);       // ITER2: R += P Khat
+                            mma8_pm_rows(p_tmR, tmem + TM_S, p_kb, kIdescPM);  // ITER2: R += P Khat
                             mma_commit(p_barR);
                         } else {                                 // OUT_O: the U_0 and V tiles (TMA)
                             wait_bar(bars + 8 * (s * B_PER_SLOT + B_LD_U), til & 1u, abort_addr);
