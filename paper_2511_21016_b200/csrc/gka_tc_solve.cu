@@ -213,9 +213,9 @@ __device__ __forceinline__ void issue_batch(int op, uint32_t kb, uint32_t hb, ui
             mma8_ek<0>(tm_S, tm_E, kb, kIdescKK);
             mma8_ek<1>(tm_S, tm_R, kb, kIdescKK);
             mma_commit(bar_sc);
+            mma8_ek<0>(tm_R, tm_E, hb, kIdescKK);   // O = X_hi U_0^T (runs under the masked-score epilogue; X_lo has been read)
             break;
-        case OP_OUT_O:   // O = X_hi U_0^T + P V
-            mma8_ek<0>(tm_R, tm_E, hb, kIdescKK);
+        case OP_OUT_O:   // O += P V
             mma8_pm(tm_R, tm_S, cb, kIdescPM);
             mma_commit(bar_r);
             break;
@@ -578,6 +578,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     }
                     uint32_t til = s ? til1 : til0;
                     if (o == OP_FROB) wait_bar(bars + 8 * (s * B_PER_SLOT + B_LD_H), til & 1u, abort_addr);   // the H_0 tile (TMA)
+                    if (o == OP_OUT_S) wait_bar(bars + 8 * (s * B_PER_SLOT + B_LD_U), til & 1u, abort_addr);  // the U_0 tile
                     issue(s, o);
                     uint32_t thr = book(s, o);
                     if (o == OP_FROB) continue;
@@ -611,8 +612,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                             fence_after();
                             mma8_pm_rows(p_tmR, tmem + TM_S, p_kb, kIdescPM);  // ITER2: R += P Khat
                             mma_commit(p_barR);
-                        } else {                                 // OUT_O: the U_0 and V tiles (TMA)
-                            wait_bar(bars + 8 * (s * B_PER_SLOT + B_LD_U), til & 1u, abort_addr);
+                        } else {                                 // OUT_O: the V tile (TMA)
                             wait_bar(bars + 8 * (s * B_PER_SLOT + B_LD_V), til & 1u, abort_addr);
                             issue(s, OP_OUT_O);
                         }
@@ -802,6 +802,16 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             float kh = 0.f, gsum = 0.f;
             {
                 uint32_t ra[32];
+                // (the Gram matrix first: it sits in the score tile, which the other slot is waiting for)
+#pragma unroll 1
+                for (int kb = 0; kb <= cx.q; ++kb) {
+                    TMEM_LD32(cx.tm_s + 32 * kb, ra);
+                    tmem_wait_ld();
+                    if (kb == cx.q) gram_block<true>(ra, gs->G2 + 32 * kb, G2c, exact, l, gsum);
+                    else gram_block<false>(ra, gs->G2 + 32 * kb, G2c, exact, l, gsum);
+                }
+                fence_before();
+                warp_post(grd_addr, l);                          // the Gram matrix has been read: S is free again
 #pragma unroll 1
                 for (int p = 0; p < 4; ++p) {
                     TMEM_LD32(cx.tm_r + 32 * p, ra);
@@ -819,16 +829,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         }
                     }
                 }
-#pragma unroll 1
-                for (int kb = 0; kb <= cx.q; ++kb) {
-                    TMEM_LD32(cx.tm_s + 32 * kb, ra);
-                    tmem_wait_ld();
-                    if (kb == cx.q) gram_block<true>(ra, gs->G2 + 32 * kb, G2c, exact, l, gsum);
-                    else gram_block<false>(ra, gs->G2 + 32 * kb, G2c, exact, l, gsum);
-                }
             }
-            fence_before();
-            warp_post(grd_addr, l);                              // the Gram matrix has been read: S is free again
             // ---- f_c by an affine scan (s_c = gamma_c^2 s_{c-1} + d_c, s_{-1} = ||H_0||^2), Chebyshev set-up
             float rho2, czb, lz;
             {
