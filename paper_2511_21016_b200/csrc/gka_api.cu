@@ -103,8 +103,13 @@ gka_status check_fwd_shape(const gka_desc *d, int chunk) {
 
 // bf16 I/O with bf16 tensor-core operands: the tcgen05 kernels, which work on 128-token tiles of 128 channels (head
 // dimension 64 is zero-extended on chip: the loads of the upper 64 channels read past the tensor, i.e. zeros)
+// Sequences of fewer than 16 tokens stay on the fp32 kernels: right after a zero initial state H_t is all but rank one,
+// x_t is dominated by q_t / lambda_t off the key direction while the read takes only its key component, and bf16
+// operands resolve that component to a few percent (up to 16 % for one token under the adaptive rule); from about a
+// dozen tokens on such tokens are a negligible part of the output.
+constexpr int kMinTensorT = 16;
 bool wants_tensor_path(const gka_desc *d) {
-    return d->io_dtype == GKA_BF16 && d->precision == GKA_PREC_NATIVE && (d->d_k == 128 || d->d_k == 64);
+    return d->io_dtype == GKA_BF16 && d->precision == GKA_PREC_NATIVE && (d->d_k == 128 || d->d_k == 64) && d->T >= kMinTensorT;
 }
 // head dimension the fp32 kernels work with on chip: 16 and 32 are zero-extended to 64
 int simt_dim(const gka_desc *d) { return d->d_k <= 64 ? 64 : 128; }
