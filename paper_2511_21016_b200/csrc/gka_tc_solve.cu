@@ -669,6 +669,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         cx.tm_r = cx.tm_e = 0u;
         const int per_tile = a.n_iter + (solve_only ? 0 : 1);
         const long long n_events = (long long)n_mine * per_tile;
+        int reads0 = 0, reads1 = 0;         // read passes seen per slot (= tiles done)
         for (long long ev = 0; ev < n_events; ++ev) {
             // The issuing thread announces an event before it issues the score product: whose scores, which pass; the
             // scalars the epilogue needs are fetched while the product runs.
@@ -692,8 +693,21 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             if (cx.l == 0 && !aborted(abort_addr) && !mbar_spin_bounded(bars + 8 * B_SC, (uint32_t)(ev & 1))) set_abort(abort_addr);
             __syncwarp();
             fence_after();
-            if (info & 2u) p_epilogue<true>(cx, gs, exact, ac_c);
-            else p_epilogue<false>(cx, gs, exact, ac_c);
+            if (info & 2u) {
+                // the score products of the read pass were the last readers of the slot's keys: the next tile's keys
+                // are loaded now, and the slot's compute warps scale them while the read runs
+                const int kdone = sl_ + kSlots * (sl_ ? reads1 : reads0);
+                if (tid == 128 && kdone + kSlots < n_mine) {
+                    const TileInfo tn = tile_info(a, t_lo + kdone + kSlots);
+                    const uint32_t bar_k = bars + 8 * (sl_ * B_PER_SLOT + B_LD_K);
+                    mbar_expect_tx(bar_k, 32768u);
+                    tma_load_tile3(&tmK, sbase + sl_ * SLOT_BYTES + BUF_A, bar_k, tn.h * a.d, tile_x_hi(tn.h, a.d, a.heads), tn.n * NT, tn.b);
+                }
+                if (sl_) ++reads1; else ++reads0;
+                p_epilogue<true>(cx, gs, exact, ac_c);
+            } else {
+                p_epilogue<false>(cx, gs, exact, ac_c);
+            }
             fence_before();
             warp_post(smem_u32(&s_req[sl_]), cx.l);          // -> ITER2 / OUT_O of that slot
         }
@@ -771,14 +785,12 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             // ||H_0||_F^2 of the tile (state kernel): fetched now, used by the scan
             const float hh = ldg_stream_f32(a.tile_hh + tile);
             // ---- gate scalars (helper warp) and the K tile (TMA) of this tile
-            wait_bar(sb + 8 * (B_GS0 + (j & 1)), (uint32_t)((j >> 1) & 1), abort_addr);
-            wait_bar(sb + 8 * B_LD_K, (uint32_t)(j & 1), abort_addr);
-            const bool exact = gs->G2[ti.ntok - 1] < -60.f;     // the tile decays below 2^-60: per-element factors
-            if (leader) sc->exact[j & 1] = exact ? 1 : 0;       // (for the score warps; published by the FROB request)
-            const float G2c = gs->G2[c];
-            {
-                // Khat: the token's key row scaled in place
-                const float fj = gs->ks[c];
+            // Khat of tile jj of this slot: gate scalars (helper warp) and K tile (TMA) awaited, the token's key row scaled
+            // in place
+            auto stage_keys = [&](int jj) {
+                wait_bar(sb + 8 * (B_GS0 + (jj & 1)), (uint32_t)((jj >> 1) & 1), abort_addr);
+                wait_bar(sb + 8 * B_LD_K, (uint32_t)(jj & 1), abort_addr);
+                const float fj = sc->g[jj & 1].ks[c];
                 const uint64_t f2 = f2_pack(fj, fj);
 #pragma unroll 1
                 for (int g = 0; g < 16; ++g) {                   // (rolled: code that runs once per tile is kept small)
@@ -792,8 +804,12 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     }
                     *reinterpret_cast<uint4 *>(bufa + tile_off(c, g)) = v;
                 }
-            }
-            fence_async_smem();
+                fence_async_smem();
+            };
+            if (j == 0 || solve_only) stage_keys(j);             // (otherwise done under the previous tile's read)
+            const bool exact = gs->G2[ti.ntok - 1] < -60.f;     // the tile decays below 2^-60: per-element factors
+            if (leader) sc->exact[j & 1] = exact ? 1 : 0;       // (for the score warps; published by the FROB request)
+            const float G2c = gs->G2[c];
             arrive_rdy();                                        // -> FROB
             wait_s();
             if (a.n_iter == 0) after_last_h0_product();
@@ -972,21 +988,23 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             arrive_rdy();                                        // -> OUT_S
             // (the score warps mask the scores and post OUT_O; the values stay as loaded: their row factor
             // sqrt(beta_j) 2^(-G_j / 2) rides on the masked scores)
+            if (more) stage_keys(j + 1);                         // the next tile's keys (loaded by a score warp at the read pass)
             wait_r();
-            load_next_k();                                       // every product of the tile is complete
-            load_next_h();
+            load_next_h();                                       // every product of the tile is complete
             // O as bf16 into the V buffer (no product reads it any more), stored by TMA
             {
-                uint32_t r[32];
-#pragma unroll 1
+                // (the iterate's registers are free by now: all four loads are in flight at once)
+                uint32_t r[4][32];
+#pragma unroll
+                for (int p = 0; p < 4; ++p) TMEM_LD32(cx.tm_r + 32 * p, r[p]);
+                tmem_wait_ld();
+#pragma unroll
                 for (int p = 0; p < 4; ++p) {
-                    TMEM_LD32(cx.tm_r + 32 * p, r);
-                    tmem_wait_ld();
 #pragma unroll
                     for (int h4 = 0; h4 < 4; ++h4) {
                         uint32_t pk[4];
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) pk[u] = pack_bf16(__uint_as_float(r[8 * h4 + 2 * u]), __uint_as_float(r[8 * h4 + 2 * u + 1]));
+                        for (int u = 0; u < 4; ++u) pk[u] = pack_bf16(__uint_as_float(r[p][8 * h4 + 2 * u]), __uint_as_float(r[p][8 * h4 + 2 * u + 1]));
                         *reinterpret_cast<uint4 *>(bufc + tile_off(c, 4 * p + h4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
                 }
