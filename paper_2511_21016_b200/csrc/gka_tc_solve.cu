@@ -51,7 +51,7 @@ constexpr int CT = kSlots * ST;            // compute threads
 // Warpgroups: 0 = helpers (gate scalars, TMA: one warp per slot, MMA issue), 1 = score warps (the masked-score
 // epilogue of both slots, one warp per TMEM lane quadrant), 2 and 3 = the compute warps of slot 0 and slot 1.
 constexpr int kThreadsSolve = 256 + CT;
-constexpr int kRegsLaunch = 128, kRegsCompute = 200, kRegsScore = 72, kRegsHelper = 40;   // register split after setmaxnreg
+constexpr int kRegsLaunch = 128, kRegsCompute = 200, kRegsScore = 64, kRegsHelper = 48;   // register split after setmaxnreg
 static_assert(kThreadsSolve * kRegsLaunch <= 65536, "launch registers");
 static_assert(CT * kRegsCompute + 128 * kRegsScore + 128 * kRegsHelper <= kThreadsSolve * kRegsLaunch, "register split exceeds the launch allocation");
 
