@@ -31,9 +31,12 @@
 // bandwidth to everything else.  Shared memory per slot: keys, H_0 (later U_0), q (later V, then the result).
 //
 // Warp roles: 4 compute warps per slot, a thread owns one token (one TMEM lane) and all 128 channels of its
-// iterate in registers; one warp prepares the gate scalars one tile ahead; one thread per slot issues that slot's
-// TMA stores and the loads that follow them; one thread issues every tcgen05.mma for both slots.  Hand-overs go
-// through mbarriers (one arrival per warp) and tcgen05.commit.
+// iterate in registers; 4 score warps (one per TMEM lane quadrant) run the masked-score epilogue of both slots; one
+// warp prepares the gate scalars one tile ahead; one thread per slot issues that slot's TMA stores and the loads that
+// follow them; one thread issues every tcgen05.mma for both slots.  Requests to the issuing thread are counters in
+// shared memory (one count per warp), completion comes back through tcgen05.commit mbarriers.  What bounds the
+// iterations is the turn of a slot on the score tile (score product, epilogue, second product); stores to tensor
+// memory (about 40 bytes per cycle per SM) are the scarce resource of the epilogues.
 #include <cuda.h>
 
 #include "gka_common.cuh"
