@@ -693,8 +693,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             const GateScalars *const gs = &scs->g[(info >> 2) & 1u];
             const bool exact = scs->exact[(info >> 2) & 1u] != 0;
             const float ac_c = gs->ac[cx.c];
-            if (cx.l == 0 && !aborted(abort_addr) && !mbar_spin_bounded(bars + 8 * B_SC, (uint32_t)(ev & 1))) set_abort(abort_addr);
-            __syncwarp();
+            wait_bar(bars + 8 * B_SC, (uint32_t)(ev & 1), abort_addr);
             fence_after();
             if (info & 2u) {
                 // the score products of the read pass were the last readers of the slot's keys: the next tile's keys
