@@ -43,11 +43,11 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_
         "r"(kDescHi), "n"(B_CONST)
         : "memory");
 }
-template <int ACC0, int KS = 0>   // both K-major, 8 k-steps over the 128 columns
+template <int ACC0, int NK = 8, int KS = 0>   // both K-major, NK k-steps over the first 16 NK columns
 __device__ __forceinline__ void mma8_kk(uint32_t d, uint32_t a_base, uint32_t b_base, uint32_t idesc) {
-    if constexpr (KS < 8) {
+    if constexpr (KS < NK) {
         mma_ss2<(KS == 0 ? ACC0 : 1), t_kmaj(0) + t_kstep(KS), t_kmaj(0) + t_kstep(KS)>(d, a_base, b_base, idesc);
-        mma8_kk<ACC0, KS + 1>(d, a_base, b_base, idesc);
+        mma8_kk<ACC0, NK, KS + 1>(d, a_base, b_base, idesc);
     }
 }
 template <int ACC0, int KS = 0>   // both MN-major, 8 k-steps over the 128 rows

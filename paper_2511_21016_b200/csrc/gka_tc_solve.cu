@@ -187,36 +187,48 @@ __device__ __forceinline__ void mma_ts_c(uint32_t d_tmem, uint32_t a_tmem, uint3
         : "memory");
 }
 // A = operand tile in TMEM (64 columns: channels 2 u, 2 u + 1 of a token in column u), B K-major
-template <int ACC0, int KS = 0>
+template <int ACC0, int NK = 8, int KS = 0>
 __device__ __forceinline__ void mma8_ek(uint32_t d, uint32_t e_tmem, uint32_t b_base, uint32_t idesc) {
-    if constexpr (KS < 8) {
+    if constexpr (KS < NK) {
         mma_ts_c<(KS == 0 ? ACC0 : 1), t_kmaj(0) + t_kstep(KS)>(d, e_tmem + 8 * KS, b_base, idesc);
-        mma8_ek<ACC0, KS + 1>(d, e_tmem, b_base, idesc);
+        mma8_ek<ACC0, NK, KS + 1>(d, e_tmem, b_base, idesc);
     }
 }
+// The contractions over the channels: with head dimension 64 (zero-extended on chip) the channels 64..127 of every
+// operand are zero, and the four k-steps over them are left out.
+template <int ACC0>
+__device__ __forceinline__ void prod_ek(bool half, uint32_t d, uint32_t e_tmem, uint32_t b_base) {
+    if (half) mma8_ek<ACC0, 4>(d, e_tmem, b_base, kIdescKK);
+    else mma8_ek<ACC0, 8>(d, e_tmem, b_base, kIdescKK);
+}
+template <int ACC0>
+__device__ __forceinline__ void prod_kk(bool half, uint32_t d, uint32_t a_base, uint32_t b_base) {
+    if (half) mma8_kk<ACC0, 4>(d, a_base, b_base, kIdescKK);
+    else mma8_kk<ACC0, 8>(d, a_base, b_base, kIdescKK);
+}
 // The products of one request.  kb, hb, cb: descriptor bases (shared address >> 4) of the slot's buffers.
-__device__ __forceinline__ void issue_batch(int op, uint32_t kb, uint32_t hb, uint32_t cb, uint32_t tm_S, uint32_t tm_R,
+__device__ __forceinline__ void issue_batch(int op, bool half, uint32_t kb, uint32_t hb, uint32_t cb, uint32_t tm_S, uint32_t tm_R,
                                             uint32_t tm_E, uint32_t bar_s, uint32_t bar_r, uint32_t bar_sc) {
     switch (op) {
         case OP_FROB:    // Gram matrix Khat Khat^T and Khat H_0
-            mma8_kk<0>(tm_S, kb, kb, kIdescKK);
-            mma8_kk<0>(tm_R, kb, hb, kIdescKK);
+            prod_kk<0>(half, tm_S, kb, kb);
+            prod_kk<0>(half, tm_R, kb, hb);
             mma_commit(bar_s);
             break;
         case OP_ITER1:   // S = E Khat^T, R += E H_0^T (the second runs under the masked-score epilogue)
-            mma8_ek<0>(tm_S, tm_E, kb, kIdescKK);
+            prod_ek<0>(half, tm_S, tm_E, kb);
             mma_commit(bar_sc);
-            mma8_ek<1>(tm_R, tm_E, hb, kIdescKK);
+            prod_ek<1>(half, tm_R, tm_E, hb);
             break;
         case OP_ITER2:   // R += P Khat
             mma8_pm_rows(tm_R, tm_S, kb, kIdescPM);
             mma_commit(bar_r);
             break;
         case OP_OUT_S:   // scores of the final iterate: S = X_hi Khat^T + X_lo Khat^T (X_lo sits in the first columns of R)
-            mma8_ek<0>(tm_S, tm_E, kb, kIdescKK);
-            mma8_ek<1>(tm_S, tm_R, kb, kIdescKK);
+            prod_ek<0>(half, tm_S, tm_E, kb);
+            prod_ek<1>(half, tm_S, tm_R, kb);
             mma_commit(bar_sc);
-            mma8_ek<0>(tm_R, tm_E, hb, kIdescKK);   // O = X_hi U_0^T (runs under the masked-score epilogue; X_lo has been read)
+            prod_ek<0>(half, tm_R, tm_E, hb);   // O = X_hi U_0^T (runs under the masked-score epilogue; X_lo has been read)
             break;
         case OP_OUT_O:   // O += P V
             mma8_pm(tm_R, tm_S, cb, kIdescPM);
@@ -343,7 +355,7 @@ __device__ __forceinline__ float affine_scan(const Ctx &cx, SlotScalars *sc, int
     return fmaf(a, s, b);
 }
 
-template <bool EXTRA>
+template <bool EXTRA, bool HALF>
 __global__ void __launch_bounds__(kThreadsSolve, 1)
 fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmO,
@@ -389,6 +401,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const float *const beta_p = EXTRA ? a.beta : nullptr;
     const float *const alpha_p = EXTRA ? a.alpha : nullptr;
     const bool mix = alpha_p != nullptr && !solve_only;   // alpha-connection: the read uses alpha x + (1 - alpha) q
+    constexpr bool half = HALF;                           // head dimension 64: channels 64..127 are zero, their k-steps are left out
 
     // The helper warps come first: when a scheduler changes warps it prefers the oldest eligible one, and the thread
     // that issues the products must not wait behind the compute warps of its scheduler.
@@ -517,7 +530,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(sinfo_addr + 4u * ((sev - 1u) & 1u)), "r"(info) : "memory");
                     }
                     fence_after();
-                    issue_batch(o, sl14 + (BUF_A >> 4), sl14 + (BUF_B >> 4), sl14 + (BUF_C >> 4), tmem + TM_S, tmem + tm_r_of(sl),
+                    issue_batch(o, half, sl14 + (BUF_A >> 4), sl14 + (BUF_B >> 4), sl14 + (BUF_C >> 4), tmem + TM_S, tmem + tm_r_of(sl),
                                 tmem + tm_e_of(sl), sbb + 8 * B_MMA_S, sbb + 8 * B_MMA_R, bars + 8 * B_SC);
                 };
                 // Bookkeeping of a request of slot sl that has just been issued, together with its follow-up (ITER2 after
@@ -638,9 +651,9 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(n_sinfo), "r"(n_info) : "memory");
                         ++sev;
                         fence_after();
-                        mma8_ek<0>(tmem + TM_S, n_tmE, n_kb, kIdescKK);        // S = E Khat^T
+                        prod_ek<0>(half, tmem + TM_S, n_tmE, n_kb);           // S = E Khat^T
                         mma_commit(bars + 8 * B_SC);
-                        mma8_ek<1>(tmem + tm_r_of(t), n_tmE, n_kb + ((BUF_B - BUF_A) >> 4), kIdescKK);   // R += E H_0^T
+                        prod_ek<1>(half, tmem + tm_r_of(t), n_tmE, n_kb + ((BUF_B - BUF_A) >> 4));   // R += E H_0^T
                         if (owner == t) {                        // (its Gram reads are done: it has asked again)
                             if (t) gthr1 += 4u; else gthr0 += 4u;
                             owner = -1;
@@ -735,6 +748,8 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         // the per-tile states and norms come from the state kernel
         asm volatile("griddepcontrol.wait;" ::: "memory");
 
+        // Head dimension 64: the passes over the channels stop at channel 64 (the rest is zero in every operand and stays so)
+        constexpr int NG16 = HALF ? 4 : 8;    // groups of 16 channels
         uint64_t xs[64];                      // -zt_c x_c: the token's 128 channels as fp32 pairs
         uint32_t n_s = 0, n_r = 0;            // completed phases of MMA_S, MMA_R
         auto wait_s = [&]() { wait_bar(sb + 8 * B_MMA_S, n_s & 1u, abort_addr); ++n_s; fence_after(); };
@@ -795,7 +810,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 const float fj = sc->g[jj & 1].ks[c];
                 const uint64_t f2 = f2_pack(fj, fj);
 #pragma unroll 1
-                for (int g = 0; g < 16; ++g) {                   // (rolled: code that runs once per tile is kept small)
+                for (int g = 0; g < 2 * NG16; ++g) {             // (rolled: code that runs once per tile is kept small)
                     uint4 v = *reinterpret_cast<const uint4 *>(bufa + tile_off(c, g));
                     uint32_t *pv = reinterpret_cast<uint32_t *>(&v);
 #pragma unroll
@@ -831,7 +846,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 fence_before();
                 warp_post(grd_addr, l);                          // the Gram matrix has been read: S is free again
 #pragma unroll 1
-                for (int p = 0; p < 4; ++p) {
+                for (int p = 0; p < NG16 / 2; ++p) {
                     TMEM_LD32(cx.tm_r + 32 * p, ra);
                     uint4 kv[4];
 #pragma unroll
@@ -868,7 +883,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             wait_bar(sb + 8 * B_LD_Q, (uint32_t)(j & 1), abort_addr);   // q tile has landed
             // ---- x_0: R = q, E_0 = czb q, xs = E_0
 #pragma unroll
-            for (int g16 = 0; g16 < 8; ++g16) {
+            for (int g16 = 0; g16 < NG16; ++g16) {
                 uint32_t rr[16], pk[8];
 #pragma unroll
                 for (int h2 = 0; h2 < 2; ++h2) {
@@ -910,12 +925,12 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     TMEM_LD8(cx.tm_e, ea);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int g = 0; g < 8; ++g) {
+                    for (int g = 0; g < NG16; ++g) {
                         uint32_t(&r)[16] = (g & 1) ? rb : ra;
                         uint32_t(&rn)[16] = (g & 1) ? ra : rb;
                         uint32_t(&e)[8] = (g & 1) ? eb : ea;
                         uint32_t(&en_)[8] = (g & 1) ? ea : eb;
-                        if (g < 7) {
+                        if (g < NG16 - 1) {
                             TMEM_LD16(cx.tm_r + 16 * (g + 1), rn);
                             TMEM_LD8(cx.tm_e + 8 * (g + 1), en_);
                         }
@@ -931,7 +946,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                             xs[i] = f2_add(xs[i], f2_pack(bf16_lo(pk[u]), bf16_hi(pk[u])));
                         }
                         TMEM_ST8(cx.tm_e + 8 * g, pk);
-                                        if (g < 7) tmem_wait_ld();
+                                        if (g < NG16 - 1) tmem_wait_ld();
                     }
                     if (!last) {
                         tmem_wait_st();
@@ -945,7 +960,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 // the solve is the result: x_c = -xs / zt_c as bf16, staged in the q buffer and stored by TMA
                 const float izc = gs->iz[c];
 #pragma unroll
-                for (int g8 = 0; g8 < 16; ++g8) {
+                for (int g8 = 0; g8 < 2 * NG16; ++g8) {
                     uint32_t pk[4];
                     pack_x(g8, false, izc, pk);
                     *reinterpret_cast<uint4 *>(bufc + tile_off(c, g8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
@@ -959,7 +974,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 // alpha-connection (Section 4.3): the read uses alpha x + (1 - alpha) q; q is still in its buffer
                 const float alc = gs->al[c], nzt = valid ? -gs->zt[c] : 0.f;
 #pragma unroll
-                for (int g8 = 0; g8 < 16; ++g8) {
+                for (int g8 = 0; g8 < 2 * NG16; ++g8) {
                     const uint4 qv = *reinterpret_cast<const uint4 *>(bufc + tile_off(c, g8));
                     const uint32_t *qq = reinterpret_cast<const uint32_t *>(&qv);
 #pragma unroll
@@ -976,7 +991,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             // of x that one bf16 rounding would lose): the leading term takes the operand columns, the remainder the
             // first columns of the accumulator, whose content is no longer needed.
 #pragma unroll
-            for (int g8 = 0; g8 < 16; g8 += 2) {
+            for (int g8 = 0; g8 < 2 * NG16; g8 += 2) {
                 uint32_t hi[8], lo[8];
                 pack_x(g8, false, 1.f, *reinterpret_cast<uint32_t(*)[4]>(&hi[0]));
                 pack_x(g8 + 1, false, 1.f, *reinterpret_cast<uint32_t(*)[4]>(&hi[4]));
@@ -998,10 +1013,10 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 // (the iterate's registers are free by now: all four loads are in flight at once)
                 uint32_t r[4][32];
 #pragma unroll
-                for (int p = 0; p < 4; ++p) TMEM_LD32(cx.tm_r + 32 * p, r[p]);
+                for (int p = 0; p < NG16 / 2; ++p) TMEM_LD32(cx.tm_r + 32 * p, r[p]);
                 tmem_wait_ld();
 #pragma unroll
-                for (int p = 0; p < 4; ++p) {
+                for (int p = 0; p < NG16 / 2; ++p) {
 #pragma unroll
                     for (int h4 = 0; h4 < 4; ++h4) {
                         uint32_t pk[4];
@@ -1039,7 +1054,9 @@ cudaError_t launch_fwd_solve(const FwdArgs &a, cudaStream_t stream) {
         !make_state_map(&tmS, a.tile_hu, (unsigned long long)ntiles * 256ull))
         return cudaErrorInvalidValue;
     const bool extra = a.beta != nullptr || a.alpha != nullptr || a.solve_only != 0;
-    auto kernel = extra ? fwd_tc_solve_kernel<true> : fwd_tc_solve_kernel<false>;
+    const bool half = a.d == 64;
+    auto kernel = extra ? (half ? fwd_tc_solve_kernel<true, true> : fwd_tc_solve_kernel<true, false>)
+                        : (half ? fwd_tc_solve_kernel<false, true> : fwd_tc_solve_kernel<false, false>);
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SOLVE_SMEM);
     if (err != cudaSuccess) return err;
     int dev = 0, sms = 0;
