@@ -37,6 +37,10 @@
 // shared memory (one count per warp), completion comes back through tcgen05.commit mbarriers.  What bounds the
 // iterations is the turn of a slot on the score tile (score product, epilogue, second product); stores to tensor
 // memory (about 40 bytes per cycle per SM) are the scarce resource of the epilogues.
+//
+// Head dimension 64 arrives zero-extended to 128 channels (the upper TMA box reads zeros).  The kernel instantiated
+// with HALF leaves out what the zero channels would contribute: contractions over the channels take four k-steps
+// instead of eight, and the passes of the compute warps over the channels stop at channel 64.
 #include <cuda.h>
 
 #include "gka_common.cuh"
