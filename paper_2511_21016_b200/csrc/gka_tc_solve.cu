@@ -222,6 +222,7 @@ __device__ __forceinline__ void issue_batch(int op, bool half, uint32_t kb, uint
         case OP_ITER1:   // S = E Khat^T, R += E H_0^T (the second runs under the masked-score epilogue)
             prod_ek<0>(half, tm_S, tm_E, kb);
             mma_commit(bar_sc);
+            if (half) mma_commit(bar_s);     // (the slot's compute warps take part in the masked-score epilogue)
             prod_ek<1>(half, tm_R, tm_E, hb);
             break;
         case OP_ITER2:   // R += P Khat
@@ -292,8 +293,29 @@ __device__ __forceinline__ void p_convert(const Ctx &cx, const GateScalars *gs, 
     TMEM_ST8(cx.tm_s + 32 * kb, pa);
     TMEM_ST8(cx.tm_s + 32 * kb + 8, pb);
 }
-template <bool EXACT, bool KEYF>
+// Head dimension 64: key blocks of the masked scores that a token's score warp converts in an iteration; the token's
+// compute warp, which has nothing else to do until the product that consumes the masked scores is complete, converts
+// the rest.
+__device__ __forceinline__ int p_split(int q) { return (q + 2) >> 1; }
+// The masked-score epilogue of an iteration for the key blocks kb0 <= kb < kb1 of this thread's token.
+template <bool EXACT>
+__device__ __forceinline__ void p_epilogue_blocks(const Ctx &cx, const GateScalars *gs, float ac_c, int kb0, int kb1) {
+#pragma unroll 1
+    for (int kb = kb0; kb < kb1; ++kb) {
+        uint32_t ra[16], rb[16];
+        TMEM_LD16(cx.tm_s + 32 * kb, ra);
+        TMEM_LD16(cx.tm_s + 32 * kb + 16, rb);
+        tmem_wait_ld();
+        p_convert<EXACT, false>(cx, gs, ac_c, kb, ra, rb);
+    }
+    tmem_wait_st();
+}
+template <bool EXACT, bool KEYF, bool SPLIT>
 __device__ __forceinline__ void p_epilogue_t(const Ctx &cx, const GateScalars *gs, float ac_c) {
+    if (!KEYF && SPLIT) {     // an iteration: the upper key blocks are left to the token's compute warp
+        p_epilogue_blocks<EXACT>(cx, gs, ac_c, 0, p_split(cx.q));
+        return;
+    }
     if (KEYF) {      // (the product of an iteration leaves out the rows whose key block is above the diagonal instead)
         uint32_t z[8];
 #pragma unroll
@@ -314,10 +336,10 @@ __device__ __forceinline__ void p_epilogue_t(const Ctx &cx, const GateScalars *g
     }
     tmem_wait_st();
 }
-template <bool KEYF>
+template <bool KEYF, bool SPLIT>
 __device__ __forceinline__ void p_epilogue(const Ctx &cx, const GateScalars *gs, bool exact, float ac_c) {
-    if (exact) p_epilogue_t<true, KEYF>(cx, gs, ac_c);
-    else p_epilogue_t<false, KEYF>(cx, gs, ac_c);
+    if (exact) p_epilogue_t<true, KEYF, SPLIT>(cx, gs, ac_c);
+    else p_epilogue_t<false, KEYF, SPLIT>(cx, gs, ac_c);
 }
 
 // Sum over one 32-key block of the squared Gram entries of the earlier keys (decayed when the keys are not
@@ -405,6 +427,9 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const float *const beta_p = EXTRA ? a.beta : nullptr;
     const float *const alpha_p = EXTRA ? a.alpha : nullptr;
     const bool mix = alpha_p != nullptr && !solve_only;   // alpha-connection: the read uses alpha x + (1 - alpha) q
+    // Head dimension 64: the slot's compute warps, idle while the slot has the score tile, convert the upper key blocks of
+    // the masked scores of an iteration (with 128 channels this measured slower: the warps come later to their update)
+    constexpr bool SPLIT = HALF;
     constexpr bool half = HALF;                           // head dimension 64: channels 64..127 are zero, their k-steps are left out
 
     // The helper warps come first: when a scheduler changes warps it prefers the oldest eligible one, and the thread
@@ -543,7 +568,8 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 auto book = [&](int sl, int o) -> uint32_t {
                     bool tile_done = false;
                     int it = sl ? it1 : it0, nop;
-                    const uint32_t thr = (sl ? thr1 : thr0) + 4u;
+                    // (the masked scores of an iteration come from the score warps and the slot's compute warps)
+                    const uint32_t thr = (sl ? thr1 : thr0) + (SPLIT && o == OP_ITER1 ? 8u : 4u);
                     if (o == OP_FROB) {
                         owner = sl;                          // until the Gram matrix has been read
                         nop = it < a.n_iter ? OP_ITER1 : OP_OUT_S;
@@ -614,6 +640,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         const bool t_iter = (t ? left1 : left0) > 0 && (t ? op1 : op0) == OP_ITER1;
                         const uint32_t thr_t = t ? thr1 : thr0;
                         const uint32_t n_kb = t14 + (BUF_A >> 4), n_tmE = tmem + tm_e_of(t);
+                        const uint32_t n_barS = bars + 8 * (t * B_PER_SLOT + B_MMA_S);
                         const uint32_t n_info = (uint32_t)t | (((t ? til1 : til0) & 1u) << 2) | ((sev + 1u) << 8);
                         const uint32_t n_sinfo = sinfo_addr + 4u * (sev & 1u);
                         uint32_t c_t = 0u;
@@ -657,6 +684,7 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         fence_after();
                         prod_ek<0>(half, tmem + TM_S, n_tmE, n_kb);           // S = E Khat^T
                         mma_commit(bars + 8 * B_SC);
+                        if (SPLIT) mma_commit(n_barS);
                         prod_ek<1>(half, tmem + tm_r_of(t), n_tmE, n_kb + ((BUF_B - BUF_A) >> 4));   // R += E H_0^T
                         if (owner == t) {                        // (its Gram reads are done: it has asked again)
                             if (t) gthr1 += 4u; else gthr0 += 4u;
@@ -723,9 +751,9 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     tma_load_tile3(&tmK, sbase + sl_ * SLOT_BYTES + BUF_A, bar_k, tn.h * a.d, tile_x_hi(tn.h, a.d, a.heads), tn.n * NT, tn.b);
                 }
                 if (sl_) ++reads1; else ++reads0;
-                p_epilogue<true>(cx, gs, exact, ac_c);
+                p_epilogue<true, SPLIT>(cx, gs, exact, ac_c);
             } else {
-                p_epilogue<false>(cx, gs, exact, ac_c);
+                p_epilogue<false, SPLIT>(cx, gs, exact, ac_c);
             }
             fence_before();
             warp_post(smem_u32(&s_req[sl_]), cx.l);          // -> ITER2 / OUT_O of that slot
@@ -919,6 +947,14 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 omega = 4.f / (4.f - rho2 * omega);              // weight schedule
                 const float beta = omega - 1.f, cz = czb * omega;
                 const uint64_t beta2 = f2_pack(beta, beta), cz2 = f2_pack(cz, cz), lz2 = f2_pack(lz, lz);
+                // this warp's share of the masked-score epilogue (the upper key blocks of its tokens)
+                if (SPLIT) {
+                    wait_s();
+                    if (exact) p_epilogue_blocks<true>(cx, gs, gs->ac[c], p_split(cx.q), cx.q + 1);
+                    else p_epilogue_blocks<false>(cx, gs, 0.f, p_split(cx.q), cx.q + 1);
+                    fence_before();
+                    arrive_rdy();                                // -> ITER2 (with the score warps' posts)
+                }
                 wait_r();
                 if (last) after_last_h0_product();
                 // e_new = beta e_old + cz (R + lz xs) as bf16, xs += e_new (the value the operand holds).  Sixteen
