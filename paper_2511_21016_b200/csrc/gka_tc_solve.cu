@@ -344,19 +344,19 @@ __device__ __forceinline__ void p_epilogue(const Ctx &cx, const GateScalars *gs,
 
 // Sum over one 32-key block of the squared Gram entries of the earlier keys (decayed when the keys are not
 // pre-scaled) and the key's own squared norm.
-template <bool DIAG>
-__device__ __forceinline__ void gram_block(const uint32_t (&r)[32], const float *G2kb, float G2j, bool exact, int l, float &gsum) {
-    float gs2 = 0.f, gd = 0.f;
+template <bool DIAG, bool EXACT>
+__device__ __forceinline__ void gram_block(const uint32_t (&r)[32], const float *G2kb, float G2j, int l, float &gsum) {
+    float acc[4] = {0.f, 0.f, 0.f, 0.f}, gd = 0.f;      // four partial sums: the additions do not wait for one another
 #pragma unroll
     for (int ii = 0; ii < 32; ++ii) {
         const float g = __uint_as_float(r[ii]);
         const float g2 = g * g;
-        if (DIAG && ii == l) gd = g2;
-        const bool in = !DIAG || ii < l;
-        if (!exact) gs2 += in ? g2 : 0.f;
-        else if (in) gs2 = fmaf(ex2_fast(G2j - G2kb[ii]), g2, gs2);
+        if (DIAG) gd = ii == l ? g2 : gd;
+        float w = EXACT ? ex2_fast(G2j - G2kb[ii]) * g2 : g2;
+        if (DIAG) w = ii < l ? w : 0.f;
+        acc[ii & 3] += w;
     }
-    gsum += 2.f * gs2 + gd;
+    gsum += 2.f * ((acc[0] + acc[1]) + (acc[2] + acc[3])) + gd;
 }
 
 // Inclusive scan over the tile's 128 tokens (the slot's four warps, one token per thread) of the affine maps
@@ -866,14 +866,20 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             // the earlier keys
             float kh = 0.f, gsum = 0.f;
             {
+                float khp[4] = {0.f, 0.f, 0.f, 0.f};
                 uint32_t ra[32];
                 // (the Gram matrix first: it sits in the score tile, which the other slot is waiting for)
 #pragma unroll 1
                 for (int kb = 0; kb <= cx.q; ++kb) {
                     TMEM_LD32(cx.tm_s + 32 * kb, ra);
                     tmem_wait_ld();
-                    if (kb == cx.q) gram_block<true>(ra, gs->G2 + 32 * kb, G2c, exact, l, gsum);
-                    else gram_block<false>(ra, gs->G2 + 32 * kb, G2c, exact, l, gsum);
+                    if (exact) {
+                        if (kb == cx.q) gram_block<true, true>(ra, gs->G2 + 32 * kb, G2c, l, gsum);
+                        else gram_block<false, true>(ra, gs->G2 + 32 * kb, G2c, l, gsum);
+                    } else {
+                        if (kb == cx.q) gram_block<true, false>(ra, gs->G2 + 32 * kb, G2c, l, gsum);
+                        else gram_block<false, false>(ra, gs->G2 + 32 * kb, G2c, l, gsum);
+                    }
                 }
                 fence_before();
                 warp_post(grd_addr, l);                          // the Gram matrix has been read: S is free again
@@ -889,11 +895,12 @@ fwd_tc_solve_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                         const uint32_t *pk = reinterpret_cast<const uint32_t *>(&kv[h4]);
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
-                            kh = fmaf(__uint_as_float(ra[8 * h4 + 2 * u]), bf16_lo(pk[u]), kh);
-                            kh = fmaf(__uint_as_float(ra[8 * h4 + 2 * u + 1]), bf16_hi(pk[u]), kh);
+                            khp[h4] = fmaf(__uint_as_float(ra[8 * h4 + 2 * u]), bf16_lo(pk[u]), khp[h4]);
+                            khp[h4] = fmaf(__uint_as_float(ra[8 * h4 + 2 * u + 1]), bf16_hi(pk[u]), khp[h4]);
                         }
                     }
                 }
+                kh = (khp[0] + khp[1]) + (khp[2] + khp[3]);
             }
             // ---- f_c by an affine scan (s_c = gamma_c^2 s_{c-1} + d_c, s_{-1} = ||H_0||^2), Chebyshev set-up
             float rho2, czb, lz;
