@@ -44,7 +44,7 @@ L2_FLUSH_BYTES = 256 << 20
 # ncu captures summarised under profiles/).  Both captures ran a half / quarter-size case of the same kernel
 # (solve kernel: 1024 of 2048 tiles; decode: 2048 of 8192 (sequence, head) pairs) and are scaled by the
 # units per launch; traffic is proportional to the units in both kernels.
-NCU_TRAFFIC_BYTES = {"fwd_solve_per_tile": (169_233_408 + 15_460_352) / 1024, "decode": 4 * 482_096_896}
+NCU_TRAFFIC_BYTES = {"fwd_solve_per_tile": (169_212_672 + 16_138_240) / 1024, "decode": 4 * 482_096_896}
 
 
 def fwd_flops(n_chunks: int, n_iter: int, C: int = 64, D: int = 128, part: str = "all") -> float:
