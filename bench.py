@@ -6,7 +6,8 @@ norms, Chebyshev iterations, output, state carry) over one batch of configuratio
 (B=4, heads=16, T=4096, d=128, chunk=64, n_iter=10, bf16 I/O).  The recurrent decode step
 (configuration 2: 256 sequences x 32 heads, fp32 state) is timed in the same run and reported
 in the "decode" object of the same JSON line, next to "fwd_r30" (the same shapes at the paper's
-setting: 30 iterations, lambda_t = 0.02 ||H_t||_F) and "fwd_long" (configuration 3, T = 131072).
+setting: 30 iterations, lambda_t = 0.02 ||H_t||_F), "fwd_d64" (the same shapes at head dimension 64) and "fwd_long"
+(configuration 3, T = 131072).
 
     python bench.py --gpus N --steps K --warmup W            # this library
     python bench.py --impl reference --steps K --warmup W    # the fp64 CPU oracle, bounded sample
@@ -405,6 +406,22 @@ def run_ours(args):
                                                    "lam": "adaptive, a = 0.02", "io_dtype": cfg.io_dtype},
                            "roofline": r30["roofline"], "gpu_launches": launches_per_step * K2}
         del r30, dev30
+        # ---- head dimension 64 on configuration 1's shapes (the tensor path's four-k-step instantiation), inputs drawn
+        # on the device; no ncu capture of this instantiation exists, so its traffic is not reported
+        if world == 1:
+            import dataclasses
+            cfg64 = dataclasses.replace(cfg, d=64)
+            K4 = min(K, 50)
+            dev64 = make_fwd_inputs_device(cfg64, device, cfg64.seed)
+            r64 = time_forward(gka, dev64, cfg64, cfg64.n_iter, 0, K4, W, peaks, stream, new_event, flush, 1, device)
+            r64["roofline"]["traffic"] = None
+            line["fwd_d64"] = {"metric": METRIC, "value": r64["value"], "unit": UNIT, "ms_per_step": r64["ms_per_step"],
+                               "steps": K4, "config": {"workload": "cfg1 shapes at head dimension 64", "B": cfg64.B,
+                                                       "heads": cfg64.heads, "T": cfg64.T, "d": 64, "n_iter": cfg64.n_iter,
+                                                       "io_dtype": cfg64.io_dtype, "inputs": "drawn on the device"},
+                               "roofline": r64["roofline"], "gpu_launches": launches_per_step * K4}
+            del r64, dev64
+            torch.cuda.empty_cache()
         # ---- long context (configuration 3), inputs drawn on the device
         if world == 1:
             cfg3 = synth.CONFIGS[3]
@@ -582,7 +599,7 @@ def main():
     ap.add_argument("--config", type=int, default=1, help="forward configuration to time (1 or 3, 4)")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-extra", action="store_true", help="skip the fwd_r30 and fwd_long objects")
+    ap.add_argument("--no-extra", action="store_true", help="skip the fwd_r30, fwd_d64 and fwd_long objects")
     ap.add_argument("--case", nargs="+", help="run one small case a few times instead of the benchmark (see run_case)")
     args = ap.parse_args()
     if args.case:
