@@ -40,7 +40,9 @@
 //
 // Head dimension 64 arrives zero-extended to 128 channels (the upper TMA box reads zeros).  The kernel instantiated
 // with HALF leaves out what the zero channels would contribute: contractions over the channels take four k-steps
-// instead of eight, and the passes of the compute warps over the channels stop at channel 64.
+// instead of eight, and the passes of the compute warps over the channels stop at channel 64.  Its turns on the score
+// tile are shorter, so the masked-score epilogue weighs more: there the slot's compute warps, idle during the turn,
+// convert the upper key blocks of their tokens and the score warps the lower ones.
 #include <cuda.h>
 
 #include "gka_common.cuh"
