@@ -157,6 +157,17 @@ int gka_fwd_num_work_items(const gka_desc *desc, int chunk) {
     const int sms = sm_count();
     if (sms <= 0) return -(int)GKA_ERR_CUDA;
     const int cap = work_items_cap(desc, chunk);
+    if (wants_tensor_path(desc)) {
+        // Fewer (sequence, head) pairs than SMs: with one range per SM nearly every range ends inside a sequence and the
+        // summary kernel reads all keys and values once more.  Whole sequences as work items need no summaries; they
+        // leave SMs idle in the state kernel and make its run of tiles longer.  Measured per 128-token tile and block:
+        // 2.94 us in the state kernel with whole sequences (2.43 us where two blocks share a sequence, one per master:
+        // at most half as many pairs as SMs), 5.12 us x pairs / SMs for the summary and state kernels with one range
+        // per SM, which also cost 28 us more per call.
+        const long long pairs = (long long)desc->B * desc->heads, n = tiles_of(desc->T);
+        const double per_tile = 2 * pairs <= sms ? 2.43 : 2.94;
+        if (pairs < sms && pairs <= cap && (double)n * (per_tile - 5.12 * (double)pairs / sms) < 28.0) return (int)pairs;
+    }
     return sms < cap ? sms : cap;
 }
 
@@ -215,6 +226,7 @@ static gka_status fwd_impl(const gka_desc *desc, const void *q, const void *k, c
     a.flags = desc->flags;
     a.solve_only = solve_only ? 1 : 0;
     a.start_from_scan = 0;
+    a.state_split = 0;
     a.after_summary = 0;
     const bool tensor_path = wants_tensor_path(desc) && fwd_tc_available();
     a.tile_hh = nullptr;

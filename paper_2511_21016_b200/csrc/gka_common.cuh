@@ -214,6 +214,7 @@ struct FwdArgs {
     unsigned flags;
     int after_summary;     // tensor path: the main kernel is launched as a programmatic dependent of the summary kernel
     int start_from_scan;   // tensor path: start states were materialised by the scan kernel (long chains of summaries)
+    int state_split;       // tensor path, no sequence cut: two blocks per work item in the state kernel, one for H, one for U
     int solve_only;        // write the solve x_t = CH(H_t + lambda_t I, q_t, r) itself instead of U_t x_t (v unused)
     WorkPlan plan;
     Workspace ws;

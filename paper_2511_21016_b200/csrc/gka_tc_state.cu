@@ -44,9 +44,10 @@ constexpr uint32_t KV_SMEM = NS * STAGE + 1024;          // + slack for the 1024
 constexpr uint32_t ST_SMEM = KV_SMEM;
 
 // rows of the K and V tiles of a stage times f[j]
-__device__ __forceinline__ void scale_kv(unsigned char *stage, const float *f, int t) {
+__device__ __forceinline__ void scale_kv(unsigned char *stage, const float *f, int t, bool with_v = true) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
+        if (i >= 4 && !with_v) break;              // (the K tile is the first half of the stage)
         const int qi = t + CT * i;                 // 16-byte group index in the 64 KB stage
         const float fj = f[(qi & 1023) >> 3];      // row of this group (K and V tiles alike)
         uint4 v = *reinterpret_cast<const uint4 *>(stage + qi * 16);
@@ -247,13 +248,14 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 // then polled looked incomplete, and the compute warps in turn waited for the load that only this thread issues.)
 enum { TB_KV0 = 0, TB_D0 = NS, TB_D1, TB_STG0, TB_COUNT = TB_STG0 + NS };
 
+template <bool SPLIT>
 __global__ void __launch_bounds__(kThreadsStateK, 1)
 fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmS, FwdArgs a) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t s_bars[TB_COUNT];
     __shared__ uint32_t s_tmem_base;
-    __shared__ float s_w[NT], s_ca[4], s_red[2][16], s_decay[2];
+    __shared__ float s_w[NT], s_ca[4], s_red[3][16], s_decay[3];
     __shared__ int s_req, s_abort;
     unsigned char *smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     const uint32_t sb = smem_u32(smem), bars = smem_u32(&s_bars[0]);
@@ -277,7 +279,11 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     fence_after();
     const uint32_t tmem = s_tmem_base;
     const WorkPlan &P = a.plan;
-    const int item = blockIdx.x;
+    // With no sequence cut and few work items the masters are split: two blocks per item, one advances H (and needs
+    // only the keys), one U.  Each handles the masters w_lo <= which < w_hi.
+    const int item = SPLIT ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int w_lo = SPLIT ? (int)(blockIdx.x & 1) : 0, w_hi = SPLIT ? w_lo + 1 : 2;
+    const bool do_h = w_lo == 0, do_u = w_hi == 2;
     const long long f_lo = P.lo(item), f_hi = P.lo(item + 1);
     const int n_mine = (int)(f_hi - f_lo);
     const uint32_t base14 = (sb >> 4) & 0x3FFF;
@@ -308,9 +314,9 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             auto issue_tma = [&](int m) {
                 const Pos p = pos_of(m);
                 const uint32_t dst = sb + (uint32_t)(m % NS) * STAGE, bar = bars + 8 * (TB_KV0 + m % NS);
-                mbar_expect_tx(bar, 65536u);
+                mbar_expect_tx(bar, do_u ? 65536u : 32768u);
                 tma_load_tile3(&tmK, dst, bar, p.h * a.d, tile_x_hi(p.h, a.d, a.heads), p.n * NT, p.b);
-                tma_load_tile3(&tmV, dst + 32768, bar, p.h * a.d, tile_x_hi(p.h, a.d, a.heads), p.n * NT, p.b);
+                if (do_u) tma_load_tile3(&tmV, dst + 32768, bar, p.h * a.d, tile_x_hi(p.h, a.d, a.heads), p.n * NT, p.b);
             };
             for (int m = 0; m < n_mine && m < NS; ++m) issue_tma(m);
             for (int m = 0; m < n_mine; ++m) {
@@ -318,7 +324,7 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 // products are complete): store them, then the stage takes the tile three further on
                 wait(TB_STG0 + m % NS, (uint32_t)((m / NS) & 1));
                 const uint32_t src = sb + (uint32_t)(m % NS) * STAGE;
-                for (int which = 0; which < 2; ++which)
+                for (int which = w_lo; which < w_hi; ++which)
                     for (int hf = 0; hf < 2; ++hf)
                         asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::
                                          "l"(reinterpret_cast<uint64_t>(&tmS)), "r"(64 * hf), "r"((int)((f_lo + m) * 256 + 128 * which)),
@@ -342,8 +348,8 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 fence_after();
                 const uint32_t kb = base14 + (uint32_t)(m % NS) * (STAGE >> 4), vb = kb + (32768u >> 4);
                 const uint32_t tm_d = tmem + 256 * (m & 1);
-                mma8_mm<0>(tm_d, kb, kb, kIdescMM);              // dH = K~^T K~
-                mma8_mm<0>(tm_d + 128, vb, kb, kIdescMM);        // dU = V~^T K~
+                if (do_h) mma8_mm<0>(tm_d, kb, kb, kIdescMM);              // dH = K~^T K~
+                if (do_u) mma8_mm<0>(tm_d + 128, vb, kb, kIdescMM);        // dU = V~^T K~
                 mma_commit(bars + 8 * (TB_D0 + (m & 1)));
             }
             __syncwarp();
@@ -393,11 +399,11 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 }
                 incl += before;
                 s_w[t] = sqrtf(bt) * exp2f(0.5f * (tile_total - incl));
-                if (t == 0) s_decay[m & 1] = exp2f(tile_total);
+                if (t == 0) s_decay[m % 3] = exp2f(tile_total);     // (three deep: thread 0 writes tile m + 2's while slower warps may still read tile m's)
             }
             wait(TB_KV0 + m % NS, (uint32_t)((m / NS) & 1));
             asm volatile("bar.sync 1, 512;" ::: "memory");       // factors are published
-            scale_kv(smem + (size_t)(m % NS) * STAGE, s_w, t);
+            scale_kv(smem + (size_t)(m % NS) * STAGE, s_w, t, do_u);
             fence_async_smem();
             fence_before();
             if (t == 0) *reinterpret_cast<volatile int *>(&s_req) = m;
@@ -434,6 +440,7 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 const bool in_ext = c < a.d && 32 * cq < a.d;
 #pragma unroll
                 for (int which = 0; which < 2; ++which) {
+                    if (which < w_lo || which >= w_hi) continue;
                     float(&mm)[32] = which ? mU : mH;
                     const size_t eo = e + which * (size_t)D * D;
 #pragma unroll
@@ -461,10 +468,11 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             // own K (V) in operand layout and goes from there to the workspace by TMA; then its increments are added
             wait(TB_D0 + (m & 1), (uint32_t)((m >> 1) & 1));     // the tile's increments are complete (posted a tile ago)
             fence_after();
-            const float decay = s_decay[m & 1];
+            const float decay = s_decay[m % 3];
             unsigned char *const stg = smem + (size_t)(m % NS) * STAGE;   // the tile's own K and V are no longer needed
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
+                if (which < w_lo || which >= w_hi) continue;
                 float(&mm)[32] = which ? mU : mH;
                 float hs = 0.f;
 #pragma unroll
@@ -481,9 +489,9 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 if (which == 0) {
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) hs += __shfl_xor_sync(0xffffffffu, hs, o);
-                    if (l == 0) s_red[m & 1][t >> 5] = hs;
+                    if (l == 0) s_red[m % 3][t >> 5] = hs;
                 }
-                if (which == 1) {
+                if (which == w_hi - 1) {
                     fence_async_smem();
                     __syncwarp();
                     if (l == 0) mbar_arrive(bars + 8 * (TB_STG0 + m % NS));  // -> the TMA thread stores both copies
@@ -504,27 +512,32 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 float *so = a.state_out + (size_t)p.seq * 2 * a.d * a.d + (size_t)c * a.d + 32 * cq;
 #pragma unroll
                 for (int which = 0; which < 2; ++which) {
+                    if (which < w_lo || which >= w_hi) continue;
                     const float(&mm)[32] = which ? mU : mH;
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
                         *reinterpret_cast<float4 *>(so + which * (size_t)a.d * a.d + 4 * i) = make_float4(mm[4 * i], mm[4 * i + 1], mm[4 * i + 2], mm[4 * i + 3]);
                 }
             }
-            // ||H_0||_F^2 of the previous tile: its per-warp sums were written before this tile's hand-over barrier
-            if (t == 0 && m >= 1) {
+            // ||H_0||_F^2 of the previous tile: its per-warp sums were written before this tile's hand-over barrier (the
+            // block's last tile has none: the sums of the last two tiles are read after the loop).  Three sets of sums,
+            // so that a warp that runs a tile ahead writes none that is still to be read.
+            if (t == 0 && m >= 1 && m + 1 < n_mine && do_h) {
                 float hh = 0.f;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) hh += s_red[(m - 1) & 1][i];
+                for (int i = 0; i < 16; ++i) hh += s_red[(m - 1) % 3][i];
                 a.tile_hh[tile - 1] = hh;
             }
         }
         if (t == 0) *reinterpret_cast<volatile int *>(&s_req) = -1;
         asm volatile("bar.sync 3, 544;" ::: "memory");           // releases the issuing warp; the last sums are published
         if (t == 0) {
-            float hh = 0.f;
+            for (int m = n_mine >= 2 ? n_mine - 2 : n_mine - 1; m < n_mine && do_h; ++m) {
+                float hh = 0.f;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) hh += s_red[(n_mine - 1) & 1][i];
-            a.tile_hh[f_lo + n_mine - 1] = hh;
+                for (int i = 0; i < 16; ++i) hh += s_red[m % 3][i];
+                a.tile_hh[f_lo + m] = hh;
+            }
             if (s_abort != 0 && a.device_status) atomicExch(a.device_status, (int)GKA_ERR_TIMEOUT);
         }
     } else {
@@ -557,6 +570,11 @@ cudaError_t launch_fwd_tc(const FwdArgs &a_in, cudaStream_t stream) {
     // work items) would make every block re-read its whole chain, so the scan kernel materialises the start
     // states once instead.
     a.start_from_scan = longest > 4 ? 1 : 0;
+    int sms_here = 0, dev_here = 0;
+    if ((err = cudaGetDevice(&dev_here)) != cudaSuccess) return err;
+    if ((err = cudaDeviceGetAttribute(&sms_here, cudaDevAttrMultiProcessorCount, dev_here)) != cudaSuccess) return err;
+    // two blocks per work item (one per master) where no sequence is cut and the blocks still fit one per SM
+    a.state_split = (!any_cut && 2 * a.plan.G <= sms_here) ? 1 : 0;
     alignas(64) CUtensorMap tmK, tmV, tmS;      // boxes of 128 tokens x 64 channels; per-tile bf16 state copies
     const int cols = a.heads * a.d;
     if (!make_tile_map(&tmK, a.k, a.B, a.T, cols, NT) || !make_tile_map(&tmV, a.v, a.B, a.T, cols, NT) ||
@@ -572,11 +590,12 @@ cudaError_t launch_fwd_tc(const FwdArgs &a_in, cudaStream_t stream) {
         }
         a.after_summary = 1;
     }
-    err = cudaFuncSetAttribute(fwd_tc_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ST_SMEM);
+    auto state_kernel = a.state_split ? fwd_tc_state_kernel<true> : fwd_tc_state_kernel<false>;
+    err = cudaFuncSetAttribute(state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ST_SMEM);
     if (err != cudaSuccess) return err;
     {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)a.plan.G);
+        cfg.gridDim = dim3((unsigned)(a.plan.G * (a.state_split ? 2 : 1)));
         cfg.blockDim = dim3(kThreadsStateK);
         cfg.dynamicSmemBytes = ST_SMEM;
         cfg.stream = stream;
@@ -585,7 +604,7 @@ cudaError_t launch_fwd_tc(const FwdArgs &a_in, cudaStream_t stream) {
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = a.after_summary ? 1 : 0;
-        err = cudaLaunchKernelEx(&cfg, fwd_tc_state_kernel, tmK, tmV, tmS, a);
+        err = cudaLaunchKernelEx(&cfg, state_kernel, tmK, tmV, tmS, a);
         if (err != cudaSuccess) return err;
     }
     return launch_fwd_solve(a, stream);

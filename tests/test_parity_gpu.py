@@ -270,6 +270,28 @@ def test_fwd_back_to_back_calls_share_a_workspace():
     assert torch.equal(alone, after) and torch.equal(st_alone, st_after)
 
 
+@pytest.mark.parametrize("B,heads,T,d", [(2, 5, 640, 128), (2, 5, 640, 64), (1, 40, 2000, 128), (8, 16, 1000, 128),
+                                         (2, 5, 3840, 128)])
+def test_fwd_bf16_native_repeated_calls_are_bit_identical(B, heads, T, d):
+    """The same problem several times over, one workspace: outputs and final states must agree bit for bit in every
+    decomposition of the state pass (whole sequences with one block per master, whole sequences with one block each,
+    ranges that cut sequences), and the first call must agree with the oracle."""
+    cfg = synth.shrink(synth.CONFIGS[1], B=B, heads=heads, T=T, d=d, n_iter=3, seed=31)
+    inp = synth.make_inputs(cfg)
+    dev = [to_dev(inp[n], n in ("q", "k", "v")) for n in ("q", "k", "v", "gate", "lam")]
+    ws = gka.alloc_workspace(B, T, heads, d, DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    first, st_first = gka.gka_fwd_chunked(*dev, 3, 64, workspace=ws, device_status=status)
+    torch.cuda.synchronize()
+    ref = oracle.fwd(inp["q"], inp["k"], inp["v"], inp["gate"], inp["lam"], 3)
+    assert rel(first.float().cpu().numpy(), ref["out"]) <= TOL_BF16
+    for _ in range(6):
+        again, st_again = gka.gka_fwd_chunked(*dev, 3, 64, workspace=ws, device_status=status)
+        torch.cuda.synchronize()
+        assert torch.equal(first, again) and torch.equal(st_first, st_again)
+    assert int(status.item()) == 0
+
+
 def test_fwd_gpu_argument_errors():
     q = torch.zeros(1, 100, 1, 64, device=DEV)
     v = torch.zeros(1, 100, 1, 128, device=DEV)
