@@ -129,6 +129,18 @@ def test_work_ranges_partition_the_chunk_list(lib, B, T, heads, G, io):
         gka.gka_fwd_work_range(B, T, heads, 128, G, G)
 
 
+@pytest.mark.parametrize("B,T,heads", [(4, 4096, 16), (2, 640, 5), (1, 2000, 40), (3, 100, 7)])
+def test_whole_sequences_as_work_items_cut_nothing(lib, B, T, heads):
+    """With as many work items as (sequence, head) pairs (the decomposition the tensor-core path takes when carrying
+    whole sequences is cheaper than cutting them) every range is one sequence: no range starts or ends inside one."""
+    N = (T + 63) // 64
+    pairs = B * heads
+    for i in range(pairs):
+        lo, hi, cin, cout = gka.gka_fwd_work_range(B, T, heads, 128, pairs, i, io_dtype=gka.GKA_BF16)
+        assert (lo, hi) == (i * N, (i + 1) * N)
+        assert not cin and not cout
+
+
 def test_missing_library_is_an_error(monkeypatch, tmp_path):
     monkeypatch.setattr(gka, "_lib", None)
     monkeypatch.setattr(gka, "LIB_PATH", str(tmp_path / "nope.so"))
