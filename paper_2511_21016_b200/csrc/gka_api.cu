@@ -158,15 +158,21 @@ int gka_fwd_num_work_items(const gka_desc *desc, int chunk) {
     if (sms <= 0) return -(int)GKA_ERR_CUDA;
     const int cap = work_items_cap(desc, chunk);
     if (wants_tensor_path(desc)) {
-        // Fewer (sequence, head) pairs than SMs: with one range per SM nearly every range ends inside a sequence and the
-        // summary kernel reads all keys and values once more.  Whole sequences as work items need no summaries; they
-        // leave SMs idle in the state kernel and make its run of tiles longer.  Measured per 128-token tile and block:
-        // 2.94 us in the state kernel with whole sequences (2.43 us where two blocks share a sequence, one per master:
-        // at most half as many pairs as SMs), 5.12 us x pairs / SMs for the summary and state kernels with one range
-        // per SM, which also cost 28 us more per call.
+        // Where the ranges cut sequences the summary kernel reads all keys and values once more.  Ranges of whole
+        // sequences (pairs / k work items of k sequences each, k the smallest divisor of the number of (sequence, head)
+        // pairs that leaves at most one item per SM) need no summaries, but may leave SMs idle in the state kernel and
+        // make its run of tiles longer.  Measured per 128-token tile and block: 2.94 us in the state kernel with whole
+        // sequences (2.43 us where two blocks share an item, one per master: at most half as many items as SMs),
+        // 5.12 us x pairs / SMs for the summary and state kernels with one range per SM, which also cost 28 us more
+        // per call.
         const long long pairs = (long long)desc->B * desc->heads, n = tiles_of(desc->T);
-        const double per_tile = 2 * pairs <= sms ? 2.43 : 2.94;
-        if (pairs < sms && pairs <= cap && (double)n * (per_tile - 5.12 * (double)pairs / sms) < 28.0) return (int)pairs;
+        for (long long k = (pairs + sms - 1) / sms; k <= pairs && k <= 64; ++k) {
+            if (pairs % k != 0 || pairs / k > cap) continue;
+            const long long items = pairs / k;
+            const double per_tile = 2 * items <= sms ? 2.43 : 2.94;
+            if ((double)n * ((double)k * per_tile - 5.12 * (double)pairs / sms) < 28.0) return (int)items;
+            break;
+        }
     }
     return sms < cap ? sms : cap;
 }

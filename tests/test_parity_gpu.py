@@ -271,11 +271,12 @@ def test_fwd_back_to_back_calls_share_a_workspace():
 
 
 @pytest.mark.parametrize("B,heads,T,d", [(2, 5, 640, 128), (2, 5, 640, 64), (1, 40, 2000, 128), (8, 16, 1000, 128),
-                                         (2, 5, 3840, 128)])
+                                         (2, 5, 3840, 128), (4, 40, 200, 128)])
 def test_fwd_bf16_native_repeated_calls_are_bit_identical(B, heads, T, d):
     """The same problem several times over, one workspace: outputs and final states must agree bit for bit in every
     decomposition of the state pass (whole sequences with one block per master, whole sequences with one block each,
-    ranges that cut sequences), and the first call must agree with the oracle."""
+    ranges that cut sequences, more pairs than SMs with two whole sequences per work item), and the first call must
+    agree with the oracle."""
     cfg = synth.shrink(synth.CONFIGS[1], B=B, heads=heads, T=T, d=d, n_iter=3, seed=31)
     inp = synth.make_inputs(cfg)
     dev = [to_dev(inp[n], n in ("q", "k", "v")) for n in ("q", "k", "v", "gate", "lam")]
