@@ -204,10 +204,10 @@ const char *gka_last_error_detail(void);
  * Work decomposition of the chunked forward, for callers that size buffers or report launch
  * counts: number of work items (contiguous ranges of the flat chunk list) of the state pass for this
  * descriptor on the current device, or a negative gka_status.  Normally one per SM (fewer for small problems).
- * On the tensor-core path with fewer (sequence, head) pairs than SMs it is the number of pairs whenever
- * carrying whole sequences is cheaper than cutting them (no range then starts or ends inside a sequence and
- * no summary or scan kernel runs); with at most half as many pairs as SMs the state kernel then runs two
- * thread blocks per work item, one per state matrix.
+ * On the tensor-core path it is pairs / k for a small divisor k of the number of (sequence, head) pairs
+ * (k = 1 with fewer pairs than SMs) whenever carrying whole sequences is cheaper than cutting them: no range then
+ * starts or ends inside a sequence and no summary or scan kernel runs; with at most half as many work items as
+ * SMs the state kernel then runs two thread blocks per work item, one per state matrix.
  */
 int gka_fwd_num_work_items(const gka_desc *desc, int chunk);
 
