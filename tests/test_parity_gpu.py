@@ -293,6 +293,25 @@ def test_fwd_bf16_native_repeated_calls_are_bit_identical(B, heads, T, d):
     assert int(status.item()) == 0
 
 
+def test_work_items_follow_the_decomposition_rule():
+    """Number of work items of the state pass on this device: whole sequences where that is cheaper than cutting them
+    (fewer pairs than SMs and short enough sequences; more pairs than SMs with a small divisor), one range per SM
+    otherwise; the fp32 path always takes one range per SM (or one per chunk for small problems)."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    n = gka.gka_fwd_num_work_items
+    assert n(4, 4096, 16, 128) == 64                       # configuration 1: the 64 pairs
+    assert n(1, 131072, 32, 128) == min(sms, 32 * 1024)    # configuration 3: long sequences are cut
+    if sms == 148:
+        assert n(16, 2048, 16, 128) == 128                 # 256 pairs: 128 items of two sequences
+        assert n(2, 3840, 5, 128) == 148                   # 10 pairs of 30 tiles: cut
+    assert n(4, 4096, 16, 128, io_dtype=gka.GKA_F32) == min(sms, 4 * 16 * 64)
+    for B, T, heads in ((4, 4096, 16), (16, 2048, 16), (2, 640, 5)):
+        G = n(B, T, heads, 128)
+        if G < sms and (B * heads) % G == 0:               # whole sequences: nothing is cut
+            for i in range(G):
+                assert gka.gka_fwd_work_range(B, T, heads, 128, G, i)[2:] == (0, 0)
+
+
 def test_fwd_gpu_argument_errors():
     q = torch.zeros(1, 100, 1, 64, device=DEV)
     v = torch.zeros(1, 100, 1, 128, device=DEV)
