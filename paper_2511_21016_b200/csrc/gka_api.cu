@@ -162,14 +162,14 @@ int gka_fwd_num_work_items(const gka_desc *desc, int chunk) {
         // sequences (pairs / k work items of k sequences each, k the smallest divisor of the number of (sequence, head)
         // pairs that leaves at most one item per SM) need no summaries, but may leave SMs idle in the state kernel and
         // make its run of tiles longer.  Measured per 128-token tile and block: 2.94 us in the state kernel with whole
-        // sequences (2.43 us where two blocks share an item, one per master: at most half as many items as SMs),
+        // sequences (2.15 us where two blocks share an item, one per master: at most half as many items as SMs),
         // 5.12 us x pairs / SMs for the summary and state kernels with one range per SM, which also cost 28 us more
         // per call.
         const long long pairs = (long long)desc->B * desc->heads, n = tiles_of(desc->T);
         for (long long k = (pairs + sms - 1) / sms; k <= pairs && k <= 64; ++k) {
             if (pairs % k != 0 || pairs / k > cap) continue;
             const long long items = pairs / k;
-            const double per_tile = 2 * items <= sms ? 2.43 : 2.94;
+            const double per_tile = 2 * items <= sms ? 2.15 : 2.94;
             if ((double)n * ((double)k * per_tile - 5.12 * (double)pairs / sms) < 28.0) return (int)items;
             break;
         }

@@ -241,7 +241,9 @@ fwd_tc_summary_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 // masters, which it keeps in registers in fp32 for a whole run.  The tensor cores compute only each tile's
 // increments dH = K~^T K~, dU = V~^T K~ into one of two TMEM buffers, one tile ahead of their use; per tile a thread
 // stores the bf16 copies of its part of the tile-initial H_0, U_0 (and adds up ||H_0||_F^2), then advances its
-// masters: H <- zeta H + dH, U <- zeta U + dU.
+// masters: H <- zeta H + dH, U <- zeta U + dU.  The warp that issues the products also turns the gates into the row
+// factors and the tile's decay, two tiles ahead, so that the compute warps meet no scan.  SPLIT: two blocks per work
+// item, one keeps H (and loads only the keys), one keeps U.
 // ------------------------------------------------------------------------------------------------------------
 // TB_STG0 + stage: one barrier per stage, like the loads.  (With a single barrier the compute warps could complete two
 // phases, tiles m + 1 and m + 2, while the TMA thread was still held up behind tile m's store; the phase parity it
@@ -255,7 +257,7 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t s_bars[TB_COUNT];
     __shared__ uint32_t s_tmem_base;
-    __shared__ float s_w[NT], s_ca[4], s_red[3][16], s_decay[3];
+    __shared__ float s_w[3][NT], s_red[3][16], s_decay[4];
     __shared__ int s_req, s_abort;
     unsigned char *smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
     const uint32_t sb = smem_u32(smem), bars = smem_u32(&s_bars[0]);
@@ -339,7 +341,57 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");    // the stores are complete
         }
     } else if (t >= CT) {
-        // ================================ MMA issuing warp ================================
+        // ================ MMA issuing warp; it also prepares the row factors, two tiles ahead ================
+        // Row factors sqrt(beta_j 2^(G_last - G_j)) (0 past the sequence) and decay of tile m: lane l has tokens l, 32 + l,
+        // 64 + l, 96 + l.  Written two hand-overs before the compute warps read them, so the hand-over barrier in between
+        // orders the two; three sets, so that no set is rewritten while a slower warp may still read it.
+        float lg[4], sb[4];          // gates and write strengths of the tile whose factors come next (loaded a hand-over ahead)
+        auto load_scalars = [&](int m, float(&lg)[4], float(&sb)[4]) {
+#pragma unroll
+            for (int grp = 0; grp < 4; ++grp) {
+                lg[grp] = 1.f;
+                sb[grp] = 0.f;
+            }
+            if (m >= n_mine) return;
+            const Pos p = pos_of(m);
+#pragma unroll
+            for (int grp = 0; grp < 4; ++grp) {
+                const int tok = 32 * grp + l;
+                if (tok < p.ntok) {
+                    lg[grp] = ldg_stream_f32(a.gate + p.tok0 + (size_t)tok * a.heads);
+                    sb[grp] = a.beta ? fmaxf(ldg_stream_f32(a.beta + p.tok0 + (size_t)tok * a.heads), 0.f) : 1.f;
+                }
+            }
+        };
+        auto factors = [&](int m, float(&lg)[4], const float(&sb)[4]) {      // from the loaded scalars of tile m
+            float before = 0.f;
+#pragma unroll
+            for (int grp = 0; grp < 4; ++grp) {
+                float incl = fmaxf(log2f(lg[grp]), -115.f);
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const float up = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (l >= o) incl += up;
+                }
+                const float tot = __shfl_sync(0xffffffffu, incl, 31);
+                lg[grp] = incl + before;             // cumulative log2 gate up to and including the token
+                before += tot;
+            }
+            const float tile_total = before;
+#pragma unroll
+            for (int grp = 0; grp < 4; ++grp) s_w[m % 3][32 * grp + l] = sqrtf(sb[grp]) * exp2f(0.5f * (tile_total - lg[grp]));
+            if (l == 0) s_decay[m & 3] = exp2f(tile_total);      // (four deep: tile m's is read after the hand-over of tile m + 1, behind which tile m + 3's is written)
+            __syncwarp();
+        };
+        if (n_mine > 0) {
+            float lg1[4], sb1[4];
+            load_scalars(0, lg, sb);
+            load_scalars(1, lg1, sb1);               // (both tiles' loads in flight together)
+            factors(0, lg, sb);
+            if (n_mine > 1) factors(1, lg1, sb1);
+            load_scalars(2, lg, sb);
+            asm volatile("bar.sync 3, 544;" ::: "memory");       // the factors of the first two tiles are published
+        }
         for (;;) {
             asm volatile("bar.sync 3, 544;" ::: "memory");
             const int m = *reinterpret_cast<const volatile int *>(&s_req);
@@ -353,6 +405,10 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 mma_commit(bars + 8 * (TB_D0 + (m & 1)));
             }
             __syncwarp();
+            if (m + 2 < n_mine) {
+                factors(m + 2, lg, sb);
+                load_scalars(m + 3, lg, sb);         // (in flight across the hand-over)
+            }
         }
     } else if (n_mine > 0) {
         // ================================= compute threads =================================
@@ -366,44 +422,10 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             chain_j0 = item - 1;
             while (P.lo(chain_j0) > seq_start) --chain_j0;
         }
-        // gate and write strength of this thread's token of tile m (threads 0..127; 1 and 0 past the sequence); returned
-        // by value so that the loads stay in registers until they are used a tile later
-        auto load_scalars = [&](int m) -> float2 {
-            float g = 1.f, bt = 0.f;
-            if (t < NT && m < n_mine) {
-                const Pos p = pos_of(m);
-                if (t < p.ntok) {
-                    g = ldg_stream_f32(a.gate + p.tok0 + (size_t)t * a.heads);
-                    bt = a.beta ? fmaxf(ldg_stream_f32(a.beta + p.tok0 + (size_t)t * a.heads), 0.f) : 1.f;
-                }
-            }
-            return make_float2(g, bt);
-        };
-        // Tile m: row factors sqrt(beta_j 2^(G_last - G_j)) (0 past the sequence), rows scaled in place, products posted.
-        // (g, bt): this thread's gate and write strength of the tile (threads 0..127).
-        auto prepare = [&](int m, float g, float bt) {
-            if (t < NT) {
-                float incl = fmaxf(log2f(g), -115.f);
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const float up = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (l >= o) incl += up;
-                }
-                if (l == 31) s_ca[t >> 5] = incl;
-                asm volatile("bar.sync 2, 128;" ::: "memory");
-                float before = 0.f, tile_total = 0.f;
-#pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    if (w < (t >> 5)) before += s_ca[w];
-                    tile_total += s_ca[w];
-                }
-                incl += before;
-                s_w[t] = sqrtf(bt) * exp2f(0.5f * (tile_total - incl));
-                if (t == 0) s_decay[m % 3] = exp2f(tile_total);     // (three deep: thread 0 writes tile m + 2's while slower warps may still read tile m's)
-            }
+        // Tile m: rows scaled in place by the row factors (prepared by the issuing warp), products posted.
+        auto prepare = [&](int m) {
             wait(TB_KV0 + m % NS, (uint32_t)((m / NS) & 1));
-            asm volatile("bar.sync 1, 512;" ::: "memory");       // factors are published
-            scale_kv(smem + (size_t)(m % NS) * STAGE, s_w, t, do_u);
+            scale_kv(smem + (size_t)(m % NS) * STAGE, s_w[m % 3], t, do_u);
             fence_async_smem();
             fence_before();
             if (t == 0) *reinterpret_cast<volatile int *>(&s_req) = m;
@@ -411,19 +433,14 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         };
 
         float mH[32], mU[32];
-        float2 nx = load_scalars(0);
-        prepare(0, nx.x, nx.y);
-        nx = load_scalars(1);
+        asm volatile("bar.sync 3, 544;" ::: "memory");           // the factors of the first two tiles are published
+        prepare(0);
         // summaries and start states are read after this point only
         asm volatile("griddepcontrol.wait;" ::: "memory");
 
         for (int m = 0; m < n_mine; ++m) {
             const Pos p = pos_of(m);
-            if (m + 1 < n_mine) {
-                const float2 cur = nx;
-                nx = load_scalars(m + 2);
-                prepare(m + 1, cur.x, cur.y);                    // its products run under this tile's passes
-            }
+            if (m + 1 < n_mine) prepare(m + 1);                  // its products run under this tile's passes
             const long long tile = f_lo + m;
             if (p.run_start) {
                 // start of a run: the caller's initial state of the sequence (or zero), carried through the summaries
@@ -468,7 +485,7 @@ fwd_tc_state_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
             // own K (V) in operand layout and goes from there to the workspace by TMA; then its increments are added
             wait(TB_D0 + (m & 1), (uint32_t)((m >> 1) & 1));     // the tile's increments are complete (posted a tile ago)
             fence_after();
-            const float decay = s_decay[m % 3];
+            const float decay = s_decay[m & 3];
             unsigned char *const stg = smem + (size_t)(m % NS) * STAGE;   // the tile's own K and V are no longer needed
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
